@@ -1,0 +1,119 @@
+/*
+ * im2win on NVIDIA B200 (sm_100a): the im2win data transformation and the
+ * im2win-based convolution, behind a plain C ABI.
+ *
+ * Notation follows the paper: input I[N][C][H][W], filter F[K][C][Fh][Fw],
+ * output O[N][K][Ho][Wo], one stride s for both directions, no padding, no
+ * dilation, no groups, no bias, no filter flip (Section II-A, Eq. 1).  All
+ * tensors are dense and row-major ("stored as a 1D array", Section I) in fp32.
+ * The im2win tensor is Ihat[N][C][Ho][W*Fh] (Section III-A, Algorithm 1).
+ *
+ * Unless a function says HOST, data pointers are DEVICE pointers owned by the
+ * caller; the library never frees or keeps them.  Shapes are passed by pointer
+ * to a plain struct in host memory that is read before the call returns.
+ * Device work is enqueued on the CUDA stream given as `cuda_stream`
+ * (a cudaStream_t cast to void*; NULL = the default stream) and the call
+ * returns without synchronising.  Every function returns IM2WIN_OK (0) or a
+ * negative im2win_status; nothing is launched when an error is returned.
+ * There is no CPU fallback: without a CUDA device the launching calls return
+ * IM2WIN_ECUDA.
+ */
+#ifndef IM2WIN_H
+#define IM2WIN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct {
+  int32_t N, C, H, W;  /* input  I[N][C][H][W]                      */
+  int32_t K, Fh, Fw;   /* filter F[K][C][Fh][Fw]                    */
+  int32_t stride;      /* s >= 1, the same in both directions       */
+} im2win_shape;
+
+/* What `src` of im2win_conv points to. */
+enum { IM2WIN_SRC_NCHW = 0,   /* the untransformed input I; the call runs the transform first   */
+       IM2WIN_SRC_IM2WIN = 1  /* an im2win tensor Ihat produced earlier by im2win_transform      */ };
+
+/* Arithmetic of the contraction.  Products are accumulated in fp32 in every mode. */
+enum { IM2WIN_MODE_TF32 = 0,  /* tensor cores, operands read as TF32 (low 13 mantissa bits unused) */
+       IM2WIN_MODE_BF16 = 1,  /* tensor cores, operands rounded to BF16 (nearest-even) on the fly  */
+       IM2WIN_MODE_FP32 = 2   /* plain fp32 FMA on the CUDA cores: a slow exact-arithmetic check    */ };
+
+typedef enum {
+  IM2WIN_OK = 0,
+  IM2WIN_EINVAL = -1,       /* null pointer, size < 1, Fh > H, Fw > W, unknown enum, size overflow */
+  IM2WIN_EALIGN = -2,       /* a device base pointer is not 16-byte aligned                        */
+  IM2WIN_EWORKSPACE = -3,   /* workspace missing or smaller than im2win_workspace_bytes            */
+  IM2WIN_EOVERLAP = -4,     /* an output range overlaps an input or workspace range                */
+  IM2WIN_ECUDA = -5,        /* a CUDA runtime call or kernel launch failed                         */
+  IM2WIN_ETIMEOUT = -6,     /* a bounded device-side wait expired (see im2win_last_device_status)  */
+  IM2WIN_EUNSUPPORTED = -7  /* shape outside what the kernels implement (see im2win_conv)          */
+} im2win_status;
+
+/* Output sizes, Ho = floor((H-Fh)/s)+1 and Wo = floor((W-Fw)/s)+1
+ * (Algorithm 1, first line; Table I fixes the division as floor). */
+int im2win_out_dims(const im2win_shape* shape, int32_t* Ho, int32_t* Wo);
+
+/* Bytes of the im2win tensor, 4*N*C*Ho*Fh*W (Section III-A: "the size of the im2win tensor is
+ * Ni x Ci x Hf x Wi x ((Hi-Hf)/s+1)").  This is the workspace im2win_conv needs when it is given
+ * the untransformed input, and the size of im2win_transform's output.  The same tight size is
+ * used when Fh <= s, where Algorithm 1 allocates the (larger or equal) input size instead. */
+int im2win_workspace_bytes(const im2win_shape* shape, size_t* bytes);
+
+/* Bytes an im2col matrix for the whole batch would take, 4*N*C*Fh*Fw*Ho*Wo (Section III-A).
+ * Reporting only: the library never builds one. */
+int im2win_im2col_bytes(const im2win_shape* shape, size_t* bytes);
+
+/* Algorithm 1:  Ihat[i][r][m][k*Fh+u] = I[i][r][m*s+u][k]  for every k in [0, W).
+ * in_nchw:    device, N*C*H*W floats, read only.
+ * out_im2win: device, N*C*Ho*W*Fh floats, every element is written; bit-exact copy of the inputs.
+ * Both bases 16-byte aligned (EALIGN); the ranges must not overlap (EOVERLAP). */
+int im2win_transform(const float* in_nchw, const im2win_shape* shape, float* out_im2win,
+                     void* cuda_stream);
+
+/* Algorithm 2 (the im2win-based convolution; its result is Eq. 1):
+ *   O[i][j][m][n] = sum_{r,u,v} Ihat[i][r][m][(n*s+v)*Fh+u] * F[j][r][u][v].
+ * (Algorithm 2 prints the strip offset as n*s*Wf+v*Hf+u, which equals the above for Hf==Wf and
+ * is the form consistent with Algorithm 1 otherwise.)
+ * src:       device.  src_kind NCHW: the input I (N*C*H*W floats); the call first runs the
+ *            transform into `workspace`, which then holds Ihat and may be reused by the caller.
+ *            src_kind IM2WIN: an im2win tensor; `workspace` is ignored and may be NULL.
+ * filter:    device, K*C*Fh*Fw floats, native K,C,Fh,Fw order (no repacking needed).
+ * mode:      IM2WIN_MODE_*.
+ * out_nchw:  device, N*K*Ho*Wo floats, every element is written.
+ * workspace: device, at least im2win_workspace_bytes(shape) bytes when src_kind is NCHW
+ *            (EWORKSPACE otherwise), 16-byte aligned.
+ * Limits of the tensor-core modes (EUNSUPPORTED beyond them): Fh*Fw <= 1024; one output row's
+ * worth of staged strips must fit in shared memory (W*Fh up to a few thousand floats).
+ * IM2WIN_MODE_FP32 has no such limits. */
+int im2win_conv(const void* src, int src_kind, const float* filter_kcfhfw,
+                const im2win_shape* shape, int mode, float* out_nchw,
+                void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* HOST-buffer convenience for callers without device memory of their own: copies the input and
+ * the filter from host memory, runs transform + convolution on an internal stream and copies the
+ * result back; returns after the result is in out_host.  Device buffers are owned by the library,
+ * grown on demand and kept for the next call (released by im2win_host_release).  Not reentrant.
+ * in_host: N*C*H*W floats; filter_host: K*C*Fh*Fw floats; out_host: N*K*Ho*Wo floats (pinned
+ * memory makes the copies faster, pageable memory is accepted). */
+int im2win_conv_host(const float* in_host, const float* filter_host, const im2win_shape* shape,
+                     int mode, float* out_host);
+int im2win_host_release(void);
+
+/* Kernels never trap.  A bounded wait that expires, or an internal range check that fails,
+ * records a code in a device-side status word and the kernel exits early (its output is then
+ * undefined).  This call synchronises `cuda_stream`, returns the word in *status (0 = clean)
+ * and clears it. */
+int im2win_last_device_status(void* cuda_stream, int32_t* status);
+
+/* English text for a status code; never NULL. */
+const char* im2win_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

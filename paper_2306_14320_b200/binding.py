@@ -1,0 +1,148 @@
+"""Thin ctypes binding of libim2win.so: same names as the C ABI (include/im2win.h), argument
+marshalling only.  Every step of the path runs in the CUDA kernels behind those calls.
+
+torch is used for device memory and streams: tensor arguments are passed as ``data_ptr()`` and the
+launch goes to ``torch.cuda.current_stream()``.  There is no fallback of any kind: if the shared
+library is missing this module raises at first use, and the launching calls raise ``Im2winError``
+when the library reports an error (for example no CUDA device).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libim2win.so")
+
+SRC_NCHW, SRC_IM2WIN = 0, 1
+MODE_TF32, MODE_BF16, MODE_FP32 = 0, 1, 2
+OK, EINVAL, EALIGN, EWORKSPACE, EOVERLAP, ECUDA, ETIMEOUT, EUNSUPPORTED = 0, -1, -2, -3, -4, -5, -6, -7
+
+EXPORTS = ("im2win_out_dims", "im2win_workspace_bytes", "im2win_im2col_bytes", "im2win_transform",
+           "im2win_conv", "im2win_conv_host", "im2win_host_release", "im2win_last_device_status",
+           "im2win_strerror")
+
+
+class Shape(ctypes.Structure):
+    """im2win_shape: N, C, H, W, K, Fh, Fw, stride (all int32)."""
+    _fields_ = [(n, ctypes.c_int32) for n in ("N", "C", "H", "W", "K", "Fh", "Fw", "stride")]
+
+    @classmethod
+    def of(cls, dims: "Shape | Sequence[int]") -> "Shape":
+        return dims if isinstance(dims, cls) else cls(*[int(d) for d in dims])
+
+
+class Im2winError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libim2win.so (built in-tree by ``paper_2306_14320_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2306_14320_b200.build` "
+                              "(there is no non-CUDA fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        sp, vp = ctypes.POINTER(Shape), ctypes.c_void_p
+        L.im2win_out_dims.argtypes = [sp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+        L.im2win_workspace_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
+        L.im2win_im2col_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
+        L.im2win_transform.argtypes = [vp, sp, vp, vp]
+        L.im2win_conv.argtypes = [vp, ctypes.c_int, vp, sp, ctypes.c_int, vp, vp, ctypes.c_size_t, vp]
+        L.im2win_conv_host.argtypes = [vp, vp, sp, ctypes.c_int, vp]
+        L.im2win_host_release.argtypes = []
+        L.im2win_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
+        L.im2win_strerror.argtypes = [ctypes.c_int]
+        L.im2win_strerror.restype = ctypes.c_char_p
+        for name in EXPORTS[:-1]:
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise Im2winError(code, where)
+
+
+def _ptr(t) -> int:
+    """Device (or host) address of a torch tensor / numpy array / int."""
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        if not t.is_contiguous():
+            raise ValueError("tensor must be contiguous")
+        return t.data_ptr()
+    if hasattr(t, "ctypes"):
+        return t.ctypes.data
+    raise TypeError(type(t))
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return int(getattr(stream, "cuda_stream", stream))
+
+
+def strerror(code: int) -> str:
+    return lib().im2win_strerror(int(code)).decode()
+
+
+def out_dims(shape) -> tuple[int, int]:
+    ho, wo = ctypes.c_int32(), ctypes.c_int32()
+    _check(lib().im2win_out_dims(ctypes.byref(Shape.of(shape)), ctypes.byref(ho), ctypes.byref(wo)), "im2win_out_dims")
+    return ho.value, wo.value
+
+
+def workspace_bytes(shape) -> int:
+    b = ctypes.c_size_t()
+    _check(lib().im2win_workspace_bytes(ctypes.byref(Shape.of(shape)), ctypes.byref(b)), "im2win_workspace_bytes")
+    return b.value
+
+
+def im2col_bytes(shape) -> int:
+    b = ctypes.c_size_t()
+    _check(lib().im2win_im2col_bytes(ctypes.byref(Shape.of(shape)), ctypes.byref(b)), "im2win_im2col_bytes")
+    return b.value
+
+
+def transform(in_nchw, shape, out_im2win, stream=None) -> None:
+    """im2win_transform on the current (or given) stream; asynchronous."""
+    _check(lib().im2win_transform(_ptr(in_nchw), ctypes.byref(Shape.of(shape)), _ptr(out_im2win), _stream(stream)),
+           "im2win_transform")
+
+
+def conv(src, src_kind: int, filter_kcfhfw, shape, mode: int, out_nchw, workspace=None,
+         workspace_nbytes: int | None = None, stream=None) -> None:
+    """im2win_conv on the current (or given) stream; asynchronous."""
+    if workspace_nbytes is None:
+        workspace_nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().im2win_conv(_ptr(src), int(src_kind), _ptr(filter_kcfhfw), ctypes.byref(Shape.of(shape)),
+                             int(mode), _ptr(out_nchw), _ptr(workspace), int(workspace_nbytes), _stream(stream)),
+           "im2win_conv")
+
+
+def conv_host(in_host, filter_host, shape, mode: int, out_host) -> None:
+    """im2win_conv_host: HOST buffers in, HOST buffer out; returns when the result is there."""
+    _check(lib().im2win_conv_host(_ptr(in_host), _ptr(filter_host), ctypes.byref(Shape.of(shape)), int(mode),
+                                  _ptr(out_host)), "im2win_conv_host")
+
+
+def host_release() -> None:
+    _check(lib().im2win_host_release(), "im2win_host_release")
+
+
+def last_device_status(stream=None) -> int:
+    st = ctypes.c_int32()
+    _check(lib().im2win_last_device_status(_stream(stream), ctypes.byref(st)), "im2win_last_device_status")
+    return st.value

@@ -1,0 +1,234 @@
+// C-ABI entry points: argument checks, size queries and dispatch to the kernels.
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace im2win {
+
+namespace {
+
+__device__ int32_t g_status_word = 0;
+
+bool mul_ok(int64_t a, int64_t b, int64_t* out) {
+  if (a < 0 || b < 0) return false;
+  if (a != 0 && b > INT64_MAX / a) return false;
+  *out = a * b;
+  return true;
+}
+
+bool prod(int64_t* out, std::initializer_list<int64_t> v) {
+  int64_t p = 1;
+  for (int64_t x : v)
+    if (!mul_ok(p, x, &p)) return false;
+  // keep byte counts (x4) and float offsets comfortably inside int64 / size_t
+  if (p > (INT64_MAX >> 4)) return false;
+  *out = p;
+  return true;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool overlap(const void* a, int64_t abytes, const void* b, int64_t bbytes) {
+  const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+  return a0 < b0 + (uintptr_t)bbytes && b0 < a0 + (uintptr_t)abytes;
+}
+
+}  // namespace
+
+int make_geometry(const im2win_shape* sh, Geometry* g) {
+  if (!sh || !g) return IM2WIN_EINVAL;
+  if (sh->N < 1 || sh->C < 1 || sh->H < 1 || sh->W < 1 || sh->K < 1 || sh->Fh < 1 || sh->Fw < 1 ||
+      sh->stride < 1)
+    return IM2WIN_EINVAL;
+  if (sh->Fh > sh->H || sh->Fw > sh->W) return IM2WIN_EINVAL;
+  g->N = sh->N; g->C = sh->C; g->H = sh->H; g->W = sh->W;
+  g->K = sh->K; g->Fh = sh->Fh; g->Fw = sh->Fw; g->s = sh->stride;
+  g->Ho = (sh->H - sh->Fh) / sh->stride + 1;
+  g->Wo = (sh->W - sh->Fw) / sh->stride + 1;
+  int64_t L, FF, sFh;
+  if (!prod(&L, {sh->W, sh->Fh}) || !prod(&FF, {sh->Fh, sh->Fw}) || !prod(&sFh, {sh->stride, sh->Fh}))
+    return IM2WIN_EINVAL;
+  if (L > INT32_MAX / 4 || FF > INT32_MAX / 4 || sFh > INT32_MAX / 4) return IM2WIN_EINVAL;
+  g->L = (int32_t)L; g->FF = (int32_t)FF; g->sFh = (int32_t)sFh;
+  if (!prod(&g->HoL, {g->Ho, L}) || !prod(&g->HoWo, {g->Ho, g->Wo}) || !prod(&g->Kg, {sh->C, FF}) ||
+      !prod(&g->Mtot, {sh->N, g->HoWo}) || !prod(&g->n_in, {sh->N, sh->C, sh->H, sh->W}) ||
+      !prod(&g->n_win, {sh->N, sh->C, g->HoL}) || !prod(&g->n_col, {sh->N, sh->C, FF, g->HoWo}) ||
+      !prod(&g->n_out, {sh->N, sh->K, g->HoWo}) || !prod(&g->n_flt, {sh->K, g->Kg}))
+    return IM2WIN_EINVAL;
+  return IM2WIN_OK;
+}
+
+int32_t* device_status_word() {
+  void* p = nullptr;
+  if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  return static_cast<int32_t*>(p);
+}
+
+}  // namespace im2win
+
+using namespace im2win;
+
+extern "C" {
+
+int im2win_out_dims(const im2win_shape* shape, int32_t* Ho, int32_t* Wo) {
+  Geometry g;
+  if (!Ho || !Wo) return IM2WIN_EINVAL;
+  int rc = make_geometry(shape, &g);
+  if (rc != IM2WIN_OK) return rc;
+  *Ho = g.Ho;
+  *Wo = g.Wo;
+  return IM2WIN_OK;
+}
+
+int im2win_workspace_bytes(const im2win_shape* shape, size_t* bytes) {
+  Geometry g;
+  if (!bytes) return IM2WIN_EINVAL;
+  int rc = make_geometry(shape, &g);
+  if (rc != IM2WIN_OK) return rc;
+  *bytes = (size_t)g.n_win * sizeof(float);
+  return IM2WIN_OK;
+}
+
+int im2win_im2col_bytes(const im2win_shape* shape, size_t* bytes) {
+  Geometry g;
+  if (!bytes) return IM2WIN_EINVAL;
+  int rc = make_geometry(shape, &g);
+  if (rc != IM2WIN_OK) return rc;
+  *bytes = (size_t)g.n_col * sizeof(float);
+  return IM2WIN_OK;
+}
+
+int im2win_transform(const float* in_nchw, const im2win_shape* shape, float* out_im2win,
+                     void* cuda_stream) {
+  Geometry g;
+  int rc = make_geometry(shape, &g);
+  if (rc != IM2WIN_OK) return rc;
+  if (!in_nchw || !out_im2win) return IM2WIN_EINVAL;
+  if (!aligned16(in_nchw) || !aligned16(out_im2win)) return IM2WIN_EALIGN;
+  if (overlap(in_nchw, g.n_in * 4, out_im2win, g.n_win * 4)) return IM2WIN_EOVERLAP;
+  return launch_transform(in_nchw, out_im2win, g, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int im2win_conv(const void* src, int src_kind, const float* filter, const im2win_shape* shape,
+                int mode, float* out_nchw, void* workspace, size_t workspace_bytes,
+                void* cuda_stream) {
+  Geometry g;
+  int rc = make_geometry(shape, &g);
+  if (rc != IM2WIN_OK) return rc;
+  if (!src || !filter || !out_nchw) return IM2WIN_EINVAL;
+  if (src_kind != IM2WIN_SRC_NCHW && src_kind != IM2WIN_SRC_IM2WIN) return IM2WIN_EINVAL;
+  if (mode != IM2WIN_MODE_TF32 && mode != IM2WIN_MODE_BF16 && mode != IM2WIN_MODE_FP32)
+    return IM2WIN_EINVAL;
+  if (!aligned16(src) || !aligned16(filter) || !aligned16(out_nchw)) return IM2WIN_EALIGN;
+  const int64_t src_bytes = (src_kind == IM2WIN_SRC_NCHW ? g.n_in : g.n_win) * 4;
+  if (overlap(out_nchw, g.n_out * 4, src, src_bytes) || overlap(out_nchw, g.n_out * 4, filter, g.n_flt * 4))
+    return IM2WIN_EOVERLAP;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const float* xhat = static_cast<const float*>(src);
+  if (src_kind == IM2WIN_SRC_NCHW) {
+    if (!workspace || workspace_bytes < (size_t)g.n_win * 4) return IM2WIN_EWORKSPACE;
+    if (!aligned16(workspace)) return IM2WIN_EALIGN;
+    if (overlap(workspace, g.n_win * 4, src, src_bytes) ||
+        overlap(workspace, g.n_win * 4, out_nchw, g.n_out * 4) ||
+        overlap(workspace, g.n_win * 4, filter, g.n_flt * 4))
+      return IM2WIN_EOVERLAP;
+    rc = launch_transform(static_cast<const float*>(src), static_cast<float*>(workspace), g, st);
+    if (rc != IM2WIN_OK) return rc;
+    xhat = static_cast<const float*>(workspace);
+  }
+  if (mode == IM2WIN_MODE_FP32) return launch_conv_fp32(xhat, filter, out_nchw, g, st);
+  return launch_conv_tc(xhat, filter, out_nchw, g, mode, st);
+}
+
+int im2win_last_device_status(void* cuda_stream, int32_t* status) {
+  if (!status) return IM2WIN_EINVAL;
+  int32_t* word = device_status_word();
+  if (!word) return IM2WIN_ECUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return IM2WIN_ECUDA;
+  int32_t v = 0;
+  if (cudaMemcpy(&v, word, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return IM2WIN_ECUDA;
+  if (v != 0 && cudaMemset(word, 0, sizeof(v)) != cudaSuccess) return IM2WIN_ECUDA;
+  *status = v;
+  return IM2WIN_OK;
+}
+
+const char* im2win_strerror(int status) {
+  switch (status) {
+    case IM2WIN_OK: return "ok";
+    case IM2WIN_EINVAL: return "invalid argument (null pointer, size < 1, filter larger than input, unknown enum or size overflow)";
+    case IM2WIN_EALIGN: return "device pointer is not 16-byte aligned";
+    case IM2WIN_EWORKSPACE: return "workspace missing or smaller than im2win_workspace_bytes";
+    case IM2WIN_EOVERLAP: return "output range overlaps an input or workspace range";
+    case IM2WIN_ECUDA: return "CUDA runtime call or kernel launch failed (no device, or see cudaGetLastError)";
+    case IM2WIN_ETIMEOUT: return "a bounded device-side wait expired";
+    case IM2WIN_EUNSUPPORTED: return "shape outside what the tensor-core kernels implement";
+    default: return "unknown im2win status";
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host-buffer convenience path.
+
+namespace {
+struct HostCtx {
+  cudaStream_t stream = nullptr;
+  float *d_in = nullptr, *d_f = nullptr, *d_out = nullptr, *d_ws = nullptr;
+  size_t b_in = 0, b_f = 0, b_out = 0, b_ws = 0;
+} g_host;
+
+int grow(float** p, size_t* have, size_t need) {
+  if (*have >= need) return IM2WIN_OK;
+  if (*p) cudaFree(*p);
+  *p = nullptr;
+  *have = 0;
+  if (cudaMalloc(reinterpret_cast<void**>(p), need) != cudaSuccess) {
+    cudaGetLastError();
+    return IM2WIN_ECUDA;
+  }
+  *have = need;
+  return IM2WIN_OK;
+}
+}  // namespace
+
+int im2win_conv_host(const float* in_host, const float* filter_host, const im2win_shape* shape,
+                     int mode, float* out_host) {
+  Geometry g;
+  int rc = make_geometry(shape, &g);
+  if (rc != IM2WIN_OK) return rc;
+  if (!in_host || !filter_host || !out_host) return IM2WIN_EINVAL;
+  if (!g_host.stream && cudaStreamCreateWithFlags(&g_host.stream, cudaStreamNonBlocking) != cudaSuccess) {
+    cudaGetLastError();
+    return IM2WIN_ECUDA;
+  }
+  if ((rc = grow(&g_host.d_in, &g_host.b_in, (size_t)g.n_in * 4)) != IM2WIN_OK) return rc;
+  if ((rc = grow(&g_host.d_f, &g_host.b_f, (size_t)g.n_flt * 4)) != IM2WIN_OK) return rc;
+  if ((rc = grow(&g_host.d_out, &g_host.b_out, (size_t)g.n_out * 4)) != IM2WIN_OK) return rc;
+  if ((rc = grow(&g_host.d_ws, &g_host.b_ws, (size_t)g.n_win * 4)) != IM2WIN_OK) return rc;
+  cudaStream_t st = g_host.stream;
+  if (cudaMemcpyAsync(g_host.d_in, in_host, (size_t)g.n_in * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(g_host.d_f, filter_host, (size_t)g.n_flt * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return IM2WIN_ECUDA;
+  rc = im2win_conv(g_host.d_in, IM2WIN_SRC_NCHW, g_host.d_f, shape, mode, g_host.d_out, g_host.d_ws,
+                   g_host.b_ws, st);
+  if (rc != IM2WIN_OK) return rc;
+  if (cudaMemcpyAsync(out_host, g_host.d_out, (size_t)g.n_out * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return IM2WIN_ECUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return IM2WIN_ECUDA;
+  return IM2WIN_OK;
+}
+
+int im2win_host_release(void) {
+  if (g_host.stream) cudaStreamSynchronize(g_host.stream);
+  for (float** p : {&g_host.d_in, &g_host.d_f, &g_host.d_out, &g_host.d_ws})
+    if (*p) { cudaFree(*p); *p = nullptr; }
+  g_host.b_in = g_host.b_f = g_host.b_out = g_host.b_ws = 0;
+  if (g_host.stream) { cudaStreamDestroy(g_host.stream); g_host.stream = nullptr; }
+  return IM2WIN_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,139 @@
+"""GPU parity, convolution: the CUDA im2win convolution against the oracle's Eq. (1) in double.
+
+Tolerances (relative L2 over the whole output): 5e-3 in TF32 mode, 2e-2 in BF16 mode (the benchmark
+definition's), 2e-6 in the fp32 CUDA-core mode.  On small-integer data every product and partial sum
+is exact in all modes, so the result must be bit-identical to the oracle: that separates layout
+mistakes from rounding."""
+import itertools
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2306_14320_b200 import binding as b
+from paper_2306_14320_b200 import workloads as wl
+from gpu_helpers import TOL, ensure_built, gpu_conv, oracle_conv, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+MODES = [b.MODE_FP32, b.MODE_TF32, b.MODE_BF16]
+MODE_ID = {b.MODE_FP32: "fp32", b.MODE_TF32: "tf32", b.MODE_BF16: "bf16"}
+
+SMALL = [
+    (1, 1, 4, 4, 2, 2, 2, 1), (2, 3, 7, 9, 4, 3, 3, 1), (1, 2, 9, 8, 3, 2, 3, 1), (2, 2, 8, 11, 2, 3, 2, 2),
+    (1, 3, 13, 12, 2, 4, 2, 3), (1, 1, 10, 10, 1, 1, 1, 1), (2, 2, 6, 6, 3, 2, 2, 2), (1, 2, 11, 7, 2, 2, 2, 3),
+    (1, 1, 12, 13, 2, 1, 3, 4), (3, 2, 5, 5, 2, 5, 5, 1),          # 1x1 outputs: a tile spans many images
+    (2, 20, 19, 23, 40, 3, 3, 1),                                     # C, K not multiples of the tile sizes
+    (1, 9, 40, 41, 300, 3, 3, 2),                                     # K > 256: two filter tiles
+    (5, 7, 9, 9, 17, 3, 3, 1),                                        # 49 positions per image: tiles straddle images
+    (2, 3, 37, 35, 24, 7, 7, 2), (1, 3, 51, 51, 32, 11, 11, 4), (1, 12, 14, 14, 16, 5, 5, 1),
+]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    ensure_built()
+
+
+def _data(dims, seed, ints=False):
+    n, c, h, w, k, fh, fw, s = dims
+    if ints:
+        x = wl.small_ints(seed, n * c * h * w).reshape(n, c, h, w)
+        f = wl.small_ints(seed + 1, k * c * fh * fw, -2, 2).reshape(k, c, fh, fw)
+    else:
+        x = wl.normal01(seed, n * c * h * w).reshape(n, c, h, w)
+        f = (wl.normal01(seed + 1, k * c * fh * fw) * np.float32(np.sqrt(2.0 / (c * fh * fw)))).reshape(k, c, fh, fw)
+    return x, f
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_ID.get)
+@pytest.mark.parametrize("dims", SMALL)
+def test_conv_small_shapes(dims, mode):
+    x, f = _data(dims, 300)
+    ref = oracle_conv(x, f, dims)
+    got = gpu_conv(x, f, dims, mode)
+    assert np.isfinite(got).all()
+    assert rel_l2(got, ref) <= TOL[mode]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_ID.get)
+@pytest.mark.parametrize("dims", SMALL)
+def test_conv_small_integers_bit_exact(dims, mode):
+    x, f = _data(dims, 400, ints=True)
+    ref = oracle_conv(x, f, dims)
+    assert np.abs(ref).max() < 2 ** 24
+    got = gpu_conv(x, f, dims, mode)
+    assert np.array_equal(got.astype(np.float64), ref)
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+def test_conv_one_hot_filters_are_strided_crops(mode):
+    dims = (2, 3, 20, 22, 18, 3, 3, 2)
+    n, c, h, w, k, fh, fw, s = dims
+    x = wl.small_ints(77, n * c * h * w).reshape(n, c, h, w)
+    f = np.zeros((k, c, fh, fw), np.float32)
+    taps = list(itertools.product(range(c), range(fh), range(fw)))[:k]
+    for j, (r, u, v) in enumerate(taps):
+        f[j, r, u, v] = 1.0
+    got = gpu_conv(x, f, dims, mode)
+    ho, wo = b.out_dims(dims)
+    for j, (r, u, v) in enumerate(taps):
+        crop = x[:, r, u:u + (ho - 1) * s + 1:s, v:v + (wo - 1) * s + 1:s]
+        assert np.array_equal(got[:, j], crop), (j, r, u, v)
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+def test_conv_from_prebuilt_im2win_tensor(mode):
+    dims = (2, 16, 30, 30, 32, 3, 3, 1)
+    x, f = _data(dims, 500)
+    xhat = oracle.im2win(x, oracle.Shape(*dims))
+    got = gpu_conv(xhat, f, dims, mode, src_kind=b.SRC_IM2WIN)
+    assert rel_l2(got, oracle_conv(x, f, dims)) <= TOL[mode]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_ID.get)
+@pytest.mark.parametrize("name,batch", [("tiny", 1), ("resnet3x3", 2), ("stem7x7", 1), ("deep3x3", 3), ("down3x3", 1)])
+def test_conv_named_configs_reduced_batch(name, batch, mode):
+    layer = wl.CONFIGS[name].with_batch(batch)
+    x, f = wl.make_input(layer), wl.make_filter(layer)
+    ref = oracle_conv(x, f, layer.dims())
+    got = gpu_conv(x, f, layer.dims(), mode)
+    err = rel_l2(got, ref)
+    assert err <= TOL[mode], err
+    if mode != b.MODE_FP32:
+        # a reduced-precision mode that is "too exact" is not the mode it claims to be
+        assert err > 1e-5
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("layer", wl.SWEEP, ids=lambda l: l.name)
+def test_conv_sweep_layers_batch1(layer, mode):
+    layer = layer.with_batch(1)
+    x, f = wl.make_input(layer), wl.make_filter(layer)
+    assert rel_l2(gpu_conv(x, f, layer.dims(), mode), oracle_conv(x, f, layer.dims())) <= TOL[mode]
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("name", ["resnet3x3", "stem7x7", "deep3x3", "down3x3"])
+def test_conv_full_batch_sampled(name, mode):
+    """Batch 128, the launch configuration the benchmark times.  The oracle evaluates Eq. (1) at 20000
+    sampled output coordinates (plus every corner of the output tensor) and at the whole first and
+    last image."""
+    layer = wl.CONFIGS[name]
+    dims = layer.dims()
+    n, c, h, w, k, fh, fw, s = dims
+    x, f = wl.make_input(layer), wl.make_filter(layer)
+    got = gpu_conv(x, f, dims, mode)
+    ho, wo = b.out_dims(dims)
+    rng = np.random.default_rng(1234)
+    idx = np.stack([rng.integers(0, n, 20000), rng.integers(0, k, 20000), rng.integers(0, ho, 20000),
+                    rng.integers(0, wo, 20000)], axis=1).astype(np.int32)
+    corners = np.array(list(itertools.product((0, n - 1), (0, k - 1), (0, ho - 1), (0, wo - 1))), dtype=np.int32)
+    idx = np.concatenate([idx, corners])
+    ref = oracle.conv_direct_points(x, f, oracle.Shape(*dims), idx)
+    sample = got[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]]
+    assert rel_l2(sample, ref) <= TOL[mode]
+    for img in (0, n - 1):
+        one = layer.with_batch(1).dims()
+        assert rel_l2(got[img:img + 1], oracle_conv(x[img:img + 1], f, one)) <= TOL[mode]
+    assert np.isfinite(got).all()

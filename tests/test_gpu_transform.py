@@ -1,0 +1,60 @@
+"""GPU parity, transform: the CUDA im2win transformation must equal the oracle's Algorithm 1 bit for bit."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2306_14320_b200 import workloads as wl
+from gpu_helpers import ensure_built, gpu_transform
+
+pytestmark = pytest.mark.gpu
+
+SMALL = [
+    (1, 1, 4, 4, 1, 2, 2, 1), (2, 3, 7, 9, 4, 3, 3, 1), (1, 2, 9, 8, 3, 2, 3, 1), (2, 2, 8, 11, 2, 3, 2, 2),
+    (1, 3, 13, 12, 2, 4, 2, 3), (1, 1, 10, 10, 1, 1, 1, 1), (2, 2, 6, 6, 3, 2, 2, 2), (1, 2, 11, 7, 2, 2, 2, 3),
+    (1, 1, 12, 13, 2, 1, 3, 4), (1, 2, 5, 5, 2, 5, 5, 1), (3, 5, 33, 37, 2, 3, 3, 1), (2, 3, 64, 64, 2, 5, 5, 2),
+    (1, 2, 130, 1031, 1, 7, 7, 2),     # rows wide enough that one CTA takes only a few output rows
+    (1, 1, 30, 5000, 1, 11, 3, 4),     # beyond the staging budget: gather fallback
+    (1, 1, 1, 1, 1, 1, 1, 1),
+]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    ensure_built()
+
+
+def _bits(a):
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).ravel()
+
+
+@pytest.mark.parametrize("dims", SMALL)
+def test_transform_bit_exact_small(dims):
+    n, c, h, w = dims[:4]
+    x = wl.normal01(100 + h * w, n * c * h * w).reshape(n, c, h, w)
+    # a few special bit patterns must survive the copy unchanged
+    flat = x.reshape(-1)
+    flat[::97] = np.float32(-0.0)
+    flat.view(np.uint32)[5::211] = 0x7FC00001  # a NaN payload
+    flat.view(np.uint32)[7::313] = 0x00000001  # a denormal
+    ref = oracle.im2win(x, oracle.Shape(*dims))
+    assert np.array_equal(_bits(gpu_transform(x, dims)), _bits(ref))
+
+
+@pytest.mark.parametrize("name,batch", [("tiny", 1), ("resnet3x3", 3), ("stem7x7", 2), ("deep3x3", 3), ("down3x3", 2)]
+                         + [(l.name, 2) for l in wl.SWEEP])
+def test_transform_bit_exact_layer_shapes(name, batch):
+    layer = wl.CONFIGS[name].with_batch(batch)
+    x = wl.make_input(layer)
+    ref = oracle.im2win(x, oracle.Shape(*layer.dims()))
+    assert np.array_equal(_bits(gpu_transform(x, layer.dims())), _bits(ref))
+
+
+@pytest.mark.parametrize("name", ["resnet3x3", "stem7x7", "deep3x3", "down3x3"])
+def test_transform_bit_exact_full_batch(name):
+    """The launch configuration the benchmark times (batch 128), every element compared."""
+    layer = wl.CONFIGS[name]
+    x = wl.make_input(layer)
+    ref = oracle.im2win(x, oracle.Shape(*layer.dims()))
+    got = gpu_transform(x, layer.dims())
+    assert got.size == ref.size
+    assert np.array_equal(_bits(got), _bits(ref))
