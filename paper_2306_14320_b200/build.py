@@ -28,20 +28,24 @@ def _stale() -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into one shared library; returns its path."""
-    if not (force or _stale()):
+def build_library(force: bool = False, verbose: bool = False, out: str | None = None,
+                  defines: tuple[str, ...] = ()) -> str:
+    """Compile every .cu under csrc/ into one shared library; returns its path.  ``out``/``defines``
+    build a variant beside the product library (e.g. -DIM2WIN_PROF, the wait-cycle counters)."""
+    target = out or LIB
+    if out is None and not (force or _stale()):
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB + f".tmp{os.getpid()}"
+    tmp = target + f".tmp{os.getpid()}"
     cmd = [nvcc, "-std=c++17", "-O3", "-lineinfo", *ARCH_FLAGS, "-Xcompiler", "-fPIC", "-shared",
+           *[f"-D{d}" for d in defines],
            "-I", os.path.join(_ROOT, "include"), "-I", CSRC, "-o", tmp, *sources()]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, target)
+    return target
 
 
 if __name__ == "__main__":

@@ -1,5 +1,6 @@
 // C-ABI entry points: argument checks, size queries and dispatch to the kernels.
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "common.cuh"
@@ -57,6 +58,18 @@ int make_geometry(const im2win_shape* sh, Geometry* g) {
       !prod(&g->n_out, {sh->N, sh->K, g->HoWo}) || !prod(&g->n_flt, {sh->K, g->Kg}))
     return IM2WIN_EINVAL;
   return IM2WIN_OK;
+}
+
+int launch_conv_tc(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
+                   cudaStream_t st) {
+  // IM2WIN_FORCE_GENERIC=1 routes every shape through the generic kernel (used by the tests to
+  // cover both kernels on the same inputs).
+  const char* force = getenv("IM2WIN_FORCE_GENERIC");
+  if (!(force && force[0] == '1')) {
+    const int rc = launch_conv_tc_persistent(xhat, f, out, g, mode, st);
+    if (rc != IM2WIN_EUNSUPPORTED) return rc;
+  }
+  return launch_conv_tc_generic(xhat, f, out, g, mode, st);
 }
 
 int32_t* device_status_word() {

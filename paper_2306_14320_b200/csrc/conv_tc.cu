@@ -1,4 +1,6 @@
-// im2win-based convolution (Algorithm 2) on the sm_100a tensor cores.
+// im2win-based convolution (Algorithm 2) on the sm_100a tensor cores: generic kernel (any Fh, Fw, C, K).
+// The persistent kernel specialised on the filter size is preferred when one applies; this one takes
+// every other shape.
 //
 // The contraction  O[i][j][m][n] = sum_{r,u,v} Ihat[i][r][m][(n*s+v)*Fh+u] * F[j][r][u][v]  is run as a
 // GEMM with M = output positions (i,m,n flattened), N = filters j, K = (r,u,v):
@@ -405,7 +407,7 @@ int32_t round_up(int32_t x, int32_t m) { return (x + m - 1) / m * m; }
 
 }  // namespace
 
-int launch_conv_tc(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
+int launch_conv_tc_generic(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
                    cudaStream_t st) {
   ConvParams P{};
   P.xhat = xhat; P.f = f; P.out = out;

@@ -1,0 +1,737 @@
+// im2win-based convolution (Algorithm 2) on the sm_100a tensor cores: persistent, specialised kernel.
+//
+// Same GEMM view as the generic kernel (M = output positions, N = filters, K = (r,u,v); A = windows in
+// TENSOR MEMORY written by tcgen05.st, B = filters in shared memory, fp32 accumulators in TMEM), with
+//   * one persistent CTA per SM walking tiles t, t+grid, ... (neighbouring CTAs work on neighbouring
+//     tiles at the same time, so the few strip floats two tiles share are L2 hits);
+//   * the filter operand either RESIDENT in shared memory for the whole kernel (built once per CTA
+//     from the native K,C,Fh,Fw order; any shape, TF32 or BF16) or STREAMED per tile by TMA tensor
+//     loads straight from the native filter viewed as a K x (C*Fh*Fw) matrix (TF32, 128-byte swizzle);
+//   * filter sizes known at compile time, so a window's elements are loads at immediate offsets from
+//     one per-thread, per-channel base address (the window is contiguous in its im2win strip);
+//   * A columns handed to the MMA thread in sub-slots of a ring in TMEM, independent of the channel
+//     grouping of the staged strips;
+//   * two accumulator buffers when they fit, so that the epilogue of one tile (tcgen05.ld -> NCHW
+//     stores) overlaps the next tile's main loop.
+// Warps: 0 strip producer (TMA bulk copies), 1 MMA issuer, 2 filter producer (TMA), 4-11 window
+// repack (two per TMEM lane quarter), 12-15 epilogue.  Every wait is bounded (status word + common teardown on expiry).
+#include <cuda.h>
+
+#include <cstdlib>
+
+#include "common.cuh"
+#include "ptx_sm100.cuh"
+
+namespace im2win {
+
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kSegMax = 8;
+constexpr int kMaxStages = 8;
+constexpr int kMaxSub = 16;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct PParams {
+  const float* xhat;
+  const float* f;
+  float* out;
+  int32_t* status;
+  int32_t C, K, Ho, Wo, L, sFh;
+  int64_t HoL, HoWo, Kg, Mtot, n_win;
+  int32_t TP, NT, n_ntiles;
+  int64_t ntiles;       // m tiles * n tiles
+  int32_t NG;           // channel groups per tile
+  int32_t SR, SB;       // raw strip stages; filter stages (streamed mode)
+  int32_t SS, NSS;      // MMA steps per A slot; slots per repack half in the TMEM ring
+  int32_t ND;           // accumulator buffers
+  int32_t chan_pitch;
+  int32_t nchunks;      // 128-byte filter chunks per tile
+  int32_t tmem_cols;
+  uint32_t idesc;
+  uint32_t off_raw, off_bar, off_misc;
+#ifdef IM2WIN_PROF
+  long long* prof;  // debug build only: per-role wait-cycle counters of the first CTAs
+#endif
+};
+
+struct PBars {
+  uint64_t raw_full[kMaxStages], raw_empty[kMaxStages];
+  uint64_t b_full[kMaxStages], b_empty[kMaxStages];
+  uint64_t a_full[kMaxSub], a_empty[kMaxSub];
+  uint64_t acc_full[2], acc_empty[2];
+};
+
+struct PMisc {
+  uint32_t tmem_base;
+  int32_t abort;
+};
+
+struct SegR {
+  int64_t start0;
+  int64_t virt_a;
+  int32_t len;
+  int32_t dst_off;
+};
+
+__device__ __forceinline__ void record(const PParams& P, PMisc* misc, int32_t code) {
+  atomicCAS(P.status, 0, code);
+  atomicExch(&misc->abort, 1);
+}
+
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+#ifdef IM2WIN_PROF
+#define PROF_DECL(n) long long prof_acc[n] = {}; const long long prof_t0 = clock64();
+#define PROF_SLOT(k) (&prof_acc[k])
+#define PROF_DUMP(role, n)                                                         \
+  if (P.prof && blockIdx.x < 8 && lane == 0) {                                     \
+    long long* o = P.prof + ((long long)blockIdx.x * 8 + (role)) * 8;              \
+    o[0] = clock64() - prof_t0;                                                    \
+    for (int z = 0; z < (n); ++z) o[1 + z] = prof_acc[z];                          \
+  }
+#else
+#define PROF_DECL(n)
+#define PROF_SLOT(k) nullptr
+#define PROF_DUMP(role, n)
+#endif
+
+__device__ __forceinline__ bool wait_bar(const PParams& P, PMisc* misc, uint64_t* bar, uint32_t parity,
+                                         int32_t code, long long* acc = nullptr) {
+  const uint32_t b = ptx::smem_u32(bar);
+#ifdef IM2WIN_PROF
+  // try_wait may block inside the instruction, so the clock brackets the first poll too
+  const long long c0 = clock64();
+  struct Fin { long long* a; long long c; __device__ ~Fin() { if (a) *a += clock64() - c; } } fin{acc, c0};
+#endif
+  if (ptx::mbar_try_wait(b, parity)) return true;
+  uint64_t t0 = 0;
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (ptx::mbar_try_wait(b, parity)) return true;
+    if ((it & 63u) == 63u) {
+      if (*reinterpret_cast<volatile int32_t*>(&misc->abort)) return false;
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > 1000000000ull) break;
+    }
+  }
+  record(P, misc, code);
+  return false;
+}
+
+__device__ __forceinline__ bool wait_bar_warp(const PParams& P, PMisc* misc, uint64_t* bar, uint32_t parity,
+                                              int32_t code, long long* acc = nullptr) {
+  return __all_sync(0xffffffffu, wait_bar(P, misc, bar, parity, code, acc));
+}
+
+// Position in a ring of n stages together with the parity of the pass over it.
+struct Ring {
+  int32_t idx = 0;
+  uint32_t phase = 0;
+  __device__ __forceinline__ void advance(int32_t n) {
+    if (++idx == n) { idx = 0; phase ^= 1u; }
+  }
+};
+// A group's S MMA steps are handed over in PARTS slots of at most 13 steps (104 TMEM columns).
+template <int S>
+struct SlotGeom {
+  static constexpr int PARTS = (S * 8 + 103) / 104;
+  static constexpr int SLOT_STEPS = (S + PARTS - 1) / PARTS;
+};
+
+// Lanes 0..nseg-1 each describe one image segment of the tile; dst_off is the exclusive prefix sum
+// of the slot sizes.  Must be called by a converged warp.
+__device__ __forceinline__ SegR compute_seg(const PParams& P, int FF, int64_t P0, int64_t Pend, int64_t i_first,
+                                            int32_t nseg, int lane) {
+  SegR s{0, 0, 0, 0};
+  int32_t slot = 0;
+  if (lane < nseg) {
+    const int64_t i = i_first + lane;
+    const int64_t qa = max(P0 - i * P.HoWo, (int64_t)0);
+    const int64_t qb = min(Pend - i * P.HoWo, P.HoWo - 1);
+    const int64_t m_a = qa / P.Wo, n_a = qa - m_a * P.Wo;
+    const int64_t m_b = qb / P.Wo, n_b = qb - m_b * P.Wo;
+    s.virt_a = m_a * P.L + n_a * P.sFh;
+    s.start0 = (i * P.C * P.Ho) * (int64_t)P.L + s.virt_a;
+    s.len = (int32_t)((m_b * P.L + n_b * P.sFh) - s.virt_a) + FF;
+    slot = (s.len + 6) & ~3;
+  }
+  int32_t incl = slot;
+#pragma unroll
+  for (int d = 1; d < kSegMax; d <<= 1) {
+    const int32_t t = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += t;
+  }
+  s.dst_off = incl - slot;
+  return s;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+template <int FH, int FW, int CB, bool BF16, bool BRES>
+__global__ void __launch_bounds__(kThreads, 1)
+conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_constant__ CUtensorMap fmap) {
+  constexpr int FF = FH * FW;
+  constexpr int KSTEP = BF16 ? 16 : 8;        // reduction elements per MMA
+  constexpr int KCHUNK = BF16 ? 64 : 32;      // reduction elements per 128-byte filter row
+  constexpr int KCG = CB * FF;                // real reduction elements per channel group
+  constexpr int KCGP = (KCG + KSTEP - 1) / KSTEP * KSTEP;
+  constexpr int S = KCGP / KSTEP;             // MMA steps per channel group
+  constexpr int PARTS = SlotGeom<S>::PARTS;   // a group's A columns go to TMEM in PARTS slots
+  constexpr int SLOT_STEPS = SlotGeom<S>::SLOT_STEPS;
+  constexpr int SLOT_COLS = SLOT_STEPS * 8;
+
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* const smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
+  uint8_t* const b_smem = smem;  // resident: nchunks * NT*128 bytes; streamed: SB stages of NT*128 bytes
+  float* const raw = reinterpret_cast<float*>(smem + P.off_raw);
+  PBars* const bars = reinterpret_cast<PBars*>(smem + P.off_bar);
+  PMisc* const misc = reinterpret_cast<PMisc*>(smem + P.off_misc);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int32_t raw_stage_floats = CB * P.chan_pitch;
+  const uint32_t b_stage_bytes = (uint32_t)P.NT * 128u;
+
+  // ------------------------------------------------------------------ prologue
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kMaxStages; ++i) {
+      ptx::mbar_init(ptx::smem_u32(&bars->raw_full[i]), 32);
+      ptx::mbar_init(ptx::smem_u32(&bars->raw_empty[i]), 4);
+      ptx::mbar_init(ptx::smem_u32(&bars->b_full[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->b_empty[i]), 1);
+    }
+    for (int i = 0; i < kMaxSub; ++i) {
+      ptx::mbar_init(ptx::smem_u32(&bars->a_full[i]), 4);
+      ptx::mbar_init(ptx::smem_u32(&bars->a_empty[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), 4);
+    }
+    ptx::fence_mbar_init();
+    misc->abort = 0;
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), (uint32_t)P.tmem_cols);
+    ptx::tmem_relinquish();
+  }
+  if constexpr (BRES) {
+    // Build the whole filter operand once: chunk c holds padded reduction indices [c*KCHUNK, +KCHUNK)
+    // for all NT filters, K-major with the 128-byte swizzle.  (A resident filter implies one n-tile.)
+    constexpr int EPP = BF16 ? 8 : 4;
+    const int32_t pieces = P.nchunks * P.NT * 8;
+    for (int32_t idx = threadIdx.x; idx < pieces; idx += kThreads) {
+      const int32_t q = idx & 7, j = (idx >> 3) % P.NT, c = (idx >> 3) / P.NT;
+      float x[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        x[e] = 0.f;
+        if (e < EPP && j < P.K) {
+          const int32_t kp = c * KCHUNK + q * EPP + e;
+          const int32_t g = kp / KCGP, kl = kp - g * KCGP;
+          const int64_t k = (int64_t)g * KCG + kl;
+          if (kl < KCG && k < P.Kg) x[e] = __ldg(P.f + (int64_t)j * P.Kg + k);
+        }
+      }
+      uint4 piece;
+      if (BF16) {
+        piece.x = ptx::pack_bf16x2(x[0], x[1]); piece.y = ptx::pack_bf16x2(x[2], x[3]);
+        piece.z = ptx::pack_bf16x2(x[4], x[5]); piece.w = ptx::pack_bf16x2(x[6], x[7]);
+      } else {
+        piece.x = __float_as_uint(x[0]); piece.y = __float_as_uint(x[1]);
+        piece.z = __float_as_uint(x[2]); piece.w = __float_as_uint(x[3]);
+      }
+      *reinterpret_cast<uint4*>(b_smem + (size_t)c * b_stage_bytes + (j >> 3) * 1024 + (j & 7) * 128 +
+                                ((q ^ (j & 7)) << 4)) = piece;
+    }
+    ptx::fence_proxy_async_smem();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = misc->tmem_base;
+  const uint32_t tmem_a0 = tmem_base + (uint32_t)(P.ND * P.NT);
+
+  if (warp == 0) {
+    // ================================================================ STRIP PRODUCER
+    Ring rr;             // raw stage being filled
+    int64_t gcount = 0;  // channel groups issued so far (all tiles)
+    bool ok = true;
+    PROF_DECL(1)
+    for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x) {
+      const int64_t tile_m = t / P.n_ntiles;
+      const int64_t P0 = tile_m * P.TP, Pend = min(P0 + P.TP, P.Mtot) - 1;
+      const int64_t i_first = P0 / P.HoWo;
+      const int32_t nseg = (int32_t)(Pend / P.HoWo - i_first) + 1;
+      const SegR seg = compute_seg(P, FF, P0, Pend, i_first, nseg, lane);
+      const int32_t npairs = CB * nseg;
+      for (int32_t g = 0; g < P.NG && ok; ++g, ++gcount, rr.advance(P.SR)) {
+        const int32_t sr = rr.idx;
+        ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0));
+        if (!ok) break;
+        const uint32_t full = ptx::smem_u32(&bars->raw_full[sr]);
+        float* stage = raw + (size_t)sr * raw_stage_floats;
+        for (int32_t idx0 = 0; idx0 < npairs; idx0 += 32) {
+          const int32_t idx = idx0 + lane;
+          const bool act = idx < npairs;
+          const int32_t rl = act ? idx / nseg : 0, sg = act ? idx - rl * nseg : 0;
+          const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
+          const int32_t s_len = __shfl_sync(0xffffffffu, seg.len, sg);
+          const int32_t s_dst = __shfl_sync(0xffffffffu, seg.dst_off, sg);
+          const int32_t r = g * CB + rl;
+          if (!act || r >= P.C) continue;
+          const int64_t start = s_start0 + (int64_t)r * P.HoL;
+          const int32_t skew = (int32_t)(start & 3);
+          const int64_t a0 = start - skew;
+          int32_t nfl = (skew + s_len + 3) & ~3;
+          float* dst = stage + rl * P.chan_pitch + s_dst;
+          if (a0 + nfl > P.n_win) {  // the last 16-byte chunk would pass the end of the tensor
+            const int32_t nbulk = (int32_t)((P.n_win - a0) & ~(int64_t)3);
+            for (int64_t e = a0 + nbulk; e < P.n_win; ++e) dst[e - a0] = __ldg(P.xhat + e);
+            nfl = nbulk;
+          }
+          if (nfl > 0) {
+            ptx::mbar_expect_tx(full, (uint32_t)nfl * 4u);
+            ptx::bulk_g2s(ptx::smem_u32(dst), P.xhat + a0, (uint32_t)nfl * 4u, full);
+          }
+        }
+        __syncwarp();
+        ptx::mbar_arrive(full);
+      }
+    }
+    PROF_DUMP(0, 1)
+    // every copy issued must have landed before the CTA exits
+    for (int64_t g = max(gcount - P.SR, (int64_t)0); g < gcount; ++g)
+      wait_bar(P, misc, &bars->raw_full[g % P.SR], (uint32_t)(g / P.SR) & 1u, DEV_TIMEOUT_DRAIN);
+  } else if (warp == 1) {
+    // ================================================================ MMA ISSUER
+    // One thread; the loop body per MMA is kept to a handful of instructions because a single
+    // thread can only issue a tcgen05.mma every few tens of cycles.
+    if (lane == 0) {
+      Ring arh[2], br, dr;  // A slot (one ring per repack half), streamed filter stage, accumulator buffer
+      uint32_t gpar = 0;    // parity of the running group count = which half produced the group
+      bool ok = true;
+      PROF_DECL(3)
+      const uint64_t desc0 = ptx::smem_desc_k_sw128(ptx::smem_u32(b_smem));
+      const uint32_t chunk16 = b_stage_bytes >> 4;  // one filter chunk / stage in descriptor units
+      for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
+        const int32_t d = dr.idx;
+        ok = wait_bar(P, misc, &bars->acc_empty[d], dr.phase ^ 1u, DEV_TIMEOUT_ACC, PROF_SLOT(2));
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(d * P.NT);
+        uint32_t accum = 0;
+        int32_t bq = 0;           // step inside the current 128-byte filter chunk
+        uint64_t b_desc = desc0;  // resident: walks the chunks of the tile
+        for (int32_t g = 0; g < P.NG && ok; ++g, gpar ^= 1u) {
+          Ring& ar = arh[gpar];
+          const int32_t slot0 = (int32_t)gpar * P.NSS;
+#pragma unroll
+          for (int h = 0; h < PARTS; ++h) {
+            const int nst = (h == PARTS - 1) ? (S - (PARTS - 1) * SLOT_STEPS) : SLOT_STEPS;
+            const int32_t slot = slot0 + ar.idx;
+            ok = wait_bar(P, misc, &bars->a_full[slot], ar.phase, DEV_TIMEOUT_A_FULL, PROF_SLOT(0));
+            if (!ok) break;
+            ptx::tc_fence_after();
+            const uint32_t a_addr = tmem_a0 + (uint32_t)(slot * SLOT_COLS);
+#pragma unroll
+            for (int j = 0; j < SLOT_STEPS; ++j) {
+              if (j < nst) {
+                if constexpr (!BRES) {
+                  if (bq == 0) {
+                    ok = wait_bar(P, misc, &bars->b_full[br.idx], br.phase, DEV_TIMEOUT_B_FULL, PROF_SLOT(1));
+                    if (!ok) break;
+                    ptx::tc_fence_after();
+                    b_desc = desc0 + (uint64_t)((uint32_t)br.idx * chunk16);
+                  }
+                }
+                if (BF16) ptx::mma_ts_f16(d_tmem, a_addr + j * 8, b_desc, P.idesc, accum);
+                else      ptx::mma_ts_tf32(d_tmem, a_addr + j * 8, b_desc, P.idesc, accum);
+                accum = 1;
+                b_desc += 2;
+                if (++bq == 4) {
+                  bq = 0;
+                  if constexpr (BRES) b_desc += chunk16 - 8;
+                  else { ptx::mma_commit(ptx::smem_u32(&bars->b_empty[br.idx])); br.advance(P.SB); }
+                }
+              }
+            }
+            if (!ok) break;
+            ptx::mma_commit(ptx::smem_u32(&bars->a_empty[slot]));
+            ar.advance(P.NSS);
+          }
+        }
+        if (!ok) break;
+        if constexpr (!BRES) {
+          if (bq != 0) { ptx::mma_commit(ptx::smem_u32(&bars->b_empty[br.idx])); br.advance(P.SB); }
+        }
+        ptx::mma_commit(ptx::smem_u32(&bars->acc_full[d]));
+      }
+      PROF_DUMP(1, 3)
+    }
+    __syncwarp();
+  } else if (warp == 2) {
+    // ================================================================ FILTER PRODUCER (streamed mode)
+    if constexpr (!BRES) {
+      if (lane == 0) {
+        int64_t bcount = 0;
+        Ring br;
+        bool ok = true;
+        for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x) {
+          const int32_t n0 = (int32_t)(t % P.n_ntiles) * P.NT;
+          for (int32_t c = 0; c < P.nchunks && ok; ++c, ++bcount, br.advance(P.SB)) {
+            const int32_t sb = br.idx;
+            ok = wait_bar(P, misc, &bars->b_empty[sb], br.phase ^ 1u, DEV_TIMEOUT_B_EMPTY);
+            if (!ok) break;
+            const uint32_t full = ptx::smem_u32(&bars->b_full[sb]);
+            ptx::mbar_expect_tx(full, b_stage_bytes);
+            tma_load_2d(ptx::smem_u32(b_smem) + (uint32_t)sb * b_stage_bytes, &fmap, c * KCHUNK, n0, full);
+            ptx::mbar_arrive(full);
+          }
+        }
+        for (int64_t c = max(bcount - P.SB, (int64_t)0); c < bcount; ++c)
+          wait_bar(P, misc, &bars->b_full[c % P.SB], (uint32_t)(c / P.SB) & 1u, DEV_TIMEOUT_DRAIN);
+      }
+      __syncwarp();
+    }
+  } else if (warp >= 4 && warp < 12) {
+    // ================================================================ WINDOW REPACK: strips -> TMEM (A)
+    // Eight warps: two per TMEM lane quarter; the two take alternate channel groups.
+    const int32_t half = (warp - 4) >> 2;
+    const int32_t q4 = (warp - 4) & 3;
+    const int32_t p = q4 * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
+    const int32_t skew_step = (int32_t)(P.HoL & 3);
+    Ring rr, ar;      // raw stage of the current group, A slot of the current part (this half's own ring)
+    const int32_t slot0 = half * P.NSS;
+    uint32_t gpar = 0;  // parity of the running group count
+    bool ok = true;
+    PROF_DECL(2)
+    for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x) {
+      const int64_t tile_m = t / P.n_ntiles;
+      const int64_t P0 = tile_m * P.TP, Pend = min(P0 + P.TP, P.Mtot) - 1;
+      const int64_t i_first = P0 / P.HoWo;
+      const int32_t nseg = (int32_t)(Pend / P.HoWo - i_first) + 1;
+      const SegR seg = compute_seg(P, FF, P0, Pend, i_first, nseg, lane);
+      const int64_t pos = P0 + p;
+      const bool valid = p < P.TP && pos <= Pend;
+      int64_t i = i_first, q = 0;
+      if (valid) { i = pos / P.HoWo; q = pos - i * P.HoWo; }
+      const int32_t sg = (int32_t)(i - i_first);
+      const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
+      const int64_t s_virt = __shfl_sync(0xffffffffu, seg.virt_a, sg);
+      const int32_t s_dst = __shfl_sync(0xffffffffu, seg.dst_off, sg);
+      int32_t base_off = 0;
+      if (valid) {
+        const int64_t m = q / P.Wo, n = q - m * P.Wo;
+        base_off = s_dst + (int32_t)((m * P.L + n * P.sFh) - s_virt);
+      }
+      const int32_t skew0 = (int32_t)(s_start0 & 3);
+
+      for (int32_t g = 0; g < P.NG && ok; ++g, gpar ^= 1u) {
+        if (gpar != (uint32_t)half) {  // the other half's group
+          rr.advance(P.SR);
+          continue;
+        }
+        const int32_t sr = rr.idx;
+        ok = wait_bar_warp(P, misc, &bars->raw_full[sr], rr.phase, DEV_TIMEOUT_RAW_FULL, PROF_SLOT(0));
+        if (!ok) break;
+        const float* stage = raw + (size_t)sr * raw_stage_floats + base_off;
+        const int32_t r0 = g * CB;
+        const bool full_group = r0 + CB <= P.C;
+        const float* cptr[CB];
+#pragma unroll
+        for (int rl = 0; rl < CB; ++rl)
+          cptr[rl] = stage + rl * P.chan_pitch + ((skew0 + (r0 + rl) * skew_step) & 3);
+        // element kl of the group: channel kl / FF, tap (u, v) = ((kl % FF) / FW, (kl % FF) % FW),
+        // stored in the strip at offset v*FH + u from the window start
+        auto elem = [&](int kl) -> float {
+          if (kl >= KCG) return 0.f;
+          const int rl = kl / FF, w = kl % FF;
+          const float x = cptr[rl][(w % FW) * FH + (w / FW)];
+          return (full_group || r0 + rl < P.C) ? x : 0.f;
+        };
+#pragma unroll
+        for (int h = 0; h < PARTS; ++h) {
+          constexpr int NB = SLOT_STEPS <= 8 ? 1 : 2;           // register batches per part
+          constexpr int BATCH = (SLOT_STEPS + NB - 1) / NB;
+          const int j0 = h * SLOT_STEPS;                         // first step of this part in the group
+          const int nst = (h == PARTS - 1) ? (S - (PARTS - 1) * SLOT_STEPS) : SLOT_STEPS;
+          const int32_t slot = slot0 + ar.idx;
+          ok = wait_bar_warp(P, misc, &bars->a_empty[slot], ar.phase ^ 1u, DEV_TIMEOUT_A_EMPTY, PROF_SLOT(1));
+          if (!ok) break;
+          ptx::tc_fence_after();
+          const uint32_t a_slot = tmem_a0 + lane_base + (uint32_t)(slot * SLOT_COLS);
+#pragma unroll
+          for (int b = 0; b < NB; ++b) {
+            uint32_t v[BATCH][8];
+#pragma unroll
+            for (int jj = 0; jj < BATCH; ++jj) {
+              const int j = b * BATCH + jj;
+              if (j < nst) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  if constexpr (BF16)
+                    v[jj][e] = ptx::pack_bf16x2(elem((j0 + j) * 16 + 2 * e), elem((j0 + j) * 16 + 2 * e + 1));
+                  else
+                    v[jj][e] = __float_as_uint(elem((j0 + j) * 8 + e));
+                }
+              }
+            }
+#pragma unroll
+            for (int jj = 0; jj < BATCH; ++jj) {
+              const int j = b * BATCH + jj;
+              if (j < nst) ptx::tmem_st_x8(a_slot + (uint32_t)(j * 8), v[jj]);
+            }
+          }
+          ptx::tmem_wait_st();
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->a_full[slot]));
+          ar.advance(P.NSS);
+        }
+        if (!ok) break;
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->raw_empty[sr]));
+        rr.advance(P.SR);
+      }
+    }
+    if (half == 0) { PROF_DUMP(2 + q4, 2) }
+  } else if (warp >= 12) {
+    // ================================================================ EPILOGUE: TMEM -> NCHW
+    const int32_t q4 = warp - 12;
+    const int32_t p = q4 * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
+    Ring dr;
+    bool ok = true;
+    PROF_DECL(1)
+    for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
+      const int64_t tile_m = t / P.n_ntiles;
+      const int32_t n0 = (int32_t)(t - tile_m * P.n_ntiles) * P.NT;
+      const int64_t P0 = tile_m * P.TP, Pend = min(P0 + P.TP, P.Mtot) - 1;
+      const int64_t pos = P0 + p;
+      const bool valid = p < P.TP && pos <= Pend;
+      float* orow = P.out;
+      if (valid) {
+        const int64_t i = pos / P.HoWo, q = pos - i * P.HoWo;
+        orow += (i * P.K + n0) * P.HoWo + q;
+      }
+      const int32_t d = dr.idx;
+      ok = wait_bar_warp(P, misc, &bars->acc_full[d], dr.phase, DEV_TIMEOUT_ACC, PROF_SLOT(0));
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)(d * P.NT);
+      for (int32_t c0 = 0; c0 < P.NT; c0 += 16) {
+        uint32_t v[16];
+        ptx::tmem_ld_x16(d_tmem + (uint32_t)c0, v);
+        ptx::tmem_wait_ld();
+        if (valid) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e)
+            if (n0 + c0 + e < P.K) orow[(int64_t)(c0 + e) * P.HoWo] = __uint_as_float(v[e]);
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->acc_empty[d]));
+    }
+    if (q4 == 0) { PROF_DUMP(6, 1) }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- host side
+
+#ifdef IM2WIN_PROF
+long long* g_prof = nullptr;
+#endif
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    else
+      cudaGetLastError();
+  }
+  return fn;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      n = 0;
+      return 148;
+    }
+  }
+  return n;
+}
+
+template <int FH, int FW, int CB, bool BF16>
+int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st) {
+  constexpr int FF = FH * FW;
+  constexpr int KSTEP = BF16 ? 16 : 8;
+  constexpr int KCG = CB * FF;
+  constexpr int KCGP = (KCG + KSTEP - 1) / KSTEP * KSTEP;
+  constexpr int S = KCGP / KSTEP;
+
+  PParams P{};
+  P.xhat = xhat; P.f = f; P.out = out;
+  P.status = device_status_word();
+  if (!P.status) return IM2WIN_ECUDA;
+#ifdef IM2WIN_PROF
+  P.prof = g_prof;
+#endif
+  P.C = g.C; P.K = g.K; P.Ho = g.Ho; P.Wo = g.Wo; P.L = g.L; P.sFh = g.sFh;
+  P.HoL = g.HoL; P.HoWo = g.HoWo; P.Kg = g.Kg; P.Mtot = g.Mtot; P.n_win = g.n_win;
+  int64_t tp = 128;
+  if ((kSegMax - 1) * g.HoWo + 1 < tp) tp = (kSegMax - 1) * g.HoWo + 1;
+  P.TP = (int32_t)tp;
+  P.n_ntiles = (g.K + 255) / 256;
+  P.NT = ((g.K + P.n_ntiles - 1) / P.n_ntiles + 15) / 16 * 16;
+  P.NG = (g.C + CB - 1) / CB;
+  const int32_t steps_tile = P.NG * S;
+  P.nchunks = (steps_tile + 3) / 4;
+  const int64_t tiles_m = (g.Mtot + P.TP - 1) / P.TP;
+  P.ntiles = tiles_m * P.n_ntiles;
+
+  // worst-case floats one channel contributes to a tile
+  const int64_t rowwrap = (int64_t)g.L - (int64_t)(g.Wo - 1) * g.sFh;
+  const int64_t wraps = (tp + g.Wo - 2) / g.Wo;
+  int64_t nseg_max = (tp - 1) / g.HoWo + 2;
+  if (nseg_max > kSegMax) nseg_max = kSegMax;
+  int64_t pitch = (tp - 1) * g.sFh + wraps * (rowwrap > g.sFh ? rowwrap - g.sFh : 0) + nseg_max * (FF + 6) + 4;
+  pitch = (pitch + 3) & ~(int64_t)3;
+  if (pitch > (1 << 20)) return IM2WIN_EUNSUPPORTED;
+  P.chan_pitch = (int32_t)pitch;
+  const int64_t raw_stage = (int64_t)CB * pitch * 4;
+
+  // filter operand: resident if it fits next to two strip stages, else streamed by TMA (TF32, dense groups)
+  const int64_t cap = 227 * 1024 - 1024 - 1024;  // alignment slack + barriers
+  const int64_t b_res = (int64_t)P.nchunks * P.NT * 128;
+  bool resident = P.n_ntiles == 1 && b_res + 2 * raw_stage <= cap;
+  const bool can_stream = !BF16 && KCG == KCGP && (g.C % CB) == 0 && (g.Kg % 4) == 0 && encode_fn() != nullptr;
+  if (!resident && !can_stream) return IM2WIN_EUNSUPPORTED;
+  int64_t b_bytes;
+  if (resident) {
+    b_bytes = b_res;
+    P.SB = 1;
+  } else {
+    P.SB = 6;
+    while (P.SB > 2 && (int64_t)P.SB * P.NT * 128 + 4 * raw_stage > cap) --P.SB;
+    b_bytes = (int64_t)P.SB * P.NT * 128;
+  }
+  // An even number of strip stages: a stage then always serves the same repack half, which sees every
+  // phase of its barrier.
+  P.SR = (int32_t)((cap - b_bytes) / raw_stage);
+  if (P.SR >= 4) P.SR = 4;
+  else if (P.SR >= 2) P.SR = 2;
+  else return IM2WIN_EUNSUPPORTED;
+
+  // TMEM: accumulators first, then the ring of A slots
+  constexpr int SLOT_COLS = SlotGeom<S>::SLOT_STEPS * 8;
+  P.ND = (2 * P.NT + 2 * SLOT_COLS <= 512) ? 2 : 1;
+  // Each repack half owns NSS slots (a barrier must be waited on by one party that sees every one of
+  // its phases, so the halves cannot share slots).
+  P.NSS = (512 - P.ND * P.NT) / SLOT_COLS / 2;
+  if (P.NSS > 4) P.NSS = 4;
+  if (P.NSS < 1) return IM2WIN_EUNSUPPORTED;
+  P.SS = SlotGeom<S>::SLOT_STEPS;
+  const int32_t cols = P.ND * P.NT + 2 * P.NSS * SLOT_COLS;
+  P.tmem_cols = 32;
+  while (P.tmem_cols < cols) P.tmem_cols *= 2;
+  P.idesc = ptx::make_idesc(128, P.NT, BF16 ? 1 : 2);
+
+  uint32_t off = (uint32_t)b_bytes;
+  P.off_raw = off; off += (uint32_t)(P.SR * raw_stage);
+  P.off_bar = off; off += (uint32_t)((sizeof(PBars) + 15) / 16 * 16);
+  P.off_misc = off; off += 64;
+  const size_t smem_bytes = off + 1024;
+
+  CUtensorMap fmap;
+  memset(&fmap, 0, sizeof(fmap));
+  if (!resident) {
+    const cuuint64_t gdim[2] = {(cuuint64_t)g.Kg, (cuuint64_t)g.K};
+    const cuuint64_t gstr[1] = {(cuuint64_t)g.Kg * 4};
+    const cuuint32_t box[2] = {32, (cuuint32_t)P.NT};
+    const cuuint32_t estr[2] = {1, 1};
+    if (encode_fn()(&fmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(f), gdim, gstr, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return IM2WIN_EUNSUPPORTED;
+  }
+  const int64_t grid = P.ntiles < sm_count() ? P.ntiles : sm_count();
+  cudaError_t e;
+  if (resident) {
+    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, true>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+    if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
+    kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap);
+  } else {
+    if constexpr (!BF16) {
+      auto kern = conv_tc_persistent_kernel<FH, FW, CB, false, false>;
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+      if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
+      kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap);
+    } else {
+      return IM2WIN_EUNSUPPORTED;
+    }
+  }
+  return cuda_status(cudaGetLastError());
+}
+
+template <int FH, int FW, int CB>
+int launch_mode(const float* xhat, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st) {
+  return mode == IM2WIN_MODE_BF16 ? launch_spec<FH, FW, CB, true>(xhat, f, out, g, st)
+                                  : launch_spec<FH, FW, CB, false>(xhat, f, out, g, st);
+}
+
+}  // namespace
+
+// Returns IM2WIN_EUNSUPPORTED when no specialisation applies (the caller then uses the generic kernel).
+int launch_conv_tc_persistent(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
+                              cudaStream_t st) {
+  if (g.Fh == 3 && g.Fw == 3) {
+    if (g.C >= 8) return launch_mode<3, 3, 8>(xhat, f, out, g, mode, st);
+    if (g.C == 3) return launch_mode<3, 3, 3>(xhat, f, out, g, mode, st);
+  }
+  if (g.Fh == 5 && g.Fw == 5 && g.C >= 8) return launch_mode<5, 5, 8>(xhat, f, out, g, mode, st);
+  if (g.Fh == 7 && g.Fw == 7 && g.C == 3) return launch_mode<7, 7, 3>(xhat, f, out, g, mode, st);
+  if (g.Fh == 11 && g.Fw == 11 && g.C <= 4) return launch_mode<11, 11, 1>(xhat, f, out, g, mode, st);
+  return IM2WIN_EUNSUPPORTED;
+}
+
+#ifdef IM2WIN_PROF
+extern "C" void im2win_debug_set_prof(long long* device_buf) { g_prof = device_buf; }
+#endif
+
+}  // namespace im2win

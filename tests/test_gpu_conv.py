@@ -35,6 +35,13 @@ def _built():
     ensure_built()
 
 
+@pytest.fixture(params=["auto", "generic"], autouse=True)
+def _kernel(request, monkeypatch):
+    """Every case runs twice: with the library's own choice of tensor-core kernel (the persistent,
+    filter-size-specialised one where it applies) and with the generic kernel forced."""
+    monkeypatch.setenv("IM2WIN_FORCE_GENERIC", "1" if request.param == "generic" else "0")
+
+
 def _data(dims, seed, ints=False):
     n, c, h, w, k, fh, fw, s = dims
     if ints:
