@@ -51,7 +51,8 @@ typedef enum {
   IM2WIN_EOVERLAP = -4,     /* an output range overlaps an input or workspace range                */
   IM2WIN_ECUDA = -5,        /* a CUDA runtime call or kernel launch failed                         */
   IM2WIN_ETIMEOUT = -6,     /* a bounded device-side wait expired (see im2win_last_device_status)  */
-  IM2WIN_EUNSUPPORTED = -7  /* shape outside what the kernels implement (see im2win_conv)          */
+  IM2WIN_EUNSUPPORTED = -7, /* shape outside what the kernels implement (see im2win_conv)          */
+  IM2WIN_ESCRATCH = -8      /* problem needs more scratch than im2win_conv_static's built-in buffer */
 } im2win_status;
 
 /* Output sizes, Ho = floor((H-Fh)/s)+1 and Wo = floor((W-Fw)/s)+1
@@ -104,6 +105,26 @@ int im2win_conv_host(const float* in_host, const float* filter_host, const im2wi
                      int mode, float* out_host);
 int im2win_host_release(void);
 
+/* No counterpart in the paper: an entry point for callers that cannot allocate device memory.
+ * Who that is: a process whose GPU memory belongs whole to some other allocator (a serving
+ * arena, a framework pool sized to the device), or code under a no-allocation-after-start-up rule
+ * (hard-real-time loops, safety-reviewed code).  im2win_conv needs a caller-supplied workspace for
+ * the im2win tensor; this variant keeps that tensor in a buffer built into the library image
+ * (IM2WIN_STATIC_SCRATCH_BYTES of device memory on every GPU that loads the library, held until
+ * the process exits) and itself calls no cudaMalloc, cudaFree or other allocating routine.
+ * Computes exactly what im2win_conv(in_nchw, IM2WIN_SRC_NCHW, ...) computes, on `cuda_stream`,
+ * asynchronously.  in_nchw / filter_kcfhfw / out_nchw: device pointers as for im2win_conv.
+ * Errors: IM2WIN_ESCRATCH when im2win_workspace_bytes(shape) exceeds the built-in buffer (nothing
+ * is launched); otherwise as im2win_conv.
+ * The first call on a device looks up the buffer's device address (a one-time set-up step, done
+ * with that device current); make that first call outside any stream capture.
+ * All calls on a device share the one buffer: two calls whose kernels can overlap on the GPU
+ * (different streams without an ordering between them) race on it and give wrong results.  The
+ * buffer keeps the previous call's im2win tensor; nothing in it needs clearing, because each call
+ * overwrites every element it later reads. */
+#define IM2WIN_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+int im2win_conv_static(const float* in_nchw, const float* filter_kcfhfw, const im2win_shape* shape,
+                       int mode, float* out_nchw, void* cuda_stream);
 /* Kernels never trap.  A bounded wait that expires, or an internal range check that fails,
  * records a code in a device-side status word and the kernel exits early (its output is then
  * undefined).  This call synchronises `cuda_stream`, returns the word in *status (0 = clean)

@@ -17,11 +17,12 @@ LIB_PATH = os.path.join(_HERE, "libim2win.so")
 
 SRC_NCHW, SRC_IM2WIN = 0, 1
 MODE_TF32, MODE_BF16, MODE_FP32 = 0, 1, 2
-OK, EINVAL, EALIGN, EWORKSPACE, EOVERLAP, ECUDA, ETIMEOUT, EUNSUPPORTED = 0, -1, -2, -3, -4, -5, -6, -7
+OK, EINVAL, EALIGN, EWORKSPACE, EOVERLAP, ECUDA, ETIMEOUT, EUNSUPPORTED, ESCRATCH = 0, -1, -2, -3, -4, -5, -6, -7, -8
 
 EXPORTS = ("im2win_out_dims", "im2win_workspace_bytes", "im2win_im2col_bytes", "im2win_transform",
-           "im2win_conv", "im2win_conv_host", "im2win_host_release", "im2win_last_device_status",
-           "im2win_strerror")
+           "im2win_conv", "im2win_conv_host", "im2win_host_release", "im2win_conv_static",
+           "im2win_last_device_status", "im2win_strerror")
+STATIC_SCRATCH_BYTES = 32 * 1024 * 1024  # IM2WIN_STATIC_SCRATCH_BYTES of include/im2win.h
 
 
 class Shape(ctypes.Structure):
@@ -58,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.im2win_conv.argtypes = [vp, ctypes.c_int, vp, sp, ctypes.c_int, vp, vp, ctypes.c_size_t, vp]
         L.im2win_conv_host.argtypes = [vp, vp, sp, ctypes.c_int, vp]
         L.im2win_host_release.argtypes = []
+        L.im2win_conv_static.argtypes = [vp, vp, sp, ctypes.c_int, vp, vp]
         L.im2win_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
         L.im2win_strerror.argtypes = [ctypes.c_int]
         L.im2win_strerror.restype = ctypes.c_char_p
@@ -136,6 +138,15 @@ def conv_host(in_host, filter_host, shape, mode: int, out_host) -> None:
     """im2win_conv_host: HOST buffers in, HOST buffer out; returns when the result is there."""
     _check(lib().im2win_conv_host(_ptr(in_host), _ptr(filter_host), ctypes.byref(Shape.of(shape)), int(mode),
                                   _ptr(out_host)), "im2win_conv_host")
+
+
+def conv_static(in_nchw, filter_kcfhfw, shape, mode: int, out_nchw, stream=None) -> None:
+    """im2win_conv_static: like conv() on the untransformed input, but the im2win tensor lives in the
+    library's built-in device buffer, so no workspace is passed and nothing is allocated.  For callers
+    that cannot allocate device memory.  Raises Im2winError(ESCRATCH) if the problem does not fit.  All
+    calls on a device share that buffer: do not let two of them overlap on the GPU."""
+    _check(lib().im2win_conv_static(_ptr(in_nchw), _ptr(filter_kcfhfw), ctypes.byref(Shape.of(shape)), int(mode),
+                                    _ptr(out_nchw), _stream(stream)), "im2win_conv_static")
 
 
 def host_release() -> None:

@@ -180,6 +180,7 @@ const char* im2win_strerror(int status) {
     case IM2WIN_ECUDA: return "CUDA runtime call or kernel launch failed (no device, or see cudaGetLastError)";
     case IM2WIN_ETIMEOUT: return "a bounded device-side wait expired";
     case IM2WIN_EUNSUPPORTED: return "shape outside what the tensor-core kernels implement";
+    case IM2WIN_ESCRATCH: return "the problem's im2win tensor is larger than the library's built-in scratch buffer";
     default: return "unknown im2win status";
   }
 }

@@ -85,9 +85,15 @@ def test_argument_checks_happen_before_any_launch():
         assert e.value.code == code, (code, e.value)
 
 
+def test_static_scratch_constant_matches_header():
+    text = open(os.path.join(ROOT, "include", "im2win.h")).read()
+    m = re.search(r"#define\s+IM2WIN_STATIC_SCRATCH_BYTES\s+\((\d+)u \* (\d+)u \* (\d+)u\)", text)
+    assert m and int(m.group(1)) * int(m.group(2)) * int(m.group(3)) == b.STATIC_SCRATCH_BYTES
+
+
 def test_strerror_covers_every_code():
-    texts = {b.strerror(c) for c in range(0, -9, -1)}
-    assert len(texts) == 9 and all(texts)
+    texts = {b.strerror(c) for c in range(0, -10, -1)}
+    assert len(texts) == 10 and all(texts)
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
