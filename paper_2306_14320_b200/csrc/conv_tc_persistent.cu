@@ -46,6 +46,8 @@ struct PParams {
   int32_t SS, NSS;      // MMA steps per A slot; slots per repack half in the TMEM ring
   int32_t ND;           // accumulator buffers
   int32_t chan_pitch;
+  int32_t box;          // 1: strips come as one 2-D TMA box per channel group, tiles never span images
+  int32_t TPI;          // box mode: tiles per image
   int32_t nchunks;      // 128-byte filter chunks per tile
   int32_t tmem_cols;
   uint32_t idesc;
@@ -88,6 +90,8 @@ __device__ __forceinline__ uint64_t global_ns() {
 #ifdef IM2WIN_PROF
 #define PROF_DECL(n) long long prof_acc[n] = {}; const long long prof_t0 = clock64();
 #define PROF_SLOT(k) (&prof_acc[k])
+#define PROF_T0(v) const long long v = clock64();
+#define PROF_ADD(k, v) prof_acc[k] += clock64() - (v);
 #define PROF_DUMP(role, n)                                                         \
   if (P.prof && blockIdx.x < 8 && lane == 0) {                                     \
     long long* o = P.prof + ((long long)blockIdx.x * 8 + (role)) * 8;              \
@@ -97,11 +101,16 @@ __device__ __forceinline__ uint64_t global_ns() {
 #else
 #define PROF_DECL(n)
 #define PROF_SLOT(k) nullptr
+#define PROF_T0(v)
+#define PROF_ADD(k, v)
 #define PROF_DUMP(role, n)
 #endif
 
+// Bounded wait (about a second).  A warp that is not ready backs off with nanosleep between polls:
+// sixteen warps share four schedulers, and a warp that spins on try_wait takes issue slots from the
+// MMA-issuing thread on its scheduler, whose instruction rate is what bounds small-N tiles.
 __device__ __forceinline__ bool wait_bar(const PParams& P, PMisc* misc, uint64_t* bar, uint32_t parity,
-                                         int32_t code, long long* acc = nullptr) {
+                                         int32_t code, long long* acc = nullptr, uint32_t sleep_ns = 64) {
   const uint32_t b = ptx::smem_u32(bar);
 #ifdef IM2WIN_PROF
   // try_wait may block inside the instruction, so the clock brackets the first poll too
@@ -111,6 +120,7 @@ __device__ __forceinline__ bool wait_bar(const PParams& P, PMisc* misc, uint64_t
   if (ptx::mbar_try_wait(b, parity)) return true;
   uint64_t t0 = 0;
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    __nanosleep(sleep_ns);
     if (ptx::mbar_try_wait(b, parity)) return true;
     if ((it & 63u) == 63u) {
       if (*reinterpret_cast<volatile int32_t*>(&misc->abort)) return false;
@@ -124,8 +134,8 @@ __device__ __forceinline__ bool wait_bar(const PParams& P, PMisc* misc, uint64_t
 }
 
 __device__ __forceinline__ bool wait_bar_warp(const PParams& P, PMisc* misc, uint64_t* bar, uint32_t parity,
-                                              int32_t code, long long* acc = nullptr) {
-  return __all_sync(0xffffffffu, wait_bar(P, misc, bar, parity, code, acc));
+                                              int32_t code, long long* acc = nullptr, uint32_t sleep_ns = 64) {
+  return __all_sync(0xffffffffu, wait_bar(P, misc, bar, parity, code, acc, sleep_ns));
 }
 
 // Position in a ring of n stages together with the parity of the pass over it.
@@ -170,6 +180,19 @@ __device__ __forceinline__ SegR compute_seg(const PParams& P, int FF, int64_t P0
   return s;
 }
 
+// First and last output position (flattened over image, row, column) of m-tile `tile_m`.
+__device__ __forceinline__ void tile_range(const PParams& P, int64_t tile_m, int64_t& P0, int64_t& Pend) {
+  if (P.box) {  // tiles are cut per image
+    const int64_t i = tile_m / P.TPI;
+    const int64_t q0 = (tile_m - i * P.TPI) * P.TP;
+    P0 = i * P.HoWo + q0;
+    Pend = min(q0 + P.TP, P.HoWo) - 1 + i * P.HoWo;
+  } else {
+    P0 = tile_m * P.TP;
+    Pend = min(P0 + P.TP, P.Mtot) - 1;
+  }
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1,
                                             uint32_t bar) {
   asm volatile(
@@ -179,7 +202,8 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 
 template <int FH, int FW, int CB, bool BF16, bool BRES>
 __global__ void __launch_bounds__(kThreads, 1)
-conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_constant__ CUtensorMap fmap) {
+conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_constant__ CUtensorMap fmap,
+                          const __grid_constant__ CUtensorMap xmap) {
   constexpr int FF = FH * FW;
   constexpr int KSTEP = BF16 ? 16 : 8;        // reduction elements per MMA
   constexpr int KCHUNK = BF16 ? 64 : 32;      // reduction elements per 128-byte filter row
@@ -204,7 +228,7 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
   // ------------------------------------------------------------------ prologue
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxStages; ++i) {
-      ptx::mbar_init(ptx::smem_u32(&bars->raw_full[i]), 32);
+      ptx::mbar_init(ptx::smem_u32(&bars->raw_full[i]), 1);
       ptx::mbar_init(ptx::smem_u32(&bars->raw_empty[i]), 4);
       ptx::mbar_init(ptx::smem_u32(&bars->b_full[i]), 1);
       ptx::mbar_init(ptx::smem_u32(&bars->b_empty[i]), 1);
@@ -225,18 +249,21 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
     ptx::tmem_relinquish();
   }
   if constexpr (BRES) {
-    // Build the whole filter operand once: chunk c holds padded reduction indices [c*KCHUNK, +KCHUNK)
-    // for all NT filters, K-major with the 128-byte swizzle.  (A resident filter implies one n-tile.)
-    constexpr int EPP = BF16 ? 8 : 4;
-    const int32_t pieces = P.nchunks * P.NT * 8;
+    // Build the whole filter operand once, one block of NT rows x 32 bytes per MMA step (padded
+    // reduction indices [s*KSTEP, +KSTEP)), K-major with the 32-byte swizzle, so that the MMA thread
+    // steps its descriptor by a constant.  (A resident filter implies one n-tile.)
+    constexpr int EPP = BF16 ? 8 : 4;  // elements per 16-byte piece
+    const int32_t nsteps_all = P.NG * S;
+    const int32_t pieces = nsteps_all * P.NT * 2;
+    const uint32_t step_bytes = (uint32_t)P.NT * 32u;
     for (int32_t idx = threadIdx.x; idx < pieces; idx += kThreads) {
-      const int32_t q = idx & 7, j = (idx >> 3) % P.NT, c = (idx >> 3) / P.NT;
+      const int32_t c = idx & 1, j = (idx >> 1) % P.NT, sidx = (idx >> 1) / P.NT;
       float x[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         x[e] = 0.f;
         if (e < EPP && j < P.K) {
-          const int32_t kp = c * KCHUNK + q * EPP + e;
+          const int32_t kp = sidx * KSTEP + c * EPP + e;
           const int32_t g = kp / KCGP, kl = kp - g * KCGP;
           const int64_t k = (int64_t)g * KCG + kl;
           if (kl < KCG && k < P.Kg) x[e] = __ldg(P.f + (int64_t)j * P.Kg + k);
@@ -250,8 +277,8 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
         piece.x = __float_as_uint(x[0]); piece.y = __float_as_uint(x[1]);
         piece.z = __float_as_uint(x[2]); piece.w = __float_as_uint(x[3]);
       }
-      *reinterpret_cast<uint4*>(b_smem + (size_t)c * b_stage_bytes + (j >> 3) * 1024 + (j & 7) * 128 +
-                                ((q ^ (j & 7)) << 4)) = piece;
+      *reinterpret_cast<uint4*>(b_smem + (size_t)sidx * step_bytes + (j >> 3) * 256 + (j & 7) * 32 +
+                                ((c ^ ((j >> 2) & 1)) << 4)) = piece;
     }
     ptx::fence_proxy_async_smem();
   }
@@ -269,43 +296,76 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
     PROF_DECL(1)
     for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x) {
       const int64_t tile_m = t / P.n_ntiles;
-      const int64_t P0 = tile_m * P.TP, Pend = min(P0 + P.TP, P.Mtot) - 1;
+      int64_t P0, Pend;
+      tile_range(P, tile_m, P0, Pend);
       const int64_t i_first = P0 / P.HoWo;
       const int32_t nseg = (int32_t)(Pend / P.HoWo - i_first) + 1;
       const SegR seg = compute_seg(P, FF, P0, Pend, i_first, nseg, lane);
-      const int32_t npairs = CB * nseg;
+      // Each lane owns up to two (channel-in-group, image segment) pairs for the whole tile; from
+      // group to group only the channel, i.e. the source address, moves (by CB planes).
+      const int32_t npairs = CB * nseg;  // <= 64
+      bool act[2];
+      int32_t rl[2], len[2], dsto[2];
+      int64_t start[2];
+#pragma unroll
+      for (int z = 0; z < 2; ++z) {
+        const int32_t idx = z * 32 + lane;
+        act[z] = idx < npairs;
+        rl[z] = act[z] ? idx / nseg : 0;
+        const int32_t sg = act[z] ? idx - rl[z] * nseg : 0;
+        const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
+        len[z] = __shfl_sync(0xffffffffu, seg.len, sg);
+        dsto[z] = rl[z] * P.chan_pitch + __shfl_sync(0xffffffffu, seg.dst_off, sg);
+        start[z] = s_start0 + (int64_t)rl[z] * P.HoL;
+      }
+      const int64_t group_step = (int64_t)CB * P.HoL;
+      // box mode: the tile lies in one image; x = first needed float of the plane rounded down to
+      // 16 bytes (in 8-byte elements), y = plane index of the group's first channel
+      const int64_t box_virt = __shfl_sync(0xffffffffu, seg.virt_a, 0);
+      const int32_t box_x = (int32_t)((box_virt & ~(int64_t)3) >> 1);
+      const int32_t box_y0 = (int32_t)(i_first * P.C);
       for (int32_t g = 0; g < P.NG && ok; ++g, ++gcount, rr.advance(P.SR)) {
         const int32_t sr = rr.idx;
-        ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0));
+        ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0), 128);
         if (!ok) break;
         const uint32_t full = ptx::smem_u32(&bars->raw_full[sr]);
         float* stage = raw + (size_t)sr * raw_stage_floats;
-        for (int32_t idx0 = 0; idx0 < npairs; idx0 += 32) {
-          const int32_t idx = idx0 + lane;
-          const bool act = idx < npairs;
-          const int32_t rl = act ? idx / nseg : 0, sg = act ? idx - rl * nseg : 0;
-          const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
-          const int32_t s_len = __shfl_sync(0xffffffffu, seg.len, sg);
-          const int32_t s_dst = __shfl_sync(0xffffffffu, seg.dst_off, sg);
-          const int32_t r = g * CB + rl;
-          if (!act || r >= P.C) continue;
-          const int64_t start = s_start0 + (int64_t)r * P.HoL;
-          const int32_t skew = (int32_t)(start & 3);
-          const int64_t a0 = start - skew;
-          int32_t nfl = (skew + s_len + 3) & ~3;
-          float* dst = stage + rl * P.chan_pitch + s_dst;
-          if (a0 + nfl > P.n_win) {  // the last 16-byte chunk would pass the end of the tensor
-            const int32_t nbulk = (int32_t)((P.n_win - a0) & ~(int64_t)3);
-            for (int64_t e = a0 + nbulk; e < P.n_win; ++e) dst[e - a0] = __ldg(P.xhat + e);
-            nfl = nbulk;
+        if (P.box) {
+          if (lane == 0) {
+            ptx::mbar_arrive_expect_tx(full, (uint32_t)raw_stage_floats * 4u);
+            tma_load_2d(ptx::smem_u32(stage), &xmap, box_x, box_y0 + g * CB, full);
           }
-          if (nfl > 0) {
-            ptx::mbar_expect_tx(full, (uint32_t)nfl * 4u);
-            ptx::bulk_g2s(ptx::smem_u32(dst), P.xhat + a0, (uint32_t)nfl * 4u, full);
-          }
+          __syncwarp();
+          continue;
         }
+        const float* src[2];
+        uint32_t dst[2], bytes[2];
+#pragma unroll
+        for (int z = 0; z < 2; ++z) {
+          bytes[z] = 0;
+          if (act[z] && g * CB + rl[z] < P.C) {
+            const int32_t skew = (int32_t)(start[z] & 3);
+            const int64_t a0 = start[z] - skew;
+            int32_t nfl = (skew + len[z] + 3) & ~3;
+            float* d = stage + dsto[z];
+            if (a0 + nfl > P.n_win) {  // the last 16-byte chunk would pass the end of the tensor
+              const int32_t nbulk = (int32_t)((P.n_win - a0) & ~(int64_t)3);
+              for (int64_t e = a0 + nbulk; e < P.n_win; ++e) d[e - a0] = __ldg(P.xhat + e);
+              nfl = nbulk;
+            }
+            src[z] = P.xhat + a0;
+            dst[z] = ptx::smem_u32(d);
+            bytes[z] = (uint32_t)nfl * 4u;
+          }
+          start[z] += group_step;
+        }
+        // one arrival carrying the byte count of the whole group, then the copies
+        const uint32_t total = __reduce_add_sync(0xffffffffu, bytes[0] + bytes[1]);
+        if (lane == 0) ptx::mbar_arrive_expect_tx(full, total);
         __syncwarp();
-        ptx::mbar_arrive(full);
+#pragma unroll
+        for (int z = 0; z < 2; ++z)
+          if (bytes[z]) ptx::bulk_g2s(dst[z], src[z], bytes[z], full);
       }
     }
     PROF_DUMP(0, 1)
@@ -320,9 +380,17 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
       Ring arh[2], br, dr;  // A slot (one ring per repack half), streamed filter stage, accumulator buffer
       uint32_t gpar = 0;    // parity of the running group count = which half produced the group
       bool ok = true;
-      PROF_DECL(3)
-      const uint64_t desc0 = ptx::smem_desc_k_sw128(ptx::smem_u32(b_smem));
+      PROF_DECL(7)
+      const uint64_t desc0 = BRES ? ptx::smem_desc_k_sw32(ptx::smem_u32(b_smem)) : ptx::smem_desc_k_sw128(ptx::smem_u32(b_smem));
+      const uint32_t desc_lo0 = (uint32_t)desc0, desc_hi = (uint32_t)(desc0 >> 32);
+      const uint32_t step16 = (uint32_t)P.NT * 2u;  // resident: one step block (NT*32 bytes) in descriptor units
+      uint32_t step_off[SLOT_STEPS];                // resident: j * step16, kept in registers
+#pragma unroll
+      for (int j = 0; j < SLOT_STEPS; ++j) step_off[j] = (uint32_t)j * step16;
       const uint32_t chunk16 = b_stage_bytes >> 4;  // one filter chunk / stage in descriptor units
+      const uint32_t a_full0 = ptx::smem_u32(&bars->a_full[0]), a_empty0 = ptx::smem_u32(&bars->a_empty[0]);
+      const uint32_t b_full0 = ptx::smem_u32(&bars->b_full[0]), b_empty0 = ptx::smem_u32(&bars->b_empty[0]);
+      (void)b_full0; (void)b_empty0;
       for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
         const int32_t d = dr.idx;
         ok = wait_bar(P, misc, &bars->acc_empty[d], dr.phase ^ 1u, DEV_TIMEOUT_ACC, PROF_SLOT(2));
@@ -330,8 +398,8 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(d * P.NT);
         uint32_t accum = 0;
-        int32_t bq = 0;           // step inside the current 128-byte filter chunk
-        uint64_t b_desc = desc0;  // resident: walks the chunks of the tile
+        uint32_t st0 = 0;             // steps of this tile issued before the current part
+        uint32_t b_lo = desc_lo0;     // streamed: descriptor of the current stage
         for (int32_t g = 0; g < P.NG && ok; ++g, gpar ^= 1u) {
           Ring& ar = arh[gpar];
           const int32_t slot0 = (int32_t)gpar * P.NSS;
@@ -339,44 +407,58 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
           for (int h = 0; h < PARTS; ++h) {
             const int nst = (h == PARTS - 1) ? (S - (PARTS - 1) * SLOT_STEPS) : SLOT_STEPS;
             const int32_t slot = slot0 + ar.idx;
-            ok = wait_bar(P, misc, &bars->a_full[slot], ar.phase, DEV_TIMEOUT_A_FULL, PROF_SLOT(0));
-            if (!ok) break;
+            if (!ptx::mbar_try_wait(a_full0 + (uint32_t)slot * 8u, ar.phase)) {  // usually ready: one poll
+              ok = wait_bar(P, misc, &bars->a_full[slot], ar.phase, DEV_TIMEOUT_A_FULL, PROF_SLOT(0), 20);
+              if (!ok) break;
+            }
+            PROF_T0(tf)
             ptx::tc_fence_after();
+            PROF_ADD(3, tf)
             const uint32_t a_addr = tmem_a0 + (uint32_t)(slot * SLOT_COLS);
+            const uint32_t lo_part = desc_lo0 + st0 * step16;
+            (void)lo_part;
+            PROF_T0(tm)
 #pragma unroll
             for (int j = 0; j < SLOT_STEPS; ++j) {
               if (j < nst) {
-                if constexpr (!BRES) {
-                  if (bq == 0) {
-                    ok = wait_bar(P, misc, &bars->b_full[br.idx], br.phase, DEV_TIMEOUT_B_FULL, PROF_SLOT(1));
-                    if (!ok) break;
+                const uint32_t st = st0 + j;  // step within the tile: chunk st >> 2, quarter st & 3
+                uint32_t lo;
+                if constexpr (BRES) {
+                  lo = lo_part + step_off[j];  // one add per MMA, no chain from step to step
+                } else {
+                  if ((st & 3u) == 0) {
+                    if (!ptx::mbar_try_wait(b_full0 + (uint32_t)br.idx * 8u, br.phase)) {
+                      ok = wait_bar(P, misc, &bars->b_full[br.idx], br.phase, DEV_TIMEOUT_B_FULL, PROF_SLOT(1), 20);
+                      if (!ok) break;
+                    }
                     ptx::tc_fence_after();
-                    b_desc = desc0 + (uint64_t)((uint32_t)br.idx * chunk16);
+                    b_lo = desc_lo0 + (uint32_t)br.idx * chunk16;
                   }
+                  lo = b_lo + (st & 3u) * 2u;
                 }
-                if (BF16) ptx::mma_ts_f16(d_tmem, a_addr + j * 8, b_desc, P.idesc, accum);
-                else      ptx::mma_ts_tf32(d_tmem, a_addr + j * 8, b_desc, P.idesc, accum);
+                ptx::mma_ts_lohi<BF16>(d_tmem, a_addr + j * 8, lo, desc_hi, P.idesc, accum);
                 accum = 1;
-                b_desc += 2;
-                if (++bq == 4) {
-                  bq = 0;
-                  if constexpr (BRES) b_desc += chunk16 - 8;
-                  else { ptx::mma_commit(ptx::smem_u32(&bars->b_empty[br.idx])); br.advance(P.SB); }
+                if constexpr (!BRES) {
+                  if ((st & 3u) == 3u) { ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u); br.advance(P.SB); }
                 }
               }
             }
             if (!ok) break;
-            ptx::mma_commit(ptx::smem_u32(&bars->a_empty[slot]));
+            PROF_ADD(4, tm)
+            st0 += nst;
+            PROF_T0(tc)
+            ptx::mma_commit(a_empty0 + (uint32_t)slot * 8u);
+            PROF_ADD(5, tc)
             ar.advance(P.NSS);
           }
         }
         if (!ok) break;
         if constexpr (!BRES) {
-          if (bq != 0) { ptx::mma_commit(ptx::smem_u32(&bars->b_empty[br.idx])); br.advance(P.SB); }
+          if ((st0 & 3u) != 0) { ptx::mma_commit(ptx::smem_u32(&bars->b_empty[br.idx])); br.advance(P.SB); }
         }
         ptx::mma_commit(ptx::smem_u32(&bars->acc_full[d]));
       }
-      PROF_DUMP(1, 3)
+      PROF_DUMP(1, 7)
     }
     __syncwarp();
   } else if (warp == 2) {
@@ -410,7 +492,7 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
     const int32_t q4 = (warp - 4) & 3;
     const int32_t p = q4 * 32 + lane;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
-    const int32_t skew_step = (int32_t)(P.HoL & 3);
+    const int32_t skew_step = P.box ? 0 : (int32_t)(P.HoL & 3);
     Ring rr, ar;      // raw stage of the current group, A slot of the current part (this half's own ring)
     const int32_t slot0 = half * P.NSS;
     uint32_t gpar = 0;  // parity of the running group count
@@ -418,7 +500,8 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
     PROF_DECL(2)
     for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x) {
       const int64_t tile_m = t / P.n_ntiles;
-      const int64_t P0 = tile_m * P.TP, Pend = min(P0 + P.TP, P.Mtot) - 1;
+      int64_t P0, Pend;
+      tile_range(P, tile_m, P0, Pend);
       const int64_t i_first = P0 / P.HoWo;
       const int32_t nseg = (int32_t)(Pend / P.HoWo - i_first) + 1;
       const SegR seg = compute_seg(P, FF, P0, Pend, i_first, nseg, lane);
@@ -435,7 +518,9 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
         const int64_t m = q / P.Wo, n = q - m * P.Wo;
         base_off = s_dst + (int32_t)((m * P.L + n * P.sFh) - s_virt);
       }
-      const int32_t skew0 = (int32_t)(s_start0 & 3);
+      // 16-byte phase of the staged range: box mode rounds inside the plane (the same for every
+      // channel, planes being multiples of 16 bytes), the bulk-copy mode per absolute address
+      const int32_t skew0 = P.box ? (int32_t)(s_virt & 3) : (int32_t)(s_start0 & 3);
 
       for (int32_t g = 0; g < P.NG && ok; ++g, gpar ^= 1u) {
         if (gpar != (uint32_t)half) {  // the other half's group
@@ -517,7 +602,8 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
     for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
       const int64_t tile_m = t / P.n_ntiles;
       const int32_t n0 = (int32_t)(t - tile_m * P.n_ntiles) * P.NT;
-      const int64_t P0 = tile_m * P.TP, Pend = min(P0 + P.TP, P.Mtot) - 1;
+      int64_t P0, Pend;
+      tile_range(P, tile_m, P0, Pend);
       const int64_t pos = P0 + p;
       const bool valid = p < P.TP && pos <= Pend;
       float* orow = P.out;
@@ -526,7 +612,7 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
         orow += (i * P.K + n0) * P.HoWo + q;
       }
       const int32_t d = dr.idx;
-      ok = wait_bar_warp(P, misc, &bars->acc_full[d], dr.phase, DEV_TIMEOUT_ACC, PROF_SLOT(0));
+      ok = wait_bar_warp(P, misc, &bars->acc_full[d], dr.phase, DEV_TIMEOUT_ACC, PROF_SLOT(0), 256);
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)(d * P.NT);
@@ -621,8 +707,6 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
   P.NG = (g.C + CB - 1) / CB;
   const int32_t steps_tile = P.NG * S;
   P.nchunks = (steps_tile + 3) / 4;
-  const int64_t tiles_m = (g.Mtot + P.TP - 1) / P.TP;
-  P.ntiles = tiles_m * P.n_ntiles;
 
   // worst-case floats one channel contributes to a tile
   const int64_t rowwrap = (int64_t)g.L - (int64_t)(g.Wo - 1) * g.sFh;
@@ -632,12 +716,30 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
   int64_t pitch = (tp - 1) * g.sFh + wraps * (rowwrap > g.sFh ? rowwrap - g.sFh : 0) + nseg_max * (FF + 6) + 4;
   pitch = (pitch + 3) & ~(int64_t)3;
   if (pitch > (1 << 20)) return IM2WIN_EUNSUPPORTED;
+  // Box mode: one 2-D TMA box (CB planes x one contiguous range) per channel group instead of CB
+  // bulk copies.  Needs planes that are multiples of 16 bytes, a range of at most 256 8-byte
+  // elements, and images large enough that cutting tiles per image wastes little.
+  {
+    const int64_t tpi = (g.HoWo + 127) / 128;
+    const int64_t one_seg = 127 * (int64_t)g.sFh + wraps * (rowwrap > g.sFh ? rowwrap - g.sFh : 0) + FF + 6 + 4;
+    const int64_t boxf = (one_seg + 3) & ~(int64_t)3;
+    const bool little_waste = tpi * 128 * 100 <= g.HoWo * 107;
+    const char* nobox = getenv("IM2WIN_NO_BOX");
+    if (CB >= 2 && (g.HoL % 4) == 0 && boxf <= 512 && little_waste && tp == 128 && encode_fn() != nullptr &&
+        (int64_t)g.N * g.C <= INT32_MAX && !(nobox && nobox[0] == '1')) {
+      P.box = 1;
+      P.TPI = (int32_t)tpi;
+      pitch = boxf;
+    }
+  }
   P.chan_pitch = (int32_t)pitch;
+  const int64_t tiles_m = P.box ? (int64_t)g.N * P.TPI : (g.Mtot + P.TP - 1) / P.TP;
+  P.ntiles = tiles_m * P.n_ntiles;
   const int64_t raw_stage = (int64_t)CB * pitch * 4;
 
   // filter operand: resident if it fits next to two strip stages, else streamed by TMA (TF32, dense groups)
   const int64_t cap = 227 * 1024 - 1024 - 1024;  // alignment slack + barriers
-  const int64_t b_res = (int64_t)P.nchunks * P.NT * 128;
+  const int64_t b_res = (int64_t)steps_tile * P.NT * 32;  // one 32-byte-swizzled block per MMA step
   bool resident = P.n_ntiles == 1 && b_res + 2 * raw_stage <= cap;
   const bool can_stream = !BF16 && KCG == KCGP && (g.C % CB) == 0 && (g.Kg % 4) == 0 && encode_fn() != nullptr;
   if (!resident && !can_stream) return IM2WIN_EUNSUPPORTED;
@@ -647,15 +749,16 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
     P.SB = 1;
   } else {
     P.SB = 6;
-    while (P.SB > 2 && (int64_t)P.SB * P.NT * 128 + 4 * raw_stage > cap) --P.SB;
+    while (P.SB > 3 && (int64_t)P.SB * P.NT * 128 + 4 * raw_stage > cap) --P.SB;
     b_bytes = (int64_t)P.SB * P.NT * 128;
   }
-  // An even number of strip stages: a stage then always serves the same repack half, which sees every
-  // phase of its barrier.
+  // An EVEN number of strip stages.  The two repack halves take alternate groups, so with an even
+  // count a stage is always read by the same half, which then sees every phase of the stage's
+  // barrier.  (A waiter that skips phases can be lapped by two and then waits on the wrong one.)
   P.SR = (int32_t)((cap - b_bytes) / raw_stage);
-  if (P.SR >= 4) P.SR = 4;
-  else if (P.SR >= 2) P.SR = 2;
-  else return IM2WIN_EUNSUPPORTED;
+  if (P.SR > kMaxStages) P.SR = kMaxStages;
+  P.SR &= ~1;
+  if (P.SR < 2) return IM2WIN_EUNSUPPORTED;
 
   // TMEM: accumulators first, then the ring of A slots
   constexpr int SLOT_COLS = SlotGeom<S>::SLOT_STEPS * 8;
@@ -689,19 +792,32 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return IM2WIN_EUNSUPPORTED;
   }
+  CUtensorMap xmap;
+  memset(&xmap, 0, sizeof(xmap));
+  if (P.box) {
+    // the im2win tensor as [N*C planes][HoL/2 8-byte elements]
+    const cuuint64_t gdim[2] = {(cuuint64_t)(g.HoL / 2), (cuuint64_t)g.N * g.C};
+    const cuuint64_t gstr[1] = {(cuuint64_t)g.HoL * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)(P.chan_pitch / 2), (cuuint32_t)CB};
+    const cuuint32_t estr[2] = {1, 1};
+    if (encode_fn()(&xmap, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<float*>(xhat), gdim, gstr, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return IM2WIN_ECUDA;
+  }
   const int64_t grid = P.ntiles < sm_count() ? P.ntiles : sm_count();
   cudaError_t e;
   if (resident) {
     auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, true>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
-    kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap);
+    kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
   } else {
     if constexpr (!BF16) {
       auto kern = conv_tc_persistent_kernel<FH, FW, CB, false, false>;
       e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
       if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
-      kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap);
+      kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
     } else {
       return IM2WIN_EUNSUPPORTED;
     }
