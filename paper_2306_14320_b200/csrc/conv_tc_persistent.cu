@@ -224,13 +224,16 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int32_t raw_stage_floats = CB * P.chan_pitch;
   const uint32_t b_stage_bytes = (uint32_t)P.NT * 128u;
+#ifdef IM2WIN_PROF
+  const long long prof_kernel_t0 = clock64();
+#endif
 
   // ------------------------------------------------------------------ prologue
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxStages; ++i) {
       ptx::mbar_init(ptx::smem_u32(&bars->raw_full[i]), 1);
       ptx::mbar_init(ptx::smem_u32(&bars->raw_empty[i]), 4);
-      ptx::mbar_init(ptx::smem_u32(&bars->b_full[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->b_full[i]), (BRES && i == 0) ? kThreads - 32 : 1);
       ptx::mbar_init(ptx::smem_u32(&bars->b_empty[i]), 1);
     }
     for (int i = 0; i < kMaxSub; ++i) {
@@ -248,43 +251,63 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
     ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), (uint32_t)P.tmem_cols);
     ptx::tmem_relinquish();
   }
-  if constexpr (BRES) {
-    // Build the whole filter operand once, one block of NT rows x 32 bytes per MMA step (padded
-    // reduction indices [s*KSTEP, +KSTEP)), K-major with the 32-byte swizzle, so that the MMA thread
-    // steps its descriptor by a constant.  (A resident filter implies one n-tile.)
-    constexpr int EPP = BF16 ? 8 : 4;  // elements per 16-byte piece
-    const int32_t nsteps_all = P.NG * S;
-    const int32_t pieces = nsteps_all * P.NT * 2;
-    const uint32_t step_bytes = (uint32_t)P.NT * 32u;
-    for (int32_t idx = threadIdx.x; idx < pieces; idx += kThreads) {
-      const int32_t c = idx & 1, j = (idx >> 1) % P.NT, sidx = (idx >> 1) / P.NT;
-      float x[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        x[e] = 0.f;
-        if (e < EPP && j < P.K) {
-          const int32_t kp = sidx * KSTEP + c * EPP + e;
-          const int32_t g = kp / KCGP, kl = kp - g * KCGP;
-          const int64_t k = (int64_t)g * KCG + kl;
-          if (kl < KCG && k < P.Kg) x[e] = __ldg(P.f + (int64_t)j * P.Kg + k);
-        }
-      }
-      uint4 piece;
-      if (BF16) {
-        piece.x = ptx::pack_bf16x2(x[0], x[1]); piece.y = ptx::pack_bf16x2(x[2], x[3]);
-        piece.z = ptx::pack_bf16x2(x[4], x[5]); piece.w = ptx::pack_bf16x2(x[6], x[7]);
-      } else {
-        piece.x = __float_as_uint(x[0]); piece.y = __float_as_uint(x[1]);
-        piece.z = __float_as_uint(x[2]); piece.w = __float_as_uint(x[3]);
-      }
-      *reinterpret_cast<uint4*>(b_smem + (size_t)sidx * step_bytes + (j >> 3) * 256 + (j & 7) * 32 +
-                                ((c ^ ((j >> 2) & 1)) << 4)) = piece;
-    }
-    ptx::fence_proxy_async_smem();
-  }
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
+  if constexpr (BRES) {
+    // Build the whole filter operand once, one block of NT rows x 32 bytes per MMA step (padded
+    // reduction indices [s*KSTEP, +KSTEP)), K-major with the 32-byte swizzle, so that the MMA thread
+    // steps its descriptor by a constant.  (A resident filter implies one n-tile.)  Every warp but
+    // the strip producer takes part; the producer already fetches strips meanwhile, and only the
+    // MMA thread waits for the build to be complete.
+    if (warp != 0) {
+      constexpr int EPP = BF16 ? 8 : 4;  // elements per 16-byte piece
+      const int32_t nsteps_all = P.NG * S;
+      const int32_t pieces = nsteps_all * P.NT * 2;
+      const uint32_t step_bytes = (uint32_t)P.NT * 32u;
+      const bool vec = (KCG == KCGP) && (P.Kg % 4) == 0;  // padded index == real index, rows 16-byte aligned
+      // piece index = [row / 8][step][row % 8][16-byte half]: 16 consecutive threads fill one
+      // contiguous 256-byte swizzle atom in shared memory and read 8 sector-sized runs of the filter
+      for (int32_t idx = (int32_t)threadIdx.x - 32; idx < pieces; idx += kThreads - 32) {
+        const int32_t c = idx & 1, jl = (idx >> 1) & 7;
+        const int32_t rest = idx >> 4;
+        const int32_t sidx = rest % nsteps_all, j = (rest / nsteps_all) * 8 + jl;
+        const int32_t kp0 = sidx * KSTEP + c * EPP;
+        float x[8];
+        if (vec && j < P.K && kp0 + EPP <= P.Kg) {
+          const float4 a = __ldg(reinterpret_cast<const float4*>(P.f + (int64_t)j * P.Kg + kp0));
+          x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+          if (EPP == 8) {
+            const float4 b = __ldg(reinterpret_cast<const float4*>(P.f + (int64_t)j * P.Kg + kp0 + 4));
+            x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            x[e] = 0.f;
+            if (e < EPP && j < P.K) {
+              const int32_t kp = kp0 + e;
+              const int32_t g = kp / KCGP, kl = kp - g * KCGP;
+              const int64_t k = (int64_t)g * KCG + kl;
+              if (kl < KCG && k < P.Kg) x[e] = __ldg(P.f + (int64_t)j * P.Kg + k);
+            }
+          }
+        }
+        uint4 piece;
+        if (BF16) {
+          piece.x = ptx::pack_bf16x2(x[0], x[1]); piece.y = ptx::pack_bf16x2(x[2], x[3]);
+          piece.z = ptx::pack_bf16x2(x[4], x[5]); piece.w = ptx::pack_bf16x2(x[6], x[7]);
+        } else {
+          piece.x = __float_as_uint(x[0]); piece.y = __float_as_uint(x[1]);
+          piece.z = __float_as_uint(x[2]); piece.w = __float_as_uint(x[3]);
+        }
+        *reinterpret_cast<uint4*>(b_smem + (size_t)sidx * step_bytes + (j >> 3) * 256 + (j & 7) * 32 +
+                                  ((c ^ ((j >> 2) & 1)) << 4)) = piece;
+      }
+      ptx::fence_proxy_async_smem();
+      ptx::mbar_arrive(ptx::smem_u32(&bars->b_full[0]));  // resident mode: b_full[0] = "filter built"
+    }
+  }
   const uint32_t tmem_base = misc->tmem_base;
   const uint32_t tmem_a0 = tmem_base + (uint32_t)(P.ND * P.NT);
 
@@ -293,7 +316,10 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
     Ring rr;             // raw stage being filled
     int64_t gcount = 0;  // channel groups issued so far (all tiles)
     bool ok = true;
-    PROF_DECL(1)
+    PROF_DECL(2)
+#ifdef IM2WIN_PROF
+    prof_acc[1] = prof_t0 - prof_kernel_t0;  // prologue (barrier init, TMEM alloc, resident filter build)
+#endif
     for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x) {
       const int64_t tile_m = t / P.n_ntiles;
       int64_t P0, Pend;
@@ -368,7 +394,7 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
           if (bytes[z]) ptx::bulk_g2s(dst[z], src[z], bytes[z], full);
       }
     }
-    PROF_DUMP(0, 1)
+    PROF_DUMP(0, 2)
     // every copy issued must have landed before the CTA exits
     for (int64_t g = max(gcount - P.SR, (int64_t)0); g < gcount; ++g)
       wait_bar(P, misc, &bars->raw_full[g % P.SR], (uint32_t)(g / P.SR) & 1u, DEV_TIMEOUT_DRAIN);
@@ -377,7 +403,7 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
     // One thread; the loop body per MMA is kept to a handful of instructions because a single
     // thread can only issue a tcgen05.mma every few tens of cycles.
     if (lane == 0) {
-      Ring arh[2], br, dr;  // A slot (one ring per repack half), streamed filter stage, accumulator buffer
+      Ring ar0, ar1, br, dr;  // A slot (one ring per repack half), streamed filter stage, accumulator buffer
       uint32_t gpar = 0;    // parity of the running group count = which half produced the group
       bool ok = true;
       PROF_DECL(7)
@@ -391,6 +417,7 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
       const uint32_t a_full0 = ptx::smem_u32(&bars->a_full[0]), a_empty0 = ptx::smem_u32(&bars->a_empty[0]);
       const uint32_t b_full0 = ptx::smem_u32(&bars->b_full[0]), b_empty0 = ptx::smem_u32(&bars->b_empty[0]);
       (void)b_full0; (void)b_empty0;
+      if constexpr (BRES) ok = wait_bar(P, misc, &bars->b_full[0], 0u, DEV_TIMEOUT_B_FULL, PROF_SLOT(1));
       for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
         const int32_t d = dr.idx;
         ok = wait_bar(P, misc, &bars->acc_empty[d], dr.phase ^ 1u, DEV_TIMEOUT_ACC, PROF_SLOT(2));
@@ -401,7 +428,8 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
         uint32_t st0 = 0;             // steps of this tile issued before the current part
         uint32_t b_lo = desc_lo0;     // streamed: descriptor of the current stage
         for (int32_t g = 0; g < P.NG && ok; ++g, gpar ^= 1u) {
-          Ring& ar = arh[gpar];
+          // the ring of the half that produced this group, held in registers (no indexed array)
+          Ring ar = gpar ? ar1 : ar0;
           const int32_t slot0 = (int32_t)gpar * P.NSS;
 #pragma unroll
           for (int h = 0; h < PARTS; ++h) {
@@ -451,6 +479,7 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
             PROF_ADD(5, tc)
             ar.advance(P.NSS);
           }
+          if (gpar) ar1 = ar; else ar0 = ar;
         }
         if (!ok) break;
         if constexpr (!BRES) {
