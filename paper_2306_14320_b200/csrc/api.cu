@@ -61,12 +61,12 @@ int make_geometry(const im2win_shape* sh, Geometry* g) {
 }
 
 int launch_conv_tc(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
-                   cudaStream_t st) {
+                   cudaStream_t st, bool may_alloc) {
   // IM2WIN_FORCE_GENERIC=1 routes every shape through the generic kernel (used by the tests to
   // cover both kernels on the same inputs).
   const char* force = getenv("IM2WIN_FORCE_GENERIC");
   if (!(force && force[0] == '1')) {
-    const int rc = launch_conv_tc_persistent(xhat, f, out, g, mode, st);
+    const int rc = launch_conv_tc_persistent(xhat, f, out, g, mode, st, may_alloc);
     if (rc != IM2WIN_EUNSUPPORTED) return rc;
   }
   return launch_conv_tc_generic(xhat, f, out, g, mode, st);

@@ -46,11 +46,12 @@ int launch_conv_fp32(const float* xhat, const float* f, float* out, const Geomet
 // Tensor-core convolution: the persistent specialised kernel when one applies (it returns
 // IM2WIN_EUNSUPPORTED otherwise), else the generic kernel.
 int launch_conv_tc_persistent(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
-                              cudaStream_t st);
+                              cudaStream_t st, bool may_alloc);
 int launch_conv_tc_generic(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
                            cudaStream_t st);
+// may_alloc = false keeps the call free of any (even stream-ordered) device allocation.
 int launch_conv_tc(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
-                   cudaStream_t st);
+                   cudaStream_t st, bool may_alloc = true);
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? IM2WIN_OK : IM2WIN_ECUDA; }
 

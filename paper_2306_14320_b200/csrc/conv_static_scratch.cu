@@ -74,7 +74,7 @@ int im2win_conv_static(const float* in_nchw, const float* filter_kcfhfw, const i
   rc = launch_transform(in_nchw, scratch, g, st);
   if (rc != IM2WIN_OK) return rc;
   if (mode == IM2WIN_MODE_FP32) return launch_conv_fp32(scratch, filter_kcfhfw, out_nchw, g, st);
-  return launch_conv_tc(scratch, filter_kcfhfw, out_nchw, g, mode, st);
+  return launch_conv_tc(scratch, filter_kcfhfw, out_nchw, g, mode, st, /*may_alloc=*/false);
 }
 
 }  // extern "C"

@@ -16,6 +16,7 @@
 // Warps: 0 strip producer (TMA bulk copies), 1 MMA issuer, 2 filter producer (TMA), 4-11 window
 // repack (two per TMEM lane quarter), 12-15 epilogue.  Every wait is bounded (status word + common teardown on expiry).
 #include <cuda.h>
+#include <cuda_bf16.h>
 
 #include <cstdlib>
 
@@ -671,6 +672,13 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
   }
 }
 
+// fp32 -> bf16 (round to nearest even) copy of the filter, for the TMA-streamed BF16 filter operand
+__global__ void __launch_bounds__(256) filter_to_bf16_kernel(const float* __restrict__ f, __nv_bfloat16* __restrict__ o,
+                                                             int64_t n) {
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (int64_t)gridDim.x * 256)
+    o[i] = __float2bfloat16_rn(f[i]);
+}
+
 // ---------------------------------------------------------------------------------------------- host side
 
 #ifdef IM2WIN_PROF
@@ -697,6 +705,28 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// Memory pool for the temporary bf16 filter copies: the library's own, with an unlimited release
+// threshold, so that after the first call the stream-ordered allocation is served from cached
+// memory instead of going back to the driver.
+cudaMemPool_t filter_pool() {
+  static cudaMemPool_t pools[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return nullptr; }
+  if (!pools[dev]) {
+    cudaMemPoolProps props = {};
+    props.allocType = cudaMemAllocationTypePinned;
+    props.handleTypes = cudaMemHandleTypeNone;
+    props.location.type = cudaMemLocationTypeDevice;
+    props.location.id = dev;
+    cudaMemPool_t pool = nullptr;
+    if (cudaMemPoolCreate(&pool, &props) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    uint64_t keep = UINT64_MAX;
+    if (cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep) != cudaSuccess) cudaGetLastError();
+    pools[dev] = pool;
+  }
+  return pools[dev];
+}
+
 int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -712,7 +742,7 @@ int sm_count() {
 }
 
 template <int FH, int FW, int CB, bool BF16>
-int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st) {
+int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc) {
   constexpr int FF = FH * FW;
   constexpr int KSTEP = BF16 ? 16 : 8;
   constexpr int KCG = CB * FF;
@@ -770,7 +800,11 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
   const int64_t cap = 227 * 1024 - 1024 - 1024;  // alignment slack + barriers
   const int64_t b_res = (int64_t)steps_tile * P.NT * 32;  // one 32-byte-swizzled block per MMA step
   bool resident = P.n_ntiles == 1 && b_res + 2 * raw_stage <= cap;
-  const bool can_stream = !BF16 && KCG == KCGP && (g.C % CB) == 0 && (g.Kg % 4) == 0 && encode_fn() != nullptr;
+  // Streaming needs dense groups (padded reduction index == real index) and 16-byte aligned filter
+  // rows.  In BF16 mode the TMA source is a bf16 copy of the filter made for the duration of the call
+  // in memory from the stream-ordered pool (only where the caller allows an allocation).
+  const bool can_stream = KCG == KCGP && (g.C % CB) == 0 && (g.Kg % (BF16 ? 8 : 4)) == 0 && encode_fn() != nullptr &&
+                          (!BF16 || may_alloc);
   if (!resident && !can_stream) return IM2WIN_EUNSUPPORTED;
   int64_t b_bytes;
   if (resident) {
@@ -811,15 +845,30 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
 
   CUtensorMap fmap;
   memset(&fmap, 0, sizeof(fmap));
+  void* f_bf16 = nullptr;  // BF16 streamed mode: temporary bf16 copy of the filter
   if (!resident) {
     const cuuint64_t gdim[2] = {(cuuint64_t)g.Kg, (cuuint64_t)g.K};
-    const cuuint64_t gstr[1] = {(cuuint64_t)g.Kg * 4};
-    const cuuint32_t box[2] = {32, (cuuint32_t)P.NT};
+    const cuuint64_t gstr[1] = {(cuuint64_t)g.Kg * (BF16 ? 2 : 4)};
+    const cuuint32_t box[2] = {BF16 ? 64u : 32u, (cuuint32_t)P.NT};  // one 128-byte row of the swizzle
     const cuuint32_t estr[2] = {1, 1};
-    if (encode_fn()(&fmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(f), gdim, gstr, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    void* base = const_cast<float*>(f);
+    if (BF16) {
+      cudaMemPool_t pool = filter_pool();
+      if (!pool || cudaMallocFromPoolAsync(&f_bf16, (size_t)g.n_flt * 2, pool, st) != cudaSuccess) {
+        cudaGetLastError();
+        return IM2WIN_EUNSUPPORTED;
+      }
+      const int64_t blocks = (g.n_flt + 255) / 256;
+      filter_to_bf16_kernel<<<(unsigned)(blocks < 148 * 8 ? blocks : 148 * 8), 256, 0, st>>>(
+          f, static_cast<__nv_bfloat16*>(f_bf16), g.n_flt);
+      base = f_bf16;
+    }
+    if (encode_fn()(&fmap, BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, gdim,
+                    gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+      if (f_bf16) cudaFreeAsync(f_bf16, st);
       return IM2WIN_EUNSUPPORTED;
+    }
   }
   CUtensorMap xmap;
   memset(&xmap, 0, sizeof(xmap));
@@ -831,8 +880,10 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
     const cuuint32_t estr[2] = {1, 1};
     if (encode_fn()(&xmap, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<float*>(xhat), gdim, gstr, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+      if (f_bf16) cudaFreeAsync(f_bf16, st);
       return IM2WIN_ECUDA;
+    }
   }
   const int64_t grid = P.ntiles < sm_count() ? P.ntiles : sm_count();
   cudaError_t e;
@@ -842,36 +893,43 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
     if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
     kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
   } else {
-    if constexpr (!BF16) {
-      auto kern = conv_tc_persistent_kernel<FH, FW, CB, false, false>;
-      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-      if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
-      kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
-    } else {
-      return IM2WIN_EUNSUPPORTED;
-    }
+    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, false>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+    if (e != cudaSuccess) { cudaGetLastError(); if (f_bf16) cudaFreeAsync(f_bf16, st); return IM2WIN_ECUDA; }
+    kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
   }
-  return cuda_status(cudaGetLastError());
-}
-
-template <int FH, int FW, int CB>
-int launch_mode(const float* xhat, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st) {
-  return mode == IM2WIN_MODE_BF16 ? launch_spec<FH, FW, CB, true>(xhat, f, out, g, st)
-                                  : launch_spec<FH, FW, CB, false>(xhat, f, out, g, st);
+  const int rc = cuda_status(cudaGetLastError());
+  if (f_bf16) cudaFreeAsync(f_bf16, st);  // stream-ordered: released after the kernel has run
+  return rc;
 }
 
 }  // namespace
 
 // Returns IM2WIN_EUNSUPPORTED when no specialisation applies (the caller then uses the generic kernel).
+// may_alloc: whether the call may take temporary device memory from the stream-ordered pool (the
+// BF16 copy of a filter that is too large to stay in shared memory).
 int launch_conv_tc_persistent(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
-                              cudaStream_t st) {
+                              cudaStream_t st, bool may_alloc) {
+  const bool bf16 = mode == IM2WIN_MODE_BF16;
   if (g.Fh == 3 && g.Fw == 3) {
-    if (g.C >= 8) return launch_mode<3, 3, 8>(xhat, f, out, g, mode, st);
-    if (g.C == 3) return launch_mode<3, 3, 3>(xhat, f, out, g, mode, st);
+    // BF16 MMAs take 16 reduction elements: sixteen channels (144 = 9 steps) leave no padding
+    if (bf16 && g.C % 16 == 0) return launch_spec<3, 3, 16, true>(xhat, f, out, g, st, may_alloc);
+    if (g.C >= 8) return bf16 ? launch_spec<3, 3, 8, true>(xhat, f, out, g, st, may_alloc)
+                              : launch_spec<3, 3, 8, false>(xhat, f, out, g, st, may_alloc);
+    if (g.C == 3) return bf16 ? launch_spec<3, 3, 3, true>(xhat, f, out, g, st, may_alloc)
+                              : launch_spec<3, 3, 3, false>(xhat, f, out, g, st, may_alloc);
   }
-  if (g.Fh == 5 && g.Fw == 5 && g.C >= 8) return launch_mode<5, 5, 8>(xhat, f, out, g, mode, st);
-  if (g.Fh == 7 && g.Fw == 7 && g.C == 3) return launch_mode<7, 7, 3>(xhat, f, out, g, mode, st);
-  if (g.Fh == 11 && g.Fw == 11 && g.C <= 4) return launch_mode<11, 11, 1>(xhat, f, out, g, mode, st);
+  if (g.Fh == 5 && g.Fw == 5) {
+    if (bf16 && g.C % 16 == 0) return launch_spec<5, 5, 16, true>(xhat, f, out, g, st, may_alloc);
+    if (g.C >= 8) return bf16 ? launch_spec<5, 5, 8, true>(xhat, f, out, g, st, may_alloc)
+                              : launch_spec<5, 5, 8, false>(xhat, f, out, g, st, may_alloc);
+  }
+  if (g.Fh == 7 && g.Fw == 7 && g.C == 3)
+    return bf16 ? launch_spec<7, 7, 3, true>(xhat, f, out, g, st, may_alloc)
+                : launch_spec<7, 7, 3, false>(xhat, f, out, g, st, may_alloc);
+  if (g.Fh == 11 && g.Fw == 11 && g.C <= 4)
+    return bf16 ? launch_spec<11, 11, 1, true>(xhat, f, out, g, st, may_alloc)
+                : launch_spec<11, 11, 1, false>(xhat, f, out, g, st, may_alloc);
   return IM2WIN_EUNSUPPORTED;
 }
 
