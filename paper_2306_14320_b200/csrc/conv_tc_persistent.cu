@@ -763,6 +763,16 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
   P.TP = (int32_t)tp;
   P.n_ntiles = (g.K + 255) / 256;
   P.NT = ((g.K + P.n_ntiles - 1) / P.n_ntiles + 15) / 16 * 16;
+  {
+    // Filter tiles stay as wide as the MMA allows (256): a unit of work costs the same number of MMA
+    // instructions and window repacks whatever its width, and narrow MMAs are bound by the issuing
+    // thread, so splitting K further to even out the last wave loses (measured).  Tuning aid only:
+    const char* fix = getenv("IM2WIN_NTILES");
+    if (fix && fix[0] >= '1' && fix[0] <= '8' && (g.K + (fix[0] - '0') - 1) / (fix[0] - '0') <= 256) {
+      P.n_ntiles = fix[0] - '0';
+      P.NT = ((g.K + P.n_ntiles - 1) / P.n_ntiles + 15) / 16 * 16;
+    }
+  }
   P.NG = (g.C + CB - 1) / CB;
   const int32_t steps_tile = P.NG * S;
   P.nchunks = (steps_tile + 3) / 4;
