@@ -21,12 +21,15 @@ struct TransformParams {
   const float* in;
   float* out;
   int32_t H, W, Fh, s, Ho, L;
-  int32_t MB;          // output rows per CTA
-  int32_t nblk;        // row blocks per plane
+  int32_t MB;          // output rows per CTA (row-block mode)
+  int32_t nblk;        // row blocks per plane (1: whole planes per CTA)
+  int32_t PB;          // planes per CTA (> 1 only with nblk == 1)
+  int64_t planes;      // N*C
   int64_t HW;          // input plane (floats)
   int64_t HoL;         // output plane (floats)
   uint64_t magic_L;    // ceil(2^32 / L)
   uint64_t magic_Fh;   // ceil(2^32 / Fh)
+  uint64_t magic_HoL;  // ceil(2^32 / HoL)
 };
 
 __device__ __forceinline__ float4 ldg_stream(const float4* p) {
@@ -36,19 +39,29 @@ __device__ __forceinline__ float4 ldg_stream(const float4* p) {
   return v;
 }
 
-// One CTA: plane p = blockIdx.x / nblk, row block b = blockIdx.x % nblk.
-__global__ void __launch_bounds__(kThreads) transform_smem_kernel(TransformParams P) {
+struct Cursor {  // position of an output element inside the CTA's range
+  int32_t base;  // shared-memory index of (plane, row m, column 0, u = 0): plane*stride + m*s*W
+  int32_t mm, k, u;
+};
+
+// One CTA: either PB whole consecutive planes (small planes), or one block of MB output rows of one
+// plane.  In both cases the input it needs and the output it writes are one contiguous range each.
+__global__ void __launch_bounds__(kThreads) transform_smem_kernel(const TransformParams P) {
   extern __shared__ __align__(16) float smem[];
   const int64_t job = blockIdx.x;
-  const int64_t plane = job / P.nblk;
-  const int32_t b = (int32_t)(job - plane * P.nblk);
+  const int64_t pg = job / P.nblk;
+  const int32_t b = (int32_t)(job - pg * P.nblk);
+  const bool whole = P.nblk == 1;
+  const int64_t plane0 = pg * P.PB;
+  const int32_t npl = whole ? (int32_t)min((int64_t)P.PB, P.planes - plane0) : 1;
   const int32_t m0 = b * P.MB;
-  const int32_t mb = min(P.MB, P.Ho - m0);
-  const int32_t rows_in = (mb - 1) * P.s + P.Fh;
-  const int32_t n_in = rows_in * P.W;
+  const int32_t mb = whole ? P.Ho : min(P.MB, P.Ho - m0);
+  const int32_t rows_in = whole ? P.H : (mb - 1) * P.s + P.Fh;
+  const int32_t plane_floats = rows_in * P.W;  // staged floats per plane
+  const int32_t n_in = npl * plane_floats;
 
   // ---- stage the input range, keeping its 16-byte phase
-  const float* src = P.in + plane * P.HW + (int64_t)m0 * P.s * P.W;
+  const float* src = P.in + plane0 * P.HW + (int64_t)m0 * P.s * P.W;
   const int32_t skew = (int32_t)((reinterpret_cast<uintptr_t>(src) >> 2) & 3);
   float* tile = smem + skew;  // tile[e] <-> src[e]
   {
@@ -64,46 +77,59 @@ __global__ void __launch_bounds__(kThreads) transform_smem_kernel(TransformParam
   __syncthreads();
 
   // ---- emit the output range
-  float* dst = P.out + plane * P.HoL + (int64_t)m0 * P.L;
-  const int32_t n_out = mb * P.L;
+  float* dst = P.out + plane0 * P.HoL + (int64_t)m0 * P.L;
+  const int32_t out_plane = mb * P.L;  // output floats per plane in this CTA
+  const int32_t n_out = npl * out_plane;
   const int32_t dskew = (int32_t)((reinterpret_cast<uintptr_t>(dst) >> 2) & 3);
   const int32_t head = min((4 - dskew) & 3, n_out);
   const int32_t nvec = (n_out - head) >> 2;
   const int32_t tail0 = head + (nvec << 2);
+  const int32_t sW = P.s * P.W;
 
-  // element e of the output range -> shared-memory index of its source
-  auto locate = [&](int32_t e, int32_t& mm, int32_t& k, int32_t& u) {
-    mm = (int32_t)(((uint64_t)(uint32_t)e * P.magic_L) >> 32);
-    const int32_t rem = e - mm * P.L;
-    k = (int32_t)(((uint64_t)(uint32_t)rem * P.magic_Fh) >> 32);
-    u = rem - k * P.Fh;
+  // element e of the output range -> cursor
+  auto locate = [&](int32_t e) -> Cursor {
+    int32_t pl = 0, rem = e;
+    if (npl > 1) {
+      pl = (int32_t)(((uint64_t)(uint32_t)e * P.magic_HoL) >> 32);
+      rem = e - pl * out_plane;
+    }
+    const int32_t mm = (int32_t)(((uint64_t)(uint32_t)rem * P.magic_L) >> 32);
+    const int32_t r2 = rem - mm * P.L;
+    Cursor c;
+    c.mm = mm;
+    c.k = (int32_t)(((uint64_t)(uint32_t)r2 * P.magic_Fh) >> 32);
+    c.u = r2 - c.k * P.Fh;
+    c.base = pl * plane_floats + mm * sW;
+    return c;
   };
-  auto fetch = [&](int32_t mm, int32_t k, int32_t u) { return tile[(mm * P.s + u) * P.W + k]; };
-  auto advance = [&](int32_t& mm, int32_t& k, int32_t& u) {
-    if (++u == P.Fh) { u = 0; if (++k == P.W) { k = 0; ++mm; } }
+  auto fetch = [&](const Cursor& c) { return tile[c.base + c.u * P.W + c.k]; };
+  auto advance = [&](Cursor c) -> Cursor {
+    if (++c.u == P.Fh) {
+      c.u = 0;
+      if (++c.k == P.W) {  // next strip: next output row, or the first row of the next plane
+        c.k = 0;
+        c.base += sW;
+        if (++c.mm == mb) {  // first row of the next plane
+          c.mm = 0;
+          c.base += plane_floats - mb * sW;
+        }
+      }
+    }
+    return c;
   };
 
-  if ((int32_t)threadIdx.x < head) {
-    int32_t mm, k, u;
-    locate(threadIdx.x, mm, k, u);
-    dst[threadIdx.x] = fetch(mm, k, u);
-  }
+  if ((int32_t)threadIdx.x < head) dst[threadIdx.x] = fetch(locate(threadIdx.x));
   float4* dst4 = reinterpret_cast<float4*>(dst + head);
   for (int32_t i = threadIdx.x; i < nvec; i += kThreads) {
-    int32_t mm, k, u;
-    locate(head + (i << 2), mm, k, u);
+    Cursor c = locate(head + (i << 2));
     float4 v;
-    v.x = fetch(mm, k, u); advance(mm, k, u);
-    v.y = fetch(mm, k, u); advance(mm, k, u);
-    v.z = fetch(mm, k, u); advance(mm, k, u);
-    v.w = fetch(mm, k, u);
+    v.x = fetch(c); c = advance(c);
+    v.y = fetch(c); c = advance(c);
+    v.z = fetch(c); c = advance(c);
+    v.w = fetch(c);
     dst4[i] = v;
   }
-  if ((int32_t)threadIdx.x < n_out - tail0) {
-    int32_t mm, k, u;
-    locate(tail0 + threadIdx.x, mm, k, u);
-    dst[tail0 + threadIdx.x] = fetch(mm, k, u);
-  }
+  if ((int32_t)threadIdx.x < n_out - tail0) dst[tail0 + threadIdx.x] = fetch(locate(tail0 + threadIdx.x));
 }
 
 // Fallback for rows too long to stage (Fh*W floats beyond the shared-memory budget): one thread
@@ -147,12 +173,25 @@ int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_
   int32_t MB = (rows_fit - g.Fh) / g.s + 1;              // output rows those feed
   if (MB < 1) MB = 1;
   if (MB > g.Ho) MB = g.Ho;
-  const int32_t nblk = (g.Ho + MB - 1) / MB;
+  int32_t nblk = (g.Ho + MB - 1) / MB;
   MB = (g.Ho + nblk - 1) / nblk;                         // balance the blocks
-  const int32_t rows_in = (MB - 1) * g.s + g.Fh;
-  const size_t smem = ((size_t)rows_in * g.W + 4) * sizeof(float);
+  // Small planes: several whole consecutive planes per CTA, so that a CTA still moves tens of KB.
+  int32_t PB = 1;
+  const int64_t hw = (int64_t)g.H * g.W;
+  if (hw <= budget) {
+    nblk = 1;
+    MB = g.Ho;
+    PB = (int32_t)(budget / hw);
+    const int64_t want_ctas = 148 * 8;                   // keep enough CTAs to fill the machine
+    if (planes / PB < want_ctas) PB = (int32_t)(planes / want_ctas > 0 ? planes / want_ctas : 1);
+    if (PB < 1) PB = 1;
+  }
+  const int32_t rows_in = nblk == 1 ? g.H : (MB - 1) * g.s + g.Fh;
+  const size_t smem = ((size_t)PB * rows_in * g.W + 4) * sizeof(float);
+  const int64_t ctas = nblk == 1 ? (planes + PB - 1) / PB : planes * nblk;
   // magic-number division is exact while (range length) * divisor < 2^32
-  if ((int64_t)MB * g.L * g.L >= ((int64_t)1 << 32) || planes * nblk > INT32_MAX) {
+  const int64_t range = (int64_t)PB * (nblk == 1 ? g.HoL : (int64_t)MB * g.L);
+  if (range * g.HoL >= ((int64_t)1 << 32) || ctas > INT32_MAX || smem > 200 * 1024) {
     const int64_t blocks = (g.n_win + kThreads - 1) / kThreads;
     const int grid = (int)(blocks < 148 * 64 ? blocks : 148 * 64);
     transform_gather_kernel<<<grid, kThreads, 0, st>>>(in, out, g.H, g.W, g.Fh, g.s, g.Ho, g.n_win);
@@ -166,11 +205,12 @@ int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_
   TransformParams P;
   P.in = in; P.out = out;
   P.H = g.H; P.W = g.W; P.Fh = g.Fh; P.s = g.s; P.Ho = g.Ho; P.L = g.L;
-  P.MB = MB; P.nblk = nblk;
-  P.HW = (int64_t)g.H * g.W; P.HoL = g.HoL;
+  P.MB = MB; P.nblk = nblk; P.PB = PB; P.planes = planes;
+  P.HW = hw; P.HoL = g.HoL;
   P.magic_L = magic_for((uint32_t)g.L);
   P.magic_Fh = magic_for((uint32_t)g.Fh);
-  transform_smem_kernel<<<(unsigned)(planes * nblk), kThreads, smem, st>>>(P);
+  P.magic_HoL = magic_for((uint32_t)g.HoL);
+  transform_smem_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(P);
   return cuda_status(cudaGetLastError());
 }
 

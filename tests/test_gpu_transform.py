@@ -15,6 +15,8 @@ SMALL = [
     (1, 2, 130, 1031, 1, 7, 7, 2),     # rows wide enough that one CTA takes only a few output rows
     (1, 1, 30, 5000, 1, 11, 3, 4),     # beyond the staging budget: gather fallback
     (1, 1, 1, 1, 1, 1, 1, 1),
+    (3, 50, 11, 11, 2, 2, 2, 4),       # many small planes per CTA, stride larger than the filter
+    (2, 700, 9, 9, 2, 3, 3, 1), (4, 300, 15, 15, 2, 3, 3, 1), (2, 130, 16, 16, 2, 3, 3, 2),
 ]
 
 
