@@ -35,6 +35,9 @@ from paper_2306_14320_b200 import workloads as wl  # noqa: E402
 METRIC = "conv TFLOP/s (transform + im2win convolution, FLOPs = 2*N*K*Ho*Wo*C*Fh*Fw)"
 UNIT = "TFLOP/s"
 NOMINAL_TF32_OVER_BF16 = 1.1 / 2.25
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (conv_tc_persistent__*.md)
+NCU_TRAFFIC_BYTES = {("resnet3x3", "tf32"): 319.53e6 + 80.16e6, ("deep3x3", "bf16"): 89.38e6 + 5.66e6}
 
 
 def _peaks():
@@ -289,7 +292,7 @@ def run_gpu(args):
     else:
         roof = {"bound": "tensor", "achieved": flops / ms_conv / 1e9, "peak": tensor_peak, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = args.traffic
+    roof["traffic"] = args.traffic if args.traffic is not None else NCU_TRAFFIC_BYTES.get((layer.name, args.mode))
     roof["kernel"] = "conv_tc_kernel"
     roof["peak_source"] = f"of {peaks['source']}" + (" (bf16 burst x nominal tf32/bf16 ratio)" if roof["bound"] == "tensor" and args.mode == "tf32" else "")
     roof["algorithmic_bytes_per_launch"] = r["conv_bytes"]
