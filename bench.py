@@ -216,6 +216,26 @@ def time_layer(layer, mode_name, steps, warmup, torch, b, flush_buf, sampler_ind
     h_used = (ho - 1) * layer.s + layer.Fh
     res["transform_bytes"] = 4.0 * layer.N * layer.C * (h_used * layer.W) + ws_bytes
     res["conv_bytes"] = float(ws_bytes + res["bytes_f"] + res["bytes_out"])
+    # the fused source kind: same result straight from the untransformed input, no im2win tensor in HBM
+    try:
+        for _ in range(3):
+            b.conv(x, b.SRC_NCHW_FUSED, f, dims, mode, out)
+        fe = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+        for k in range(steps):
+            flush_buf.zero_()
+            fe[k][0].record(stream)
+            b.conv(x, b.SRC_NCHW_FUSED, f, dims, mode, out)
+            fe[k][1].record(stream)
+        torch.cuda.synchronize()
+        if b.last_device_status() != 0:
+            raise RuntimeError("device status word set during the fused timing")
+        tf_ = [e[0].elapsed_time(e[1]) for e in fe]
+        res["ms_fused"], res["ms_fused_best"] = sum(tf_) / steps, min(tf_)
+        res["fused_bytes"] = float(res["bytes_in"] + res["bytes_f"] + res["bytes_out"])
+    except b.Im2winError as exc:
+        if exc.code != b.EUNSUPPORTED:
+            raise
+        res["ms_fused"] = None
     if e2e:
         out_host = torch.empty((layer.N, layer.K, ho, wo), dtype=torch.float32).pin_memory()
         n_e2e = max(3, min(steps, 10))
@@ -262,7 +282,10 @@ def run_gpu(args):
                             "transform_gbs": r["transform_bytes"] / r["ms_transform"] / 1e6,
                             "transform_frac_hbm": r["transform_bytes"] / r["ms_transform"] / 1e6 / peaks["hbm_gbs"],
                             "step_tflops": r["flops"] / r["ms_step"] / 1e9, "ms_conv": r["ms_conv"], "ms_transform": r["ms_transform"],
-                            "workspace_bytes": r["workspace_bytes"], "im2col_bytes": r["im2col_bytes"], "peaks": peaks["source"]}
+                            "workspace_bytes": r["workspace_bytes"], "im2col_bytes": r["im2col_bytes"], "peaks": peaks["source"],
+                            "ms_fused": r.get("ms_fused"),
+                            "fused_tflops": (r["flops"] / r["ms_fused"] / 1e9) if r.get("ms_fused") else None,
+                            "fused_frac_hbm": (r["fused_bytes"] / r["ms_fused"] / 1e6 / peaks["hbm_gbs"]) if r.get("ms_fused") else None}
                     print(json.dumps(line), file=sys.stderr, flush=True)
         return
 

@@ -36,7 +36,9 @@ typedef struct {
 
 /* What `src` of im2win_conv points to. */
 enum { IM2WIN_SRC_NCHW = 0,   /* the untransformed input I; the call runs the transform first   */
-       IM2WIN_SRC_IM2WIN = 1  /* an im2win tensor Ihat produced earlier by im2win_transform      */ };
+       IM2WIN_SRC_IM2WIN = 1, /* an im2win tensor Ihat produced earlier by im2win_transform      */
+       IM2WIN_SRC_NCHW_FUSED = 2 /* the untransformed input I; each tile's window rows are built
+                                    on the fly in shared memory, no im2win tensor reaches memory   */ };
 
 /* Arithmetic of the contraction.  Products are accumulated in fp32 in every mode. */
 enum { IM2WIN_MODE_TF32 = 0,  /* tensor cores, operands read as TF32 (low 13 mantissa bits unused) */
@@ -83,6 +85,11 @@ int im2win_transform(const float* in_nchw, const im2win_shape* shape, float* out
  * src:       device.  src_kind NCHW: the input I (N*C*H*W floats); the call first runs the
  *            transform into `workspace`, which then holds Ihat and may be reused by the caller.
  *            src_kind IM2WIN: an im2win tensor; `workspace` is ignored and may be NULL.
+ *            src_kind NCHW_FUSED: the input I; the tensor-core kernel stages the input rows a tile
+ *            needs and reads the windows from them, so nothing of size Ihat is written (workspace
+ *            0 bytes).  Same result as the other two kinds.  Shapes without a fused specialisation
+ *            (see below) fall back to transform + convolution if a sufficient `workspace` is
+ *            given, else EUNSUPPORTED; IM2WIN_MODE_FP32 always takes that fallback.
  * filter:    device, K*C*Fh*Fw floats, native K,C,Fh,Fw order (no repacking needed).
  * mode:      IM2WIN_MODE_*.
  * out_nchw:  device, N*K*Ho*Wo floats, every element is written.

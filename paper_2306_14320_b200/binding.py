@@ -15,7 +15,7 @@ from typing import Sequence
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libim2win.so")
 
-SRC_NCHW, SRC_IM2WIN = 0, 1
+SRC_NCHW, SRC_IM2WIN, SRC_NCHW_FUSED = 0, 1, 2
 MODE_TF32, MODE_BF16, MODE_FP32 = 0, 1, 2
 OK, EINVAL, EALIGN, EWORKSPACE, EOVERLAP, ECUDA, ETIMEOUT, EUNSUPPORTED, ESCRATCH = 0, -1, -2, -3, -4, -5, -6, -7, -8
 

@@ -133,15 +133,28 @@ int im2win_conv(const void* src, int src_kind, const float* filter, const im2win
   int rc = make_geometry(shape, &g);
   if (rc != IM2WIN_OK) return rc;
   if (!src || !filter || !out_nchw) return IM2WIN_EINVAL;
-  if (src_kind != IM2WIN_SRC_NCHW && src_kind != IM2WIN_SRC_IM2WIN) return IM2WIN_EINVAL;
+  if (src_kind != IM2WIN_SRC_NCHW && src_kind != IM2WIN_SRC_IM2WIN && src_kind != IM2WIN_SRC_NCHW_FUSED)
+    return IM2WIN_EINVAL;
   if (mode != IM2WIN_MODE_TF32 && mode != IM2WIN_MODE_BF16 && mode != IM2WIN_MODE_FP32)
     return IM2WIN_EINVAL;
   if (!aligned16(src) || !aligned16(filter) || !aligned16(out_nchw)) return IM2WIN_EALIGN;
-  const int64_t src_bytes = (src_kind == IM2WIN_SRC_NCHW ? g.n_in : g.n_win) * 4;
+  const int64_t src_bytes = (src_kind == IM2WIN_SRC_IM2WIN ? g.n_win : g.n_in) * 4;
   if (overlap(out_nchw, g.n_out * 4, src, src_bytes) || overlap(out_nchw, g.n_out * 4, filter, g.n_flt * 4))
     return IM2WIN_EOVERLAP;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const float* xhat = static_cast<const float*>(src);
+  if (src_kind == IM2WIN_SRC_NCHW_FUSED) {
+    if (mode != IM2WIN_MODE_FP32) {
+      const char* force = getenv("IM2WIN_FORCE_GENERIC");
+      if (!(force && force[0] == '1')) {
+        rc = launch_conv_tc_persistent(xhat, filter, out_nchw, g, mode, st, /*may_alloc=*/true, /*fused=*/true);
+        if (rc != IM2WIN_EUNSUPPORTED) return rc;
+      }
+    }
+    // no fused kernel for this shape or mode: the unfused path, if the caller supplied a workspace
+    if (!workspace || workspace_bytes < (size_t)g.n_win * 4) return IM2WIN_EUNSUPPORTED;
+    src_kind = IM2WIN_SRC_NCHW;
+  }
   if (src_kind == IM2WIN_SRC_NCHW) {
     if (!workspace || workspace_bytes < (size_t)g.n_win * 4) return IM2WIN_EWORKSPACE;
     if (!aligned16(workspace)) return IM2WIN_EALIGN;

@@ -38,8 +38,14 @@ struct PParams {
   const float* f;
   float* out;
   int32_t* status;
-  int32_t C, K, Ho, Wo, L, sFh;
-  int64_t HoL, HoWo, Kg, Mtot, n_win;
+  int32_t C, K, Ho, Wo;
+  int32_t row_mul;      // source floats from one output row to the next: W*Fh (im2win strips) or s*W (raw rows)
+  int32_t col_mul;      // source floats from one output column to the next: s*Fh or s
+  int32_t win_span;     // floats from a window's first to one past its last element: Fh*Fw or (Fh-1)*W+Fw
+  int32_t W;            // input row length (fused source addressing)
+  int64_t plane;        // floats per (image, channel) plane of the source: Ho*W*Fh or H*W
+  int32_t HoWo;         // output positions per image (fits 32 bits; checked on the host)
+  int64_t Kg, Mtot, n_src;
   int32_t TP, NT, n_ntiles;
   int64_t ntiles;       // m tiles * n tiles
   int32_t NG;           // channel groups per tile
@@ -52,7 +58,7 @@ struct PParams {
   int32_t nchunks;      // 128-byte filter chunks per tile
   int32_t tmem_cols;
   uint32_t idesc;
-  uint32_t off_raw, off_bar, off_misc;
+  uint32_t off_raw, off_zero, off_bar, off_misc;  // shared-memory offsets in bytes
 #ifdef IM2WIN_PROF
   long long* prof;  // debug build only: per-role wait-cycle counters of the first CTAs
 #endif
@@ -154,21 +160,59 @@ struct SlotGeom {
   static constexpr int SLOT_STEPS = (S + PARTS - 1) / PARTS;
 };
 
+// Where an m-tile lies: image of its first position, that position's index inside the image, how
+// many positions it has, how many images it touches.  One 64-bit division per tile at most; all
+// other per-tile arithmetic is 32-bit (a tile holds at most 128 positions and 8 images).
+struct TileInfo {
+  int64_t i_first;
+  int32_t q_first, npos, nseg;
+};
+
+__device__ __forceinline__ TileInfo tile_info(const PParams& P, int32_t tile_m) {
+  TileInfo ti;
+  if (P.box) {  // tiles are cut per image
+    const int32_t i = tile_m / P.TPI;
+    ti.i_first = i;
+    ti.q_first = (tile_m - i * P.TPI) * P.TP;
+    ti.npos = min(P.TP, P.HoWo - ti.q_first);
+    ti.nseg = 1;
+  } else if (P.Mtot <= 0x7fffffff) {  // the usual case: 32-bit arithmetic throughout
+    const uint32_t P0 = (uint32_t)tile_m * (uint32_t)P.TP;
+    const uint32_t i = P0 / (uint32_t)P.HoWo;
+    ti.i_first = i;
+    ti.q_first = (int32_t)(P0 - i * (uint32_t)P.HoWo);
+    ti.npos = min(P.TP, (int32_t)((uint32_t)P.Mtot - P0));
+    ti.nseg = (ti.q_first + ti.npos - 1) / P.HoWo + 1;
+  } else {
+    const int64_t P0 = (int64_t)tile_m * P.TP;
+    ti.i_first = P0 / P.HoWo;
+    ti.q_first = (int32_t)(P0 - ti.i_first * P.HoWo);
+    ti.npos = (int32_t)min((int64_t)P.TP, P.Mtot - P0);
+    ti.nseg = (ti.q_first + ti.npos - 1) / P.HoWo + 1;
+  }
+  return ti;
+}
+
+// Row p of the tile: image (as an offset from the tile's first image) and position inside it.
+__device__ __forceinline__ void tile_row(const PParams& P, const TileInfo& ti, int32_t p, int32_t& i_off, int32_t& q) {
+  q = ti.q_first + p;
+  i_off = 0;
+  while (q >= P.HoWo) { q -= P.HoWo; ++i_off; }
+}
+
 // Lanes 0..nseg-1 each describe one image segment of the tile; dst_off is the exclusive prefix sum
 // of the slot sizes.  Must be called by a converged warp.
-__device__ __forceinline__ SegR compute_seg(const PParams& P, int FF, int64_t P0, int64_t Pend, int64_t i_first,
-                                            int32_t nseg, int lane) {
+__device__ __forceinline__ SegR compute_seg(const PParams& P, const TileInfo& ti, int lane) {
   SegR s{0, 0, 0, 0};
   int32_t slot = 0;
-  if (lane < nseg) {
-    const int64_t i = i_first + lane;
-    const int64_t qa = max(P0 - i * P.HoWo, (int64_t)0);
-    const int64_t qb = min(Pend - i * P.HoWo, P.HoWo - 1);
-    const int64_t m_a = qa / P.Wo, n_a = qa - m_a * P.Wo;
-    const int64_t m_b = qb / P.Wo, n_b = qb - m_b * P.Wo;
-    s.virt_a = m_a * P.L + n_a * P.sFh;
-    s.start0 = (i * P.C * P.Ho) * (int64_t)P.L + s.virt_a;
-    s.len = (int32_t)((m_b * P.L + n_b * P.sFh) - s.virt_a) + FF;
+  if (lane < ti.nseg) {
+    const int32_t qa = lane == 0 ? ti.q_first : 0;
+    const int32_t qb = min(ti.q_first + ti.npos - 1 - lane * P.HoWo, P.HoWo - 1);
+    const int32_t m_a = qa / P.Wo, n_a = qa - m_a * P.Wo;
+    const int32_t m_b = qb / P.Wo, n_b = qb - m_b * P.Wo;
+    s.virt_a = (int64_t)m_a * P.row_mul + (int64_t)n_a * P.col_mul;
+    s.start0 = ((ti.i_first + lane) * P.C) * P.plane + s.virt_a;
+    s.len = (int32_t)(((int64_t)m_b * P.row_mul + (int64_t)n_b * P.col_mul) - s.virt_a) + P.win_span;
     slot = (s.len + 6) & ~3;
   }
   int32_t incl = slot;
@@ -181,19 +225,6 @@ __device__ __forceinline__ SegR compute_seg(const PParams& P, int FF, int64_t P0
   return s;
 }
 
-// First and last output position (flattened over image, row, column) of m-tile `tile_m`.
-__device__ __forceinline__ void tile_range(const PParams& P, int64_t tile_m, int64_t& P0, int64_t& Pend) {
-  if (P.box) {  // tiles are cut per image
-    const int64_t i = tile_m / P.TPI;
-    const int64_t q0 = (tile_m - i * P.TPI) * P.TP;
-    P0 = i * P.HoWo + q0;
-    Pend = min(q0 + P.TP, P.HoWo) - 1 + i * P.HoWo;
-  } else {
-    P0 = tile_m * P.TP;
-    Pend = min(P0 + P.TP, P.Mtot) - 1;
-  }
-}
-
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1,
                                             uint32_t bar) {
   asm volatile(
@@ -201,9 +232,9 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
 
-template <int FH, int FW, int CB, bool BF16, bool BRES>
+template <int FH, int FW, int CB, bool BF16, bool BRES, bool FUSED>
 __global__ void __launch_bounds__(kThreads, 1)
-conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_constant__ CUtensorMap fmap,
+conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap fmap,
                           const __grid_constant__ CUtensorMap xmap) {
   constexpr int FF = FH * FW;
   constexpr int KSTEP = BF16 ? 16 : 8;        // reduction elements per MMA
@@ -219,6 +250,7 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
   uint8_t* const smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   uint8_t* const b_smem = smem;  // resident: nchunks * NT*128 bytes; streamed: SB stages of NT*128 bytes
   float* const raw = reinterpret_cast<float*>(smem + P.off_raw);
+  const float* const zero_pad = reinterpret_cast<const float*>(smem + P.off_zero);  // win_span + 8 zeros
   PBars* const bars = reinterpret_cast<PBars*>(smem + P.off_bar);
   PMisc* const misc = reinterpret_cast<PMisc*>(smem + P.off_misc);
 
@@ -242,12 +274,13 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
       ptx::mbar_init(ptx::smem_u32(&bars->a_empty[i]), 1);
     }
     for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), BRES ? 2 : 1);  // one commit per MMA-issuing thread
       ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), 4);
     }
     ptx::fence_mbar_init();
     misc->abort = 0;
   }
+  for (int32_t i = threadIdx.x; i < P.win_span + 8; i += kThreads) reinterpret_cast<float*>(smem + P.off_zero)[i] = 0.f;
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), (uint32_t)P.tmem_cols);
     ptx::tmem_relinquish();
@@ -321,13 +354,11 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
 #ifdef IM2WIN_PROF
     prof_acc[1] = prof_t0 - prof_kernel_t0;  // prologue (barrier init, TMEM alloc, resident filter build)
 #endif
-    for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x) {
-      const int64_t tile_m = t / P.n_ntiles;
-      int64_t P0, Pend;
-      tile_range(P, tile_m, P0, Pend);
-      const int64_t i_first = P0 / P.HoWo;
-      const int32_t nseg = (int32_t)(Pend / P.HoWo - i_first) + 1;
-      const SegR seg = compute_seg(P, FF, P0, Pend, i_first, nseg, lane);
+    for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
+      const TileInfo ti = tile_info(P, t / P.n_ntiles);
+      const int64_t i_first = ti.i_first;
+      const int32_t nseg = ti.nseg;
+      const SegR seg = compute_seg(P, ti, lane);
       // Each lane owns up to two (channel-in-group, image segment) pairs for the whole tile; from
       // group to group only the channel, i.e. the source address, moves (by CB planes).
       const int32_t npairs = CB * nseg;  // <= 64
@@ -343,9 +374,9 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
         const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
         len[z] = __shfl_sync(0xffffffffu, seg.len, sg);
         dsto[z] = rl[z] * P.chan_pitch + __shfl_sync(0xffffffffu, seg.dst_off, sg);
-        start[z] = s_start0 + (int64_t)rl[z] * P.HoL;
+        start[z] = s_start0 + (int64_t)rl[z] * P.plane;
       }
-      const int64_t group_step = (int64_t)CB * P.HoL;
+      const int64_t group_step = (int64_t)CB * P.plane;
       // box mode: the tile lies in one image; x = first needed float of the plane rounded down to
       // 16 bytes (in 8-byte elements), y = plane index of the group's first channel
       const int64_t box_virt = __shfl_sync(0xffffffffu, seg.virt_a, 0);
@@ -375,9 +406,9 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
             const int64_t a0 = start[z] - skew;
             int32_t nfl = (skew + len[z] + 3) & ~3;
             float* d = stage + dsto[z];
-            if (a0 + nfl > P.n_win) {  // the last 16-byte chunk would pass the end of the tensor
-              const int32_t nbulk = (int32_t)((P.n_win - a0) & ~(int64_t)3);
-              for (int64_t e = a0 + nbulk; e < P.n_win; ++e) d[e - a0] = __ldg(P.xhat + e);
+            if (a0 + nfl > P.n_src) {  // the last 16-byte chunk would pass the end of the tensor
+              const int32_t nbulk = (int32_t)((P.n_src - a0) & ~(int64_t)3);
+              for (int64_t e = a0 + nbulk; e < P.n_src; ++e) d[e - a0] = __ldg(P.xhat + e);
               nfl = nbulk;
             }
             src[z] = P.xhat + a0;
@@ -399,10 +430,16 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
     // every copy issued must have landed before the CTA exits
     for (int64_t g = max(gcount - P.SR, (int64_t)0); g < gcount; ++g)
       wait_bar(P, misc, &bars->raw_full[g % P.SR], (uint32_t)(g / P.SR) & 1u, DEV_TIMEOUT_DRAIN);
-  } else if (warp == 1) {
-    // ================================================================ MMA ISSUER
-    // One thread; the loop body per MMA is kept to a handful of instructions because a single
-    // thread can only issue a tcgen05.mma every few tens of cycles.
+  } else if (warp == 1 || (BRES && warp == 3)) {
+    // ================================================================ MMA ISSUER(S)
+    // The loop body per MMA is kept to a handful of instructions because a single thread can only
+    // issue a tcgen05.mma every few tens of cycles -- more than a narrow (N = 64) MMA takes to run.
+    // With a resident filter nothing orders the groups of a tile among themselves (every MMA
+    // accumulates onto an accumulator the epilogue has zeroed), so two threads, in warps 1 and 3,
+    // issue alternate channel groups: each serves the groups of one repack half.  With a streamed
+    // filter the stages are consumed in order by the one thread in warp 1.
+    const uint32_t me = warp == 3 ? 1u : 0u;
+    (void)me;
     if (lane == 0) {
       Ring ar0, ar1, br, dr;  // A slot (one ring per repack half), streamed filter stage, accumulator buffer
       uint32_t gpar = 0;    // parity of the running group count = which half produced the group
@@ -419,16 +456,20 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
       const uint32_t b_full0 = ptx::smem_u32(&bars->b_full[0]), b_empty0 = ptx::smem_u32(&bars->b_empty[0]);
       (void)b_full0; (void)b_empty0;
       if constexpr (BRES) ok = wait_bar(P, misc, &bars->b_full[0], 0u, DEV_TIMEOUT_B_FULL, PROF_SLOT(1));
-      for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
+      for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
         const int32_t d = dr.idx;
-        ok = wait_bar(P, misc, &bars->acc_empty[d], dr.phase ^ 1u, DEV_TIMEOUT_ACC, PROF_SLOT(2));
+        // the epilogue hands the buffer over zeroed (also before its first use)
+        ok = wait_bar(P, misc, &bars->acc_empty[d], dr.phase, DEV_TIMEOUT_ACC, PROF_SLOT(2));
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(d * P.NT);
-        uint32_t accum = 0;
-        uint32_t st0 = 0;             // steps of this tile issued before the current part
+        const uint32_t accum = 1;
+        uint32_t st0 = 0;             // steps of this tile before the current part
         uint32_t b_lo = desc_lo0;     // streamed: descriptor of the current stage
         for (int32_t g = 0; g < P.NG && ok; ++g, gpar ^= 1u) {
+          if constexpr (BRES) {
+            if (gpar != me) { st0 += S; continue; }  // the other issuer's group
+          }
           // the ring of the half that produced this group, held in registers (no indexed array)
           Ring ar = gpar ? ar1 : ar0;
           const int32_t slot0 = (int32_t)gpar * P.NSS;
@@ -466,7 +507,6 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
                   lo = b_lo + (st & 3u) * 2u;
                 }
                 ptx::mma_ts_lohi<BF16>(d_tmem, a_addr + j * 8, lo, desc_hi, P.idesc, accum);
-                accum = 1;
                 if constexpr (!BRES) {
                   if ((st & 3u) == 3u) { ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u); br.advance(P.SB); }
                 }
@@ -488,7 +528,7 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
         }
         ptx::mma_commit(ptx::smem_u32(&bars->acc_full[d]));
       }
-      PROF_DUMP(1, 7)
+      if (me == 0) { PROF_DUMP(1, 7) }
     }
     __syncwarp();
   } else if (warp == 2) {
@@ -498,8 +538,8 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
         int64_t bcount = 0;
         Ring br;
         bool ok = true;
-        for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x) {
-          const int32_t n0 = (int32_t)(t % P.n_ntiles) * P.NT;
+        for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
+          const int32_t n0 = (t % P.n_ntiles) * P.NT;
           for (int32_t c = 0; c < P.nchunks && ok; ++c, ++bcount, br.advance(P.SB)) {
             const int32_t sb = br.idx;
             ok = wait_bar(P, misc, &bars->b_empty[sb], br.phase ^ 1u, DEV_TIMEOUT_B_EMPTY);
@@ -522,35 +562,31 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
     const int32_t q4 = (warp - 4) & 3;
     const int32_t p = q4 * 32 + lane;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
-    const int32_t skew_step = P.box ? 0 : (int32_t)(P.HoL & 3);
+    const int32_t skew_step = P.box ? 0 : (int32_t)(P.plane & 3);
     Ring rr, ar;      // raw stage of the current group, A slot of the current part (this half's own ring)
     const int32_t slot0 = half * P.NSS;
     uint32_t gpar = 0;  // parity of the running group count
     bool ok = true;
-    PROF_DECL(2)
-    for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x) {
-      const int64_t tile_m = t / P.n_ntiles;
-      int64_t P0, Pend;
-      tile_range(P, tile_m, P0, Pend);
-      const int64_t i_first = P0 / P.HoWo;
-      const int32_t nseg = (int32_t)(Pend / P.HoWo - i_first) + 1;
-      const SegR seg = compute_seg(P, FF, P0, Pend, i_first, nseg, lane);
-      const int64_t pos = P0 + p;
-      const bool valid = p < P.TP && pos <= Pend;
-      int64_t i = i_first, q = 0;
-      if (valid) { i = pos / P.HoWo; q = pos - i * P.HoWo; }
-      const int32_t sg = (int32_t)(i - i_first);
+    PROF_DECL(6)
+    for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
+      PROF_T0(tt)
+      const TileInfo ti = tile_info(P, t / P.n_ntiles);
+      const SegR seg = compute_seg(P, ti, lane);
+      const bool valid = p < ti.npos;
+      int32_t sg = 0, q = 0;
+      if (valid) tile_row(P, ti, p, sg, q);
       const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
       const int64_t s_virt = __shfl_sync(0xffffffffu, seg.virt_a, sg);
       const int32_t s_dst = __shfl_sync(0xffffffffu, seg.dst_off, sg);
       int32_t base_off = 0;
       if (valid) {
-        const int64_t m = q / P.Wo, n = q - m * P.Wo;
-        base_off = s_dst + (int32_t)((m * P.L + n * P.sFh) - s_virt);
+        const int32_t m = q / P.Wo, n = q - m * P.Wo;
+        base_off = s_dst + (int32_t)(((int64_t)m * P.row_mul + (int64_t)n * P.col_mul) - s_virt);
       }
       // 16-byte phase of the staged range: box mode rounds inside the plane (the same for every
       // channel, planes being multiples of 16 bytes), the bulk-copy mode per absolute address
       const int32_t skew0 = P.box ? (int32_t)(s_virt & 3) : (int32_t)(s_start0 & 3);
+      PROF_ADD(2, tt)
 
       for (int32_t g = 0; g < P.NG && ok; ++g, gpar ^= 1u) {
         if (gpar != (uint32_t)half) {  // the other half's group
@@ -569,11 +605,19 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
           cptr[rl] = stage + rl * P.chan_pitch + ((skew0 + (r0 + rl) * skew_step) & 3);
         // element kl of the group: channel kl / FF, tap (u, v) = ((kl % FF) / FW, (kl % FF) % FW),
         // stored in the strip at offset v*FH + u from the window start
+        // (fused source: the raw input rows are staged instead, and tap (u, v) is at u*W + v)
+        const int32_t Wsrc = P.W;
+        // channels past C (last group of a C that CB does not divide) read as zero: their pointers
+        // are parked on a zeroed pad so that the hot loop carries no per-element select
+        if (!full_group) {
+#pragma unroll
+          for (int rl = 0; rl < CB; ++rl)
+            if (r0 + rl >= P.C) cptr[rl] = zero_pad;
+        }
         auto elem = [&](int kl) -> float {
           if (kl >= KCG) return 0.f;
           const int rl = kl / FF, w = kl % FF;
-          const float x = cptr[rl][(w % FW) * FH + (w / FW)];
-          return (full_group || r0 + rl < P.C) ? x : 0.f;
+          return FUSED ? cptr[rl][(w / FW) * Wsrc + (w % FW)] : cptr[rl][(w % FW) * FH + (w / FW)];
         };
 #pragma unroll
         for (int h = 0; h < PARTS; ++h) {
@@ -586,6 +630,7 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t a_slot = tmem_a0 + lane_base + (uint32_t)(slot * SLOT_COLS);
+          PROF_T0(tl)
 #pragma unroll
           for (int b = 0; b < NB; ++b) {
             uint32_t v[BATCH][8];
@@ -608,10 +653,13 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
               if (j < nst) ptx::tmem_st_x8(a_slot + (uint32_t)(j * 8), v[jj]);
             }
           }
+          PROF_ADD(3, tl)
+          PROF_T0(tw)
           ptx::tmem_wait_st();
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->a_full[slot]));
+          PROF_ADD(4, tw)
           ar.advance(P.NSS);
         }
         if (!ok) break;
@@ -620,7 +668,7 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
         rr.advance(P.SR);
       }
     }
-    if (half == 0) { PROF_DUMP(2 + q4, 2) }
+    if (half == 0) { PROF_DUMP(2 + q4, 6) }
   } else if (warp >= 12) {
     // ================================================================ EPILOGUE: TMEM -> NCHW
     const int32_t q4 = warp - 12;
@@ -628,39 +676,63 @@ conv_tc_persistent_kernel(const __grid_constant__ PParams P, const __grid_consta
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
     Ring dr;
     bool ok = true;
-    PROF_DECL(1)
-    for (int64_t t = blockIdx.x; t < P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
-      const int64_t tile_m = t / P.n_ntiles;
-      const int32_t n0 = (int32_t)(t - tile_m * P.n_ntiles) * P.NT;
-      int64_t P0, Pend;
-      tile_range(P, tile_m, P0, Pend);
-      const int64_t pos = P0 + p;
-      const bool valid = p < P.TP && pos <= Pend;
-      float* orow = P.out;
-      if (valid) {
-        const int64_t i = pos / P.HoWo, q = pos - i * P.HoWo;
-        orow += (i * P.K + n0) * P.HoWo + q;
-      }
-      const int32_t d = dr.idx;
-      ok = wait_bar_warp(P, misc, &bars->acc_full[d], dr.phase, DEV_TIMEOUT_ACC, PROF_SLOT(0), 256);
-      if (!ok) break;
-      ptx::tc_fence_after();
-      const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)(d * P.NT);
-      for (int32_t c0 = 0; c0 < P.NT; c0 += 16) {
-        uint32_t v[16];
-        ptx::tmem_ld_x16(d_tmem + (uint32_t)c0, v);
-        ptx::tmem_wait_ld();
-        if (valid) {
-#pragma unroll
-          for (int e = 0; e < 16; ++e)
-            if (n0 + c0 + e < P.K) orow[(int64_t)(c0 + e) * P.HoWo] = __uint_as_float(v[e]);
-        }
-      }
+    PROF_DECL(6)
+    const int32_t eK = P.K, eNT = P.NT, eHoWo = P.HoWo;  // kept in registers for the store loop
+    // hand both accumulator buffers to the MMA side zeroed: every MMA accumulates
+    for (int32_t d = 0; d < P.ND; ++d) {
+      for (int32_t c0 = 0; c0 < P.NT; c0 += 16) ptx::tmem_zero_x16(tmem_base + lane_base + (uint32_t)(d * P.NT + c0));
+      ptx::tmem_wait_st();
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->acc_empty[d]));
     }
-    if (q4 == 0) { PROF_DUMP(6, 1) }
+    for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
+      PROF_T0(tp)
+      const int32_t tile_m = t / P.n_ntiles;
+      const int32_t n0 = (t - tile_m * P.n_ntiles) * P.NT;
+      const TileInfo ti = tile_info(P, tile_m);
+      const bool valid = p < ti.npos;
+      float* orow = P.out;
+      if (valid) {
+        int32_t i_off, q;
+        tile_row(P, ti, p, i_off, q);
+        orow += ((ti.i_first + i_off) * P.K + n0) * (int64_t)P.HoWo + q;
+      }
+      const int32_t d = dr.idx;
+      PROF_ADD(1, tp)
+      ok = wait_bar_warp(P, misc, &bars->acc_full[d], dr.phase, DEV_TIMEOUT_ACC, PROF_SLOT(0), 256);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)(d * P.NT);
+      // 16 columns per trip.  Deliberately a rolled loop with a small body: this code runs once per
+      // tile, and a fully unrolled store sequence (hundreds of instructions executed once) spent its
+      // time on instruction fetch, the other roles' code having evicted it in between.
+#pragma unroll 1
+      for (int32_t c0 = 0; c0 < eNT; c0 += 16) {
+        uint32_t v[16];
+        PROF_T0(t1)
+        ptx::tmem_ld_x16(d_tmem + (uint32_t)c0, v);
+        ptx::tmem_wait_ld();
+        PROF_ADD(2, t1)
+        ptx::tmem_zero_x16(d_tmem + (uint32_t)c0);  // leave the columns zeroed for the next tile
+        PROF_T0(t3)
+        if (valid) {
+          float* o = orow + (int64_t)c0 * eHoWo;
+          const int32_t left = eK - n0 - c0;  // filters of this block that exist
+#pragma unroll
+          for (int e = 0; e < 16; ++e)
+            if (e < left) o[(int64_t)e * eHoWo] = __uint_as_float(v[e]);
+        }
+        PROF_ADD(4, t3)
+      }
+      PROF_T0(t4)
+      ptx::tmem_wait_st();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->acc_empty[d]));
+      PROF_ADD(5, t4)
+    }
+    if (q4 == 0) { PROF_DUMP(6, 6) }
   }
 
   // ------------------------------------------------------------------ teardown
@@ -741,8 +813,8 @@ int sm_count() {
   return n;
 }
 
-template <int FH, int FW, int CB, bool BF16>
-int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc) {
+template <int FH, int FW, int CB, bool BF16, bool FUSED>
+int launch_spec_impl(const float* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc) {
   constexpr int FF = FH * FW;
   constexpr int KSTEP = BF16 ? 16 : 8;
   constexpr int KCG = CB * FF;
@@ -756,8 +828,16 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
 #ifdef IM2WIN_PROF
   P.prof = g_prof;
 #endif
-  P.C = g.C; P.K = g.K; P.Ho = g.Ho; P.Wo = g.Wo; P.L = g.L; P.sFh = g.sFh;
-  P.HoL = g.HoL; P.HoWo = g.HoWo; P.Kg = g.Kg; P.Mtot = g.Mtot; P.n_win = g.n_win;
+  P.C = g.C; P.K = g.K; P.Ho = g.Ho; P.Wo = g.Wo; P.W = g.W;
+  if (g.HoWo > (1 << 30)) return IM2WIN_EUNSUPPORTED;
+  P.HoWo = (int32_t)g.HoWo; P.Kg = g.Kg; P.Mtot = g.Mtot;
+  if (FUSED) {  // source = the untransformed input: windows are read from Fh staged rows
+    P.row_mul = g.s * g.W; P.col_mul = g.s; P.win_span = (g.Fh - 1) * g.W + g.Fw;
+    P.plane = (int64_t)g.H * g.W; P.n_src = g.n_in;
+  } else {      // source = the im2win tensor: a window is Fh*Fw contiguous floats of its strip
+    P.row_mul = g.L; P.col_mul = g.sFh; P.win_span = FF;
+    P.plane = g.HoL; P.n_src = g.n_win;
+  }
   int64_t tp = 128;
   if ((kSegMax - 1) * g.HoWo + 1 < tp) tp = (kSegMax - 1) * g.HoWo + 1;
   P.TP = (int32_t)tp;
@@ -778,11 +858,11 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
   P.nchunks = (steps_tile + 3) / 4;
 
   // worst-case floats one channel contributes to a tile
-  const int64_t rowwrap = (int64_t)g.L - (int64_t)(g.Wo - 1) * g.sFh;
+  const int64_t rowwrap = (int64_t)P.row_mul - (int64_t)(g.Wo - 1) * P.col_mul;
   const int64_t wraps = (tp + g.Wo - 2) / g.Wo;
   int64_t nseg_max = (tp - 1) / g.HoWo + 2;
   if (nseg_max > kSegMax) nseg_max = kSegMax;
-  int64_t pitch = (tp - 1) * g.sFh + wraps * (rowwrap > g.sFh ? rowwrap - g.sFh : 0) + nseg_max * (FF + 6) + 4;
+  int64_t pitch = (tp - 1) * P.col_mul + wraps * (rowwrap > P.col_mul ? rowwrap - P.col_mul : 0) + nseg_max * (P.win_span + 6) + 4;
   pitch = (pitch + 3) & ~(int64_t)3;
   if (pitch > (1 << 20)) return IM2WIN_EUNSUPPORTED;
   // Box mode: one 2-D TMA box (CB planes x one contiguous range) per channel group instead of CB
@@ -790,11 +870,11 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
   // elements, and images large enough that cutting tiles per image wastes little.
   {
     const int64_t tpi = (g.HoWo + 127) / 128;
-    const int64_t one_seg = 127 * (int64_t)g.sFh + wraps * (rowwrap > g.sFh ? rowwrap - g.sFh : 0) + FF + 6 + 4;
+    const int64_t one_seg = 127 * (int64_t)P.col_mul + wraps * (rowwrap > P.col_mul ? rowwrap - P.col_mul : 0) + P.win_span + 6 + 4;
     const int64_t boxf = (one_seg + 3) & ~(int64_t)3;
     const bool little_waste = tpi * 128 * 100 <= g.HoWo * 107;
     const char* nobox = getenv("IM2WIN_NO_BOX");
-    if (CB >= 2 && (g.HoL % 4) == 0 && boxf <= 512 && little_waste && tp == 128 && encode_fn() != nullptr &&
+    if (CB >= 2 && (P.plane % 4) == 0 && boxf <= 512 && little_waste && tp == 128 && encode_fn() != nullptr &&
         (int64_t)g.N * g.C <= INT32_MAX && !(nobox && nobox[0] == '1')) {
       P.box = 1;
       P.TPI = (int32_t)tpi;
@@ -807,7 +887,7 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
   const int64_t raw_stage = (int64_t)CB * pitch * 4;
 
   // filter operand: resident if it fits next to two strip stages, else streamed by TMA (TF32, dense groups)
-  const int64_t cap = 227 * 1024 - 1024 - 1024;  // alignment slack + barriers
+  const int64_t cap = 227 * 1024 - 1024 - 1024 - ((int64_t)(P.win_span + 8) * 4 + 16);  // alignment slack, barriers, zero pad
   const int64_t b_res = (int64_t)steps_tile * P.NT * 32;  // one 32-byte-swizzled block per MMA step
   bool resident = P.n_ntiles == 1 && b_res + 2 * raw_stage <= cap;
   // Streaming needs dense groups (padded reduction index == real index) and 16-byte aligned filter
@@ -849,6 +929,7 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
 
   uint32_t off = (uint32_t)b_bytes;
   P.off_raw = off; off += (uint32_t)(P.SR * raw_stage);
+  P.off_zero = off; off += (uint32_t)(((P.win_span + 8) * 4 + 15) / 16 * 16);
   P.off_bar = off; off += (uint32_t)((sizeof(PBars) + 15) / 16 * 16);
   P.off_misc = off; off += 64;
   const size_t smem_bytes = off + 1024;
@@ -884,8 +965,8 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
   memset(&xmap, 0, sizeof(xmap));
   if (P.box) {
     // the im2win tensor as [N*C planes][HoL/2 8-byte elements]
-    const cuuint64_t gdim[2] = {(cuuint64_t)(g.HoL / 2), (cuuint64_t)g.N * g.C};
-    const cuuint64_t gstr[1] = {(cuuint64_t)g.HoL * 4};
+    const cuuint64_t gdim[2] = {(cuuint64_t)(P.plane / 2), (cuuint64_t)g.N * g.C};
+    const cuuint64_t gstr[1] = {(cuuint64_t)P.plane * 4};
     const cuuint32_t box[2] = {(cuuint32_t)(P.chan_pitch / 2), (cuuint32_t)CB};
     const cuuint32_t estr[2] = {1, 1};
     if (encode_fn()(&xmap, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<float*>(xhat), gdim, gstr, box, estr,
@@ -898,12 +979,12 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
   const int64_t grid = P.ntiles < sm_count() ? P.ntiles : sm_count();
   cudaError_t e;
   if (resident) {
-    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, true>;
+    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, true, FUSED>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
     kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
   } else {
-    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, false>;
+    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, false, FUSED>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) { cudaGetLastError(); if (f_bf16) cudaFreeAsync(f_bf16, st); return IM2WIN_ECUDA; }
     kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
@@ -913,33 +994,42 @@ int launch_spec(const float* xhat, const float* f, float* out, const Geometry& g
   return rc;
 }
 
+template <int FH, int FW, int CB, bool BF16>
+int launch_spec(const float* src, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc,
+                bool fused) {
+  return fused ? launch_spec_impl<FH, FW, CB, BF16, true>(src, f, out, g, st, may_alloc)
+               : launch_spec_impl<FH, FW, CB, BF16, false>(src, f, out, g, st, may_alloc);
+}
+
 }  // namespace
 
 // Returns IM2WIN_EUNSUPPORTED when no specialisation applies (the caller then uses the generic kernel).
 // may_alloc: whether the call may take temporary device memory from the stream-ordered pool (the
 // BF16 copy of a filter that is too large to stay in shared memory).
+// fused: `xhat` is the untransformed NCHW input and the windows are built from staged input rows
+// (no im2win tensor exists in global memory).
 int launch_conv_tc_persistent(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
-                              cudaStream_t st, bool may_alloc) {
+                              cudaStream_t st, bool may_alloc, bool fused) {
   const bool bf16 = mode == IM2WIN_MODE_BF16;
   if (g.Fh == 3 && g.Fw == 3) {
     // BF16 MMAs take 16 reduction elements: sixteen channels (144 = 9 steps) leave no padding
-    if (bf16 && g.C % 16 == 0) return launch_spec<3, 3, 16, true>(xhat, f, out, g, st, may_alloc);
-    if (g.C >= 8) return bf16 ? launch_spec<3, 3, 8, true>(xhat, f, out, g, st, may_alloc)
-                              : launch_spec<3, 3, 8, false>(xhat, f, out, g, st, may_alloc);
-    if (g.C == 3) return bf16 ? launch_spec<3, 3, 3, true>(xhat, f, out, g, st, may_alloc)
-                              : launch_spec<3, 3, 3, false>(xhat, f, out, g, st, may_alloc);
+    if (bf16 && g.C % 16 == 0) return launch_spec<3, 3, 16, true>(xhat, f, out, g, st, may_alloc, fused);
+    if (g.C >= 8) return bf16 ? launch_spec<3, 3, 8, true>(xhat, f, out, g, st, may_alloc, fused)
+                              : launch_spec<3, 3, 8, false>(xhat, f, out, g, st, may_alloc, fused);
+    if (g.C == 3) return bf16 ? launch_spec<3, 3, 3, true>(xhat, f, out, g, st, may_alloc, fused)
+                              : launch_spec<3, 3, 3, false>(xhat, f, out, g, st, may_alloc, fused);
   }
   if (g.Fh == 5 && g.Fw == 5) {
-    if (bf16 && g.C % 16 == 0) return launch_spec<5, 5, 16, true>(xhat, f, out, g, st, may_alloc);
-    if (g.C >= 8) return bf16 ? launch_spec<5, 5, 8, true>(xhat, f, out, g, st, may_alloc)
-                              : launch_spec<5, 5, 8, false>(xhat, f, out, g, st, may_alloc);
+    if (bf16 && g.C % 16 == 0) return launch_spec<5, 5, 16, true>(xhat, f, out, g, st, may_alloc, fused);
+    if (g.C >= 8) return bf16 ? launch_spec<5, 5, 8, true>(xhat, f, out, g, st, may_alloc, fused)
+                              : launch_spec<5, 5, 8, false>(xhat, f, out, g, st, may_alloc, fused);
   }
   if (g.Fh == 7 && g.Fw == 7 && g.C == 3)
-    return bf16 ? launch_spec<7, 7, 3, true>(xhat, f, out, g, st, may_alloc)
-                : launch_spec<7, 7, 3, false>(xhat, f, out, g, st, may_alloc);
+    return bf16 ? launch_spec<7, 7, 3, true>(xhat, f, out, g, st, may_alloc, fused)
+                : launch_spec<7, 7, 3, false>(xhat, f, out, g, st, may_alloc, fused);
   if (g.Fh == 11 && g.Fw == 11 && g.C <= 4)
-    return bf16 ? launch_spec<11, 11, 1, true>(xhat, f, out, g, st, may_alloc)
-                : launch_spec<11, 11, 1, false>(xhat, f, out, g, st, may_alloc);
+    return bf16 ? launch_spec<11, 11, 1, true>(xhat, f, out, g, st, may_alloc, fused)
+                : launch_spec<11, 11, 1, false>(xhat, f, out, g, st, may_alloc, fused);
   return IM2WIN_EUNSUPPORTED;
 }
 

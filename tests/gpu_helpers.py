@@ -50,7 +50,7 @@ def gpu_conv(x: np.ndarray, f: np.ndarray, dims, mode: int, src_kind: int = b.SR
     xd = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda()
     fd = torch.from_numpy(np.ascontiguousarray(f, dtype=np.float32)).cuda()
     out = Guarded(n * k * ho * wo)
-    ws = Guarded(b.workspace_bytes(dims) // 4) if src_kind == b.SRC_NCHW else None
+    ws = Guarded(b.workspace_bytes(dims) // 4) if src_kind in (b.SRC_NCHW, b.SRC_NCHW_FUSED) else None
     b.conv(xd, src_kind, fd, dims, mode, out.view, None if ws is None else ws.view,
            0 if ws is None else ws.n * 4)
     status = b.last_device_status()

@@ -65,6 +65,43 @@ def test_conv_small_shapes(dims, mode):
     assert rel_l2(got, ref) <= TOL[mode]
 
 
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("dims", SMALL + [(3, 16, 30, 30, 32, 3, 3, 1), (2, 32, 21, 25, 24, 5, 5, 1), (3, 8, 20, 22, 40, 3, 3, 2)])
+def test_conv_fused_source_small_shapes(dims, mode):
+    """src_kind NCHW_FUSED: windows built from staged input rows, no im2win tensor in memory (shapes
+    without a fused specialisation take the documented fallback through the workspace)."""
+    x, f = _data(dims, 600)
+    got = gpu_conv(x, f, dims, mode, src_kind=b.SRC_NCHW_FUSED)
+    assert rel_l2(got, oracle_conv(x, f, dims)) <= TOL[mode]
+    xi, fi = _data(dims, 700, ints=True)
+    assert np.array_equal(gpu_conv(xi, fi, dims, mode, src_kind=b.SRC_NCHW_FUSED).astype(np.float64), oracle_conv(xi, fi, dims))
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("name,batch", [("tiny", 1), ("resnet3x3", 3), ("stem7x7", 1), ("deep3x3", 3), ("down3x3", 2)]
+                         + [(l.name, 1) for l in wl.SWEEP])
+def test_conv_fused_source_layer_shapes(name, batch, mode):
+    layer = wl.CONFIGS[name].with_batch(batch)
+    x, f = wl.make_input(layer), wl.make_filter(layer)
+    got = gpu_conv(x, f, layer.dims(), mode, src_kind=b.SRC_NCHW_FUSED)
+    assert rel_l2(got, oracle_conv(x, f, layer.dims())) <= TOL[mode]
+
+
+def test_conv_fused_source_needs_no_workspace(request):
+    import torch
+    if "generic" in request.node.name:
+        pytest.skip("the generic kernel has no fused source; that fallback needs a workspace")
+    layer = wl.CONFIGS["resnet3x3"].with_batch(2)
+    dims = layer.dims()
+    x, f = wl.make_input(layer), wl.make_filter(layer)
+    ho, wo = b.out_dims(dims)
+    xd, fd = torch.from_numpy(x).cuda(), torch.from_numpy(f).cuda()
+    out = torch.zeros((2, layer.K, ho, wo), dtype=torch.float32, device="cuda")
+    b.conv(xd, b.SRC_NCHW_FUSED, fd, dims, b.MODE_TF32, out, None, 0)
+    assert b.last_device_status() == 0
+    assert rel_l2(out.cpu().numpy(), oracle_conv(x, f, dims)) <= TOL[b.MODE_TF32]
+
+
 @pytest.mark.parametrize("mode", MODES, ids=MODE_ID.get)
 @pytest.mark.parametrize("dims", SMALL)
 def test_conv_small_integers_bit_exact(dims, mode):
