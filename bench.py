@@ -249,6 +249,23 @@ def time_layer(layer, mode_name, steps, warmup, torch, b, flush_buf, sampler_ind
     return res
 
 
+def max_over_ranks(values, dist, device="cpu"):
+    """Element-wise maximum of a list of per-rank timings over all ranks (the slowest rank defines the
+    job's time); identity when torch.distributed is not initialised.  Used for every multi-GPU number."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.barrier()
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def job_value(flops_per_rank, world, ms_step_max):
+    """Whole-job TFLOP/s under weak scaling: every rank did `flops_per_rank` in the slowest rank's time."""
+    return world * flops_per_rank / ms_step_max / 1e9
+
+
 def run_gpu(args):
     import torch
     from paper_2306_14320_b200 import binding as b, build
@@ -267,7 +284,12 @@ def run_gpu(args):
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
 
     if args.sweep:
-        names = list(wl.CONFIGS) if args.sweep == "all" else args.sweep.split(",")
+        if args.sweep == "all":
+            names = [n for n in wl.CONFIGS if not n.startswith("table1_")]
+        elif args.sweep == "table1":
+            names = [l.name for l in wl.TABLE_I_LAYERS]
+        else:
+            names = args.sweep.split(",")
         for name in names:
             for n_batch in ([128] if not args.sweep_batches else [int(v) for v in args.sweep_batches.split(",")]):
                 layer = wl.CONFIGS[name]
@@ -295,18 +317,15 @@ def run_gpu(args):
     torch.cuda.synchronize()
     r = time_layer(layer, args.mode, args.steps, args.warmup, torch, b, flush_buf, local, e2e=True)
     torch.cuda.synchronize()
-    ms = torch.tensor([r["ms_step"], r["e2e_s"] * 1e3, r["ms_conv"], r["ms_transform"]], dtype=torch.float64, device="cuda")
-    if dist:
-        dist.barrier()
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    ms_step, ms_e2e, ms_conv, ms_tr = [float(v) for v in ms.cpu()]
+    ms_step, ms_e2e, ms_conv, ms_tr = max_over_ranks([r["ms_step"], r["e2e_s"] * 1e3, r["ms_conv"], r["ms_transform"]],
+                                                     dist, device="cuda")
     if rank != 0:
         if dist:
             dist.destroy_process_group()
         return
 
     flops = r["flops"]
-    value = world * flops / ms_step / 1e9
+    value = job_value(flops, world, ms_step)
     tensor_peak = peaks["bf16_tflops"] * (NOMINAL_TF32_OVER_BF16 if args.mode == "tf32" else 1.0)
     t_hbm = r["conv_bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_tensor = flops / (tensor_peak * 1e12)
@@ -316,7 +335,7 @@ def run_gpu(args):
         roof = {"bound": "tensor", "achieved": flops / ms_conv / 1e9, "peak": tensor_peak, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = args.traffic if args.traffic is not None else NCU_TRAFFIC_BYTES.get((layer.name, args.mode))
-    roof["kernel"] = "conv_tc_kernel"
+    roof["kernel"] = "conv_tc_persistent_kernel"
     roof["peak_source"] = f"of {peaks['source']}" + (" (bf16 burst x nominal tf32/bf16 ratio)" if roof["bound"] == "tensor" and args.mode == "tf32" else "")
     roof["algorithmic_bytes_per_launch"] = r["conv_bytes"]
     roof["kernel_ms"] = ms_conv
@@ -337,6 +356,10 @@ def run_gpu(args):
         "transform": {"gbs": r["transform_bytes"] / ms_tr / 1e6, "frac_hbm": r["transform_bytes"] / ms_tr / 1e6 / peaks["hbm_gbs"],
                       "ms": ms_tr, "algorithmic_bytes": r["transform_bytes"], "peak_source": f"of {peaks['source']}"},
         "workspace_bytes": r["workspace_bytes"], "im2col_bytes": r["im2col_bytes"],
+        "fused": ({"value": world * flops / r["ms_fused"] / 1e9, "unit": UNIT, "ms": r["ms_fused"],
+                   "what": "im2win_conv with src_kind NCHW_FUSED: same result from the untransformed input in one kernel, "
+                           "no im2win tensor written (workspace 0 bytes); not part of `value`",
+                   "frac_hbm": r["fused_bytes"] / r["ms_fused"] / 1e6 / peaks["hbm_gbs"]} if r.get("ms_fused") else None),
         "e2e": {"value": world * flops / ms_e2e / 1e9, "unit": UNIT, "h2d_bytes_per_step": r["bytes_in"] + r["bytes_f"],
                 "d2h_bytes_per_step": r["bytes_out"], "ms_per_step": ms_e2e,
                 "how": "im2win_conv_host: pinned host buffers in, pinned host buffer out, wall clock per call"},
@@ -353,7 +376,7 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--mode", default="tf32", choices=["tf32", "bf16"])
@@ -367,7 +390,7 @@ def main():
     if args.warmup < 3 and args.impl == "b200":
         args.warmup = 3
     if args.impl == "reference":
-        if args.steps == 100:
+        if args.steps == 200:
             args.steps = 5
         run_reference(args)
     else:

@@ -199,13 +199,18 @@ const char* im2win_strerror(int status) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Host-buffer convenience path.
+// Host-buffer convenience path: the batch is cut into chunks of images that flow through three
+// streams (host->device copy, kernels, device->host copy), so that the two copy directions and the
+// compute overlap; images are independent, so a chunk is a complete problem of its own.
 
 namespace {
+constexpr int kHostChunks = 8;
 struct HostCtx {
-  cudaStream_t stream = nullptr;
+  cudaStream_t s_in = nullptr, s_cmp = nullptr, s_out = nullptr;
+  cudaEvent_t ev_in[kHostChunks + 1] = {}, ev_cmp[kHostChunks] = {};
   float *d_in = nullptr, *d_f = nullptr, *d_out = nullptr, *d_ws = nullptr;
   size_t b_in = 0, b_f = 0, b_out = 0, b_ws = 0;
+  bool ready = false;
 } g_host;
 
 int grow(float** p, size_t* have, size_t need) {
@@ -220,6 +225,18 @@ int grow(float** p, size_t* have, size_t need) {
   *have = need;
   return IM2WIN_OK;
 }
+
+int host_ctx_init() {
+  if (g_host.ready) return IM2WIN_OK;
+  for (cudaStream_t* st : {&g_host.s_in, &g_host.s_cmp, &g_host.s_out})
+    if (cudaStreamCreateWithFlags(st, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
+  for (cudaEvent_t& e : g_host.ev_in)
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
+  for (cudaEvent_t& e : g_host.ev_cmp)
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
+  g_host.ready = true;
+  return IM2WIN_OK;
+}
 }  // namespace
 
 int im2win_conv_host(const float* in_host, const float* filter_host, const im2win_shape* shape,
@@ -228,33 +245,66 @@ int im2win_conv_host(const float* in_host, const float* filter_host, const im2wi
   int rc = make_geometry(shape, &g);
   if (rc != IM2WIN_OK) return rc;
   if (!in_host || !filter_host || !out_host) return IM2WIN_EINVAL;
-  if (!g_host.stream && cudaStreamCreateWithFlags(&g_host.stream, cudaStreamNonBlocking) != cudaSuccess) {
-    cudaGetLastError();
-    return IM2WIN_ECUDA;
-  }
+  if ((rc = host_ctx_init()) != IM2WIN_OK) return rc;
+  const int64_t in_img = g.n_in / g.N, out_img = g.n_out / g.N, win_img = g.n_win / g.N;
+  // images per chunk: about an eighth of the batch, and such that every chunk starts on a
+  // 16-byte boundary of the device input and output buffers (the kernels require aligned bases)
+  auto need = [](int64_t img_floats) { return img_floats % 4 == 0 ? 1 : (img_floats % 2 == 0 ? 2 : 4); };
+  const int mult = need(in_img) > need(out_img) ? need(in_img) : need(out_img);
+  int per = (g.N + kHostChunks - 1) / kHostChunks;
+  per = (per + mult - 1) / mult * mult;
+  const int nchunks = (g.N + per - 1) / per;
   if ((rc = grow(&g_host.d_in, &g_host.b_in, (size_t)g.n_in * 4)) != IM2WIN_OK) return rc;
   if ((rc = grow(&g_host.d_f, &g_host.b_f, (size_t)g.n_flt * 4)) != IM2WIN_OK) return rc;
   if ((rc = grow(&g_host.d_out, &g_host.b_out, (size_t)g.n_out * 4)) != IM2WIN_OK) return rc;
-  if ((rc = grow(&g_host.d_ws, &g_host.b_ws, (size_t)g.n_win * 4)) != IM2WIN_OK) return rc;
-  cudaStream_t st = g_host.stream;
-  if (cudaMemcpyAsync(g_host.d_in, in_host, (size_t)g.n_in * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(g_host.d_f, filter_host, (size_t)g.n_flt * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+  // workspace for one chunk: only the shapes without a fused kernel use it
+  if ((rc = grow(&g_host.d_ws, &g_host.b_ws, (size_t)win_img * per * 4)) != IM2WIN_OK) return rc;
+  if (cudaMemcpyAsync(g_host.d_f, filter_host, (size_t)g.n_flt * 4, cudaMemcpyHostToDevice, g_host.s_in) != cudaSuccess ||
+      cudaEventRecord(g_host.ev_in[kHostChunks], g_host.s_in) != cudaSuccess ||
+      cudaStreamWaitEvent(g_host.s_cmp, g_host.ev_in[kHostChunks], 0) != cudaSuccess)
     return IM2WIN_ECUDA;
-  rc = im2win_conv(g_host.d_in, IM2WIN_SRC_NCHW, g_host.d_f, shape, mode, g_host.d_out, g_host.d_ws,
-                   g_host.b_ws, st);
-  if (rc != IM2WIN_OK) return rc;
-  if (cudaMemcpyAsync(out_host, g_host.d_out, (size_t)g.n_out * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-    return IM2WIN_ECUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return IM2WIN_ECUDA;
+  for (int c = 0; c < nchunks; ++c) {
+    const int i0 = c * per, n = (i0 + per <= g.N ? per : g.N - i0);
+    if (n <= 0) break;
+    im2win_shape sh = *shape;
+    sh.N = n;
+    const float* hin = in_host + (int64_t)i0 * in_img;
+    float* din = g_host.d_in + (int64_t)i0 * in_img;
+    float* dout = g_host.d_out + (int64_t)i0 * out_img;
+    if (cudaMemcpyAsync(din, hin, (size_t)n * in_img * 4, cudaMemcpyHostToDevice, g_host.s_in) != cudaSuccess ||
+        cudaEventRecord(g_host.ev_in[c], g_host.s_in) != cudaSuccess ||
+        cudaStreamWaitEvent(g_host.s_cmp, g_host.ev_in[c], 0) != cudaSuccess)
+      return IM2WIN_ECUDA;
+    // fused where a specialisation exists (the workspace then stays untouched), else transform + convolution
+    rc = im2win_conv(din, IM2WIN_SRC_NCHW_FUSED, g_host.d_f, &sh, mode, dout, g_host.d_ws, g_host.b_ws, g_host.s_cmp);
+    if (rc != IM2WIN_OK) return rc;
+    if (cudaEventRecord(g_host.ev_cmp[c], g_host.s_cmp) != cudaSuccess ||
+        cudaStreamWaitEvent(g_host.s_out, g_host.ev_cmp[c], 0) != cudaSuccess ||
+        cudaMemcpyAsync(out_host + (int64_t)i0 * out_img, dout, (size_t)n * out_img * 4, cudaMemcpyDeviceToHost,
+                        g_host.s_out) != cudaSuccess)
+      return IM2WIN_ECUDA;
+  }
+  if (cudaStreamSynchronize(g_host.s_out) != cudaSuccess) return IM2WIN_ECUDA;
   return IM2WIN_OK;
 }
 
 int im2win_host_release(void) {
-  if (g_host.stream) cudaStreamSynchronize(g_host.stream);
+  if (g_host.ready) {
+    cudaStreamSynchronize(g_host.s_in);
+    cudaStreamSynchronize(g_host.s_cmp);
+    cudaStreamSynchronize(g_host.s_out);
+  }
   for (float** p : {&g_host.d_in, &g_host.d_f, &g_host.d_out, &g_host.d_ws})
     if (*p) { cudaFree(*p); *p = nullptr; }
   g_host.b_in = g_host.b_f = g_host.b_out = g_host.b_ws = 0;
-  if (g_host.stream) { cudaStreamDestroy(g_host.stream); g_host.stream = nullptr; }
+  if (g_host.ready) {
+    for (cudaEvent_t& e : g_host.ev_in) cudaEventDestroy(e);
+    for (cudaEvent_t& e : g_host.ev_cmp) cudaEventDestroy(e);
+    cudaStreamDestroy(g_host.s_in);
+    cudaStreamDestroy(g_host.s_cmp);
+    cudaStreamDestroy(g_host.s_out);
+    g_host = HostCtx{};
+  }
   return IM2WIN_OK;
 }
 

@@ -871,7 +871,9 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
   {
     const int64_t tpi = (g.HoWo + 127) / 128;
     const int64_t one_seg = 127 * (int64_t)P.col_mul + wraps * (rowwrap > P.col_mul ? rowwrap - P.col_mul : 0) + P.win_span + 6 + 4;
-    const int64_t boxf = (one_seg + 3) & ~(int64_t)3;
+    // rows of the box are a multiple of 128 bytes, so that every stage (CB rows) starts on the
+    // 128-byte boundary a tiled TMA destination needs, whatever CB is
+    const int64_t boxf = (one_seg + 31) & ~(int64_t)31;
     const bool little_waste = tpi * 128 * 100 <= g.HoWo * 107;
     const char* nobox = getenv("IM2WIN_NO_BOX");
     if (CB >= 2 && (P.plane % 4) == 0 && boxf <= 512 && little_waste && tp == 128 && encode_fn() != nullptr &&
@@ -1023,6 +1025,10 @@ int launch_conv_tc_persistent(const float* xhat, const float* f, float* out, con
     if (bf16 && g.C % 16 == 0) return launch_spec<5, 5, 16, true>(xhat, f, out, g, st, may_alloc, fused);
     if (g.C >= 8) return bf16 ? launch_spec<5, 5, 8, true>(xhat, f, out, g, st, may_alloc, fused)
                               : launch_spec<5, 5, 8, false>(xhat, f, out, g, st, may_alloc, fused);
+  }
+  if (g.Fh == 7 && g.Fw == 7 && g.C % 8 == 0) {
+    if (bf16 && g.C % 16 == 0) return launch_spec<7, 7, 16, true>(xhat, f, out, g, st, may_alloc, fused);
+    if (!bf16) return launch_spec<7, 7, 8, false>(xhat, f, out, g, st, may_alloc, fused);
   }
   if (g.Fh == 7 && g.Fw == 7 && g.C == 3)
     return bf16 ? launch_spec<7, 7, 3, true>(xhat, f, out, g, st, may_alloc, fused)

@@ -152,8 +152,18 @@ SWEEP: list[Layer] = _sweep()
 for _l in SWEEP:
     CONFIGS[_l.name] = _l
 
+def _table1() -> list[Layer]:
+    return [Layer(f"table1_Conv{i}", 128, c, h, h, k, f, f, s, pad=0, seed=80 + i)
+            for i, (c, h, k, f, s) in enumerate(TABLE_I, start=1)]
+
+
 # The twelve layer shapes of the paper's Table I (unpadded; batch 128 in its experiments) as
 # (C, H=W, K, Fh=Fw, s).  The output sizes the table prints live in tests/golden/.
 TABLE_I = [(3, 227, 96, 11, 4), (3, 231, 96, 11, 4), (3, 227, 64, 7, 2), (64, 224, 64, 7, 2),
            (96, 24, 256, 5, 1), (256, 12, 512, 3, 1), (3, 224, 64, 3, 1), (64, 112, 128, 3, 1),
            (64, 56, 64, 3, 1), (128, 28, 128, 3, 1), (256, 14, 256, 3, 1), (512, 7, 512, 3, 1)]
+
+# The same twelve as unpadded benchmark layers (batch 128, N(0,1) inputs, Kaiming-normal filters).
+TABLE_I_LAYERS: list[Layer] = _table1()
+for _l in TABLE_I_LAYERS:
+    CONFIGS[_l.name] = _l

@@ -160,6 +160,15 @@ def test_conv_sweep_layers_batch1(layer, mode):
 
 
 @pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("layer", wl.TABLE_I_LAYERS, ids=lambda l: l.name)
+def test_conv_table1_layers_batch1(layer, mode):
+    """The paper's own twelve layers (Table I, unpadded), one image each."""
+    layer = layer.with_batch(1)
+    x, f = wl.make_input(layer), wl.make_filter(layer)
+    assert rel_l2(gpu_conv(x, f, layer.dims(), mode), oracle_conv(x, f, layer.dims())) <= TOL[mode]
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
 @pytest.mark.parametrize("name", ["resnet3x3", "stem7x7", "deep3x3", "down3x3"])
 def test_conv_full_batch_sampled(name, mode):
     """Batch 128, the launch configuration the benchmark times.  The oracle evaluates Eq. (1) at 20000
@@ -183,3 +192,18 @@ def test_conv_full_batch_sampled(name, mode):
         one = layer.with_batch(1).dims()
         assert rel_l2(got[img:img + 1], oracle_conv(x[img:img + 1], f, one)) <= TOL[mode]
     assert np.isfinite(got).all()
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16, b.MODE_FP32], ids=MODE_ID.get)
+@pytest.mark.parametrize("dims", [(19, 16, 30, 30, 32, 3, 3, 1), (3, 5, 17, 19, 7, 2, 3, 2), (1, 3, 32, 32, 16, 3, 3, 1)])
+def test_conv_host_buffers(dims, mode):
+    """im2win_conv_host: host buffers in and out (the batch is pipelined through the GPU in chunks)."""
+    import torch
+    n, c, h, w, k, fh, fw, s = dims
+    x, f = _data(dims, 900)
+    ho, wo = b.out_dims(dims)
+    out = torch.full((n, k, ho, wo), float("nan"), dtype=torch.float32).pin_memory()
+    for _ in range(2):
+        b.conv_host(torch.from_numpy(x).pin_memory(), torch.from_numpy(f), dims, mode, out)
+    assert rel_l2(out.numpy(), oracle_conv(x, f, dims)) <= TOL[mode]
+    b.host_release()

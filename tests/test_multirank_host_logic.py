@@ -1,0 +1,58 @@
+"""The N>1 path of the benchmark has no collective on the data path (images are independent, every
+rank runs its own batch); what it does across ranks is a barrier and a MAX reduction of the timings.
+That host logic runs here as two gloo ranks on CPU."""
+import os
+import socket
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        mine = [1.0 + rank, 10.0 - rank, 5.0]            # rank 1 is slower on the first, faster on the second
+        got = bench.max_over_ranks(mine, dist, device="cpu")
+        assert got == [2.0, 10.0, 5.0], got
+        value = bench.job_value(flops_per_rank=3.0e12, world=world, ms_step_max=got[0])
+        assert value == pytest.approx(world * 3.0e12 / 2.0 / 1e9)
+        with open(os.path.join(out_dir, f"ok{rank}"), "w") as fh:
+            fh.write("ok")
+    finally:
+        dist.destroy_process_group()
+
+
+def test_max_over_ranks_and_job_value_two_gloo_ranks(tmp_path):
+    port = _free_port()
+    mp.spawn(_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    assert sorted(os.listdir(tmp_path)) == ["ok0", "ok1"]
+
+
+def test_single_rank_is_identity():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks([1.5, 2.5], None) == [1.5, 2.5]
+    assert bench.job_value(2.0e12, 1, 4.0) == pytest.approx(0.5e3)
+
+
+def test_reference_arm_runs_on_rank0_only(monkeypatch, capsys):
+    sys.path.insert(0, ROOT)
+    import bench
+    monkeypatch.setenv("RANK", "1")
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--impl", "reference", "--steps", "1", "--warmup", "0"])
+    bench.main()
+    assert capsys.readouterr().out == ""

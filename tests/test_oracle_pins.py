@@ -85,7 +85,6 @@ def test_table1_mean_size_ratio_2p93():
 # ---------------------------------------------------------------- closed forms (Section III-A)
 def _all_layers():
     out = [(l.name, Shape(*l.dims())) for l in wl.CONFIGS.values()]
-    out += [(f"table1_{i}", Shape(128, c, h, h, k, f, f, s)) for i, (c, h, k, f, s) in enumerate(wl.TABLE_I)]
     return out
 
 

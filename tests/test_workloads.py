@@ -43,3 +43,4 @@ def test_named_configs_cover_the_benchmark_definition():
         (1, 3, 32, 32, 16, 3, 3, 1), (128, 64, 58, 58, 64, 3, 3, 1), (128, 3, 230, 230, 64, 7, 7, 2),
         (128, 256, 16, 16, 256, 3, 3, 1), (128, 128, 58, 58, 256, 3, 3, 2)]
     assert len(wl.SWEEP) == 12 and wl.SWEEP[8].dims() == wl.CONFIGS["resnet3x3"].dims()
+    assert [l.dims()[1:] for l in wl.TABLE_I_LAYERS] == [(c, h, h, k, f, f, s) for c, h, k, f, s in wl.TABLE_I]
