@@ -571,21 +571,30 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
       PROF_T0(tt)
       const TileInfo ti = tile_info(P, t / P.n_ntiles);
-      const SegR seg = compute_seg(P, ti, lane);
       const bool valid = p < ti.npos;
-      int32_t sg = 0, q = 0;
-      if (valid) tile_row(P, ti, p, sg, q);
-      const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
-      const int64_t s_virt = __shfl_sync(0xffffffffu, seg.virt_a, sg);
-      const int32_t s_dst = __shfl_sync(0xffffffffu, seg.dst_off, sg);
-      int32_t base_off = 0;
-      if (valid) {
-        const int32_t m = q / P.Wo, n = q - m * P.Wo;
-        base_off = s_dst + (int32_t)(((int64_t)m * P.row_mul + (int64_t)n * P.col_mul) - s_virt);
+      int32_t base_off = 0, skew0 = 0;
+      if (P.box) {
+        // one image, one segment: everything follows from the tile's first position
+        const int32_t m_a = ti.q_first / P.Wo, n_a = ti.q_first - m_a * P.Wo;
+        const int32_t virt_a = m_a * P.row_mul + n_a * P.col_mul;  // box mode: a plane fits 32 bits (host check)
+        if (valid) {
+          const int32_t q = ti.q_first + p;
+          const int32_t m = q / P.Wo, n = q - m * P.Wo;
+          base_off = m * P.row_mul + n * P.col_mul - (virt_a & ~3);  // includes the 16-byte phase
+        }
+      } else {
+        const SegR seg = compute_seg(P, ti, lane);
+        int32_t sg = 0, q = 0;
+        if (valid) tile_row(P, ti, p, sg, q);
+        const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
+        const int64_t s_virt = __shfl_sync(0xffffffffu, seg.virt_a, sg);
+        const int32_t s_dst = __shfl_sync(0xffffffffu, seg.dst_off, sg);
+        if (valid) {
+          const int32_t m = q / P.Wo, n = q - m * P.Wo;
+          base_off = s_dst + (int32_t)(((int64_t)m * P.row_mul + (int64_t)n * P.col_mul) - s_virt);
+        }
+        skew0 = (int32_t)(s_start0 & 3);  // 16-byte phase of the staged range, per absolute address
       }
-      // 16-byte phase of the staged range: box mode rounds inside the plane (the same for every
-      // channel, planes being multiples of 16 bytes), the bulk-copy mode per absolute address
-      const int32_t skew0 = P.box ? (int32_t)(s_virt & 3) : (int32_t)(s_start0 & 3);
       PROF_ADD(2, tt)
 
       for (int32_t g = 0; g < P.NG && ok; ++g, gpar ^= 1u) {
@@ -600,9 +609,14 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         const int32_t r0 = g * CB;
         const bool full_group = r0 + CB <= P.C;
         const float* cptr[CB];
+        if (skew_step == 0) {  // every plane starts on a 16-byte boundary: one phase for all channels
 #pragma unroll
-        for (int rl = 0; rl < CB; ++rl)
-          cptr[rl] = stage + rl * P.chan_pitch + ((skew0 + (r0 + rl) * skew_step) & 3);
+          for (int rl = 0; rl < CB; ++rl) cptr[rl] = stage + rl * P.chan_pitch + skew0;
+        } else {
+#pragma unroll
+          for (int rl = 0; rl < CB; ++rl)
+            cptr[rl] = stage + rl * P.chan_pitch + ((skew0 + (r0 + rl) * skew_step) & 3);
+        }
         // element kl of the group: channel kl / FF, tap (u, v) = ((kl % FF) / FW, (kl % FF) % FW),
         // stored in the strip at offset v*FH + u from the window start
         // (fused source: the raw input rows are staged instead, and tap (u, v) is at u*W + v)
@@ -877,7 +891,7 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
     const bool little_waste = tpi * 128 * 100 <= g.HoWo * 107;
     const char* nobox = getenv("IM2WIN_NO_BOX");
     if (CB >= 2 && (P.plane % 4) == 0 && boxf <= 512 && little_waste && tp == 128 && encode_fn() != nullptr &&
-        (int64_t)g.N * g.C <= INT32_MAX && !(nobox && nobox[0] == '1')) {
+        (int64_t)g.N * g.C <= INT32_MAX && P.plane < ((int64_t)1 << 30) && !(nobox && nobox[0] == '1')) {
       P.box = 1;
       P.TPI = (int32_t)tpi;
       pitch = boxf;
