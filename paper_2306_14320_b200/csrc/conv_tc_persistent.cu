@@ -29,7 +29,7 @@ namespace {
 
 constexpr int kThreads = 512;
 constexpr int kSegMax = 8;
-constexpr int kMaxStages = 8;
+constexpr int kMaxStages = 12;
 constexpr int kMaxSub = 16;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
@@ -53,9 +53,12 @@ struct PParams {
   int32_t SS, NSS;      // MMA steps per A slot; slots per repack half in the TMEM ring
   int32_t ND;           // accumulator buffers
   int32_t chan_pitch;
-  int32_t box;          // 1: strips come as one 2-D TMA box per channel group, tiles never span images
-  int32_t TPI;          // box mode: tiles per image
+  int32_t pim;          // 1: tiles are cut per image (a tile never spans two images)
+  int32_t box;          // 1 (implies pim): strips come as one 2-D TMA box per channel group
+  int32_t TPI;          // pim: tiles per image
+  uint64_t magic_TPI, magic_Wo;  // pim: ceil(2^32 / d); n / d == (n * magic) >> 32 while n * d < 2^32 (host check)
   int32_t nchunks;      // 128-byte filter chunks per tile
+  int32_t b_tma;        // resident filter fetched by TMA (TF32, dense groups) instead of built by the threads
   int32_t tmem_cols;
   uint32_t idesc;
   uint32_t off_raw, off_zero, off_bar, off_misc;  // shared-memory offsets in bytes
@@ -160,6 +163,16 @@ struct SlotGeom {
   static constexpr int SLOT_STEPS = (S + PARTS - 1) / PARTS;
 };
 
+// n / d for the divisors with a precomputed magic (exact while n * d < 2^32: checked on the host)
+__device__ __forceinline__ int32_t fast_div(int32_t n, uint64_t magic) {
+  return (int32_t)(((uint64_t)(uint32_t)n * magic) >> 32);
+}
+
+// m-tile of work unit t (units are numbered m-tile major, n-tile minor; usually there is one n-tile)
+__device__ __forceinline__ int32_t tile_of(const PParams& P, int32_t t) {
+  return P.n_ntiles == 1 ? t : t / P.n_ntiles;
+}
+
 // Where an m-tile lies: image of its first position, that position's index inside the image, how
 // many positions it has, how many images it touches.  One 64-bit division per tile at most; all
 // other per-tile arithmetic is 32-bit (a tile holds at most 128 positions and 8 images).
@@ -170,8 +183,8 @@ struct TileInfo {
 
 __device__ __forceinline__ TileInfo tile_info(const PParams& P, int32_t tile_m) {
   TileInfo ti;
-  if (P.box) {  // tiles are cut per image
-    const int32_t i = tile_m / P.TPI;
+  if (P.pim) {  // tiles are cut per image
+    const int32_t i = fast_div(tile_m, P.magic_TPI);
     ti.i_first = i;
     ti.q_first = (tile_m - i * P.TPI) * P.TP;
     ti.npos = min(P.TP, P.HoWo - ti.q_first);
@@ -259,6 +272,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
   const uint32_t b_stage_bytes = (uint32_t)P.NT * 128u;
 #ifdef IM2WIN_PROF
   const long long prof_kernel_t0 = clock64();
+  if (P.prof && threadIdx.x == 0) { P.prof[512 + blockIdx.x * 4] = (long long)global_ns(); P.prof[512 + blockIdx.x * 4 + 2] = prof_kernel_t0; }
 #endif
 
   // ------------------------------------------------------------------ prologue
@@ -266,7 +280,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     for (int i = 0; i < kMaxStages; ++i) {
       ptx::mbar_init(ptx::smem_u32(&bars->raw_full[i]), 1);
       ptx::mbar_init(ptx::smem_u32(&bars->raw_empty[i]), 4);
-      ptx::mbar_init(ptx::smem_u32(&bars->b_full[i]), (BRES && i == 0) ? kThreads - 32 : 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->b_full[i]), (BRES && i == 0 && !P.b_tma) ? kThreads - 32 : 1);
       ptx::mbar_init(ptx::smem_u32(&bars->b_empty[i]), 1);
     }
     for (int i = 0; i < kMaxSub; ++i) {
@@ -294,7 +308,19 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     // steps its descriptor by a constant.  (A resident filter implies one n-tile.)  Every warp but
     // the strip producer takes part; the producer already fetches strips meanwhile, and only the
     // MMA thread waits for the build to be complete.
-    if (warp != 0) {
+    if (P.b_tma) {
+      // TF32 with dense groups: the operand is the native filter itself, so one TMA box per MMA step
+      // (NT rows x 32 bytes, 32-byte swizzle) lays it out; the lanes of the otherwise idle warp 2
+      // issue them, and no thread waits except the MMA issuers.
+      if (warp == 2) {
+        const int32_t nsteps_all = P.NG * S;
+        const uint32_t full = ptx::smem_u32(&bars->b_full[0]);
+        if (lane == 0) ptx::mbar_arrive_expect_tx(full, (uint32_t)nsteps_all * (uint32_t)P.NT * 32u);
+        __syncwarp();
+        for (int32_t st = lane; st < nsteps_all; st += 32)
+          tma_load_2d(ptx::smem_u32(b_smem) + (uint32_t)st * (uint32_t)P.NT * 32u, &fmap, st * KSTEP, 0, full);
+      }
+    } else if (warp != 0) {
       constexpr int EPP = BF16 ? 8 : 4;  // elements per 16-byte piece
       const int32_t nsteps_all = P.NG * S;
       const int32_t pieces = nsteps_all * P.NT * 2;
@@ -302,41 +328,59 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
       const bool vec = (KCG == KCGP) && (P.Kg % 4) == 0;  // padded index == real index, rows 16-byte aligned
       // piece index = [row / 8][step][row % 8][16-byte half]: 16 consecutive threads fill one
       // contiguous 256-byte swizzle atom in shared memory and read 8 sector-sized runs of the filter
-      for (int32_t idx = (int32_t)threadIdx.x - 32; idx < pieces; idx += kThreads - 32) {
-        const int32_t c = idx & 1, jl = (idx >> 1) & 7;
-        const int32_t rest = idx >> 4;
-        const int32_t sidx = rest % nsteps_all, j = (rest / nsteps_all) * 8 + jl;
-        const int32_t kp0 = sidx * KSTEP + c * EPP;
-        float x[8];
-        if (vec && j < P.K && kp0 + EPP <= P.Kg) {
-          const float4 a = __ldg(reinterpret_cast<const float4*>(P.f + (int64_t)j * P.Kg + kp0));
-          x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
-          if (EPP == 8) {
-            const float4 b = __ldg(reinterpret_cast<const float4*>(P.f + (int64_t)j * P.Kg + kp0 + 4));
-            x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
-          }
-        } else {
+      // Four pieces per thread and trip: all loads of a trip are issued before the first store, so
+      // that a thread has four requests in flight (every CTA reads the same filter at the same
+      // time, and a trip costs one L2 round trip under that load).
+      constexpr int U = 4;
+      for (int32_t base = (int32_t)threadIdx.x - 32; base < pieces; base += U * (kThreads - 32)) {
+        float x[U][8];
+        int32_t dst[U];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            x[e] = 0.f;
-            if (e < EPP && j < P.K) {
-              const int32_t kp = kp0 + e;
-              const int32_t g = kp / KCGP, kl = kp - g * KCGP;
-              const int64_t k = (int64_t)g * KCG + kl;
-              if (kl < KCG && k < P.Kg) x[e] = __ldg(P.f + (int64_t)j * P.Kg + k);
+        for (int u = 0; u < U; ++u) {
+          const int32_t idx = base + u * (kThreads - 32);
+          dst[u] = -1;
+          if (idx < pieces) {
+            const int32_t c = idx & 1, jl = (idx >> 1) & 7;
+            const int32_t rest = idx >> 4;
+            const int32_t jb = rest / nsteps_all;
+            const int32_t sidx = rest - jb * nsteps_all, j = jb * 8 + jl;
+            const int32_t kp0 = sidx * KSTEP + c * EPP;
+            dst[u] = sidx * (int32_t)step_bytes + (j >> 3) * 256 + (j & 7) * 32 + ((c ^ ((j >> 2) & 1)) << 4);
+            if (vec && j < P.K && kp0 + EPP <= P.Kg) {
+              const float4 a = __ldg(reinterpret_cast<const float4*>(P.f + (int64_t)j * P.Kg + kp0));
+              x[u][0] = a.x; x[u][1] = a.y; x[u][2] = a.z; x[u][3] = a.w;
+              if (EPP == 8) {
+                const float4 b = __ldg(reinterpret_cast<const float4*>(P.f + (int64_t)j * P.Kg + kp0 + 4));
+                x[u][4] = b.x; x[u][5] = b.y; x[u][6] = b.z; x[u][7] = b.w;
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                x[u][e] = 0.f;
+                if (e < EPP && j < P.K) {
+                  const int32_t kp = kp0 + e;
+                  const int32_t g = kp / KCGP, kl = kp - g * KCGP;
+                  const int64_t k = (int64_t)g * KCG + kl;
+                  if (kl < KCG && k < P.Kg) x[u][e] = __ldg(P.f + (int64_t)j * P.Kg + k);
+                }
+              }
             }
           }
         }
-        uint4 piece;
-        if (BF16) {
-          piece.x = ptx::pack_bf16x2(x[0], x[1]); piece.y = ptx::pack_bf16x2(x[2], x[3]);
-          piece.z = ptx::pack_bf16x2(x[4], x[5]); piece.w = ptx::pack_bf16x2(x[6], x[7]);
-        } else {
-          piece.x = __float_as_uint(x[0]); piece.y = __float_as_uint(x[1]);
-          piece.z = __float_as_uint(x[2]); piece.w = __float_as_uint(x[3]);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          if (dst[u] >= 0) {
+            uint4 piece;
+            if (BF16) {
+              piece.x = ptx::pack_bf16x2(x[u][0], x[u][1]); piece.y = ptx::pack_bf16x2(x[u][2], x[u][3]);
+              piece.z = ptx::pack_bf16x2(x[u][4], x[u][5]); piece.w = ptx::pack_bf16x2(x[u][6], x[u][7]);
+            } else {
+              piece.x = __float_as_uint(x[u][0]); piece.y = __float_as_uint(x[u][1]);
+              piece.z = __float_as_uint(x[u][2]); piece.w = __float_as_uint(x[u][3]);
+            }
+            *reinterpret_cast<uint4*>(b_smem + dst[u]) = piece;
+          }
         }
-        *reinterpret_cast<uint4*>(b_smem + (size_t)sidx * step_bytes + (j >> 3) * 256 + (j & 7) * 32 +
-                                  ((c ^ ((j >> 2) & 1)) << 4)) = piece;
       }
       ptx::fence_proxy_async_smem();
       ptx::mbar_arrive(ptx::smem_u32(&bars->b_full[0]));  // resident mode: b_full[0] = "filter built"
@@ -350,83 +394,144 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     Ring rr;             // raw stage being filled
     int64_t gcount = 0;  // channel groups issued so far (all tiles)
     bool ok = true;
-    PROF_DECL(2)
+    PROF_DECL(7)
 #ifdef IM2WIN_PROF
     prof_acc[1] = prof_t0 - prof_kernel_t0;  // prologue (barrier init, TMEM alloc, resident filter build)
 #endif
-    for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
-      const TileInfo ti = tile_info(P, t / P.n_ntiles);
-      const int64_t i_first = ti.i_first;
-      const int32_t nseg = ti.nseg;
-      const SegR seg = compute_seg(P, ti, lane);
-      // Each lane owns up to two (channel-in-group, image segment) pairs for the whole tile; from
-      // group to group only the channel, i.e. the source address, moves (by CB planes).
-      const int32_t npairs = CB * nseg;  // <= 64
-      bool act[2];
-      int32_t rl[2], len[2], dsto[2];
-      int64_t start[2];
-#pragma unroll
-      for (int z = 0; z < 2; ++z) {
-        const int32_t idx = z * 32 + lane;
-        act[z] = idx < npairs;
-        rl[z] = act[z] ? idx / nseg : 0;
-        const int32_t sg = act[z] ? idx - rl[z] * nseg : 0;
-        const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
-        len[z] = __shfl_sync(0xffffffffu, seg.len, sg);
-        dsto[z] = rl[z] * P.chan_pitch + __shfl_sync(0xffffffffu, seg.dst_off, sg);
-        start[z] = s_start0 + (int64_t)rl[z] * P.plane;
-      }
-      const int64_t group_step = (int64_t)CB * P.plane;
-      // box mode: the tile lies in one image; x = first needed float of the plane rounded down to
-      // 16 bytes (in 8-byte elements), y = plane index of the group's first channel
-      const int64_t box_virt = __shfl_sync(0xffffffffu, seg.virt_a, 0);
-      const int32_t box_x = (int32_t)((box_virt & ~(int64_t)3) >> 1);
-      const int32_t box_y0 = (int32_t)(i_first * P.C);
-      for (int32_t g = 0; g < P.NG && ok; ++g, ++gcount, rr.advance(P.SR)) {
-        const int32_t sr = rr.idx;
-        ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0), 128);
-        if (!ok) break;
-        const uint32_t full = ptx::smem_u32(&bars->raw_full[sr]);
-        float* stage = raw + (size_t)sr * raw_stage_floats;
-        if (P.box) {
+    if (P.box) {
+      // One 2-D box per channel group.  The tile lies in one image: x = first needed float of the
+      // plane rounded down to 16 bytes (in 8-byte elements), y = plane index of the group's first
+      // channel.  Nothing else is needed per tile, and only one lane works.
+      for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
+        PROF_T0(pa)
+        const int32_t tile_m = tile_of(P, t);
+        const int32_t i = fast_div(tile_m, P.magic_TPI);
+        const int32_t q_first = (tile_m - i * P.TPI) * P.TP;
+        const int32_t m_a = fast_div(q_first, P.magic_Wo), n_a = q_first - m_a * P.Wo;
+        const int32_t box_x = ((m_a * P.row_mul + n_a * P.col_mul) & ~3) >> 1;
+        const int32_t box_y0 = i * P.C;
+        PROF_ADD(2, pa)
+        for (int32_t g = 0; g < P.NG && ok; ++g, ++gcount, rr.advance(P.SR)) {
+          PROF_T0(pb)
+          const int32_t sr = rr.idx;
+          ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0), 128);
+          if (!ok) break;
+          PROF_ADD(3, pb)
+          PROF_T0(pc)
           if (lane == 0) {
+            const uint32_t full = ptx::smem_u32(&bars->raw_full[sr]);
             ptx::mbar_arrive_expect_tx(full, (uint32_t)raw_stage_floats * 4u);
-            tma_load_2d(ptx::smem_u32(stage), &xmap, box_x, box_y0 + g * CB, full);
+            tma_load_2d(ptx::smem_u32(raw + (size_t)sr * raw_stage_floats), &xmap, box_x, box_y0 + g * CB, full);
           }
+          PROF_ADD(4, pc)
+          PROF_T0(pd)
           __syncwarp();
-          continue;
+          PROF_ADD(5, pd)
         }
-        const float* src[2];
-        uint32_t dst[2], bytes[2];
-#pragma unroll
-        for (int z = 0; z < 2; ++z) {
-          bytes[z] = 0;
-          if (act[z] && g * CB + rl[z] < P.C) {
-            const int32_t skew = (int32_t)(start[z] & 3);
-            const int64_t a0 = start[z] - skew;
-            int32_t nfl = (skew + len[z] + 3) & ~3;
-            float* d = stage + dsto[z];
+      }
+    } else if (P.pim) {
+      // Tiles cut per image, strips by bulk copies: lane rl < CB copies the one contiguous range of
+      // channel rl that the tile needs; from group to group only the plane moves.
+      const int64_t group_step = (int64_t)CB * P.plane;
+      for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
+        const int32_t tile_m = tile_of(P, t);
+        const int32_t i = fast_div(tile_m, P.magic_TPI);
+        const int32_t q_first = (tile_m - i * P.TPI) * P.TP;
+        const int32_t q_last = min(q_first + P.TP, P.HoWo) - 1;
+        const int32_t m_a = fast_div(q_first, P.magic_Wo), n_a = q_first - m_a * P.Wo;
+        const int32_t m_b = fast_div(q_last, P.magic_Wo), n_b = q_last - m_b * P.Wo;
+        const int32_t virt_a = m_a * P.row_mul + n_a * P.col_mul;
+        const int32_t len = m_b * P.row_mul + n_b * P.col_mul - virt_a + P.win_span;
+        int64_t start = ((int64_t)i * P.C + lane) * P.plane + virt_a;
+        for (int32_t g = 0; g < P.NG && ok; ++g, ++gcount, rr.advance(P.SR)) {
+          const int32_t sr = rr.idx;
+          ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0), 128);
+          if (!ok) break;
+          const uint32_t full = ptx::smem_u32(&bars->raw_full[sr]);
+          const float* src = nullptr;
+          uint32_t dst = 0, bytes = 0;
+          if (lane < CB && g * CB + lane < P.C) {
+            const int32_t skew = (int32_t)(start & 3);
+            const int64_t a0 = start - skew;
+            int32_t nfl = (skew + len + 3) & ~3;
+            float* d = raw + (size_t)sr * raw_stage_floats + lane * P.chan_pitch;
             if (a0 + nfl > P.n_src) {  // the last 16-byte chunk would pass the end of the tensor
               const int32_t nbulk = (int32_t)((P.n_src - a0) & ~(int64_t)3);
               for (int64_t e = a0 + nbulk; e < P.n_src; ++e) d[e - a0] = __ldg(P.xhat + e);
               nfl = nbulk;
             }
-            src[z] = P.xhat + a0;
-            dst[z] = ptx::smem_u32(d);
-            bytes[z] = (uint32_t)nfl * 4u;
+            src = P.xhat + a0;
+            dst = ptx::smem_u32(d);
+            bytes = (uint32_t)nfl * 4u;
           }
-          start[z] += group_step;
+          start += group_step;
+          const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+          if (lane == 0) ptx::mbar_arrive_expect_tx(full, total);
+          __syncwarp();
+          if (bytes) ptx::bulk_g2s(dst, src, bytes, full);
         }
-        // one arrival carrying the byte count of the whole group, then the copies
-        const uint32_t total = __reduce_add_sync(0xffffffffu, bytes[0] + bytes[1]);
-        if (lane == 0) ptx::mbar_arrive_expect_tx(full, total);
-        __syncwarp();
+      }
+    } else {
+      for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
+        const TileInfo ti = tile_info(P, tile_of(P, t));
+        const int32_t nseg = ti.nseg;
+        const SegR seg = compute_seg(P, ti, lane);
+        // Each lane owns up to two (channel-in-group, image segment) pairs for the whole tile; from
+        // group to group only the channel, i.e. the source address, moves (by CB planes).
+        const int32_t npairs = CB * nseg;  // <= 64
+        bool act[2];
+        int32_t rl[2], len[2], dsto[2];
+        int64_t start[2];
 #pragma unroll
-        for (int z = 0; z < 2; ++z)
-          if (bytes[z]) ptx::bulk_g2s(dst[z], src[z], bytes[z], full);
+        for (int z = 0; z < 2; ++z) {
+          const int32_t idx = z * 32 + lane;
+          act[z] = idx < npairs;
+          rl[z] = act[z] ? idx / nseg : 0;
+          const int32_t sg = act[z] ? idx - rl[z] * nseg : 0;
+          const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
+          len[z] = __shfl_sync(0xffffffffu, seg.len, sg);
+          dsto[z] = rl[z] * P.chan_pitch + __shfl_sync(0xffffffffu, seg.dst_off, sg);
+          start[z] = s_start0 + (int64_t)rl[z] * P.plane;
+        }
+        const int64_t group_step = (int64_t)CB * P.plane;
+        for (int32_t g = 0; g < P.NG && ok; ++g, ++gcount, rr.advance(P.SR)) {
+          const int32_t sr = rr.idx;
+          ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0), 128);
+          if (!ok) break;
+          const uint32_t full = ptx::smem_u32(&bars->raw_full[sr]);
+          float* stage = raw + (size_t)sr * raw_stage_floats;
+          const float* src[2];
+          uint32_t dst[2], bytes[2];
+#pragma unroll
+          for (int z = 0; z < 2; ++z) {
+            bytes[z] = 0;
+            if (act[z] && g * CB + rl[z] < P.C) {
+              const int32_t skew = (int32_t)(start[z] & 3);
+              const int64_t a0 = start[z] - skew;
+              int32_t nfl = (skew + len[z] + 3) & ~3;
+              float* d = stage + dsto[z];
+              if (a0 + nfl > P.n_src) {  // the last 16-byte chunk would pass the end of the tensor
+                const int32_t nbulk = (int32_t)((P.n_src - a0) & ~(int64_t)3);
+                for (int64_t e = a0 + nbulk; e < P.n_src; ++e) d[e - a0] = __ldg(P.xhat + e);
+                nfl = nbulk;
+              }
+              src[z] = P.xhat + a0;
+              dst[z] = ptx::smem_u32(d);
+              bytes[z] = (uint32_t)nfl * 4u;
+            }
+            start[z] += group_step;
+          }
+          // one arrival carrying the byte count of the whole group, then the copies
+          const uint32_t total = __reduce_add_sync(0xffffffffu, bytes[0] + bytes[1]);
+          if (lane == 0) ptx::mbar_arrive_expect_tx(full, total);
+          __syncwarp();
+#pragma unroll
+          for (int z = 0; z < 2; ++z)
+            if (bytes[z]) ptx::bulk_g2s(dst[z], src[z], bytes[z], full);
+        }
       }
     }
-    PROF_DUMP(0, 2)
+    PROF_DUMP(0, 7)
     // every copy issued must have landed before the CTA exits
     for (int64_t g = max(gcount - P.SR, (int64_t)0); g < gcount; ++g)
       wait_bar(P, misc, &bars->raw_full[g % P.SR], (uint32_t)(g / P.SR) & 1u, DEV_TIMEOUT_DRAIN);
@@ -533,6 +638,11 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     __syncwarp();
   } else if (warp == 2) {
     // ================================================================ FILTER PRODUCER (streamed mode)
+    if constexpr (BRES) {
+      // resident filter by TMA: the copies this warp issued must have landed before the CTA exits
+      if (P.b_tma && lane == 0) wait_bar(P, misc, &bars->b_full[0], 0u, DEV_TIMEOUT_DRAIN, nullptr, 1024);
+      __syncwarp();
+    }
     if constexpr (!BRES) {
       if (lane == 0) {
         int64_t bcount = 0;
@@ -567,21 +677,24 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     const int32_t slot0 = half * P.NSS;
     uint32_t gpar = 0;  // parity of the running group count
     bool ok = true;
-    PROF_DECL(6)
+    PROF_DECL(7)
     for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
       PROF_T0(tt)
-      const TileInfo ti = tile_info(P, t / P.n_ntiles);
+      const TileInfo ti = tile_info(P, tile_of(P, t));
       const bool valid = p < ti.npos;
       int32_t base_off = 0, skew0 = 0;
-      if (P.box) {
+      if (P.pim) {
         // one image, one segment: everything follows from the tile's first position
-        const int32_t m_a = ti.q_first / P.Wo, n_a = ti.q_first - m_a * P.Wo;
-        const int32_t virt_a = m_a * P.row_mul + n_a * P.col_mul;  // box mode: a plane fits 32 bits (host check)
+        const int32_t m_a = fast_div(ti.q_first, P.magic_Wo), n_a = ti.q_first - m_a * P.Wo;
+        const int32_t virt_a = m_a * P.row_mul + n_a * P.col_mul;  // a plane fits 32 bits (host check)
         if (valid) {
           const int32_t q = ti.q_first + p;
-          const int32_t m = q / P.Wo, n = q - m * P.Wo;
-          base_off = m * P.row_mul + n * P.col_mul - (virt_a & ~3);  // includes the 16-byte phase
+          const int32_t m = fast_div(q, P.magic_Wo), n = q - m * P.Wo;
+          // box: the staged range starts at the 16-byte boundary below the first float (same phase
+          // in every plane); bulk copies: the phase is per channel, added to the pointers below
+          base_off = m * P.row_mul + n * P.col_mul - (P.box ? (virt_a & ~3) : virt_a);
         }
+        if (!P.box) skew0 = (int32_t)((ti.i_first * P.C * P.plane + virt_a) & 3);
       } else {
         const SegR seg = compute_seg(P, ti, lane);
         int32_t sg = 0, q = 0;
@@ -603,8 +716,10 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           continue;
         }
         const int32_t sr = rr.idx;
+        PROF_T0(twhole)
         ok = wait_bar_warp(P, misc, &bars->raw_full[sr], rr.phase, DEV_TIMEOUT_RAW_FULL, PROF_SLOT(0));
         if (!ok) break;
+        PROF_T0(ts)
         const float* stage = raw + (size_t)sr * raw_stage_floats + base_off;
         const int32_t r0 = g * CB;
         const bool full_group = r0 + CB <= P.C;
@@ -640,6 +755,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           const int j0 = h * SLOT_STEPS;                         // first step of this part in the group
           const int nst = (h == PARTS - 1) ? (S - (PARTS - 1) * SLOT_STEPS) : SLOT_STEPS;
           const int32_t slot = slot0 + ar.idx;
+          if (h == 0) { PROF_ADD(5, ts) }
           ok = wait_bar_warp(P, misc, &bars->a_empty[slot], ar.phase ^ 1u, DEV_TIMEOUT_A_EMPTY, PROF_SLOT(1));
           if (!ok) break;
           ptx::tc_fence_after();
@@ -680,9 +796,10 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->raw_empty[sr]));
         rr.advance(P.SR);
+        PROF_ADD(6, twhole)
       }
     }
-    if (half == 0) { PROF_DUMP(2 + q4, 6) }
+    if (half == 0) { PROF_DUMP(2 + q4, 7) }
   } else if (warp >= 12) {
     // ================================================================ EPILOGUE: TMEM -> NCHW
     const int32_t q4 = warp - 12;
@@ -702,7 +819,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     }
     for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
       PROF_T0(tp)
-      const int32_t tile_m = t / P.n_ntiles;
+      const int32_t tile_m = tile_of(P, t);
       const int32_t n0 = (t - tile_m * P.n_ntiles) * P.NT;
       const TileInfo ti = tile_info(P, tile_m);
       const bool valid = p < ti.npos;
@@ -752,6 +869,9 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
   // ------------------------------------------------------------------ teardown
   ptx::tc_fence_before();
   __syncthreads();
+#ifdef IM2WIN_PROF
+  if (P.prof && threadIdx.x == 0) { P.prof[512 + blockIdx.x * 4 + 1] = (long long)global_ns(); P.prof[512 + blockIdx.x * 4 + 3] = clock64(); }
+#endif
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols);
@@ -879,26 +999,39 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
   int64_t pitch = (tp - 1) * P.col_mul + wraps * (rowwrap > P.col_mul ? rowwrap - P.col_mul : 0) + nseg_max * (P.win_span + 6) + 4;
   pitch = (pitch + 3) & ~(int64_t)3;
   if (pitch > (1 << 20)) return IM2WIN_EUNSUPPORTED;
-  // Box mode: one 2-D TMA box (CB planes x one contiguous range) per channel group instead of CB
-  // bulk copies.  Needs planes that are multiples of 16 bytes, a range of at most 256 8-byte
-  // elements, and images large enough that cutting tiles per image wastes little.
+  // Per-image tiling: where images are large enough that cutting tiles per image wastes little, a
+  // tile lies in one image and needs one contiguous range per channel; the per-tile index work of
+  // every role then is a few multiplications (divisions by precomputed reciprocals).
+  // Box mode (on top of it): one 2-D TMA box (CB planes x one contiguous range) per channel group
+  // instead of CB bulk copies.  Needs planes that are multiples of 16 bytes and a range of at most
+  // 256 8-byte elements.
   {
     const int64_t tpi = (g.HoWo + 127) / 128;
     const int64_t one_seg = 127 * (int64_t)P.col_mul + wraps * (rowwrap > P.col_mul ? rowwrap - P.col_mul : 0) + P.win_span + 6 + 4;
-    // rows of the box are a multiple of 128 bytes, so that every stage (CB rows) starts on the
-    // 128-byte boundary a tiled TMA destination needs, whatever CB is
-    const int64_t boxf = (one_seg + 31) & ~(int64_t)31;
+    // A box row is a whole number of 16-byte units, and CB rows (one stage) a whole number of 128
+    // bytes, so that every stage starts on the 128-byte boundary a tiled TMA destination needs.
+    int64_t row_align = 4;
+    while ((CB * row_align) % 32 != 0) row_align *= 2;
+    const int64_t boxf = (one_seg + row_align - 1) / row_align * row_align;
     const bool little_waste = tpi * 128 * 100 <= g.HoWo * 107;
     const char* nobox = getenv("IM2WIN_NO_BOX");
-    if (CB >= 2 && (P.plane % 4) == 0 && boxf <= 512 && little_waste && tp == 128 && encode_fn() != nullptr &&
-        (int64_t)g.N * g.C <= INT32_MAX && P.plane < ((int64_t)1 << 30) && !(nobox && nobox[0] == '1')) {
-      P.box = 1;
+    const char* nopim = getenv("IM2WIN_NO_PIM");
+    if (little_waste && tp == 128 && P.plane < ((int64_t)1 << 30) && (g.HoWo + 128) * g.Wo < ((int64_t)1 << 32) &&
+        (int64_t)g.N * tpi * tpi < ((int64_t)1 << 32) && one_seg <= (1 << 20) && !(nopim && nopim[0] == '1')) {
+      P.pim = 1;
       P.TPI = (int32_t)tpi;
-      pitch = boxf;
+      P.magic_TPI = (((uint64_t)1 << 32) + (uint64_t)tpi - 1) / (uint64_t)tpi;
+      P.magic_Wo = (((uint64_t)1 << 32) + (uint64_t)g.Wo - 1) / (uint64_t)g.Wo;
+      pitch = (one_seg + 3) & ~(int64_t)3;
+      if (CB >= 2 && (P.plane % 4) == 0 && boxf <= 512 && encode_fn() != nullptr && (int64_t)g.N * g.C <= INT32_MAX &&
+          !(nobox && nobox[0] == '1')) {
+        P.box = 1;
+        pitch = boxf;
+      }
     }
   }
   P.chan_pitch = (int32_t)pitch;
-  const int64_t tiles_m = P.box ? (int64_t)g.N * P.TPI : (g.Mtot + P.TP - 1) / P.TP;
+  const int64_t tiles_m = P.pim ? (int64_t)g.N * P.TPI : (g.Mtot + P.TP - 1) / P.TP;
   P.ntiles = tiles_m * P.n_ntiles;
   const int64_t raw_stage = (int64_t)CB * pitch * 4;
 
@@ -953,6 +1086,18 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
   CUtensorMap fmap;
   memset(&fmap, 0, sizeof(fmap));
   void* f_bf16 = nullptr;  // BF16 streamed mode: temporary bf16 copy of the filter
+  if (resident && !BF16 && KCG == KCGP && (g.C % CB) == 0 && (g.Kg % 4) == 0 && encode_fn() != nullptr &&
+      !(getenv("IM2WIN_NO_BTMA") && getenv("IM2WIN_NO_BTMA")[0] == '1')) {
+    // the native filter as a K x Kg matrix, fetched one MMA step (8 reduction elements) at a time
+    const cuuint64_t gdim[2] = {(cuuint64_t)g.Kg, (cuuint64_t)g.K};
+    const cuuint64_t gstr[1] = {(cuuint64_t)g.Kg * 4};
+    const cuuint32_t box[2] = {8u, (cuuint32_t)P.NT};
+    const cuuint32_t estr[2] = {1, 1};
+    if (encode_fn()(&fmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(f), gdim, gstr, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+      P.b_tma = 1;
+  }
   if (!resident) {
     const cuuint64_t gdim[2] = {(cuuint64_t)g.Kg, (cuuint64_t)g.K};
     const cuuint64_t gstr[1] = {(cuuint64_t)g.Kg * (BF16 ? 2 : 4)};
