@@ -13,8 +13,10 @@
 //     grouping of the staged strips;
 //   * two accumulator buffers when they fit, so that the epilogue of one tile (tcgen05.ld -> NCHW
 //     stores) overlaps the next tile's main loop.
-// Warps: 0 strip producer (TMA bulk copies), 1 MMA issuer, 2 filter producer (TMA), 4-11 window
-// repack (two per TMEM lane quarter), 12-15 epilogue.  Every wait is bounded (status word + common teardown on expiry).
+// Warps (20): 0 strip producer (TMA); 1-3 MMA issuers, one per repack set (resident filter), or 1 MMA
+// issuer and 2 filter producer (streamed filter); 4-15 window repack in up to three sets of four
+// (one warp per TMEM lane quarter), the sets taking channel groups in turn; 16-19 epilogue.
+// Every wait is bounded (status word + common teardown on expiry).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -27,7 +29,10 @@ namespace im2win {
 
 namespace {
 
-constexpr int kThreads = 512;
+constexpr int kThreads = 640;       // 20 warps: see the role list above the kernel
+constexpr int kMaxSets = 3;         // repack warp sets (and MMA-issuing threads with a resident filter)
+constexpr int kRepackWarp0 = 4;     // first repack warp: sets of four (one per TMEM lane quarter)
+constexpr int kEpiWarp0 = kRepackWarp0 + 4 * kMaxSets;
 constexpr int kSegMax = 8;
 constexpr int kMaxStages = 12;
 constexpr int kMaxSub = 16;
@@ -50,7 +55,8 @@ struct PParams {
   int64_t ntiles;       // m tiles * n tiles
   int32_t NG;           // channel groups per tile
   int32_t SR, SB;       // raw strip stages; filter stages (streamed mode)
-  int32_t SS, NSS;      // MMA steps per A slot; slots per repack half in the TMEM ring
+  int32_t NSETS;        // repack warp sets taking channel groups in turn (2 or 3)
+  int32_t SS, NSS;      // MMA steps per A slot; slots per repack set in the TMEM ring
   int32_t ND;           // accumulator buffers
   int32_t chan_pitch;
   int32_t pim;          // 1: tiles are cut per image (a tile never spans two images)
@@ -58,6 +64,7 @@ struct PParams {
   int32_t TPI;          // pim: tiles per image
   uint64_t magic_TPI, magic_Wo;  // pim: ceil(2^32 / d); n / d == (n * magic) >> 32 while n * d < 2^32 (host check)
   int32_t nchunks;      // 128-byte filter chunks per tile
+  int32_t l2_ahead;     // box mode: request the next tile's boxes into L2 one tile ahead
   int32_t b_tma;        // resident filter fetched by TMA (TF32, dense groups) instead of built by the threads
   int32_t tmem_cols;
   uint32_t idesc;
@@ -119,9 +126,8 @@ __device__ __forceinline__ uint64_t global_ns() {
 // Bounded wait (about a second).  A warp that is not ready backs off with nanosleep between polls:
 // sixteen warps share four schedulers, and a warp that spins on try_wait takes issue slots from the
 // MMA-issuing thread on its scheduler, whose instruction rate is what bounds small-N tiles.
-__device__ __forceinline__ bool wait_bar(const PParams& P, PMisc* misc, uint64_t* bar, uint32_t parity,
-                                         int32_t code, long long* acc = nullptr, uint32_t sleep_ns = 64) {
-  const uint32_t b = ptx::smem_u32(bar);
+__device__ __forceinline__ bool wait_bar_a(const PParams& P, PMisc* misc, uint32_t b, uint32_t parity,
+                                           int32_t code, long long* acc = nullptr, uint32_t sleep_ns = 64) {
 #ifdef IM2WIN_PROF
   // try_wait may block inside the instruction, so the clock brackets the first poll too
   const long long c0 = clock64();
@@ -143,9 +149,27 @@ __device__ __forceinline__ bool wait_bar(const PParams& P, PMisc* misc, uint64_t
   return false;
 }
 
+__device__ __forceinline__ bool wait_bar(const PParams& P, PMisc* misc, uint64_t* bar, uint32_t parity,
+                                         int32_t code, long long* acc = nullptr, uint32_t sleep_ns = 64) {
+  return wait_bar_a(P, misc, ptx::smem_u32(bar), parity, code, acc, sleep_ns);
+}
+
 __device__ __forceinline__ bool wait_bar_warp(const PParams& P, PMisc* misc, uint64_t* bar, uint32_t parity,
                                               int32_t code, long long* acc = nullptr, uint32_t sleep_ns = 64) {
   return __all_sync(0xffffffffu, wait_bar(P, misc, bar, parity, code, acc, sleep_ns));
+}
+
+__device__ __forceinline__ bool wait_bar_warp_a(const PParams& P, PMisc* misc, uint32_t b, uint32_t parity,
+                                                int32_t code, long long* acc = nullptr, uint32_t sleep_ns = 64) {
+  return __all_sync(0xffffffffu, wait_bar_a(P, misc, b, parity, code, acc, sleep_ns));
+}
+
+// 32-bit load from a shared-space byte address (kept in program order with the waits and the
+// tcgen05 stores around it)
+__device__ __forceinline__ uint32_t lds_u32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+  return v;
 }
 
 // Position in a ring of n stages together with the parity of the pass over it.
@@ -156,10 +180,15 @@ struct Ring {
     if (++idx == n) { idx = 0; phase ^= 1u; }
   }
 };
-// A group's S MMA steps are handed over in PARTS slots of at most 13 steps (104 TMEM columns).
-template <int S>
+// A group's S MMA steps are handed over in PARTS slots.  With a resident filter, short groups (up
+// to 10 steps) use slots of at most 5 steps (40 TMEM columns): small slots let three repack sets
+// own two or more slots each, so that a set never waits for the MMAs of the part it has just
+// handed over.  Otherwise slots hold up to 13 steps (104 columns), which keeps the number of
+// hand-overs per group low for the single MMA-issuing thread of the streamed-filter mode.
+template <int S, bool BRES>
 struct SlotGeom {
-  static constexpr int PARTS = (S * 8 + 103) / 104;
+  static constexpr int MAXS = (BRES && S <= 10) ? 5 : 13;
+  static constexpr int PARTS = (S + MAXS - 1) / MAXS;
   static constexpr int SLOT_STEPS = (S + PARTS - 1) / PARTS;
 };
 
@@ -245,6 +274,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
 
+// Ask for a box to be brought into L2 (no shared-memory destination, nothing to wait for).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int32_t c0, int32_t c1) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
+}
+
 template <int FH, int FW, int CB, bool BF16, bool BRES, bool FUSED>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap fmap,
@@ -255,8 +289,8 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
   constexpr int KCG = CB * FF;                // real reduction elements per channel group
   constexpr int KCGP = (KCG + KSTEP - 1) / KSTEP * KSTEP;
   constexpr int S = KCGP / KSTEP;             // MMA steps per channel group
-  constexpr int PARTS = SlotGeom<S>::PARTS;   // a group's A columns go to TMEM in PARTS slots
-  constexpr int SLOT_STEPS = SlotGeom<S>::SLOT_STEPS;
+  constexpr int PARTS = SlotGeom<S, BRES>::PARTS;   // a group's A columns go to TMEM in PARTS slots
+  constexpr int SLOT_STEPS = SlotGeom<S, BRES>::SLOT_STEPS;
   constexpr int SLOT_COLS = SLOT_STEPS * 8;
 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -288,7 +322,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
       ptx::mbar_init(ptx::smem_u32(&bars->a_empty[i]), 1);
     }
     for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), BRES ? 2 : 1);  // one commit per MMA-issuing thread
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), BRES ? P.NSETS : 1);  // one commit per MMA-issuing thread
       ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), 4);
     }
     ptx::fence_mbar_init();
@@ -394,7 +428,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     Ring rr;             // raw stage being filled
     int64_t gcount = 0;  // channel groups issued so far (all tiles)
     bool ok = true;
-    PROF_DECL(7)
+    PROF_DECL(2)
 #ifdef IM2WIN_PROF
     prof_acc[1] = prof_t0 - prof_kernel_t0;  // prologue (barrier init, TMEM alloc, resident filter build)
 #endif
@@ -402,31 +436,37 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
       // One 2-D box per channel group.  The tile lies in one image: x = first needed float of the
       // plane rounded down to 16 bytes (in 8-byte elements), y = plane index of the group's first
       // channel.  Nothing else is needed per tile, and only one lane works.
+      // The boxes of this CTA's next tile are requested into L2 one tile ahead, group by group, so
+      // that the copies into the few shared-memory stages later meet L2 latency, not DRAM's.
       for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
-        PROF_T0(pa)
         const int32_t tile_m = tile_of(P, t);
         const int32_t i = fast_div(tile_m, P.magic_TPI);
         const int32_t q_first = (tile_m - i * P.TPI) * P.TP;
         const int32_t m_a = fast_div(q_first, P.magic_Wo), n_a = q_first - m_a * P.Wo;
         const int32_t box_x = ((m_a * P.row_mul + n_a * P.col_mul) & ~3) >> 1;
         const int32_t box_y0 = i * P.C;
-        PROF_ADD(2, pa)
+        const int32_t tn = t + (int32_t)gridDim.x;
+        const bool pf = P.l2_ahead && tn < (int32_t)P.ntiles;
+        int32_t pf_x = 0, pf_y0 = 0;
+        if (pf) {
+          const int32_t tm2 = tile_of(P, tn);
+          const int32_t i2 = fast_div(tm2, P.magic_TPI);
+          const int32_t q2 = (tm2 - i2 * P.TPI) * P.TP;
+          const int32_t m2 = fast_div(q2, P.magic_Wo), n2 = q2 - m2 * P.Wo;
+          pf_x = ((m2 * P.row_mul + n2 * P.col_mul) & ~3) >> 1;
+          pf_y0 = i2 * P.C;
+        }
         for (int32_t g = 0; g < P.NG && ok; ++g, ++gcount, rr.advance(P.SR)) {
-          PROF_T0(pb)
           const int32_t sr = rr.idx;
+          if (pf && lane == 0) tma_prefetch_2d(&xmap, pf_x, pf_y0 + g * CB);
           ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0), 128);
           if (!ok) break;
-          PROF_ADD(3, pb)
-          PROF_T0(pc)
           if (lane == 0) {
             const uint32_t full = ptx::smem_u32(&bars->raw_full[sr]);
             ptx::mbar_arrive_expect_tx(full, (uint32_t)raw_stage_floats * 4u);
             tma_load_2d(ptx::smem_u32(raw + (size_t)sr * raw_stage_floats), &xmap, box_x, box_y0 + g * CB, full);
           }
-          PROF_ADD(4, pc)
-          PROF_T0(pd)
           __syncwarp();
-          PROF_ADD(5, pd)
         }
       }
     } else if (P.pim) {
@@ -531,23 +571,24 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         }
       }
     }
-    PROF_DUMP(0, 7)
+    PROF_DUMP(0, 2)
     // every copy issued must have landed before the CTA exits
     for (int64_t g = max(gcount - P.SR, (int64_t)0); g < gcount; ++g)
       wait_bar(P, misc, &bars->raw_full[g % P.SR], (uint32_t)(g / P.SR) & 1u, DEV_TIMEOUT_DRAIN);
-  } else if (warp == 1 || (BRES && warp == 3)) {
+  } else if (warp == 1 || (BRES && warp >= 2 && warp <= P.NSETS)) {
     // ================================================================ MMA ISSUER(S)
     // The loop body per MMA is kept to a handful of instructions because a single thread can only
     // issue a tcgen05.mma every few tens of cycles -- more than a narrow (N = 64) MMA takes to run.
     // With a resident filter nothing orders the groups of a tile among themselves (every MMA
-    // accumulates onto an accumulator the epilogue has zeroed), so two threads, in warps 1 and 3,
-    // issue alternate channel groups: each serves the groups of one repack half.  With a streamed
-    // filter the stages are consumed in order by the one thread in warp 1.
-    const uint32_t me = warp == 3 ? 1u : 0u;
+    // accumulates onto an accumulator the epilogue has zeroed), so one thread per repack set, in
+    // warps 1, 2, (3), issues the groups that set produced.  With a streamed filter the stages are
+    // consumed in order by the one thread in warp 1.
+    const uint32_t me = (uint32_t)(warp - 1);
     (void)me;
     if (lane == 0) {
-      Ring ar0, ar1, br, dr;  // A slot (one ring per repack half), streamed filter stage, accumulator buffer
-      uint32_t gpar = 0;    // parity of the running group count = which half produced the group
+      Ring ar0, ar1, ar2, br, dr;  // A slot (one ring per repack set), streamed filter stage, accumulator buffer
+      uint32_t gset = 0;    // running group count modulo the number of sets = which set produced the group
+      const uint32_t nsets = (uint32_t)P.NSETS;
       bool ok = true;
       PROF_DECL(7)
       const uint64_t desc0 = BRES ? ptx::smem_desc_k_sw32(ptx::smem_u32(b_smem)) : ptx::smem_desc_k_sw128(ptx::smem_u32(b_smem));
@@ -571,13 +612,13 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         const uint32_t accum = 1;
         uint32_t st0 = 0;             // steps of this tile before the current part
         uint32_t b_lo = desc_lo0;     // streamed: descriptor of the current stage
-        for (int32_t g = 0; g < P.NG && ok; ++g, gpar ^= 1u) {
+        for (int32_t g = 0; g < P.NG && ok; ++g, gset = (gset + 1u == nsets) ? 0u : gset + 1u) {
           if constexpr (BRES) {
-            if (gpar != me) { st0 += S; continue; }  // the other issuer's group
+            if (gset != me) { st0 += S; continue; }  // another issuer's group
           }
-          // the ring of the half that produced this group, held in registers (no indexed array)
-          Ring ar = gpar ? ar1 : ar0;
-          const int32_t slot0 = (int32_t)gpar * P.NSS;
+          // the ring of the set that produced this group, held in registers (no indexed array)
+          Ring ar = gset == 0 ? ar0 : (gset == 1 ? ar1 : ar2);
+          const int32_t slot0 = (int32_t)gset * P.NSS;
 #pragma unroll
           for (int h = 0; h < PARTS; ++h) {
             const int nst = (h == PARTS - 1) ? (S - (PARTS - 1) * SLOT_STEPS) : SLOT_STEPS;
@@ -625,7 +666,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
             PROF_ADD(5, tc)
             ar.advance(P.NSS);
           }
-          if (gpar) ar1 = ar; else ar0 = ar;
+          if (gset == 0) ar0 = ar; else if (gset == 1) ar1 = ar; else ar2 = ar;
         }
         if (!ok) break;
         if constexpr (!BRES) {
@@ -638,11 +679,8 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     __syncwarp();
   } else if (warp == 2) {
     // ================================================================ FILTER PRODUCER (streamed mode)
-    if constexpr (BRES) {
-      // resident filter by TMA: the copies this warp issued must have landed before the CTA exits
-      if (P.b_tma && lane == 0) wait_bar(P, misc, &bars->b_full[0], 0u, DEV_TIMEOUT_DRAIN, nullptr, 1024);
-      __syncwarp();
-    }
+    // (with a resident filter this warp is an MMA issuer, and the copies it issued in the prologue
+    // have landed before its first MMA)
     if constexpr (!BRES) {
       if (lane == 0) {
         int64_t bcount = 0;
@@ -665,17 +703,22 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
       }
       __syncwarp();
     }
-  } else if (warp >= 4 && warp < 12) {
+  } else if (warp >= kRepackWarp0 && warp < kRepackWarp0 + 4 * P.NSETS) {
     // ================================================================ WINDOW REPACK: strips -> TMEM (A)
-    // Eight warps: two per TMEM lane quarter; the two take alternate channel groups.
-    const int32_t half = (warp - 4) >> 2;
-    const int32_t q4 = (warp - 4) & 3;
+    // Sets of four warps (one per TMEM lane quarter); the sets take channel groups in turn.
+    const int32_t set = (warp - kRepackWarp0) >> 2;
+    const int32_t q4 = (warp - kRepackWarp0) & 3;
     const int32_t p = q4 * 32 + lane;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
     const int32_t skew_step = P.box ? 0 : (int32_t)(P.plane & 3);
-    Ring rr, ar;      // raw stage of the current group, A slot of the current part (this half's own ring)
-    const int32_t slot0 = half * P.NSS;
-    uint32_t gpar = 0;  // parity of the running group count
+    Ring rr, ar;      // raw stage of the current group, A slot of the current part (this set's own ring)
+    const uint32_t slot0 = (uint32_t)(set * P.NSS);
+    const uint32_t raw_a = ptx::smem_u32(raw), zero_a = ptx::smem_u32(zero_pad);
+    const uint32_t W4 = (uint32_t)P.W * 4u;
+    (void)W4;
+    const uint32_t raw_full0 = ptx::smem_u32(&bars->raw_full[0]), raw_empty0 = ptx::smem_u32(&bars->raw_empty[0]);
+    const uint32_t a_full0 = ptx::smem_u32(&bars->a_full[0]), a_empty0 = ptx::smem_u32(&bars->a_empty[0]);
+    int32_t gset = 0;  // running group count modulo the number of sets
     bool ok = true;
     PROF_DECL(7)
     for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
@@ -710,57 +753,56 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
       }
       PROF_ADD(2, tt)
 
-      for (int32_t g = 0; g < P.NG && ok; ++g, gpar ^= 1u) {
-        if (gpar != (uint32_t)half) {  // the other half's group
+      for (int32_t g = 0; g < P.NG && ok; ++g, gset = (gset + 1 == P.NSETS) ? 0 : gset + 1) {
+        if (gset != set) {  // another set's group
           rr.advance(P.SR);
           continue;
         }
         const int32_t sr = rr.idx;
         PROF_T0(twhole)
-        ok = wait_bar_warp(P, misc, &bars->raw_full[sr], rr.phase, DEV_TIMEOUT_RAW_FULL, PROF_SLOT(0));
+        ok = wait_bar_warp_a(P, misc, raw_full0 + (uint32_t)sr * 8u, rr.phase, DEV_TIMEOUT_RAW_FULL, PROF_SLOT(0));
         if (!ok) break;
         PROF_T0(ts)
-        const float* stage = raw + (size_t)sr * raw_stage_floats + base_off;
-        const int32_t r0 = g * CB;
-        const bool full_group = r0 + CB <= P.C;
-        const float* cptr[CB];
-        if (skew_step == 0) {  // every plane starts on a 16-byte boundary: one phase for all channels
-#pragma unroll
-          for (int rl = 0; rl < CB; ++rl) cptr[rl] = stage + rl * P.chan_pitch + skew0;
-        } else {
-#pragma unroll
-          for (int rl = 0; rl < CB; ++rl)
-            cptr[rl] = stage + rl * P.chan_pitch + ((skew0 + (r0 + rl) * skew_step) & 3);
-        }
+        // Shared-space byte address of this lane's window start in each channel of the group.
         // element kl of the group: channel kl / FF, tap (u, v) = ((kl % FF) / FW, (kl % FF) % FW),
         // stored in the strip at offset v*FH + u from the window start
         // (fused source: the raw input rows are staged instead, and tap (u, v) is at u*W + v)
-        const int32_t Wsrc = P.W;
-        // channels past C (last group of a C that CB does not divide) read as zero: their pointers
-        // are parked on a zeroed pad so that the hot loop carries no per-element select
-        if (!full_group) {
+        const int32_t r0 = g * CB;
+        const uint32_t stage_a = raw_a + (uint32_t)(sr * raw_stage_floats + base_off) * 4u;
+        uint32_t ca[CB];
+        if (skew_step == 0) {  // every plane starts on a 16-byte boundary: one phase for all channels
+#pragma unroll
+          for (int rl = 0; rl < CB; ++rl) ca[rl] = stage_a + (uint32_t)(rl * P.chan_pitch + skew0) * 4u;
+        } else {
 #pragma unroll
           for (int rl = 0; rl < CB; ++rl)
-            if (r0 + rl >= P.C) cptr[rl] = zero_pad;
+            ca[rl] = stage_a + (uint32_t)(rl * P.chan_pitch + ((skew0 + (r0 + rl) * skew_step) & 3)) * 4u;
         }
-        auto elem = [&](int kl) -> float {
-          if (kl >= KCG) return 0.f;
+        // channels past C (last group of a C that CB does not divide) read as zero: their addresses
+        // are parked on a zeroed pad so that the hot loop carries no per-element select
+        if (r0 + CB > P.C) {
+#pragma unroll
+          for (int rl = 0; rl < CB; ++rl)
+            if (r0 + rl >= P.C) ca[rl] = zero_a;
+        }
+        auto elem = [&](int kl) -> uint32_t {
+          if (kl >= KCG) return 0u;
           const int rl = kl / FF, w = kl % FF;
-          return FUSED ? cptr[rl][(w / FW) * Wsrc + (w % FW)] : cptr[rl][(w % FW) * FH + (w / FW)];
+          return lds_u32(FUSED ? ca[rl] + (uint32_t)(w / FW) * W4 + (uint32_t)((w % FW) * 4)
+                               : ca[rl] + (uint32_t)(((w % FW) * FH + (w / FW)) * 4));
         };
 #pragma unroll
         for (int h = 0; h < PARTS; ++h) {
-          constexpr int NB = SLOT_STEPS <= 8 ? 1 : 2;           // register batches per part
-          constexpr int BATCH = (SLOT_STEPS + NB - 1) / NB;
           const int j0 = h * SLOT_STEPS;                         // first step of this part in the group
           const int nst = (h == PARTS - 1) ? (S - (PARTS - 1) * SLOT_STEPS) : SLOT_STEPS;
-          const int32_t slot = slot0 + ar.idx;
+          const uint32_t slot = slot0 + (uint32_t)ar.idx;
           if (h == 0) { PROF_ADD(5, ts) }
-          ok = wait_bar_warp(P, misc, &bars->a_empty[slot], ar.phase ^ 1u, DEV_TIMEOUT_A_EMPTY, PROF_SLOT(1));
-          if (!ok) break;
-          ptx::tc_fence_after();
-          const uint32_t a_slot = tmem_a0 + lane_base + (uint32_t)(slot * SLOT_COLS);
           PROF_T0(tl)
+          // In register batches of at most 7 steps; the first batch's windows are loaded before the
+          // slot is waited for (the slot is only needed for the stores).
+          constexpr int NB = (SLOT_STEPS + 6) / 7;
+          constexpr int BATCH = (SLOT_STEPS + NB - 1) / NB;
+          uint32_t a_slot = 0;
 #pragma unroll
           for (int b = 0; b < NB; ++b) {
             uint32_t v[BATCH][8];
@@ -771,11 +813,18 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                   if constexpr (BF16)
-                    v[jj][e] = ptx::pack_bf16x2(elem((j0 + j) * 16 + 2 * e), elem((j0 + j) * 16 + 2 * e + 1));
+                    v[jj][e] = ptx::pack_bf16x2(__uint_as_float(elem((j0 + j) * 16 + 2 * e)),
+                                                __uint_as_float(elem((j0 + j) * 16 + 2 * e + 1)));
                   else
-                    v[jj][e] = __float_as_uint(elem((j0 + j) * 8 + e));
+                    v[jj][e] = elem((j0 + j) * 8 + e);
                 }
               }
+            }
+            if (b == 0) {
+              ok = wait_bar_warp_a(P, misc, a_empty0 + slot * 8u, ar.phase ^ 1u, DEV_TIMEOUT_A_EMPTY, PROF_SLOT(1));
+              if (!ok) break;
+              ptx::tc_fence_after();
+              a_slot = tmem_a0 + lane_base + slot * (uint32_t)SLOT_COLS;
             }
 #pragma unroll
             for (int jj = 0; jj < BATCH; ++jj) {
@@ -783,26 +832,29 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
               if (j < nst) ptx::tmem_st_x8(a_slot + (uint32_t)(j * 8), v[jj]);
             }
           }
+          if (!ok) break;
           PROF_ADD(3, tl)
           PROF_T0(tw)
           ptx::tmem_wait_st();
           ptx::tc_fence_before();
           __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->a_full[slot]));
+          if (lane == 0) {
+            ptx::mbar_arrive(a_full0 + slot * 8u);
+            // every lane's loads of the stage are done too (their values went into the stores)
+            if (h == PARTS - 1) ptx::mbar_arrive(raw_empty0 + (uint32_t)sr * 8u);
+          }
           PROF_ADD(4, tw)
           ar.advance(P.NSS);
         }
         if (!ok) break;
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->raw_empty[sr]));
         rr.advance(P.SR);
         PROF_ADD(6, twhole)
       }
     }
-    if (half == 0) { PROF_DUMP(2 + q4, 7) }
-  } else if (warp >= 12) {
+    if (set == 0) { PROF_DUMP(2 + q4, 7) }
+  } else if (warp >= kEpiWarp0) {
     // ================================================================ EPILOGUE: TMEM -> NCHW
-    const int32_t q4 = warp - 12;
+    const int32_t q4 = warp - kEpiWarp0;
     const int32_t p = q4 * 32 + lane;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
     Ring dr;
@@ -1026,6 +1078,7 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
       if (CB >= 2 && (P.plane % 4) == 0 && boxf <= 512 && encode_fn() != nullptr && (int64_t)g.N * g.C <= INT32_MAX &&
           !(nobox && nobox[0] == '1')) {
         P.box = 1;
+        P.l2_ahead = !(getenv("IM2WIN_NO_L2AHEAD") && getenv("IM2WIN_NO_L2AHEAD")[0] == '1');
         pitch = boxf;
       }
     }
@@ -1054,24 +1107,30 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
     while (P.SB > 3 && (int64_t)P.SB * P.NT * 128 + 4 * raw_stage > cap) --P.SB;
     b_bytes = (int64_t)P.SB * P.NT * 128;
   }
-  // An EVEN number of strip stages.  The two repack halves take alternate groups, so with an even
-  // count a stage is always read by the same half, which then sees every phase of the stage's
-  // barrier.  (A waiter that skips phases can be lapped by two and then waits on the wrong one.)
-  P.SR = (int32_t)((cap - b_bytes) / raw_stage);
-  if (P.SR > kMaxStages) P.SR = kMaxStages;
-  P.SR &= ~1;
+  // Repack sets and strip stages.  The sets take groups in turn, so with a stage count that is a
+  // multiple of the number of sets a stage is always read by the same set, which then sees every
+  // phase of the stage's barrier.  (A waiter that skips phases can poll before the previous phase
+  // has completed and would take it for its own.)  Three sets where that leaves at least six
+  // stages in flight, else two.
+  const int SLOT_STEPS = resident ? SlotGeom<S, true>::SLOT_STEPS : SlotGeom<S, false>::SLOT_STEPS;
+  const int SLOT_COLS = SLOT_STEPS * 8;
+  int32_t sr_max = (int32_t)((cap - b_bytes) / raw_stage);
+  if (sr_max > kMaxStages) sr_max = kMaxStages;
+  P.NSETS = (sr_max / 3 * 3 >= 6 || sr_max == 3) ? 3 : 2;
+  if (const char* fix = getenv("IM2WIN_NSETS")) {
+    if (fix[0] == '2' || fix[0] == '3') P.NSETS = fix[0] - '0';
+  }
+  // TMEM: accumulators first, then the rings of A slots, one ring of NSS slots per set (a barrier
+  // must be waited on by one party that sees every one of its phases, so the sets cannot share slots)
+  P.ND = (2 * P.NT + P.NSETS * SLOT_COLS <= 512) ? 2 : 1;
+  if (P.ND * P.NT + P.NSETS * SLOT_COLS > 512) P.NSETS = 2;
+  P.SR = sr_max / P.NSETS * P.NSETS;
   if (P.SR < 2) return IM2WIN_EUNSUPPORTED;
-
-  // TMEM: accumulators first, then the ring of A slots
-  constexpr int SLOT_COLS = SlotGeom<S>::SLOT_STEPS * 8;
-  P.ND = (2 * P.NT + 2 * SLOT_COLS <= 512) ? 2 : 1;
-  // Each repack half owns NSS slots (a barrier must be waited on by one party that sees every one of
-  // its phases, so the halves cannot share slots).
-  P.NSS = (512 - P.ND * P.NT) / SLOT_COLS / 2;
+  P.NSS = (512 - P.ND * P.NT) / SLOT_COLS / P.NSETS;
   if (P.NSS > 4) P.NSS = 4;
   if (P.NSS < 1) return IM2WIN_EUNSUPPORTED;
-  P.SS = SlotGeom<S>::SLOT_STEPS;
-  const int32_t cols = P.ND * P.NT + 2 * P.NSS * SLOT_COLS;
+  P.SS = SLOT_STEPS;
+  const int32_t cols = P.ND * P.NT + P.NSETS * P.NSS * SLOT_COLS;
   P.tmem_cols = 32;
   while (P.tmem_cols < cols) P.tmem_cols *= 2;
   P.idesc = ptx::make_idesc(128, P.NT, BF16 ? 1 : 2);
