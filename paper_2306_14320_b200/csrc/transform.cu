@@ -9,7 +9,10 @@
 //      memory (an Fh x W -> W x Fh transposition per strip) and writing one 128-bit store.
 // Every needed input row is read from HBM once per row block (the Fh-s halo rows between
 // neighbouring blocks come from L2), every output element is written exactly once.
+#include <cstdlib>
+
 #include "common.cuh"
+#include "ptx_sm100.cuh"
 
 namespace im2win {
 
@@ -132,6 +135,155 @@ __global__ void __launch_bounds__(kThreads) transform_smem_kernel(const Transfor
   if ((int32_t)threadIdx.x < n_out - tail0) dst[tail0 + threadIdx.x] = fetch(locate(tail0 + threadIdx.x));
 }
 
+// ------------------------------------------------------------------------------------------------
+// Tile kernel: the same jobs (whole planes, or a block of output rows of one plane), but all global
+// traffic is two TMA bulk copies.  The input range comes into shared memory with one
+// cp.async.bulk; the threads transpose it shared -> shared into a second buffer that holds the
+// job's output range in its final order; one cp.async.bulk stores that buffer.  A thread handles
+// four input columns of one strip at a time: FH vector loads (4 consecutive floats of a row) and
+// 4*FH contiguous output floats, i.e. a few instructions per 16 bytes instead of a gather per
+// element.  Both buffers keep the 16-byte phase of their global ranges, so the bulk copies move
+// aligned chunks; the at most 3 + 3 floats outside the aligned part are copied by threads.
+struct TileParams {
+  const float* in;
+  float* out;
+  int32_t* status;
+  int32_t H, W, s, Ho, L;
+  int32_t MB, nblk, PB;
+  int32_t QW;           // column quads per row: ceil(W / 4)
+  int64_t planes, HW, HoL, n_in_total;
+  uint64_t magic_QW;    // ceil(2^32 / QW)
+  uint64_t magic_MQ;    // ceil(2^32 / (rows per plane in the job * QW))
+  uint32_t off_out;     // byte offset of the output buffer in shared memory
+  uint32_t off_bar;     // byte offset of the mbarrier
+};
+
+template <int FH>
+__global__ void __launch_bounds__(kThreads) transform_tile_kernel(const TileParams P) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  float* const tin0 = reinterpret_cast<float*>(smem_raw);
+  float* const tout0 = reinterpret_cast<float*>(smem_raw + P.off_out);
+  uint64_t* const bar = reinterpret_cast<uint64_t*>(smem_raw + P.off_bar);
+
+  const int64_t job = blockIdx.x;
+  const int64_t pg = job / P.nblk;
+  const int32_t b = (int32_t)(job - pg * P.nblk);
+  const bool whole = P.nblk == 1;
+  const int64_t plane0 = pg * P.PB;
+  const int32_t npl = whole ? (int32_t)min((int64_t)P.PB, P.planes - plane0) : 1;
+  const int32_t m0 = b * P.MB;
+  const int32_t mb = whole ? P.Ho : min(P.MB, P.Ho - m0);
+  const int32_t rows_in = whole ? P.H : (mb - 1) * P.s + FH;
+  const int32_t plane_floats = rows_in * P.W;
+  const int32_t n_in = npl * plane_floats;
+  const int32_t out_plane = mb * P.L;
+  const int32_t n_out = npl * out_plane;
+
+  // ---- input range -> shared memory (one bulk copy of the enclosing aligned range)
+  const int64_t src0 = plane0 * P.HW + (int64_t)m0 * P.s * P.W;  // first float of the range
+  const int32_t skew = (int32_t)(src0 & 3);                      // P.in is 16-byte aligned
+  const float* const tin = tin0 + skew;                           // tin[e] <-> in[src0 + e]
+  const int64_t a0 = src0 - skew;
+  int32_t nfl = (skew + n_in + 3) & ~3;
+  int32_t ntail = 0;                                              // floats past the last whole chunk
+  if (a0 + nfl > P.n_in_total) {                                  // the last chunk would pass the tensor's end
+    nfl = (int32_t)((P.n_in_total - a0) & ~(int64_t)3);
+    ntail = (int32_t)(P.n_in_total - a0) - nfl;
+  }
+  const uint32_t bar_a = ptx::smem_u32(bar);
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(bar_a, 1);
+    ptx::fence_mbar_init();
+    ptx::mbar_arrive_expect_tx(bar_a, (uint32_t)nfl * 4u);
+    if (nfl > 0) ptx::bulk_g2s(ptx::smem_u32(tin0), P.in + a0, (uint32_t)nfl * 4u, bar_a);
+  }
+  if ((int32_t)threadIdx.x < ntail) tin0[nfl + threadIdx.x] = __ldg(P.in + a0 + nfl + threadIdx.x);
+  __syncthreads();  // the barrier is initialised for everyone; the tail floats are in place
+  {
+    bool landed = false;
+    for (uint32_t it = 0; it < (1u << 24) && !landed; ++it) {
+      landed = ptx::mbar_try_wait(bar_a, 0u);
+      if (!landed && it > 64) __nanosleep(64);
+    }
+    if (!__all_sync(0xffffffffu, landed)) {  // about a second without the copy: report and leave
+      if ((threadIdx.x & 31) == 0) atomicCAS(P.status, 0, (int32_t)DEV_TIMEOUT_DRAIN);
+      return;
+    }
+  }
+
+  // ---- transpose shared -> shared
+  const int64_t dst0 = plane0 * P.HoL + (int64_t)m0 * P.L;       // first float of the output range
+  const int32_t dskew = (int32_t)(dst0 & 3);                      // P.out is 16-byte aligned
+  float* const tout = tout0 + dskew;                              // tout[e] <-> out[dst0 + e]
+  const int32_t sW = P.s * P.W;
+  const int32_t units_plane = mb * P.QW;
+  const int32_t nunits = npl * units_plane;
+  const bool in_even = ((P.W | skew) & 1) == 0;                  // every row start is 8-byte aligned
+  for (int32_t q = threadIdx.x; q < nunits; q += kThreads) {
+    int32_t pl = 0, rem = q;
+    if (npl > 1) {
+      pl = (int32_t)(((uint64_t)(uint32_t)q * P.magic_MQ) >> 32);
+      rem = q - pl * units_plane;
+    }
+    const int32_t mm = (int32_t)(((uint64_t)(uint32_t)rem * P.magic_QW) >> 32);
+    const int32_t k0 = (rem - mm * P.QW) * 4;
+    const float* src = tin + pl * plane_floats + mm * sW + k0;
+    const int32_t oe = pl * out_plane + mm * P.L + k0 * FH;
+    float* dst = tout + oe;
+    if (k0 + 4 <= P.W) {
+      float r[4 * FH];  // r[c*FH + u] = I[m*s + u][k0 + c]: the 4*FH output floats in order
+      if (in_even) {
+#pragma unroll
+        for (int u = 0; u < FH; ++u) {
+          const float2 x = *reinterpret_cast<const float2*>(src + u * P.W);
+          const float2 y = *reinterpret_cast<const float2*>(src + u * P.W + 2);
+          r[0 * FH + u] = x.x; r[1 * FH + u] = x.y; r[2 * FH + u] = y.x; r[3 * FH + u] = y.y;
+        }
+      } else {
+#pragma unroll
+        for (int u = 0; u < FH; ++u) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) r[c * FH + u] = src[u * P.W + c];
+        }
+      }
+      const int32_t a = (dskew + oe) & 3;  // 16-byte phase of the run in the output buffer
+      if (a == 0) {
+#pragma unroll
+        for (int j = 0; j < FH; ++j)
+          reinterpret_cast<float4*>(dst)[j] = make_float4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+      } else if (a == 2) {
+        *reinterpret_cast<float2*>(dst) = make_float2(r[0], r[1]);
+#pragma unroll
+        for (int j = 0; j < FH - 1; ++j)
+          *reinterpret_cast<float4*>(dst + 2 + 4 * j) = make_float4(r[4 * j + 2], r[4 * j + 3], r[4 * j + 4], r[4 * j + 5]);
+        *reinterpret_cast<float2*>(dst + 4 * FH - 2) = make_float2(r[4 * FH - 2], r[4 * FH - 1]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4 * FH; ++j) dst[j] = r[j];
+      }
+    } else {  // the last, partial quad of a row
+      for (int32_t c = 0; k0 + c < P.W; ++c)
+#pragma unroll
+        for (int u = 0; u < FH; ++u) dst[c * FH + u] = src[u * P.W + c];
+    }
+  }
+  ptx::fence_proxy_async_smem();  // the buffer is about to be read by the bulk copy
+  __syncthreads();
+
+  // ---- output buffer -> global: one bulk copy of the aligned part, threads for the ragged ends
+  const int32_t head = min((4 - dskew) & 3, n_out);
+  const int32_t nvec = (n_out - head) >> 2;
+  const int32_t tail0 = head + (nvec << 2);
+  float* const gout = P.out + dst0;
+  if (threadIdx.x == 0 && nvec > 0) {
+    ptx::bulk_s2g(gout + head, ptx::smem_u32(tout + head), (uint32_t)nvec * 16u);
+    ptx::bulk_s2g_commit();
+  }
+  if ((int32_t)threadIdx.x < head) gout[threadIdx.x] = tout[threadIdx.x];
+  if ((int32_t)threadIdx.x < n_out - tail0) gout[tail0 + threadIdx.x] = tout[tail0 + threadIdx.x];
+  if (threadIdx.x == 0 && nvec > 0) ptx::bulk_s2g_wait_read();  // shared memory must outlive the copy's reads
+}
+
 // Fallback for rows too long to stage (Fh*W floats beyond the shared-memory budget): one thread
 // per output element, reads through L1/L2.  Correct for every shape, not tuned.
 __global__ void __launch_bounds__(kThreads) transform_gather_kernel(const float* __restrict__ in,
@@ -154,7 +306,82 @@ uint64_t magic_for(uint32_t d) { return ((uint64_t)1 << 32) / d + ((((uint64_t)1
 
 }  // namespace
 
+template <int FH>
+int launch_tile_fh(const TileParams& P, int64_t ctas, size_t smem, cudaStream_t st) {
+  auto kern = transform_tile_kernel<FH>;
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    cudaGetLastError();
+    return IM2WIN_ECUDA;
+  }
+  kern<<<(unsigned)ctas, kThreads, smem, st>>>(P);
+  return cuda_status(cudaGetLastError());
+}
+
+// Tile kernel where a job's input and output ranges fit one shared-memory budget together (a sixth
+// of an SM's shared memory, so that six CTAs overlap their loads, transposes and stores);
+// IM2WIN_EUNSUPPORTED otherwise (the caller then uses the staged-gather kernel).
+int launch_transform_tile(const float* in, float* out, const Geometry& g, cudaStream_t st) {
+  if (g.Fh != 1 && g.Fh != 2 && g.Fh != 3 && g.Fh != 4 && g.Fh != 5 && g.Fh != 7 && g.Fh != 11) return IM2WIN_EUNSUPPORTED;
+  constexpr int64_t kBudget = 8704 - 16;  // floats for input + output ranges: 34 KB with the phase skews, six CTAs per SM
+  const int64_t planes = (int64_t)g.N * g.C;
+  const int64_t hw = (int64_t)g.H * g.W;
+  int32_t PB = 1, MB = g.Ho, nblk = 1;
+  if (hw + g.HoL <= kBudget) {
+    PB = (int32_t)(kBudget / (hw + g.HoL));
+    const int64_t want_ctas = 148 * 8;  // keep enough CTAs to fill the machine
+    if (planes / PB < want_ctas) PB = (int32_t)(planes / want_ctas > 0 ? planes / want_ctas : 1);
+    if (PB < 1) PB = 1;
+  } else {
+    const int64_t mbmax = (kBudget - (int64_t)(g.Fh - g.s) * g.W) / ((int64_t)g.s * g.W + g.L);
+    if (mbmax < 1) return IM2WIN_EUNSUPPORTED;
+    MB = (int32_t)(mbmax < g.Ho ? mbmax : g.Ho);
+    nblk = (g.Ho + MB - 1) / MB;
+    MB = (g.Ho + nblk - 1) / nblk;  // balance the blocks
+    // neighbouring blocks re-read Fh - s rows each; with the output buffer taking most of the
+    // budget, wide rows leave blocks so short that this would dominate: leave those to the
+    // staged-gather kernel, which stages the input only
+    if ((int64_t)(g.Fh - g.s) * 8 > (int64_t)(MB - 1) * g.s + g.Fh) return IM2WIN_EUNSUPPORTED;
+  }
+  const int64_t ctas = nblk == 1 ? (planes + PB - 1) / PB : planes * nblk;
+  if (ctas > INT32_MAX) return IM2WIN_EUNSUPPORTED;
+  const int32_t rows_in = nblk == 1 ? g.H : (MB - 1) * g.s + g.Fh;
+  const int64_t in_floats = (int64_t)PB * rows_in * g.W + 8;                       // + phase skew and rounding
+  const int64_t out_floats = (int64_t)PB * (nblk == 1 ? g.HoL : (int64_t)MB * g.L) + 8;
+  TileParams P;
+  P.in = in; P.out = out;
+  P.status = device_status_word();
+  if (!P.status) return IM2WIN_ECUDA;
+  P.H = g.H; P.W = g.W; P.s = g.s; P.Ho = g.Ho; P.L = g.L;
+  P.MB = MB; P.nblk = nblk; P.PB = PB;
+  P.QW = (g.W + 3) / 4;
+  P.planes = planes; P.HW = hw; P.HoL = g.HoL; P.n_in_total = g.n_in;
+  const int64_t units_plane = (int64_t)(nblk == 1 ? g.Ho : MB) * P.QW;
+  if (units_plane * PB * units_plane >= ((int64_t)1 << 32)) return IM2WIN_EUNSUPPORTED;  // reciprocal division exact
+  P.magic_QW = magic_for((uint32_t)P.QW);
+  P.magic_MQ = magic_for((uint32_t)units_plane);
+  P.off_out = (uint32_t)((in_floats * 4 + 127) / 128 * 128);
+  P.off_bar = P.off_out + (uint32_t)((out_floats * 4 + 15) / 16 * 16);
+  const size_t smem = P.off_bar + 16;
+  switch (g.Fh) {
+    case 1: return launch_tile_fh<1>(P, ctas, smem, st);
+    case 2: return launch_tile_fh<2>(P, ctas, smem, st);
+    case 3: return launch_tile_fh<3>(P, ctas, smem, st);
+    case 4: return launch_tile_fh<4>(P, ctas, smem, st);
+    case 5: return launch_tile_fh<5>(P, ctas, smem, st);
+    case 7: return launch_tile_fh<7>(P, ctas, smem, st);
+    default: return launch_tile_fh<11>(P, ctas, smem, st);
+  }
+}
+
 int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_t st) {
+  {
+    const char* old = getenv("IM2WIN_TRANSFORM_GATHER");
+    if (!(old && old[0] == '1')) {
+      const int rc = launch_transform_tile(in, out, g, st);
+      if (rc != IM2WIN_EUNSUPPORTED) return rc;
+    }
+  }
   // Shared-memory budget for the staged input rows.  Small enough for several CTAs per SM so that
   // one CTA's loads overlap another's stores.
   constexpr int32_t kTileFloats = 8192 - 4;      // 32 KB including the phase skew

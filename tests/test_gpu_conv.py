@@ -35,13 +35,15 @@ def _built():
     ensure_built()
 
 
-@pytest.fixture(params=["auto", "nobox", "generic"], autouse=True)
+@pytest.fixture(params=["auto", "nobox", "nopim", "generic"], autouse=True)
 def _kernel(request, monkeypatch):
-    """Every case runs three times: with the library's own choice of tensor-core kernel (the persistent,
-    filter-size-specialised one where it applies, strips staged by 2-D TMA boxes where they qualify),
-    with the box staging switched off (bulk copies), and with the generic kernel forced."""
+    """Every case runs four times: with the library's own choice of tensor-core kernel (the persistent,
+    filter-size-specialised one where it applies, tiles cut per image and strips staged by 2-D TMA
+    boxes where they qualify), with the box staging switched off (per-image tiles, bulk copies), with
+    per-image tiling switched off as well (tiles that span images), and with the generic kernel forced."""
     monkeypatch.setenv("IM2WIN_FORCE_GENERIC", "1" if request.param == "generic" else "0")
     monkeypatch.setenv("IM2WIN_NO_BOX", "1" if request.param == "nobox" else "0")
+    monkeypatch.setenv("IM2WIN_NO_PIM", "1" if request.param == "nopim" else "0")
 
 
 def _data(dims, seed, ints=False):

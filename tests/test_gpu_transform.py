@@ -25,6 +25,13 @@ def _built():
     ensure_built()
 
 
+@pytest.fixture(params=["auto", "gather"], autouse=True)
+def _kernel(request, monkeypatch):
+    """Every case runs twice: with the library's own choice of kernel (the TMA tile kernel where a job's
+    input and output ranges fit its shared-memory budget), and with the staged-gather kernel forced."""
+    monkeypatch.setenv("IM2WIN_TRANSFORM_GATHER", "1" if request.param == "gather" else "0")
+
+
 def _bits(a):
     return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).ravel()
 
