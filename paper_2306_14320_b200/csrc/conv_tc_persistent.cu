@@ -126,14 +126,10 @@ __device__ __forceinline__ uint64_t global_ns() {
 // Bounded wait (about a second).  A warp that is not ready backs off with nanosleep between polls:
 // sixteen warps share four schedulers, and a warp that spins on try_wait takes issue slots from the
 // MMA-issuing thread on its scheduler, whose instruction rate is what bounds small-N tiles.
-__device__ __forceinline__ bool wait_bar_a(const PParams& P, PMisc* misc, uint32_t b, uint32_t parity,
-                                           int32_t code, long long* acc = nullptr, uint32_t sleep_ns = 64) {
-#ifdef IM2WIN_PROF
-  // try_wait may block inside the instruction, so the clock brackets the first poll too
-  const long long c0 = clock64();
-  struct Fin { long long* a; long long c; __device__ ~Fin() { if (a) *a += clock64() - c; } } fin{acc, c0};
-#endif
-  if (ptx::mbar_try_wait(b, parity)) return true;
+// The polling loop lives in one out-of-line copy: the call sites keep only the first poll, which
+// keeps the roles' hot loops short (instruction fetch is a visible cost in this kernel).
+__device__ __noinline__ bool wait_bar_slow(int32_t* status, PMisc* misc, uint32_t b, uint32_t parity, int32_t code,
+                                           uint32_t sleep_ns) {
   uint64_t t0 = 0;
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     __nanosleep(sleep_ns);
@@ -145,8 +141,20 @@ __device__ __forceinline__ bool wait_bar_a(const PParams& P, PMisc* misc, uint32
       else if (now - t0 > 1000000000ull) break;
     }
   }
-  record(P, misc, code);
+  atomicCAS(status, 0, code);
+  atomicExch(&misc->abort, 1);
   return false;
+}
+
+__device__ __forceinline__ bool wait_bar_a(const PParams& P, PMisc* misc, uint32_t b, uint32_t parity,
+                                           int32_t code, long long* acc = nullptr, uint32_t sleep_ns = 64) {
+#ifdef IM2WIN_PROF
+  // try_wait may block inside the instruction, so the clock brackets the first poll too
+  const long long c0 = clock64();
+  struct Fin { long long* a; long long c; __device__ ~Fin() { if (a) *a += clock64() - c; } } fin{acc, c0};
+#endif
+  if (ptx::mbar_try_wait(b, parity)) return true;
+  return wait_bar_slow(P.status, misc, b, parity, code, sleep_ns);
 }
 
 __device__ __forceinline__ bool wait_bar(const PParams& P, PMisc* misc, uint64_t* bar, uint32_t parity,
@@ -1122,6 +1130,10 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
   }
   // TMEM: accumulators first, then the rings of A slots, one ring of NSS slots per set (a barrier
   // must be waited on by one party that sees every one of its phases, so the sets cannot share slots)
+  P.ND = (2 * P.NT + P.NSETS * SLOT_COLS <= 512) ? 2 : 1;
+  // a third set only pays where every set still owns at least two slots (a set with one slot waits
+  // for the MMAs of each part before it can store the next)
+  if ((512 - P.ND * P.NT) / SLOT_COLS / P.NSETS < 2 && !getenv("IM2WIN_NSETS")) P.NSETS = 2;
   P.ND = (2 * P.NT + P.NSETS * SLOT_COLS <= 512) ? 2 : 1;
   if (P.ND * P.NT + P.NSETS * SLOT_COLS > 512) P.NSETS = 2;
   P.SR = sr_max / P.NSETS * P.NSETS;
