@@ -21,6 +21,7 @@
 #include <cuda_bf16.h>
 
 #include <cstdlib>
+#include <type_traits>
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
@@ -52,6 +53,8 @@ struct PParams {
   int32_t HoWo;         // output positions per image (fits 32 bits; checked on the host)
   int64_t Kg, Mtot, n_src;
   int32_t TP, NT, n_ntiles;
+  int32_t Z, GZ;        // reduction slices per (m-tile, n-tile) and channel groups per slice (Z > 1: results are added into a zeroed output)
+  int32_t usub;         // work units per m-tile: n_ntiles * Z
   int64_t ntiles;       // m tiles * n tiles
   int32_t NG;           // channel groups per tile
   int32_t SR, SB;       // raw strip stages; filter stages (streamed mode)
@@ -205,9 +208,18 @@ __device__ __forceinline__ int32_t fast_div(int32_t n, uint64_t magic) {
   return (int32_t)(((uint64_t)(uint32_t)n * magic) >> 32);
 }
 
-// m-tile of work unit t (units are numbered m-tile major, n-tile minor; usually there is one n-tile)
+// Work unit t = (m-tile, n-tile, reduction slice), the slice fastest (usually one n-tile, one slice).
 __device__ __forceinline__ int32_t tile_of(const PParams& P, int32_t t) {
-  return P.n_ntiles == 1 ? t : t / P.n_ntiles;
+  return P.usub == 1 ? t : t / P.usub;
+}
+// n-tile and first / one-past-last channel group of unit t
+__device__ __forceinline__ void unit_range(const PParams& P, int32_t t, int32_t& nt, int32_t& g0, int32_t& g1) {
+  if (__builtin_expect(P.usub == 1, 1)) { nt = 0; g0 = 0; g1 = P.NG; return; }
+  const int32_t sub = t - (t / P.usub) * P.usub;
+  nt = P.Z == 1 ? sub : sub / P.Z;
+  const int32_t z = sub - nt * P.Z;
+  g0 = z * P.GZ;
+  g1 = min(g0 + P.GZ, P.NG);
 }
 
 // Where an m-tile lies: image of its first position, that position's index inside the image, how
@@ -218,29 +230,37 @@ struct TileInfo {
   int32_t q_first, npos, nseg;
 };
 
-__device__ __forceinline__ TileInfo tile_info(const PParams& P, int32_t tile_m) {
+// Tiles that may span images (small images).  Out of line: the per-image case below is the hot one.
+__device__ __noinline__ TileInfo tile_info_general(int32_t TP, int32_t HoWo, int64_t Mtot, int32_t tile_m) {
   TileInfo ti;
-  if (P.pim) {  // tiles are cut per image
+  if (Mtot <= 0x7fffffff) {  // the usual case: 32-bit arithmetic throughout
+    const uint32_t P0 = (uint32_t)tile_m * (uint32_t)TP;
+    const uint32_t i = P0 / (uint32_t)HoWo;
+    ti.i_first = i;
+    ti.q_first = (int32_t)(P0 - i * (uint32_t)HoWo);
+    ti.npos = min(TP, (int32_t)((uint32_t)Mtot - P0));
+    ti.nseg = (ti.q_first + ti.npos - 1) / HoWo + 1;
+  } else {
+    const int64_t P0 = (int64_t)tile_m * TP;
+    ti.i_first = P0 / HoWo;
+    ti.q_first = (int32_t)(P0 - ti.i_first * HoWo);
+    ti.npos = (int32_t)min((int64_t)TP, Mtot - P0);
+    ti.nseg = (ti.q_first + ti.npos - 1) / HoWo + 1;
+  }
+  return ti;
+}
+
+__device__ __forceinline__ TileInfo tile_info(const PParams& P, int32_t tile_m) {
+  if (__builtin_expect(P.pim, 1)) {  // tiles are cut per image
+    TileInfo ti;
     const int32_t i = fast_div(tile_m, P.magic_TPI);
     ti.i_first = i;
     ti.q_first = (tile_m - i * P.TPI) * P.TP;
     ti.npos = min(P.TP, P.HoWo - ti.q_first);
     ti.nseg = 1;
-  } else if (P.Mtot <= 0x7fffffff) {  // the usual case: 32-bit arithmetic throughout
-    const uint32_t P0 = (uint32_t)tile_m * (uint32_t)P.TP;
-    const uint32_t i = P0 / (uint32_t)P.HoWo;
-    ti.i_first = i;
-    ti.q_first = (int32_t)(P0 - i * (uint32_t)P.HoWo);
-    ti.npos = min(P.TP, (int32_t)((uint32_t)P.Mtot - P0));
-    ti.nseg = (ti.q_first + ti.npos - 1) / P.HoWo + 1;
-  } else {
-    const int64_t P0 = (int64_t)tile_m * P.TP;
-    ti.i_first = P0 / P.HoWo;
-    ti.q_first = (int32_t)(P0 - ti.i_first * P.HoWo);
-    ti.npos = (int32_t)min((int64_t)P.TP, P.Mtot - P0);
-    ti.nseg = (ti.q_first + ti.npos - 1) / P.HoWo + 1;
+    return ti;
   }
-  return ti;
+  return tile_info_general(P.TP, P.HoWo, P.Mtot, tile_m);
 }
 
 // Row p of the tile: image (as an offset from the tile's first image) and position inside it.
@@ -273,6 +293,25 @@ __device__ __forceinline__ SegR compute_seg(const PParams& P, const TileInfo& ti
   }
   s.dst_off = incl - slot;
   return s;
+}
+
+// Repack warps, tiles that may span images: where lane's window starts in a staged channel row, and
+// the 16-byte phase of the staged range.  (Kept inline: an out-of-line copy would take the kernel
+// parameters by address, which turns every later read of them into a memory load.)
+__device__ __forceinline__ void repack_prologue_general(const PParams& P, const TileInfo& ti, int32_t p, int lane,
+                                                     bool valid, int32_t& base_off, int32_t& skew0) {
+  const SegR seg = compute_seg(P, ti, lane);
+  int32_t sg = 0, q = 0;
+  if (valid) tile_row(P, ti, p, sg, q);
+  const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
+  const int64_t s_virt = __shfl_sync(0xffffffffu, seg.virt_a, sg);
+  const int32_t s_dst = __shfl_sync(0xffffffffu, seg.dst_off, sg);
+  base_off = 0;
+  if (valid) {
+    const int32_t m = q / P.Wo, n = q - m * P.Wo;
+    base_off = s_dst + (int32_t)(((int64_t)m * P.row_mul + (int64_t)n * P.col_mul) - s_virt);
+  }
+  skew0 = (int32_t)(s_start0 & 3);  // 16-byte phase of the staged range, per absolute address
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1,
@@ -464,7 +503,10 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           pf_x = ((m2 * P.row_mul + n2 * P.col_mul) & ~3) >> 1;
           pf_y0 = i2 * P.C;
         }
-        for (int32_t g = 0; g < P.NG && ok; ++g, ++gcount, rr.advance(P.SR)) {
+        int32_t nt_, g0, g1;
+        unit_range(P, t, nt_, g0, g1);
+        (void)nt_;
+        for (int32_t g = g0; g < g1 && ok; ++g, ++gcount, rr.advance(P.SR)) {
           const int32_t sr = rr.idx;
           if (pf && lane == 0) tma_prefetch_2d(&xmap, pf_x, pf_y0 + g * CB);
           ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0), 128);
@@ -490,8 +532,11 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         const int32_t m_b = fast_div(q_last, P.magic_Wo), n_b = q_last - m_b * P.Wo;
         const int32_t virt_a = m_a * P.row_mul + n_a * P.col_mul;
         const int32_t len = m_b * P.row_mul + n_b * P.col_mul - virt_a + P.win_span;
-        int64_t start = ((int64_t)i * P.C + lane) * P.plane + virt_a;
-        for (int32_t g = 0; g < P.NG && ok; ++g, ++gcount, rr.advance(P.SR)) {
+        int32_t nt_, g0, g1;
+        unit_range(P, t, nt_, g0, g1);
+        (void)nt_;
+        int64_t start = ((int64_t)i * P.C + (int64_t)g0 * CB + lane) * P.plane + virt_a;
+        for (int32_t g = g0; g < g1 && ok; ++g, ++gcount, rr.advance(P.SR)) {
           const int32_t sr = rr.idx;
           ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0), 128);
           if (!ok) break;
@@ -542,7 +587,12 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           start[z] = s_start0 + (int64_t)rl[z] * P.plane;
         }
         const int64_t group_step = (int64_t)CB * P.plane;
-        for (int32_t g = 0; g < P.NG && ok; ++g, ++gcount, rr.advance(P.SR)) {
+        int32_t nt_, g0, g1;
+        unit_range(P, t, nt_, g0, g1);
+        (void)nt_;
+        start[0] += g0 * group_step;
+        start[1] += g0 * group_step;
+        for (int32_t g = g0; g < g1 && ok; ++g, ++gcount, rr.advance(P.SR)) {
           const int32_t sr = rr.idx;
           ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0), 128);
           if (!ok) break;
@@ -618,9 +668,12 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(d * P.NT);
         const uint32_t accum = 1;
-        uint32_t st0 = 0;             // steps of this tile before the current part
-        uint32_t b_lo = desc_lo0;     // streamed: descriptor of the current stage
-        for (int32_t g = 0; g < P.NG && ok; ++g, gset = (gset + 1u == nsets) ? 0u : gset + 1u) {
+        int32_t nt_, g0, g1;
+        unit_range(P, t, nt_, g0, g1);
+        (void)nt_;
+        uint32_t st0 = (uint32_t)(g0 * S);  // steps of this tile before the current part
+        uint32_t b_lo = desc_lo0;           // streamed: descriptor of the current stage
+        for (int32_t g = g0; g < g1 && ok; ++g, gset = (gset + 1u == nsets) ? 0u : gset + 1u) {
           if constexpr (BRES) {
             if (gset != me) { st0 += S; continue; }  // another issuer's group
           }
@@ -695,8 +748,12 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         Ring br;
         bool ok = true;
         for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
-          const int32_t n0 = (t % P.n_ntiles) * P.NT;
-          for (int32_t c = 0; c < P.nchunks && ok; ++c, ++bcount, br.advance(P.SB)) {
+          int32_t nt, g0, g1;
+          unit_range(P, t, nt, g0, g1);
+          const int32_t n0 = nt * P.NT;
+          // the slice's 128-byte filter chunks (a slice starts on a chunk boundary: host check)
+          const int32_t c0 = (g0 * S) >> 2, c1 = (g1 * S + 3) >> 2;
+          for (int32_t c = c0; c < c1 && ok; ++c, ++bcount, br.advance(P.SB)) {
             const int32_t sb = br.idx;
             ok = wait_bar(P, misc, &bars->b_empty[sb], br.phase ^ 1u, DEV_TIMEOUT_B_EMPTY);
             if (!ok) break;
@@ -747,21 +804,14 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         }
         if (!P.box) skew0 = (int32_t)((ti.i_first * P.C * P.plane + virt_a) & 3);
       } else {
-        const SegR seg = compute_seg(P, ti, lane);
-        int32_t sg = 0, q = 0;
-        if (valid) tile_row(P, ti, p, sg, q);
-        const int64_t s_start0 = __shfl_sync(0xffffffffu, seg.start0, sg);
-        const int64_t s_virt = __shfl_sync(0xffffffffu, seg.virt_a, sg);
-        const int32_t s_dst = __shfl_sync(0xffffffffu, seg.dst_off, sg);
-        if (valid) {
-          const int32_t m = q / P.Wo, n = q - m * P.Wo;
-          base_off = s_dst + (int32_t)(((int64_t)m * P.row_mul + (int64_t)n * P.col_mul) - s_virt);
-        }
-        skew0 = (int32_t)(s_start0 & 3);  // 16-byte phase of the staged range, per absolute address
+        repack_prologue_general(P, ti, p, lane, valid, base_off, skew0);
       }
       PROF_ADD(2, tt)
 
-      for (int32_t g = 0; g < P.NG && ok; ++g, gset = (gset + 1 == P.NSETS) ? 0 : gset + 1) {
+      int32_t nt_, g0, g1;
+      unit_range(P, t, nt_, g0, g1);
+      (void)nt_;
+      for (int32_t g = g0; g < g1 && ok; ++g, gset = (gset + 1 == P.NSETS) ? 0 : gset + 1) {
         if (gset != set) {  // another set's group
           rr.advance(P.SR);
           continue;
@@ -865,64 +915,79 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     const int32_t q4 = warp - kEpiWarp0;
     const int32_t p = q4 * 32 + lane;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
-    Ring dr;
-    bool ok = true;
+    // The role exists in two copies, chosen once: plain stores, or (reduction slices, Z > 1) additions
+    // into the zeroed output.  A choice inside the store loop, or an out-of-line call next to it,
+    // slowed the C = 3 stem layers, which this loop bounds, by 20 %.
     PROF_DECL(6)
-    const int32_t eK = P.K, eNT = P.NT, eHoWo = P.HoWo;  // kept in registers for the store loop
-    // hand both accumulator buffers to the MMA side zeroed: every MMA accumulates
-    for (int32_t d = 0; d < P.ND; ++d) {
-      for (int32_t c0 = 0; c0 < P.NT; c0 += 16) ptx::tmem_zero_x16(tmem_base + lane_base + (uint32_t)(d * P.NT + c0));
-      ptx::tmem_wait_st();
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->acc_empty[d]));
-    }
-    for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
-      PROF_T0(tp)
-      const int32_t tile_m = tile_of(P, t);
-      const int32_t n0 = (t - tile_m * P.n_ntiles) * P.NT;
-      const TileInfo ti = tile_info(P, tile_m);
-      const bool valid = p < ti.npos;
-      float* orow = P.out;
-      if (valid) {
-        int32_t i_off, q;
-        tile_row(P, ti, p, i_off, q);
-        orow += ((ti.i_first + i_off) * P.K + n0) * (int64_t)P.HoWo + q;
+    auto epilogue_role = [&](auto reduce_tag) {
+      constexpr bool REDUCE = decltype(reduce_tag)::value;
+      Ring dr;
+      bool ok = true;
+      const int32_t eK = P.K, eNT = P.NT, eHoWo = P.HoWo;  // kept in registers for the store loop
+      // hand both accumulator buffers to the MMA side zeroed: every MMA accumulates
+      for (int32_t d = 0; d < P.ND; ++d) {
+        for (int32_t c0 = 0; c0 < P.NT; c0 += 16) ptx::tmem_zero_x16(tmem_base + lane_base + (uint32_t)(d * P.NT + c0));
+        ptx::tmem_wait_st();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->acc_empty[d]));
       }
-      const int32_t d = dr.idx;
-      PROF_ADD(1, tp)
-      ok = wait_bar_warp(P, misc, &bars->acc_full[d], dr.phase, DEV_TIMEOUT_ACC, PROF_SLOT(0), 256);
-      if (!ok) break;
-      ptx::tc_fence_after();
-      const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)(d * P.NT);
-      // 16 columns per trip.  Deliberately a rolled loop with a small body: this code runs once per
-      // tile, and a fully unrolled store sequence (hundreds of instructions executed once) spent its
-      // time on instruction fetch, the other roles' code having evicted it in between.
-#pragma unroll 1
-      for (int32_t c0 = 0; c0 < eNT; c0 += 16) {
-        uint32_t v[16];
-        PROF_T0(t1)
-        ptx::tmem_ld_x16(d_tmem + (uint32_t)c0, v);
-        ptx::tmem_wait_ld();
-        PROF_ADD(2, t1)
-        ptx::tmem_zero_x16(d_tmem + (uint32_t)c0);  // leave the columns zeroed for the next tile
-        PROF_T0(t3)
+      for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
+        PROF_T0(tp)
+        const int32_t tile_m = tile_of(P, t);
+        int32_t nt, g0_, g1_;
+        unit_range(P, t, nt, g0_, g1_);
+        (void)g0_; (void)g1_;
+        const int32_t n0 = nt * P.NT;
+        const TileInfo ti = tile_info(P, tile_m);
+        const bool valid = p < ti.npos;
+        float* orow = P.out;
         if (valid) {
-          float* o = orow + (int64_t)c0 * eHoWo;
-          const int32_t left = eK - n0 - c0;  // filters of this block that exist
-#pragma unroll
-          for (int e = 0; e < 16; ++e)
-            if (e < left) o[(int64_t)e * eHoWo] = __uint_as_float(v[e]);
+          int32_t i_off, q;
+          tile_row(P, ti, p, i_off, q);
+          orow += ((ti.i_first + i_off) * P.K + n0) * (int64_t)P.HoWo + q;
         }
-        PROF_ADD(4, t3)
+        const int32_t d = dr.idx;
+        PROF_ADD(1, tp)
+        ok = wait_bar_warp(P, misc, &bars->acc_full[d], dr.phase, DEV_TIMEOUT_ACC, PROF_SLOT(0), 256);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)(d * P.NT);
+        // 16 columns per trip.  Deliberately a rolled loop with a small body: this code runs once per
+        // tile, and a fully unrolled store sequence (hundreds of instructions executed once) spent its
+        // time on instruction fetch, the other roles' code having evicted it in between.
+  #pragma unroll 1
+        for (int32_t c0 = 0; c0 < eNT; c0 += 16) {
+          uint32_t v[16];
+          PROF_T0(t1)
+          ptx::tmem_ld_x16(d_tmem + (uint32_t)c0, v);
+          ptx::tmem_wait_ld();
+          PROF_ADD(2, t1)
+          ptx::tmem_zero_x16(d_tmem + (uint32_t)c0);  // leave the columns zeroed for the next tile
+          PROF_T0(t3)
+          if (valid) {
+            float* o = orow + (int64_t)c0 * eHoWo;
+            const int32_t left = eK - n0 - c0;  // filters of this block that exist
+  #pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              if (e < left) {
+                if constexpr (REDUCE) atomicAdd(o + (int64_t)e * eHoWo, __uint_as_float(v[e]));  // fp32 reduction in L2
+                else o[(int64_t)e * eHoWo] = __uint_as_float(v[e]);
+              }
+            }
+          }
+          PROF_ADD(4, t3)
+        }
+        PROF_T0(t4)
+        ptx::tmem_wait_st();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->acc_empty[d]));
+        PROF_ADD(5, t4)
       }
-      PROF_T0(t4)
-      ptx::tmem_wait_st();
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->acc_empty[d]));
-      PROF_ADD(5, t4)
-    }
+    };
+    if (P.Z == 1) epilogue_role(std::false_type{});
+    else epilogue_role(std::true_type{});
     if (q4 == 0) { PROF_DUMP(6, 6) }
   }
 
@@ -1142,6 +1207,43 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
   if (P.NSS > 4) P.NSS = 4;
   if (P.NSS < 1) return IM2WIN_EUNSUPPORTED;
   P.SS = SLOT_STEPS;
+
+  // Reduction slices.  When the (m-tile, n-tile) units do not fill the SMs evenly -- few tiles at
+  // small batch, or a last wave that is mostly idle -- a unit's channel groups are cut into Z slices
+  // that run as separate units and add their partial sums into the zeroed output.  Z is picked with
+  // a small cost model: waves x (groups per slice x cycles per group + per-unit overhead), where a
+  // group costs its MMA time (or the repack floor) and the overhead is the pipeline fill plus, with a
+  // single accumulator buffer, the epilogue that nothing overlaps; a split also pays for zeroing the
+  // output.  A slice of a streamed filter must start on a 128-byte filter chunk (4 MMA steps).
+  P.Z = 1; P.GZ = P.NG;
+  {
+    const int64_t units1 = P.ntiles;
+    const int nsm = sm_count();
+    const double group_cyc = (double)S * P.NT * 0.7 > 600.0 ? (double)S * P.NT * 0.7 : 600.0;
+    const double ov_cyc = (P.ND == 1 ? P.NT * 31.0 : 0.0) + 3000.0;
+    const double zero_cyc = 5000.0 + (double)g.n_out * 4.0 / 1600.0;  // the extra launch that zeroes the output
+    auto cost = [&](int64_t z_eff, int32_t gz) {
+      const int64_t waves = (units1 * z_eff + nsm - 1) / nsm;
+      const double c = (double)waves * (gz * group_cyc + ov_cyc);
+      return z_eff > 1 ? c * 1.05 + zero_cyc : c;
+    };
+    int32_t gmul = 1;
+    if (!resident) while ((gmul * S) % 4 != 0) ++gmul;
+    double best = cost(1, P.NG) * 0.92;  // a split must win clearly
+    int forced = -1;
+    if (const char* fix = getenv("IM2WIN_SPLITK")) forced = atoi(fix);
+    for (int32_t z = 2; z <= 16 && z <= P.NG; ++z) {
+      int32_t gz = (P.NG + z - 1) / z;
+      gz = (gz + gmul - 1) / gmul * gmul;
+      const int32_t z_eff = (P.NG + gz - 1) / gz;
+      if (z_eff < 2) continue;
+      const double c = cost(z_eff, gz);
+      if (forced >= 0 ? z == forced : c < best) { best = c; P.Z = z_eff; P.GZ = gz; }
+    }
+    if (forced == 0 || forced == 1) { P.Z = 1; P.GZ = P.NG; }
+  }
+  P.usub = P.n_ntiles * P.Z;
+  P.ntiles *= P.Z;
   const int32_t cols = P.ND * P.NT + P.NSETS * P.NSS * SLOT_COLS;
   P.tmem_cols = 32;
   while (P.tmem_cols < cols) P.tmem_cols *= 2;
@@ -1210,6 +1312,11 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
   }
   const int64_t grid = P.ntiles < sm_count() ? P.ntiles : sm_count();
   cudaError_t e;
+  if (P.Z > 1 && cudaMemsetAsync(out, 0, (size_t)g.n_out * 4, st) != cudaSuccess) {
+    cudaGetLastError();
+    if (f_bf16) cudaFreeAsync(f_bf16, st);
+    return IM2WIN_ECUDA;
+  }
   if (resident) {
     auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, true, FUSED>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
