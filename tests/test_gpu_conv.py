@@ -35,15 +35,21 @@ def _built():
     ensure_built()
 
 
-@pytest.fixture(params=["auto", "nobox", "nopim", "generic"], autouse=True)
+@pytest.fixture(params=["auto", "nobox", "nopim", "split3", "generic"], autouse=True)
 def _kernel(request, monkeypatch):
-    """Every case runs four times: with the library's own choice of tensor-core kernel (the persistent,
+    """Every case runs five times: with the library's own choice of tensor-core kernel (the persistent,
     filter-size-specialised one where it applies, tiles cut per image and strips staged by 2-D TMA
-    boxes where they qualify), with the box staging switched off (per-image tiles, bulk copies), with
-    per-image tiling switched off as well (tiles that span images), and with the generic kernel forced."""
+    boxes where they qualify, reduction slices where its cost model wants them), with the box staging
+    switched off (per-image tiles, bulk copies), with per-image tiling switched off as well (tiles
+    that span images), with three reduction slices forced wherever a layer has that many channel
+    groups (partial sums added into the zeroed output), and with the generic kernel forced."""
     monkeypatch.setenv("IM2WIN_FORCE_GENERIC", "1" if request.param == "generic" else "0")
     monkeypatch.setenv("IM2WIN_NO_BOX", "1" if request.param == "nobox" else "0")
     monkeypatch.setenv("IM2WIN_NO_PIM", "1" if request.param == "nopim" else "0")
+    if request.param == "split3":
+        monkeypatch.setenv("IM2WIN_SPLITK", "3")
+    else:
+        monkeypatch.delenv("IM2WIN_SPLITK", raising=False)
 
 
 def _data(dims, seed, ints=False):
