@@ -236,6 +236,31 @@ def time_layer(layer, mode_name, steps, warmup, torch, b, flush_buf, sampler_ind
         if exc.code != b.EUNSUPPORTED:
             raise
         res["ms_fused"] = None
+    # the bf16 storage variant of the im2win tensor (BF16 mode only; layers with per-image tiling)
+    res["ms_transform_bf16"] = res["ms_conv_bf16src"] = None
+    if mode == b.MODE_BF16:
+        ws16 = torch.empty(b.workspace_bytes_bf16(dims) // 2, dtype=torch.int16, device="cuda")
+        try:
+            for _ in range(3):
+                b.transform_bf16(x, dims, ws16)
+                b.conv(ws16, b.SRC_IM2WIN_BF16, f, dims, mode, out)
+            be = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+            for k in range(steps):
+                flush_buf.zero_()
+                be[k][0].record(stream)
+                b.transform_bf16(x, dims, ws16)
+                be[k][1].record(stream)
+                b.conv(ws16, b.SRC_IM2WIN_BF16, f, dims, mode, out)
+                be[k][2].record(stream)
+            torch.cuda.synchronize()
+            if b.last_device_status() != 0:
+                raise RuntimeError("device status word set during the bf16-storage timing")
+            res["ms_transform_bf16"] = sum(e[0].elapsed_time(e[1]) for e in be) / steps
+            res["ms_conv_bf16src"] = sum(e[1].elapsed_time(e[2]) for e in be) / steps
+        except b.Im2winError as exc:
+            if exc.code != b.EUNSUPPORTED:
+                raise
+        del ws16
     if e2e:
         out_host = torch.empty((layer.N, layer.K, ho, wo), dtype=torch.float32).pin_memory()
         n_e2e = max(3, min(steps, 10))
@@ -305,6 +330,7 @@ def run_gpu(args):
                             "transform_frac_hbm": r["transform_bytes"] / r["ms_transform"] / 1e6 / peaks["hbm_gbs"],
                             "step_tflops": r["flops"] / r["ms_step"] / 1e9, "ms_conv": r["ms_conv"], "ms_transform": r["ms_transform"],
                             "workspace_bytes": r["workspace_bytes"], "im2col_bytes": r["im2col_bytes"], "peaks": peaks["source"],
+                            "ms_transform_bf16": r.get("ms_transform_bf16"), "ms_conv_bf16src": r.get("ms_conv_bf16src"),
                             "ms_fused": r.get("ms_fused"),
                             "fused_tflops": (r["flops"] / r["ms_fused"] / 1e9) if r.get("ms_fused") else None,
                             "fused_frac_hbm": (r["fused_bytes"] / r["ms_fused"] / 1e6 / peaks["hbm_gbs"]) if r.get("ms_fused") else None}
@@ -360,6 +386,10 @@ def run_gpu(args):
                    "what": "im2win_conv with src_kind NCHW_FUSED: same result from the untransformed input in one kernel, "
                            "no im2win tensor written (workspace 0 bytes); not part of `value`",
                    "frac_hbm": r["fused_bytes"] / r["ms_fused"] / 1e6 / peaks["hbm_gbs"]} if r.get("ms_fused") else None),
+        "bf16_storage": ({"ms_transform": r["ms_transform_bf16"], "ms_conv": r["ms_conv_bf16src"],
+                          "what": "the im2win tensor stored as bf16 (im2win_transform_bf16, src_kind IM2WIN_BF16): "
+                                  "half the workspace; BF16 mode only; not part of `value`"}
+                         if r.get("ms_conv_bf16src") else None),
         "e2e": {"value": world * flops / ms_e2e / 1e9, "unit": UNIT, "h2d_bytes_per_step": r["bytes_in"] + r["bytes_f"],
                 "d2h_bytes_per_step": r["bytes_out"], "ms_per_step": ms_e2e,
                 "how": "im2win_conv_host: pinned host buffers in, pinned host buffer out, wall clock per call"},

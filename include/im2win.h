@@ -37,8 +37,10 @@ typedef struct {
 /* What `src` of im2win_conv points to. */
 enum { IM2WIN_SRC_NCHW = 0,   /* the untransformed input I; the call runs the transform first   */
        IM2WIN_SRC_IM2WIN = 1, /* an im2win tensor Ihat produced earlier by im2win_transform      */
-       IM2WIN_SRC_NCHW_FUSED = 2 /* the untransformed input I; each tile's window rows are built
-                                    on the fly in shared memory, no im2win tensor reaches memory   */ };
+       IM2WIN_SRC_NCHW_FUSED = 2, /* the untransformed input I; each tile's window rows are built
+                                    on the fly in shared memory, no im2win tensor reaches memory   */
+       IM2WIN_SRC_IM2WIN_BF16 = 3 /* an im2win tensor stored as bf16 by im2win_transform_bf16
+                                    (a storage variant of this build, not in the paper)            */ };
 
 /* Arithmetic of the contraction.  Products are accumulated in fp32 in every mode. */
 enum { IM2WIN_MODE_TF32 = 0,  /* tensor cores, operands read as TF32 (low 13 mantissa bits unused) */
@@ -78,6 +80,17 @@ int im2win_im2col_bytes(const im2win_shape* shape, size_t* bytes);
 int im2win_transform(const float* in_nchw, const im2win_shape* shape, float* out_im2win,
                      void* cuda_stream);
 
+/* Storage variant of Algorithm 1 (no counterpart in the paper, which stores fp32 only):
+ *   Ihat16[i][r][m][k*Fh+u] = bf16(I[i][r][m*s+u][k]),  round to nearest even,
+ * i.e. the same tensor at 2 bytes per element, for IM2WIN_MODE_BF16 convolutions, whose operands
+ * are rounded to bf16 anyway: it halves what the transform writes and what the convolution reads.
+ * in_nchw:         device, N*C*H*W floats, read only.
+ * out_im2win_bf16: device, N*C*Ho*W*Fh 16-bit words (im2win_workspace_bytes_bf16), all written.
+ * Both bases 16-byte aligned (EALIGN); the ranges must not overlap (EOVERLAP). */
+int im2win_workspace_bytes_bf16(const im2win_shape* shape, size_t* bytes);  /* 2*N*C*Ho*Fh*W */
+int im2win_transform_bf16(const float* in_nchw, const im2win_shape* shape, uint16_t* out_im2win_bf16,
+                          void* cuda_stream);
+
 /* Algorithm 2 (the im2win-based convolution; its result is Eq. 1):
  *   O[i][j][m][n] = sum_{r,u,v} Ihat[i][r][m][(n*s+v)*Fh+u] * F[j][r][u][v].
  * (Algorithm 2 prints the strip offset as n*s*Wf+v*Hf+u, which equals the above for Hf==Wf and
@@ -90,6 +103,11 @@ int im2win_transform(const float* in_nchw, const im2win_shape* shape, float* out
  *            0 bytes).  Same result as the other two kinds.  Shapes without a fused specialisation
  *            (see below) fall back to transform + convolution if a sufficient `workspace` is
  *            given, else EUNSUPPORTED; IM2WIN_MODE_FP32 always takes that fallback.
+ *            src_kind IM2WIN_BF16: a bf16 im2win tensor from im2win_transform_bf16; mode must be
+ *            IM2WIN_MODE_BF16 (EINVAL otherwise); `workspace` is ignored.  The MMA operands are
+ *            the same bf16 values as from an fp32 im2win tensor.  Implemented for layers with a
+ *            filter-size specialisation whose images have roughly a thousand output positions or
+ *            more (tiles cut per image); EUNSUPPORTED otherwise.
  * filter:    device, K*C*Fh*Fw floats, native K,C,Fh,Fw order (no repacking needed).
  * mode:      IM2WIN_MODE_*.
  * out_nchw:  device, N*K*Ho*Wo floats, every element is written.

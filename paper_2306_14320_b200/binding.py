@@ -15,12 +15,12 @@ from typing import Sequence
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libim2win.so")
 
-SRC_NCHW, SRC_IM2WIN, SRC_NCHW_FUSED = 0, 1, 2
+SRC_NCHW, SRC_IM2WIN, SRC_NCHW_FUSED, SRC_IM2WIN_BF16 = 0, 1, 2, 3
 MODE_TF32, MODE_BF16, MODE_FP32 = 0, 1, 2
 OK, EINVAL, EALIGN, EWORKSPACE, EOVERLAP, ECUDA, ETIMEOUT, EUNSUPPORTED, ESCRATCH = 0, -1, -2, -3, -4, -5, -6, -7, -8
 
 EXPORTS = ("im2win_out_dims", "im2win_workspace_bytes", "im2win_im2col_bytes", "im2win_transform",
-           "im2win_conv", "im2win_conv_host", "im2win_host_release", "im2win_conv_static",
+           "im2win_workspace_bytes_bf16", "im2win_transform_bf16", "im2win_conv", "im2win_conv_host", "im2win_host_release", "im2win_conv_static",
            "im2win_last_device_status", "im2win_strerror")
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024  # IM2WIN_STATIC_SCRATCH_BYTES of include/im2win.h
 
@@ -56,6 +56,8 @@ def lib() -> ctypes.CDLL:
         L.im2win_workspace_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
         L.im2win_im2col_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
         L.im2win_transform.argtypes = [vp, sp, vp, vp]
+        L.im2win_workspace_bytes_bf16.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
+        L.im2win_transform_bf16.argtypes = [vp, sp, vp, vp]
         L.im2win_conv.argtypes = [vp, ctypes.c_int, vp, sp, ctypes.c_int, vp, vp, ctypes.c_size_t, vp]
         L.im2win_conv_host.argtypes = [vp, vp, sp, ctypes.c_int, vp]
         L.im2win_host_release.argtypes = []
@@ -122,6 +124,19 @@ def transform(in_nchw, shape, out_im2win, stream=None) -> None:
     """im2win_transform on the current (or given) stream; asynchronous."""
     _check(lib().im2win_transform(_ptr(in_nchw), ctypes.byref(Shape.of(shape)), _ptr(out_im2win), _stream(stream)),
            "im2win_transform")
+
+
+def workspace_bytes_bf16(shape) -> int:
+    b = ctypes.c_size_t()
+    _check(lib().im2win_workspace_bytes_bf16(ctypes.byref(Shape.of(shape)), ctypes.byref(b)),
+           "im2win_workspace_bytes_bf16")
+    return b.value
+
+
+def transform_bf16(in_nchw, shape, out_im2win_bf16, stream=None) -> None:
+    """im2win_transform_bf16 (the im2win tensor stored as bf16) on the current (or given) stream."""
+    _check(lib().im2win_transform_bf16(_ptr(in_nchw), ctypes.byref(Shape.of(shape)), _ptr(out_im2win_bf16),
+                                       _stream(stream)), "im2win_transform_bf16")
 
 
 def conv(src, src_kind: int, filter_kcfhfw, shape, mode: int, out_nchw, workspace=None,

@@ -126,6 +126,26 @@ int im2win_transform(const float* in_nchw, const im2win_shape* shape, float* out
   return launch_transform(in_nchw, out_im2win, g, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int im2win_workspace_bytes_bf16(const im2win_shape* shape, size_t* bytes) {
+  Geometry g;
+  const int rc = make_geometry(shape, &g);
+  if (rc != IM2WIN_OK) return rc;
+  if (!bytes) return IM2WIN_EINVAL;
+  *bytes = (size_t)g.n_win * 2;
+  return IM2WIN_OK;
+}
+
+int im2win_transform_bf16(const float* in_nchw, const im2win_shape* shape, uint16_t* out_im2win_bf16,
+                          void* cuda_stream) {
+  Geometry g;
+  int rc = make_geometry(shape, &g);
+  if (rc != IM2WIN_OK) return rc;
+  if (!in_nchw || !out_im2win_bf16) return IM2WIN_EINVAL;
+  if (!aligned16(in_nchw) || !aligned16(out_im2win_bf16)) return IM2WIN_EALIGN;
+  if (overlap(in_nchw, g.n_in * 4, out_im2win_bf16, g.n_win * 2)) return IM2WIN_EOVERLAP;
+  return launch_transform_bf16(in_nchw, out_im2win_bf16, g, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int im2win_conv(const void* src, int src_kind, const float* filter, const im2win_shape* shape,
                 int mode, float* out_nchw, void* workspace, size_t workspace_bytes,
                 void* cuda_stream) {
@@ -133,15 +153,21 @@ int im2win_conv(const void* src, int src_kind, const float* filter, const im2win
   int rc = make_geometry(shape, &g);
   if (rc != IM2WIN_OK) return rc;
   if (!src || !filter || !out_nchw) return IM2WIN_EINVAL;
-  if (src_kind != IM2WIN_SRC_NCHW && src_kind != IM2WIN_SRC_IM2WIN && src_kind != IM2WIN_SRC_NCHW_FUSED)
+  if (src_kind != IM2WIN_SRC_NCHW && src_kind != IM2WIN_SRC_IM2WIN && src_kind != IM2WIN_SRC_NCHW_FUSED &&
+      src_kind != IM2WIN_SRC_IM2WIN_BF16)
     return IM2WIN_EINVAL;
+  if (src_kind == IM2WIN_SRC_IM2WIN_BF16 && mode != IM2WIN_MODE_BF16) return IM2WIN_EINVAL;
   if (mode != IM2WIN_MODE_TF32 && mode != IM2WIN_MODE_BF16 && mode != IM2WIN_MODE_FP32)
     return IM2WIN_EINVAL;
   if (!aligned16(src) || !aligned16(filter) || !aligned16(out_nchw)) return IM2WIN_EALIGN;
-  const int64_t src_bytes = (src_kind == IM2WIN_SRC_IM2WIN ? g.n_win : g.n_in) * 4;
+  const int64_t src_bytes = src_kind == IM2WIN_SRC_IM2WIN_BF16 ? g.n_win * 2
+                                                                : (src_kind == IM2WIN_SRC_IM2WIN ? g.n_win : g.n_in) * 4;
   if (overlap(out_nchw, g.n_out * 4, src, src_bytes) || overlap(out_nchw, g.n_out * 4, filter, g.n_flt * 4))
     return IM2WIN_EOVERLAP;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (src_kind == IM2WIN_SRC_IM2WIN_BF16)  // no generic-kernel fallback for this storage variant
+    return launch_conv_tc_persistent(src, filter, out_nchw, g, mode, st, /*may_alloc=*/true, /*fused=*/false,
+                                     /*src_bf16=*/true);
   const float* xhat = static_cast<const float*>(src);
   if (src_kind == IM2WIN_SRC_NCHW_FUSED) {
     if (mode != IM2WIN_MODE_FP32) {

@@ -42,11 +42,12 @@ int32_t* device_status_word();  // device address of the status word (nullptr if
 
 // Launchers (all asynchronous on `st`; return a cudaError_t-derived im2win status).
 int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_t st);
+int launch_transform_bf16(const float* in, uint16_t* out, const Geometry& g, cudaStream_t st);
 int launch_conv_fp32(const float* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st);
 // Tensor-core convolution: the persistent specialised kernel when one applies (it returns
 // IM2WIN_EUNSUPPORTED otherwise), else the generic kernel.
-int launch_conv_tc_persistent(const float* src, const float* f, float* out, const Geometry& g, int mode,
-                              cudaStream_t st, bool may_alloc, bool fused = false);
+int launch_conv_tc_persistent(const void* src, const float* f, float* out, const Geometry& g, int mode,
+                              cudaStream_t st, bool may_alloc, bool fused = false, bool src_bf16 = false);
 int launch_conv_tc_generic(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
                            cudaStream_t st);
 // may_alloc = false keeps the call free of any (even stream-ordered) device allocation.

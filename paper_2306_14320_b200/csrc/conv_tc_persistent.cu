@@ -40,7 +40,7 @@ constexpr int kMaxSub = 16;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 struct PParams {
-  const float* xhat;
+  const void* xhat;     // strip source: fp32 im2win tensor / untransformed input, or a bf16 im2win tensor
   const float* f;
   float* out;
   int32_t* status;
@@ -177,6 +177,18 @@ __device__ __forceinline__ bool wait_bar_warp_a(const PParams& P, PMisc* misc, u
 
 // 32-bit load from a shared-space byte address (kept in program order with the waits and the
 // tcgen05 stores around it)
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a) {
+  uint32_t v;
+  asm volatile("{\n.reg .b16 h;\nld.shared.u16 h, [%1];\ncvt.u32.u16 %0, h;\n}" : "=r"(v) : "r"(a) : "memory");
+  return v;
+}
+// two 16-bit loads packed into one register (low half = first address)
+__device__ __forceinline__ uint32_t lds_u16x2(uint32_t a_lo, uint32_t a_hi) {
+  uint32_t v;
+  asm volatile("{\n.reg .b16 l, h;\nld.shared.u16 l, [%1];\nld.shared.u16 h, [%2];\nmov.b32 %0, {l, h};\n}"
+               : "=r"(v) : "r"(a_lo), "r"(a_hi) : "memory");
+  return v;
+}
 __device__ __forceinline__ uint32_t lds_u32(uint32_t a) {
   uint32_t v;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
@@ -326,11 +338,16 @@ __device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int32_t 
   asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
 }
 
-template <int FH, int FW, int CB, bool BF16, bool BRES, bool FUSED>
+template <int FH, int FW, int CB, bool BF16, bool BRES, bool FUSED, bool SRC16>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap fmap,
                           const __grid_constant__ CUtensorMap xmap) {
   constexpr int FF = FH * FW;
+  // SRC16: the staged source is an im2win tensor stored as bf16 (per-image tiling only; BF16 mode).
+  // Source lengths and offsets are in elements; ES bytes each, EPC elements per 16-byte chunk.
+  static_assert(!SRC16 || (BF16 && !FUSED), "a 16-bit source is an im2win tensor consumed in BF16 mode");
+  constexpr uint32_t ES = SRC16 ? 2u : 4u;
+  constexpr int32_t EPC = SRC16 ? 8 : 4;
   constexpr int KSTEP = BF16 ? 16 : 8;        // reduction elements per MMA
   constexpr int KCHUNK = BF16 ? 64 : 32;      // reduction elements per 128-byte filter row
   constexpr int KCG = CB * FF;                // real reduction elements per channel group
@@ -349,7 +366,11 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
   PMisc* const misc = reinterpret_cast<PMisc*>(smem + P.off_misc);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int32_t raw_stage_floats = CB * P.chan_pitch;
+  const int32_t raw_stage_floats = CB * P.chan_pitch;  // source elements per strip stage
+  using SrcT = typename std::conditional<SRC16, uint16_t, float>::type;
+  const SrcT* const xsrc = reinterpret_cast<const SrcT*>(P.xhat);
+  const uint32_t raw_sa = ptx::smem_u32(raw);
+  (void)xsrc; (void)raw_sa;
   const uint32_t b_stage_bytes = (uint32_t)P.NT * 128u;
 #ifdef IM2WIN_PROF
   const long long prof_kernel_t0 = clock64();
@@ -490,7 +511,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         const int32_t i = fast_div(tile_m, P.magic_TPI);
         const int32_t q_first = (tile_m - i * P.TPI) * P.TP;
         const int32_t m_a = fast_div(q_first, P.magic_Wo), n_a = q_first - m_a * P.Wo;
-        const int32_t box_x = ((m_a * P.row_mul + n_a * P.col_mul) & ~3) >> 1;
+        const int32_t box_x = ((m_a * P.row_mul + n_a * P.col_mul) & ~(EPC - 1)) / (EPC / 2);  // in 8-byte units
         const int32_t box_y0 = i * P.C;
         const int32_t tn = t + (int32_t)gridDim.x;
         const bool pf = P.l2_ahead && tn < (int32_t)P.ntiles;
@@ -500,7 +521,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           const int32_t i2 = fast_div(tm2, P.magic_TPI);
           const int32_t q2 = (tm2 - i2 * P.TPI) * P.TP;
           const int32_t m2 = fast_div(q2, P.magic_Wo), n2 = q2 - m2 * P.Wo;
-          pf_x = ((m2 * P.row_mul + n2 * P.col_mul) & ~3) >> 1;
+          pf_x = ((m2 * P.row_mul + n2 * P.col_mul) & ~(EPC - 1)) / (EPC / 2);
           pf_y0 = i2 * P.C;
         }
         int32_t nt_, g0, g1;
@@ -513,8 +534,8 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           if (!ok) break;
           if (lane == 0) {
             const uint32_t full = ptx::smem_u32(&bars->raw_full[sr]);
-            ptx::mbar_arrive_expect_tx(full, (uint32_t)raw_stage_floats * 4u);
-            tma_load_2d(ptx::smem_u32(raw + (size_t)sr * raw_stage_floats), &xmap, box_x, box_y0 + g * CB, full);
+            ptx::mbar_arrive_expect_tx(full, (uint32_t)raw_stage_floats * ES);
+            tma_load_2d(raw_sa + (uint32_t)(sr * raw_stage_floats) * ES, &xmap, box_x, box_y0 + g * CB, full);
           }
           __syncwarp();
         }
@@ -541,21 +562,21 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           ok = wait_bar_warp(P, misc, &bars->raw_empty[sr], rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, PROF_SLOT(0), 128);
           if (!ok) break;
           const uint32_t full = ptx::smem_u32(&bars->raw_full[sr]);
-          const float* src = nullptr;
+          const SrcT* src = nullptr;
           uint32_t dst = 0, bytes = 0;
           if (lane < CB && g * CB + lane < P.C) {
-            const int32_t skew = (int32_t)(start & 3);
+            const int32_t skew = (int32_t)(start & (EPC - 1));
             const int64_t a0 = start - skew;
-            int32_t nfl = (skew + len + 3) & ~3;
-            float* d = raw + (size_t)sr * raw_stage_floats + lane * P.chan_pitch;
+            int32_t nfl = (skew + len + EPC - 1) & ~(EPC - 1);
+            SrcT* d = reinterpret_cast<SrcT*>(raw) + (size_t)sr * raw_stage_floats + lane * P.chan_pitch;
             if (a0 + nfl > P.n_src) {  // the last 16-byte chunk would pass the end of the tensor
-              const int32_t nbulk = (int32_t)((P.n_src - a0) & ~(int64_t)3);
-              for (int64_t e = a0 + nbulk; e < P.n_src; ++e) d[e - a0] = __ldg(P.xhat + e);
+              const int32_t nbulk = (int32_t)((P.n_src - a0) & ~(int64_t)(EPC - 1));
+              for (int64_t e = a0 + nbulk; e < P.n_src; ++e) d[e - a0] = __ldg(xsrc + e);
               nfl = nbulk;
             }
-            src = P.xhat + a0;
+            src = xsrc + a0;
             dst = ptx::smem_u32(d);
-            bytes = (uint32_t)nfl * 4u;
+            bytes = (uint32_t)nfl * ES;
           }
           start += group_step;
           const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
@@ -564,7 +585,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           if (bytes) ptx::bulk_g2s(dst, src, bytes, full);
         }
       }
-    } else {
+    } else if constexpr (!SRC16) {
       for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
         const TileInfo ti = tile_info(P, tile_of(P, t));
         const int32_t nseg = ti.nseg;
@@ -610,10 +631,10 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
               float* d = stage + dsto[z];
               if (a0 + nfl > P.n_src) {  // the last 16-byte chunk would pass the end of the tensor
                 const int32_t nbulk = (int32_t)((P.n_src - a0) & ~(int64_t)3);
-                for (int64_t e = a0 + nbulk; e < P.n_src; ++e) d[e - a0] = __ldg(P.xhat + e);
+                for (int64_t e = a0 + nbulk; e < P.n_src; ++e) d[e - a0] = __ldg(xsrc + e);
                 nfl = nbulk;
               }
-              src[z] = P.xhat + a0;
+              src[z] = xsrc + a0;
               dst[z] = ptx::smem_u32(d);
               bytes[z] = (uint32_t)nfl * 4u;
             }
@@ -775,7 +796,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     const int32_t q4 = (warp - kRepackWarp0) & 3;
     const int32_t p = q4 * 32 + lane;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
-    const int32_t skew_step = P.box ? 0 : (int32_t)(P.plane & 3);
+    const int32_t skew_step = P.box ? 0 : (int32_t)(P.plane & (EPC - 1));
     Ring rr, ar;      // raw stage of the current group, A slot of the current part (this set's own ring)
     const uint32_t slot0 = (uint32_t)(set * P.NSS);
     const uint32_t raw_a = ptx::smem_u32(raw), zero_a = ptx::smem_u32(zero_pad);
@@ -800,9 +821,9 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           const int32_t m = fast_div(q, P.magic_Wo), n = q - m * P.Wo;
           // box: the staged range starts at the 16-byte boundary below the first float (same phase
           // in every plane); bulk copies: the phase is per channel, added to the pointers below
-          base_off = m * P.row_mul + n * P.col_mul - (P.box ? (virt_a & ~3) : virt_a);
+          base_off = m * P.row_mul + n * P.col_mul - (P.box ? (virt_a & ~(EPC - 1)) : virt_a);
         }
-        if (!P.box) skew0 = (int32_t)((ti.i_first * P.C * P.plane + virt_a) & 3);
+        if (!P.box) skew0 = (int32_t)((ti.i_first * P.C * P.plane + virt_a) & (EPC - 1));
       } else {
         repack_prologue_general(P, ti, p, lane, valid, base_off, skew0);
       }
@@ -826,15 +847,15 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         // stored in the strip at offset v*FH + u from the window start
         // (fused source: the raw input rows are staged instead, and tap (u, v) is at u*W + v)
         const int32_t r0 = g * CB;
-        const uint32_t stage_a = raw_a + (uint32_t)(sr * raw_stage_floats + base_off) * 4u;
+        const uint32_t stage_a = raw_a + (uint32_t)(sr * raw_stage_floats + base_off) * ES;
         uint32_t ca[CB];
         if (skew_step == 0) {  // every plane starts on a 16-byte boundary: one phase for all channels
 #pragma unroll
-          for (int rl = 0; rl < CB; ++rl) ca[rl] = stage_a + (uint32_t)(rl * P.chan_pitch + skew0) * 4u;
+          for (int rl = 0; rl < CB; ++rl) ca[rl] = stage_a + (uint32_t)(rl * P.chan_pitch + skew0) * ES;
         } else {
 #pragma unroll
           for (int rl = 0; rl < CB; ++rl)
-            ca[rl] = stage_a + (uint32_t)(rl * P.chan_pitch + ((skew0 + (r0 + rl) * skew_step) & 3)) * 4u;
+            ca[rl] = stage_a + (uint32_t)(rl * P.chan_pitch + ((skew0 + (r0 + rl) * skew_step) & (EPC - 1))) * ES;
         }
         // channels past C (last group of a C that CB does not divide) read as zero: their addresses
         // are parked on a zeroed pad so that the hot loop carries no per-element select
@@ -843,11 +864,23 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           for (int rl = 0; rl < CB; ++rl)
             if (r0 + rl >= P.C) ca[rl] = zero_a;
         }
+        // (16-bit source) shared address of element kl, and a packed pair of consecutive elements
+        auto addr16 = [&](int kl) -> uint32_t {
+          const int rl = kl / FF, w = kl % FF;
+          return ca[rl] + (uint32_t)(((w % FW) * FH + (w / FW)) * 2);
+        };
+        auto pair16 = [&](int kl) -> uint32_t {
+          if (kl >= KCG) return 0u;
+          if (kl + 1 >= KCG) return lds_u16(addr16(kl));
+          return lds_u16x2(addr16(kl), addr16(kl + 1));
+        };
+        (void)pair16;
         auto elem = [&](int kl) -> uint32_t {
           if (kl >= KCG) return 0u;
           const int rl = kl / FF, w = kl % FF;
-          return lds_u32(FUSED ? ca[rl] + (uint32_t)(w / FW) * W4 + (uint32_t)((w % FW) * 4)
-                               : ca[rl] + (uint32_t)(((w % FW) * FH + (w / FW)) * 4));
+          if constexpr (SRC16) return lds_u16(ca[rl] + (uint32_t)(((w % FW) * FH + (w / FW)) * 2));  // bf16 bits
+          else return lds_u32(FUSED ? ca[rl] + (uint32_t)(w / FW) * W4 + (uint32_t)((w % FW) * 4)
+                                    : ca[rl] + (uint32_t)(((w % FW) * FH + (w / FW)) * 4));
         };
 #pragma unroll
         for (int h = 0; h < PARTS; ++h) {
@@ -870,7 +903,9 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
               if (j < nst) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                  if constexpr (BF16)
+                  if constexpr (SRC16)  // already bf16: low half = even k
+                    v[jj][e] = pair16((j0 + j) * 16 + 2 * e);
+                  else if constexpr (BF16)
                     v[jj][e] = ptx::pack_bf16x2(__uint_as_float(elem((j0 + j) * 16 + 2 * e)),
                                                 __uint_as_float(elem((j0 + j) * 16 + 2 * e + 1)));
                   else
@@ -1072,9 +1107,11 @@ int sm_count() {
   return n;
 }
 
-template <int FH, int FW, int CB, bool BF16, bool FUSED>
-int launch_spec_impl(const float* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc) {
+template <int FH, int FW, int CB, bool BF16, bool FUSED, bool SRC16 = false>
+int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc) {
   constexpr int FF = FH * FW;
+  constexpr int64_t ES = SRC16 ? 2 : 4;    // bytes per source element
+  constexpr int64_t EPC = 16 / ES;         // source elements per 16-byte chunk
   constexpr int KSTEP = BF16 ? 16 : 8;
   constexpr int KCG = CB * FF;
   constexpr int KCGP = (KCG + KSTEP - 1) / KSTEP * KSTEP;
@@ -1132,11 +1169,13 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
   // 256 8-byte elements.
   {
     const int64_t tpi = (g.HoWo + 127) / 128;
-    const int64_t one_seg = 127 * (int64_t)P.col_mul + wraps * (rowwrap > P.col_mul ? rowwrap - P.col_mul : 0) + P.win_span + 6 + 4;
+    // (+ the 16-byte phase in front and the rounding up to whole 16-byte chunks behind)
+    const int64_t one_seg = 127 * (int64_t)P.col_mul + wraps * (rowwrap > P.col_mul ? rowwrap - P.col_mul : 0) +
+                            P.win_span + 2 * (EPC - 1) + EPC;
     // A box row is a whole number of 16-byte units, and CB rows (one stage) a whole number of 128
     // bytes, so that every stage starts on the 128-byte boundary a tiled TMA destination needs.
-    int64_t row_align = 4;
-    while ((CB * row_align) % 32 != 0) row_align *= 2;
+    int64_t row_align = EPC;
+    while ((CB * row_align * ES) % 128 != 0) row_align *= 2;
     const int64_t boxf = (one_seg + row_align - 1) / row_align * row_align;
     const bool little_waste = tpi * 128 * 100 <= g.HoWo * 107;
     const char* nobox = getenv("IM2WIN_NO_BOX");
@@ -1147,8 +1186,8 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
       P.TPI = (int32_t)tpi;
       P.magic_TPI = (((uint64_t)1 << 32) + (uint64_t)tpi - 1) / (uint64_t)tpi;
       P.magic_Wo = (((uint64_t)1 << 32) + (uint64_t)g.Wo - 1) / (uint64_t)g.Wo;
-      pitch = (one_seg + 3) & ~(int64_t)3;
-      if (CB >= 2 && (P.plane % 4) == 0 && boxf <= 512 && encode_fn() != nullptr && (int64_t)g.N * g.C <= INT32_MAX &&
+      pitch = (one_seg + EPC - 1) / EPC * EPC;
+      if (CB >= 2 && (P.plane % EPC) == 0 && boxf * ES <= 2048 && encode_fn() != nullptr && (int64_t)g.N * g.C <= INT32_MAX &&
           !(nobox && nobox[0] == '1')) {
         P.box = 1;
         P.l2_ahead = !(getenv("IM2WIN_NO_L2AHEAD") && getenv("IM2WIN_NO_L2AHEAD")[0] == '1');
@@ -1156,10 +1195,11 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
       }
     }
   }
+  if (SRC16 && !P.pim) return IM2WIN_EUNSUPPORTED;  // the 16-bit source is implemented for per-image tiling only
   P.chan_pitch = (int32_t)pitch;
   const int64_t tiles_m = P.pim ? (int64_t)g.N * P.TPI : (g.Mtot + P.TP - 1) / P.TP;
   P.ntiles = tiles_m * P.n_ntiles;
-  const int64_t raw_stage = (int64_t)CB * pitch * 4;
+  const int64_t raw_stage = (int64_t)CB * pitch * ES;
 
   // filter operand: resident if it fits next to two strip stages, else streamed by TMA (TF32, dense groups)
   const int64_t cap = 227 * 1024 - 1024 - 1024 - ((int64_t)(P.win_span + 8) * 4 + 16);  // alignment slack, barriers, zero pad
@@ -1298,12 +1338,12 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
   CUtensorMap xmap;
   memset(&xmap, 0, sizeof(xmap));
   if (P.box) {
-    // the im2win tensor as [N*C planes][HoL/2 8-byte elements]
-    const cuuint64_t gdim[2] = {(cuuint64_t)(P.plane / 2), (cuuint64_t)g.N * g.C};
-    const cuuint64_t gstr[1] = {(cuuint64_t)P.plane * 4};
-    const cuuint32_t box[2] = {(cuuint32_t)(P.chan_pitch / 2), (cuuint32_t)CB};
+    // the source as [N*C planes][plane bytes / 8 8-byte elements]
+    const cuuint64_t gdim[2] = {(cuuint64_t)(P.plane * ES / 8), (cuuint64_t)g.N * g.C};
+    const cuuint64_t gstr[1] = {(cuuint64_t)P.plane * ES};
+    const cuuint32_t box[2] = {(cuuint32_t)(P.chan_pitch * ES / 8), (cuuint32_t)CB};
     const cuuint32_t estr[2] = {1, 1};
-    if (encode_fn()(&xmap, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<float*>(xhat), gdim, gstr, box, estr,
+    if (encode_fn()(&xmap, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(xhat), gdim, gstr, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
       if (f_bf16) cudaFreeAsync(f_bf16, st);
@@ -1318,12 +1358,12 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
     return IM2WIN_ECUDA;
   }
   if (resident) {
-    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, true, FUSED>;
+    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, true, FUSED, SRC16>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
     kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
   } else {
-    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, false, FUSED>;
+    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, false, FUSED, SRC16>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) { cudaGetLastError(); if (f_bf16) cudaFreeAsync(f_bf16, st); return IM2WIN_ECUDA; }
     kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
@@ -1333,11 +1373,16 @@ int launch_spec_impl(const float* xhat, const float* f, float* out, const Geomet
   return rc;
 }
 
+// src_kind: 0 = im2win tensor (fp32), 1 = untransformed input consumed fused, 2 = im2win tensor stored as bf16
 template <int FH, int FW, int CB, bool BF16>
-int launch_spec(const float* src, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc,
-                bool fused) {
-  return fused ? launch_spec_impl<FH, FW, CB, BF16, true>(src, f, out, g, st, may_alloc)
-               : launch_spec_impl<FH, FW, CB, BF16, false>(src, f, out, g, st, may_alloc);
+int launch_spec(const void* src, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc,
+                int src_kind) {
+  if (src_kind == 2) {
+    if constexpr (BF16) return launch_spec_impl<FH, FW, CB, true, false, true>(src, f, out, g, st, may_alloc);
+    else return IM2WIN_EUNSUPPORTED;
+  }
+  return src_kind == 1 ? launch_spec_impl<FH, FW, CB, BF16, true>(src, f, out, g, st, may_alloc)
+                       : launch_spec_impl<FH, FW, CB, BF16, false>(src, f, out, g, st, may_alloc);
 }
 
 }  // namespace
@@ -1347,32 +1392,34 @@ int launch_spec(const float* src, const float* f, float* out, const Geometry& g,
 // BF16 copy of a filter that is too large to stay in shared memory).
 // fused: `xhat` is the untransformed NCHW input and the windows are built from staged input rows
 // (no im2win tensor exists in global memory).
-int launch_conv_tc_persistent(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
-                              cudaStream_t st, bool may_alloc, bool fused) {
+int launch_conv_tc_persistent(const void* xhat, const float* f, float* out, const Geometry& g, int mode,
+                              cudaStream_t st, bool may_alloc, bool fused, bool src_bf16) {
+  const int kind = src_bf16 ? 2 : (fused ? 1 : 0);
+  if (src_bf16 && (fused || mode != IM2WIN_MODE_BF16)) return IM2WIN_EUNSUPPORTED;
   const bool bf16 = mode == IM2WIN_MODE_BF16;
   if (g.Fh == 3 && g.Fw == 3) {
     // BF16 MMAs take 16 reduction elements: sixteen channels (144 = 9 steps) leave no padding
-    if (bf16 && g.C % 16 == 0) return launch_spec<3, 3, 16, true>(xhat, f, out, g, st, may_alloc, fused);
-    if (g.C >= 8) return bf16 ? launch_spec<3, 3, 8, true>(xhat, f, out, g, st, may_alloc, fused)
-                              : launch_spec<3, 3, 8, false>(xhat, f, out, g, st, may_alloc, fused);
-    if (g.C == 3) return bf16 ? launch_spec<3, 3, 3, true>(xhat, f, out, g, st, may_alloc, fused)
-                              : launch_spec<3, 3, 3, false>(xhat, f, out, g, st, may_alloc, fused);
+    if (bf16 && g.C % 16 == 0) return launch_spec<3, 3, 16, true>(xhat, f, out, g, st, may_alloc, kind);
+    if (g.C >= 8) return bf16 ? launch_spec<3, 3, 8, true>(xhat, f, out, g, st, may_alloc, kind)
+                              : launch_spec<3, 3, 8, false>(xhat, f, out, g, st, may_alloc, kind);
+    if (g.C == 3) return bf16 ? launch_spec<3, 3, 3, true>(xhat, f, out, g, st, may_alloc, kind)
+                              : launch_spec<3, 3, 3, false>(xhat, f, out, g, st, may_alloc, kind);
   }
   if (g.Fh == 5 && g.Fw == 5) {
-    if (bf16 && g.C % 16 == 0) return launch_spec<5, 5, 16, true>(xhat, f, out, g, st, may_alloc, fused);
-    if (g.C >= 8) return bf16 ? launch_spec<5, 5, 8, true>(xhat, f, out, g, st, may_alloc, fused)
-                              : launch_spec<5, 5, 8, false>(xhat, f, out, g, st, may_alloc, fused);
+    if (bf16 && g.C % 16 == 0) return launch_spec<5, 5, 16, true>(xhat, f, out, g, st, may_alloc, kind);
+    if (g.C >= 8) return bf16 ? launch_spec<5, 5, 8, true>(xhat, f, out, g, st, may_alloc, kind)
+                              : launch_spec<5, 5, 8, false>(xhat, f, out, g, st, may_alloc, kind);
   }
   if (g.Fh == 7 && g.Fw == 7 && g.C % 8 == 0) {
-    if (bf16 && g.C % 16 == 0) return launch_spec<7, 7, 16, true>(xhat, f, out, g, st, may_alloc, fused);
-    if (!bf16) return launch_spec<7, 7, 8, false>(xhat, f, out, g, st, may_alloc, fused);
+    if (bf16 && g.C % 16 == 0) return launch_spec<7, 7, 16, true>(xhat, f, out, g, st, may_alloc, kind);
+    if (!bf16) return launch_spec<7, 7, 8, false>(xhat, f, out, g, st, may_alloc, kind);
   }
   if (g.Fh == 7 && g.Fw == 7 && g.C == 3)
-    return bf16 ? launch_spec<7, 7, 3, true>(xhat, f, out, g, st, may_alloc, fused)
-                : launch_spec<7, 7, 3, false>(xhat, f, out, g, st, may_alloc, fused);
+    return bf16 ? launch_spec<7, 7, 3, true>(xhat, f, out, g, st, may_alloc, kind)
+                : launch_spec<7, 7, 3, false>(xhat, f, out, g, st, may_alloc, kind);
   if (g.Fh == 11 && g.Fw == 11 && g.C <= 4)
-    return bf16 ? launch_spec<11, 11, 1, true>(xhat, f, out, g, st, may_alloc, fused)
-                : launch_spec<11, 11, 1, false>(xhat, f, out, g, st, may_alloc, fused);
+    return bf16 ? launch_spec<11, 11, 1, true>(xhat, f, out, g, st, may_alloc, kind)
+                : launch_spec<11, 11, 1, false>(xhat, f, out, g, st, may_alloc, kind);
   return IM2WIN_EUNSUPPORTED;
 }
 

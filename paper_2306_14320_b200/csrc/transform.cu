@@ -10,6 +10,7 @@
 // Every needed input row is read from HBM once per row block (the Fh-s halo rows between
 // neighbouring blocks come from L2), every output element is written exactly once.
 #include <cstdlib>
+#include <type_traits>
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
@@ -135,6 +136,117 @@ __global__ void __launch_bounds__(kThreads) transform_smem_kernel(const Transfor
   if ((int32_t)threadIdx.x < n_out - tail0) dst[tail0 + threadIdx.x] = fetch(locate(tail0 + threadIdx.x));
 }
 
+// bf16 storage variant of the staged-gather kernel: same jobs and staging, the output range walked
+// in 16-byte chunks of eight bf16 (round to nearest even), one 128-bit store each.
+__device__ __forceinline__ uint32_t bf16x2_rn(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ uint16_t bf16_rn(float x) { return (uint16_t)(bf16x2_rn(x, 0.f) & 0xffffu); }
+
+__global__ void __launch_bounds__(kThreads) transform_smem_bf16_kernel(const TransformParams P, uint16_t* out16) {
+  extern __shared__ __align__(16) float smem[];
+  const int64_t job = blockIdx.x;
+  const int64_t pg = job / P.nblk;
+  const int32_t b = (int32_t)(job - pg * P.nblk);
+  const bool whole = P.nblk == 1;
+  const int64_t plane0 = pg * P.PB;
+  const int32_t npl = whole ? (int32_t)min((int64_t)P.PB, P.planes - plane0) : 1;
+  const int32_t m0 = b * P.MB;
+  const int32_t mb = whole ? P.Ho : min(P.MB, P.Ho - m0);
+  const int32_t rows_in = whole ? P.H : (mb - 1) * P.s + P.Fh;
+  const int32_t plane_floats = rows_in * P.W;
+  const int32_t n_in = npl * plane_floats;
+
+  const float* src = P.in + plane0 * P.HW + (int64_t)m0 * P.s * P.W;
+  const int32_t skew = (int32_t)((reinterpret_cast<uintptr_t>(src) >> 2) & 3);
+  float* tile = smem + skew;
+  {
+    const int32_t head = min((4 - skew) & 3, n_in);
+    const int32_t nvec = (n_in - head) >> 2;
+    const int32_t tail0 = head + (nvec << 2);
+    if ((int32_t)threadIdx.x < head) tile[threadIdx.x] = __ldg(src + threadIdx.x);
+    const float4* src4 = reinterpret_cast<const float4*>(src + head);
+    float4* dst4 = reinterpret_cast<float4*>(tile + head);
+    for (int32_t i = threadIdx.x; i < nvec; i += kThreads) dst4[i] = ldg_stream(src4 + i);
+    if ((int32_t)threadIdx.x < n_in - tail0) tile[tail0 + threadIdx.x] = __ldg(src + tail0 + threadIdx.x);
+  }
+  __syncthreads();
+
+  uint16_t* dst = out16 + plane0 * P.HoL + (int64_t)m0 * P.L;
+  const int32_t out_plane = mb * P.L;
+  const int32_t n_out = npl * out_plane;
+  const int32_t dskew = (int32_t)((reinterpret_cast<uintptr_t>(dst) >> 1) & 7);  // 16-byte phase in elements
+  const int32_t head = min((8 - dskew) & 7, n_out);
+  const int32_t nvec = (n_out - head) >> 3;
+  const int32_t tail0 = head + (nvec << 3);
+  const int32_t sW = P.s * P.W;
+  auto locate = [&](int32_t e) -> Cursor {
+    int32_t pl = 0, rem = e;
+    if (npl > 1) {
+      pl = (int32_t)(((uint64_t)(uint32_t)e * P.magic_HoL) >> 32);
+      rem = e - pl * out_plane;
+    }
+    const int32_t mm = (int32_t)(((uint64_t)(uint32_t)rem * P.magic_L) >> 32);
+    const int32_t r2 = rem - mm * P.L;
+    Cursor c;
+    c.mm = mm;
+    c.k = (int32_t)(((uint64_t)(uint32_t)r2 * P.magic_Fh) >> 32);
+    c.u = r2 - c.k * P.Fh;
+    c.base = pl * plane_floats + mm * sW;
+    return c;
+  };
+  auto fetch = [&](const Cursor& c) { return tile[c.base + c.u * P.W + c.k]; };
+  auto advance = [&](Cursor c) -> Cursor {
+    if (++c.u == P.Fh) {
+      c.u = 0;
+      if (++c.k == P.W) {
+        c.k = 0;
+        c.base += sW;
+        if (++c.mm == mb) {
+          c.mm = 0;
+          c.base += plane_floats - mb * sW;
+        }
+      }
+    }
+    return c;
+  };
+  if ((int32_t)threadIdx.x < head) dst[threadIdx.x] = bf16_rn(fetch(locate(threadIdx.x)));
+  uint4* dst4 = reinterpret_cast<uint4*>(dst + head);
+  for (int32_t i = threadIdx.x; i < nvec; i += kThreads) {
+    Cursor c = locate(head + (i << 3));
+    float x[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      x[j] = fetch(c);
+      if (j < 7) c = advance(c);
+    }
+    uint4 v;
+    v.x = bf16x2_rn(x[0], x[1]); v.y = bf16x2_rn(x[2], x[3]);
+    v.z = bf16x2_rn(x[4], x[5]); v.w = bf16x2_rn(x[6], x[7]);
+    dst4[i] = v;
+  }
+  if ((int32_t)threadIdx.x < n_out - tail0) dst[tail0 + threadIdx.x] = bf16_rn(fetch(locate(tail0 + threadIdx.x)));
+}
+
+// one thread per element; any shape
+__global__ void __launch_bounds__(kThreads) transform_gather_bf16_kernel(const float* __restrict__ in,
+                                                                          uint16_t* __restrict__ out,
+                                                                          int32_t H, int32_t W, int32_t Fh,
+                                                                          int32_t s, int32_t Ho, int64_t total) {
+  const int64_t L = (int64_t)W * Fh;
+  for (int64_t e = (int64_t)blockIdx.x * kThreads + threadIdx.x; e < total;
+       e += (int64_t)gridDim.x * kThreads) {
+    const int64_t strip = e / L;
+    const int32_t rem = (int32_t)(e - strip * L);
+    const int32_t k = rem / Fh, u = rem - k * Fh;
+    const int64_t plane = strip / Ho;
+    const int32_t m = (int32_t)(strip - plane * Ho);
+    out[e] = bf16_rn(__ldg(in + (plane * H + (int64_t)m * s + u) * W + k));
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Tile kernel: the same jobs (whole planes, or a block of output rows of one plane), but all global
 // traffic is two TMA bulk copies.  The input range comes into shared memory with one
@@ -146,7 +258,7 @@ __global__ void __launch_bounds__(kThreads) transform_smem_kernel(const Transfor
 // aligned chunks; the at most 3 + 3 floats outside the aligned part are copied by threads.
 struct TileParams {
   const float* in;
-  float* out;
+  void* out;            // fp32 im2win tensor, or 16-bit words for the bf16 storage variant
   int32_t* status;
   int32_t H, W, s, Ho, L;
   int32_t MB, nblk, PB;
@@ -158,11 +270,14 @@ struct TileParams {
   uint32_t off_bar;     // byte offset of the mbarrier
 };
 
-template <int FH>
+// OUT16: the output is the bf16 storage variant (P.out then points at 16-bit words).
+template <int FH, bool OUT16>
 __global__ void __launch_bounds__(kThreads) transform_tile_kernel(const TileParams P) {
+  using OutT = typename std::conditional<OUT16, uint16_t, float>::type;
+  constexpr int32_t OPC = OUT16 ? 8 : 4;  // output elements per 16-byte chunk
   extern __shared__ __align__(128) uint8_t smem_raw[];
   float* const tin0 = reinterpret_cast<float*>(smem_raw);
-  float* const tout0 = reinterpret_cast<float*>(smem_raw + P.off_out);
+  OutT* const tout0 = reinterpret_cast<OutT*>(smem_raw + P.off_out);
   uint64_t* const bar = reinterpret_cast<uint64_t*>(smem_raw + P.off_bar);
 
   const int64_t job = blockIdx.x;
@@ -212,9 +327,9 @@ __global__ void __launch_bounds__(kThreads) transform_tile_kernel(const TilePara
   }
 
   // ---- transpose shared -> shared
-  const int64_t dst0 = plane0 * P.HoL + (int64_t)m0 * P.L;       // first float of the output range
-  const int32_t dskew = (int32_t)(dst0 & 3);                      // P.out is 16-byte aligned
-  float* const tout = tout0 + dskew;                              // tout[e] <-> out[dst0 + e]
+  const int64_t dst0 = plane0 * P.HoL + (int64_t)m0 * P.L;       // first element of the output range
+  const int32_t dskew = (int32_t)(dst0 & (OPC - 1));              // P.out is 16-byte aligned
+  OutT* const tout = tout0 + dskew;                               // tout[e] <-> out[dst0 + e]
   const int32_t sW = P.s * P.W;
   const int32_t units_plane = mb * P.QW;
   const int32_t nunits = npl * units_plane;
@@ -229,7 +344,7 @@ __global__ void __launch_bounds__(kThreads) transform_tile_kernel(const TilePara
     const int32_t k0 = (rem - mm * P.QW) * 4;
     const float* src = tin + pl * plane_floats + mm * sW + k0;
     const int32_t oe = pl * out_plane + mm * P.L + k0 * FH;
-    float* dst = tout + oe;
+    OutT* dst = tout + oe;
     if (k0 + 4 <= P.W) {
       float r[4 * FH];  // r[c*FH + u] = I[m*s + u][k0 + c]: the 4*FH output floats in order
       if (in_even) {
@@ -246,35 +361,52 @@ __global__ void __launch_bounds__(kThreads) transform_tile_kernel(const TilePara
           for (int c = 0; c < 4; ++c) r[c * FH + u] = src[u * P.W + c];
         }
       }
+      if constexpr (OUT16) {
+        // 4*FH bf16 in order: 32-bit stores of rounded pairs where the run starts on a 4-byte
+        // boundary, else element by element
+        if (((dskew + oe) & 1) == 0) {
+#pragma unroll
+          for (int j = 0; j < 2 * FH; ++j) reinterpret_cast<uint32_t*>(dst)[j] = bf16x2_rn(r[2 * j], r[2 * j + 1]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4 * FH; ++j) dst[j] = bf16_rn(r[j]);
+        }
+        continue;
+      }
       const int32_t a = (dskew + oe) & 3;  // 16-byte phase of the run in the output buffer
-      if (a == 0) {
+      if constexpr (!OUT16) {
+        if (a == 0) {
 #pragma unroll
-        for (int j = 0; j < FH; ++j)
-          reinterpret_cast<float4*>(dst)[j] = make_float4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-      } else if (a == 2) {
-        *reinterpret_cast<float2*>(dst) = make_float2(r[0], r[1]);
+          for (int j = 0; j < FH; ++j)
+            reinterpret_cast<float4*>(dst)[j] = make_float4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        } else if (a == 2) {
+          *reinterpret_cast<float2*>(dst) = make_float2(r[0], r[1]);
 #pragma unroll
-        for (int j = 0; j < FH - 1; ++j)
-          *reinterpret_cast<float4*>(dst + 2 + 4 * j) = make_float4(r[4 * j + 2], r[4 * j + 3], r[4 * j + 4], r[4 * j + 5]);
-        *reinterpret_cast<float2*>(dst + 4 * FH - 2) = make_float2(r[4 * FH - 2], r[4 * FH - 1]);
-      } else {
+          for (int j = 0; j < FH - 1; ++j)
+            *reinterpret_cast<float4*>(dst + 2 + 4 * j) = make_float4(r[4 * j + 2], r[4 * j + 3], r[4 * j + 4], r[4 * j + 5]);
+          *reinterpret_cast<float2*>(dst + 4 * FH - 2) = make_float2(r[4 * FH - 2], r[4 * FH - 1]);
+        } else {
 #pragma unroll
-        for (int j = 0; j < 4 * FH; ++j) dst[j] = r[j];
+          for (int j = 0; j < 4 * FH; ++j) dst[j] = r[j];
+        }
       }
     } else {  // the last, partial quad of a row
       for (int32_t c = 0; k0 + c < P.W; ++c)
 #pragma unroll
-        for (int u = 0; u < FH; ++u) dst[c * FH + u] = src[u * P.W + c];
+        for (int u = 0; u < FH; ++u) {
+          if constexpr (OUT16) dst[c * FH + u] = bf16_rn(src[u * P.W + c]);
+          else dst[c * FH + u] = src[u * P.W + c];
+        }
     }
   }
   ptx::fence_proxy_async_smem();  // the buffer is about to be read by the bulk copy
   __syncthreads();
 
   // ---- output buffer -> global: one bulk copy of the aligned part, threads for the ragged ends
-  const int32_t head = min((4 - dskew) & 3, n_out);
-  const int32_t nvec = (n_out - head) >> 2;
-  const int32_t tail0 = head + (nvec << 2);
-  float* const gout = P.out + dst0;
+  const int32_t head = min((OPC - dskew) & (OPC - 1), n_out);
+  const int32_t nvec = (n_out - head) / OPC;
+  const int32_t tail0 = head + nvec * OPC;
+  OutT* const gout = reinterpret_cast<OutT*>(P.out) + dst0;
   if (threadIdx.x == 0 && nvec > 0) {
     ptx::bulk_s2g(gout + head, ptx::smem_u32(tout + head), (uint32_t)nvec * 16u);
     ptx::bulk_s2g_commit();
@@ -306,9 +438,9 @@ uint64_t magic_for(uint32_t d) { return ((uint64_t)1 << 32) / d + ((((uint64_t)1
 
 }  // namespace
 
-template <int FH>
+template <int FH, bool OUT16>
 int launch_tile_fh(const TileParams& P, int64_t ctas, size_t smem, cudaStream_t st) {
-  auto kern = transform_tile_kernel<FH>;
+  auto kern = transform_tile_kernel<FH, OUT16>;
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
     cudaGetLastError();
@@ -321,7 +453,7 @@ int launch_tile_fh(const TileParams& P, int64_t ctas, size_t smem, cudaStream_t 
 // Tile kernel where a job's input and output ranges fit one shared-memory budget together (a sixth
 // of an SM's shared memory, so that six CTAs overlap their loads, transposes and stores);
 // IM2WIN_EUNSUPPORTED otherwise (the caller then uses the staged-gather kernel).
-int launch_transform_tile(const float* in, float* out, const Geometry& g, cudaStream_t st) {
+int launch_transform_tile(const float* in, void* out, bool out16, const Geometry& g, cudaStream_t st) {
   if (g.Fh != 1 && g.Fh != 2 && g.Fh != 3 && g.Fh != 4 && g.Fh != 5 && g.Fh != 7 && g.Fh != 11) return IM2WIN_EUNSUPPORTED;
   constexpr int64_t kBudget = 8704 - 16;  // floats for input + output ranges: 34 KB with the phase skews, six CTAs per SM
   const int64_t planes = (int64_t)g.N * g.C;
@@ -361,27 +493,22 @@ int launch_transform_tile(const float* in, float* out, const Geometry& g, cudaSt
   P.magic_QW = magic_for((uint32_t)P.QW);
   P.magic_MQ = magic_for((uint32_t)units_plane);
   P.off_out = (uint32_t)((in_floats * 4 + 127) / 128 * 128);
-  P.off_bar = P.off_out + (uint32_t)((out_floats * 4 + 15) / 16 * 16);
+  P.off_bar = P.off_out + (uint32_t)((out_floats * (out16 ? 2 : 4) + 15) / 16 * 16);
   const size_t smem = P.off_bar + 16;
   switch (g.Fh) {
-    case 1: return launch_tile_fh<1>(P, ctas, smem, st);
-    case 2: return launch_tile_fh<2>(P, ctas, smem, st);
-    case 3: return launch_tile_fh<3>(P, ctas, smem, st);
-    case 4: return launch_tile_fh<4>(P, ctas, smem, st);
-    case 5: return launch_tile_fh<5>(P, ctas, smem, st);
-    case 7: return launch_tile_fh<7>(P, ctas, smem, st);
-    default: return launch_tile_fh<11>(P, ctas, smem, st);
+    case 1: return out16 ? launch_tile_fh<1, true>(P, ctas, smem, st) : launch_tile_fh<1, false>(P, ctas, smem, st);
+    case 2: return out16 ? launch_tile_fh<2, true>(P, ctas, smem, st) : launch_tile_fh<2, false>(P, ctas, smem, st);
+    case 3: return out16 ? launch_tile_fh<3, true>(P, ctas, smem, st) : launch_tile_fh<3, false>(P, ctas, smem, st);
+    case 4: return out16 ? launch_tile_fh<4, true>(P, ctas, smem, st) : launch_tile_fh<4, false>(P, ctas, smem, st);
+    case 5: return out16 ? launch_tile_fh<5, true>(P, ctas, smem, st) : launch_tile_fh<5, false>(P, ctas, smem, st);
+    case 7: return out16 ? launch_tile_fh<7, true>(P, ctas, smem, st) : launch_tile_fh<7, false>(P, ctas, smem, st);
+    default: return out16 ? launch_tile_fh<11, true>(P, ctas, smem, st) : launch_tile_fh<11, false>(P, ctas, smem, st);
   }
 }
 
-int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_t st) {
-  {
-    const char* old = getenv("IM2WIN_TRANSFORM_GATHER");
-    if (!(old && old[0] == '1')) {
-      const int rc = launch_transform_tile(in, out, g, st);
-      if (rc != IM2WIN_EUNSUPPORTED) return rc;
-    }
-  }
+// Staged-gather path (and, for rows too long to stage, the per-element kernel), writing fp32 (`out`)
+// or, when `out16` is given, the bf16 storage variant.
+static int launch_transform_staged(const float* in, float* out, uint16_t* out16, const Geometry& g, cudaStream_t st) {
   // Shared-memory budget for the staged input rows.  Small enough for several CTAs per SM so that
   // one CTA's loads overlap another's stores.
   constexpr int32_t kTileFloats = 8192 - 4;      // 32 KB including the phase skew
@@ -392,7 +519,8 @@ int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_
   if (row_floats > kTileFloatsMax) {
     const int64_t blocks = (g.n_win + kThreads - 1) / kThreads;
     const int grid = (int)(blocks < 148 * 64 ? blocks : 148 * 64);
-    transform_gather_kernel<<<grid, kThreads, 0, st>>>(in, out, g.H, g.W, g.Fh, g.s, g.Ho, g.n_win);
+    if (out16) transform_gather_bf16_kernel<<<grid, kThreads, 0, st>>>(in, out16, g.H, g.W, g.Fh, g.s, g.Ho, g.n_win);
+    else transform_gather_kernel<<<grid, kThreads, 0, st>>>(in, out, g.H, g.W, g.Fh, g.s, g.Ho, g.n_win);
     return cuda_status(cudaGetLastError());
   }
   const int32_t budget = row_floats > kTileFloats ? kTileFloatsMax : kTileFloats;
@@ -421,12 +549,13 @@ int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_
   if (range * g.HoL >= ((int64_t)1 << 32) || ctas > INT32_MAX || smem > 200 * 1024) {
     const int64_t blocks = (g.n_win + kThreads - 1) / kThreads;
     const int grid = (int)(blocks < 148 * 64 ? blocks : 148 * 64);
-    transform_gather_kernel<<<grid, kThreads, 0, st>>>(in, out, g.H, g.W, g.Fh, g.s, g.Ho, g.n_win);
+    if (out16) transform_gather_bf16_kernel<<<grid, kThreads, 0, st>>>(in, out16, g.H, g.W, g.Fh, g.s, g.Ho, g.n_win);
+    else transform_gather_kernel<<<grid, kThreads, 0, st>>>(in, out, g.H, g.W, g.Fh, g.s, g.Ho, g.n_win);
     return cuda_status(cudaGetLastError());
   }
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(transform_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    cudaError_t e = out16 ? cudaFuncSetAttribute(transform_smem_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                          : cudaFuncSetAttribute(transform_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return IM2WIN_ECUDA;
   }
   TransformParams P;
@@ -437,8 +566,31 @@ int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_
   P.magic_L = magic_for((uint32_t)g.L);
   P.magic_Fh = magic_for((uint32_t)g.Fh);
   P.magic_HoL = magic_for((uint32_t)g.HoL);
-  transform_smem_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(P);
+  if (out16) transform_smem_bf16_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(P, out16);
+  else transform_smem_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(P);
   return cuda_status(cudaGetLastError());
+}
+
+int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_t st) {
+  {
+    const char* old = getenv("IM2WIN_TRANSFORM_GATHER");
+    if (!(old && old[0] == '1')) {
+      const int rc = launch_transform_tile(in, out, false, g, st);
+      if (rc != IM2WIN_EUNSUPPORTED) return rc;
+    }
+  }
+  return launch_transform_staged(in, out, nullptr, g, st);
+}
+
+int launch_transform_bf16(const float* in, uint16_t* out, const Geometry& g, cudaStream_t st) {
+  {
+    const char* old = getenv("IM2WIN_TRANSFORM_GATHER");
+    if (!(old && old[0] == '1')) {
+      const int rc = launch_transform_tile(in, out, true, g, st);
+      if (rc != IM2WIN_EUNSUPPORTED) return rc;
+    }
+  }
+  return launch_transform_staged(in, nullptr, out, g, st);
 }
 
 }  // namespace im2win
