@@ -37,7 +37,7 @@ UNIT = "TFLOP/s"
 NOMINAL_TF32_OVER_BF16 = 1.1 / 2.25
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (conv_tc_persistent__*.md)
-NCU_TRAFFIC_BYTES = {("resnet3x3", "tf32"): 319.51e6 + 79.85e6, ("deep3x3", "bf16"): 89.36e6 + 3.90e6, ("stem7x7", "tf32"): 277.08e6 + 350.73e6, ("down3x3", "tf32"): 323.06e6 + 74.49e6}
+NCU_TRAFFIC_BYTES = {("resnet3x3", "tf32"): 319.57e6 + 81.23e6, ("deep3x3", "bf16"): 89.40e6 + 4.28e6, ("stem7x7", "tf32"): 277.09e6 + 352.88e6, ("down3x3", "tf32"): 322.88e6 + 73.69e6}
 
 
 def _peaks():
