@@ -2,11 +2,17 @@
 //
 // Same GEMM view as the generic kernel (M = output positions, N = filters, K = (r,u,v); A = windows in
 // TENSOR MEMORY written by tcgen05.st, B = filters in shared memory, fp32 accumulators in TMEM), with
-//   * one persistent CTA per SM walking tiles t, t+grid, ... (neighbouring CTAs work on neighbouring
-//     tiles at the same time, so the few strip floats two tiles share are L2 hits);
-//   * the filter operand either RESIDENT in shared memory for the whole kernel (built once per CTA
-//     from the native K,C,Fh,Fw order; any shape, TF32 or BF16) or STREAMED per tile by TMA tensor
-//     loads straight from the native filter viewed as a K x (C*Fh*Fw) matrix (TF32, 128-byte swizzle);
+//   * one persistent CTA per SM walking work units t, t+grid, ... (neighbouring CTAs work on
+//     neighbouring tiles at the same time, so the few strip floats two tiles share are L2 hits);
+//     tiles are cut per image where that wastes little (one contiguous source range per channel,
+//     one 2-D TMA box per channel group where it fits), else they may span images;
+//   * the filter operand either RESIDENT in shared memory for the whole kernel (fetched by TMA with
+//     the 32-byte swizzle where the native order serves as is, else built once per CTA from the
+//     native K,C,Fh,Fw order; any shape, TF32 or BF16) or STREAMED per tile by TMA tensor loads
+//     straight from the native filter viewed as a K x (C*Fh*Fw) matrix (128-byte swizzle);
+//   * a unit's channel groups optionally cut into reduction slices that add into a zeroed output
+//     (under-filled launches); the strip source optionally a bf16 im2win tensor or (fused) the
+//     untransformed input;
 //   * filter sizes known at compile time, so a window's elements are loads at immediate offsets from
 //     one per-thread, per-channel base address (the window is contiguous in its im2win strip);
 //   * A columns handed to the MMA thread in sub-slots of a ring in TMEM, independent of the channel
