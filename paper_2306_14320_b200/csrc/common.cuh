@@ -36,6 +36,7 @@ enum : int32_t {
   DEV_TIMEOUT_B_EMPTY = 106,    // filter loaders waiting for a free stage
   DEV_TIMEOUT_ACC = 107,        // epilogue waiting for the accumulator
   DEV_TIMEOUT_DRAIN = 108,      // teardown waiting for copies in flight
+  DEV_TIMEOUT_COPY = 109,       // transform waiting for the bulk copy of its input range
   DEV_RANGE = 201               // an internal index check failed
 };
 int32_t* device_status_word();  // device address of the status word (nullptr if no device)

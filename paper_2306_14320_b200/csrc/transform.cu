@@ -266,6 +266,7 @@ struct TileParams {
   int64_t planes, HW, HoL, n_in_total;
   uint64_t magic_QW;    // ceil(2^32 / QW)
   uint64_t magic_MQ;    // ceil(2^32 / (rows per plane in the job * QW))
+  int32_t test_skip_copy;  // test hook, see the kernel
   uint32_t off_out;     // byte offset of the output buffer in shared memory
   uint32_t off_bar;     // byte offset of the mbarrier
 };
@@ -310,18 +311,28 @@ __global__ void __launch_bounds__(kThreads) transform_tile_kernel(const TilePara
     ptx::mbar_init(bar_a, 1);
     ptx::fence_mbar_init();
     ptx::mbar_arrive_expect_tx(bar_a, (uint32_t)nfl * 4u);
-    if (nfl > 0) ptx::bulk_g2s(ptx::smem_u32(tin0), P.in + a0, (uint32_t)nfl * 4u, bar_a);
+    // (test hook: with test_skip_copy the copy is announced but never issued, so that the expiry
+    // path of the bounded wait below can be exercised by a kernel that neither faults nor hangs)
+    if (nfl > 0 && !P.test_skip_copy) ptx::bulk_g2s(ptx::smem_u32(tin0), P.in + a0, (uint32_t)nfl * 4u, bar_a);
   }
   if ((int32_t)threadIdx.x < ntail) tin0[nfl + threadIdx.x] = __ldg(P.in + a0 + nfl + threadIdx.x);
   __syncthreads();  // the barrier is initialised for everyone; the tail floats are in place
   {
-    bool landed = false;
-    for (uint32_t it = 0; it < (1u << 24) && !landed; ++it) {
+    // bounded wait: about a second by the global timer (and an iteration cap), then report and leave
+    bool landed = ptx::mbar_try_wait(bar_a, 0u);
+    uint64_t t0 = 0;
+    for (uint32_t it = 0; it < (1u << 22) && !landed; ++it) {
+      __nanosleep(64);
       landed = ptx::mbar_try_wait(bar_a, 0u);
-      if (!landed && it > 64) __nanosleep(64);
+      if ((it & 63u) == 63u && !landed) {
+        uint64_t now;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > 1000000000ull) break;
+      }
     }
-    if (!__all_sync(0xffffffffu, landed)) {  // about a second without the copy: report and leave
-      if ((threadIdx.x & 31) == 0) atomicCAS(P.status, 0, (int32_t)DEV_TIMEOUT_DRAIN);
+    if (!__all_sync(0xffffffffu, landed)) {
+      if ((threadIdx.x & 31) == 0) atomicCAS(P.status, 0, (int32_t)DEV_TIMEOUT_COPY);
       return;
     }
   }
@@ -487,6 +498,11 @@ int launch_transform_tile(const float* in, void* out, bool out16, const Geometry
   P.H = g.H; P.W = g.W; P.s = g.s; P.Ho = g.Ho; P.L = g.L;
   P.MB = MB; P.nblk = nblk; P.PB = PB;
   P.QW = (g.W + 3) / 4;
+  {
+    // honoured for single-CTA problems only: every CTA would wait out its own second otherwise
+    const char* hook = getenv("IM2WIN_TEST_SKIP_COPY");
+    P.test_skip_copy = (hook && hook[0] == '1' && ctas == 1) ? 1 : 0;
+  }
   P.planes = planes; P.HW = hw; P.HoL = g.HoL; P.n_in_total = g.n_in;
   const int64_t units_plane = (int64_t)(nblk == 1 ? g.Ho : MB) * P.QW;
   if (units_plane * PB * units_plane >= ((int64_t)1 << 32)) return IM2WIN_EUNSUPPORTED;  // reciprocal division exact
