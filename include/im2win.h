@@ -120,6 +120,17 @@ int im2win_conv(const void* src, int src_kind, const float* filter_kcfhfw,
                 const im2win_shape* shape, int mode, float* out_nchw,
                 void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Output-storage variant of im2win_conv (no counterpart in the paper, whose outputs are fp32):
+ * the same result rounded to bf16 (nearest even) from the fp32 accumulators, NCHW, 2 bytes per
+ * element: half the output footprint and half the bytes written.
+ * out_nchw_bf16: device, N*K*Ho*Wo 16-bit words, every element is written; 16-byte aligned.
+ * Everything else as im2win_conv.  Tensor-core modes only (IM2WIN_MODE_FP32: EINVAL), and only
+ * shapes with a filter-size specialisation (EUNSUPPORTED otherwise: the generic kernel has no
+ * bf16 epilogue). */
+int im2win_conv_bf16out(const void* src, int src_kind, const float* filter_kcfhfw,
+                        const im2win_shape* shape, int mode, uint16_t* out_nchw_bf16,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* HOST-buffer convenience for callers without device memory of their own: copies the input and
  * the filter from host memory, runs transform + convolution on an internal stream and copies the
  * result back; returns after the result is in out_host.  Device buffers are owned by the library,

@@ -146,9 +146,13 @@ int im2win_transform_bf16(const float* in_nchw, const im2win_shape* shape, uint1
   return launch_transform_bf16(in_nchw, out_im2win_bf16, g, static_cast<cudaStream_t>(cuda_stream));
 }
 
-int im2win_conv(const void* src, int src_kind, const float* filter, const im2win_shape* shape,
-                int mode, float* out_nchw, void* workspace, size_t workspace_bytes,
-                void* cuda_stream) {
+// Shared body of im2win_conv (fp32 output) and im2win_conv_bf16out (out16: `out` holds 16-bit words;
+// tensor-core modes and the specialised kernel only).
+static int conv_impl(const void* src, int src_kind, const float* filter, const im2win_shape* shape,
+                     int mode, void* out, bool out16, void* workspace, size_t workspace_bytes,
+                     void* cuda_stream) {
+  float* const out_nchw = static_cast<float*>(out);
+  const int64_t out_es = out16 ? 2 : 4;
   Geometry g;
   int rc = make_geometry(shape, &g);
   if (rc != IM2WIN_OK) return rc;
@@ -159,21 +163,23 @@ int im2win_conv(const void* src, int src_kind, const float* filter, const im2win
   if (src_kind == IM2WIN_SRC_IM2WIN_BF16 && mode != IM2WIN_MODE_BF16) return IM2WIN_EINVAL;
   if (mode != IM2WIN_MODE_TF32 && mode != IM2WIN_MODE_BF16 && mode != IM2WIN_MODE_FP32)
     return IM2WIN_EINVAL;
+  if (out16 && mode == IM2WIN_MODE_FP32) return IM2WIN_EINVAL;
   if (!aligned16(src) || !aligned16(filter) || !aligned16(out_nchw)) return IM2WIN_EALIGN;
   const int64_t src_bytes = src_kind == IM2WIN_SRC_IM2WIN_BF16 ? g.n_win * 2
                                                                 : (src_kind == IM2WIN_SRC_IM2WIN ? g.n_win : g.n_in) * 4;
-  if (overlap(out_nchw, g.n_out * 4, src, src_bytes) || overlap(out_nchw, g.n_out * 4, filter, g.n_flt * 4))
+  if (overlap(out_nchw, g.n_out * out_es, src, src_bytes) || overlap(out_nchw, g.n_out * out_es, filter, g.n_flt * 4))
     return IM2WIN_EOVERLAP;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (src_kind == IM2WIN_SRC_IM2WIN_BF16)  // no generic-kernel fallback for this storage variant
     return launch_conv_tc_persistent(src, filter, out_nchw, g, mode, st, /*may_alloc=*/true, /*fused=*/false,
-                                     /*src_bf16=*/true);
+                                     /*src_bf16=*/true, out16);
   const float* xhat = static_cast<const float*>(src);
   if (src_kind == IM2WIN_SRC_NCHW_FUSED) {
     if (mode != IM2WIN_MODE_FP32) {
       const char* force = getenv("IM2WIN_FORCE_GENERIC");
       if (!(force && force[0] == '1')) {
-        rc = launch_conv_tc_persistent(xhat, filter, out_nchw, g, mode, st, /*may_alloc=*/true, /*fused=*/true);
+        rc = launch_conv_tc_persistent(xhat, filter, out_nchw, g, mode, st, /*may_alloc=*/true, /*fused=*/true,
+                                       /*src_bf16=*/false, out16);
         if (rc != IM2WIN_EUNSUPPORTED) return rc;
       }
     }
@@ -185,15 +191,30 @@ int im2win_conv(const void* src, int src_kind, const float* filter, const im2win
     if (!workspace || workspace_bytes < (size_t)g.n_win * 4) return IM2WIN_EWORKSPACE;
     if (!aligned16(workspace)) return IM2WIN_EALIGN;
     if (overlap(workspace, g.n_win * 4, src, src_bytes) ||
-        overlap(workspace, g.n_win * 4, out_nchw, g.n_out * 4) ||
+        overlap(workspace, g.n_win * 4, out_nchw, g.n_out * out_es) ||
         overlap(workspace, g.n_win * 4, filter, g.n_flt * 4))
       return IM2WIN_EOVERLAP;
     rc = launch_transform(static_cast<const float*>(src), static_cast<float*>(workspace), g, st);
     if (rc != IM2WIN_OK) return rc;
     xhat = static_cast<const float*>(workspace);
   }
+  if (out16)  // only the specialised kernel has the bf16 epilogue
+    return launch_conv_tc_persistent(xhat, filter, out_nchw, g, mode, st, /*may_alloc=*/true, /*fused=*/false,
+                                     /*src_bf16=*/false, true);
   if (mode == IM2WIN_MODE_FP32) return launch_conv_fp32(xhat, filter, out_nchw, g, st);
   return launch_conv_tc(xhat, filter, out_nchw, g, mode, st);
+}
+
+int im2win_conv(const void* src, int src_kind, const float* filter, const im2win_shape* shape,
+                int mode, float* out_nchw, void* workspace, size_t workspace_bytes,
+                void* cuda_stream) {
+  return conv_impl(src, src_kind, filter, shape, mode, out_nchw, false, workspace, workspace_bytes, cuda_stream);
+}
+
+int im2win_conv_bf16out(const void* src, int src_kind, const float* filter, const im2win_shape* shape,
+                        int mode, uint16_t* out_nchw_bf16, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+  return conv_impl(src, src_kind, filter, shape, mode, out_nchw_bf16, true, workspace, workspace_bytes, cuda_stream);
 }
 
 int im2win_last_device_status(void* cuda_stream, int32_t* status) {

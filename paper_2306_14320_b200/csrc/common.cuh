@@ -48,7 +48,7 @@ int launch_conv_fp32(const float* xhat, const float* f, float* out, const Geomet
 // Tensor-core convolution: the persistent specialised kernel when one applies (it returns
 // IM2WIN_EUNSUPPORTED otherwise), else the generic kernel.
 int launch_conv_tc_persistent(const void* src, const float* f, float* out, const Geometry& g, int mode,
-                              cudaStream_t st, bool may_alloc, bool fused = false, bool src_bf16 = false);
+                              cudaStream_t st, bool may_alloc, bool fused = false, bool src_bf16 = false, bool out_bf16 = false);
 int launch_conv_tc_generic(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
                            cudaStream_t st);
 // may_alloc = false keeps the call free of any (even stream-ordered) device allocation.

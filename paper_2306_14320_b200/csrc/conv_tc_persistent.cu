@@ -102,11 +102,6 @@ struct SegR {
   int32_t dst_off;
 };
 
-__device__ __forceinline__ void record(const PParams& P, PMisc* misc, int32_t code) {
-  atomicCAS(P.status, 0, code);
-  atomicExch(&misc->abort, 1);
-}
-
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -344,7 +339,7 @@ __device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int32_t 
   asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
 }
 
-template <int FH, int FW, int CB, bool BF16, bool BRES, bool FUSED, bool SRC16>
+template <int FH, int FW, int CB, bool BF16, bool BRES, bool FUSED, bool SRC16, bool OUT16>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap fmap,
                           const __grid_constant__ CUtensorMap xmap) {
@@ -960,8 +955,9 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     // into the zeroed output.  A choice inside the store loop, or an out-of-line call next to it,
     // slowed the C = 3 stem layers, which this loop bounds, by 20 %.
     PROF_DECL(6)
-    auto epilogue_role = [&](auto reduce_tag) {
-      constexpr bool REDUCE = decltype(reduce_tag)::value;
+    auto epilogue_role = [&](auto kind_tag) {
+      constexpr int EK = decltype(kind_tag)::value;  // 0 fp32 stores, 1 fp32 reductions, 2 bf16 stores
+      constexpr bool REDUCE = EK == 1;
       Ring dr;
       bool ok = true;
       const int32_t eK = P.K, eNT = P.NT, eHoWo = P.HoWo;  // kept in registers for the store loop
@@ -1006,6 +1002,21 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           PROF_ADD(2, t1)
           ptx::tmem_zero_x16(d_tmem + (uint32_t)c0);  // leave the columns zeroed for the next tile
           PROF_T0(t3)
+          if constexpr (EK == 2) {
+            // bf16 output: every lane rounds its own value and stores 16 bits; the 32 lanes of a
+            // warp write 64 contiguous bytes per filter.  (Pairing neighbouring positions into 32-bit
+            // stores through shuffles was slower: this loop is bound by its instruction count.)
+            if (valid) {
+              uint16_t* const o16 = reinterpret_cast<uint16_t*>(P.out) + (orow - P.out) + (int64_t)c0 * eHoWo;
+              const int32_t left = eK - n0 - c0;
+#pragma unroll
+              for (int e = 0; e < 16; e += 2) {
+                const uint32_t pk = ptx::pack_bf16x2(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+                if (e < left) o16[(int64_t)e * eHoWo] = (uint16_t)(pk & 0xffffu);
+                if (e + 1 < left) o16[(int64_t)(e + 1) * eHoWo] = (uint16_t)(pk >> 16);
+              }
+            }
+          } else
           if (valid) {
             float* o = orow + (int64_t)c0 * eHoWo;
             const int32_t left = eK - n0 - c0;  // filters of this block that exist
@@ -1027,8 +1038,12 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         PROF_ADD(5, t4)
       }
     };
-    if (P.Z == 1) epilogue_role(std::false_type{});
-    else epilogue_role(std::true_type{});
+    if constexpr (OUT16) {  // (separate instantiations: the fp32 kernels' code is not touched by this variant)
+      epilogue_role(std::integral_constant<int, 2>{});
+    } else {
+      if (P.Z == 1) epilogue_role(std::integral_constant<int, 0>{});
+      else epilogue_role(std::integral_constant<int, 1>{});
+    }
     if (q4 == 0) { PROF_DUMP(6, 6) }
   }
 
@@ -1113,8 +1128,9 @@ int sm_count() {
   return n;
 }
 
-template <int FH, int FW, int CB, bool BF16, bool FUSED, bool SRC16 = false>
+template <int FH, int FW, int CB, bool BF16, bool FUSED, bool SRC16 = false, bool OUT16 = false>
 int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc) {
+  constexpr bool out16 = OUT16;
   constexpr int FF = FH * FW;
   constexpr int64_t ES = SRC16 ? 2 : 4;    // bytes per source element
   constexpr int64_t EPC = 16 / ES;         // source elements per 16-byte chunk
@@ -1124,7 +1140,7 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   constexpr int S = KCGP / KSTEP;
 
   PParams P{};
-  P.xhat = xhat; P.f = f; P.out = out;
+  P.xhat = xhat; P.f = f; P.out = out;  // (OUT16: `out` points at 16-bit words)
   P.status = device_status_word();
   if (!P.status) return IM2WIN_ECUDA;
 #ifdef IM2WIN_PROF
@@ -1278,6 +1294,7 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
     double best = cost(1, P.NG) * 0.92;  // a split must win clearly
     int forced = -1;
     if (const char* fix = getenv("IM2WIN_SPLITK")) forced = atoi(fix);
+    if (out16) forced = 1;  // partial sums cannot be added into a bf16 output
     for (int32_t z = 2; z <= 16 && z <= P.NG; ++z) {
       int32_t gz = (P.NG + z - 1) / z;
       gz = (gz + gmul - 1) / gmul * gmul;
@@ -1358,18 +1375,18 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   }
   const int64_t grid = P.ntiles < sm_count() ? P.ntiles : sm_count();
   cudaError_t e;
-  if (P.Z > 1 && cudaMemsetAsync(out, 0, (size_t)g.n_out * 4, st) != cudaSuccess) {
+  if (P.Z > 1 && cudaMemsetAsync(out, 0, (size_t)g.n_out * 4, st) != cudaSuccess) {  // (Z > 1 implies an fp32 output)
     cudaGetLastError();
     if (f_bf16) cudaFreeAsync(f_bf16, st);
     return IM2WIN_ECUDA;
   }
   if (resident) {
-    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, true, FUSED, SRC16>;
+    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, true, FUSED, SRC16, OUT16>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
     kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
   } else {
-    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, false, FUSED, SRC16>;
+    auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, false, FUSED, SRC16, OUT16>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) { cudaGetLastError(); if (f_bf16) cudaFreeAsync(f_bf16, st); return IM2WIN_ECUDA; }
     kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
@@ -1382,7 +1399,15 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
 // src_kind: 0 = im2win tensor (fp32), 1 = untransformed input consumed fused, 2 = im2win tensor stored as bf16
 template <int FH, int FW, int CB, bool BF16>
 int launch_spec(const void* src, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc,
-                int src_kind) {
+                int src_kind, bool out16) {
+  if (out16) {  // the bf16 epilogue exists for the unfused sources
+    if (src_kind == 1) return IM2WIN_EUNSUPPORTED;
+    if (src_kind == 2) {
+      if constexpr (BF16) return launch_spec_impl<FH, FW, CB, true, false, true, true>(src, f, out, g, st, may_alloc);
+      else return IM2WIN_EUNSUPPORTED;
+    }
+    return launch_spec_impl<FH, FW, CB, BF16, false, false, true>(src, f, out, g, st, may_alloc);
+  }
   if (src_kind == 2) {
     if constexpr (BF16) return launch_spec_impl<FH, FW, CB, true, false, true>(src, f, out, g, st, may_alloc);
     else return IM2WIN_EUNSUPPORTED;
@@ -1398,39 +1423,74 @@ int launch_spec(const void* src, const float* f, float* out, const Geometry& g, 
 // BF16 copy of a filter that is too large to stay in shared memory).
 // fused: `xhat` is the untransformed NCHW input and the windows are built from staged input rows
 // (no im2win tensor exists in global memory).
+// The filter-size families are separate functions so that the build can compile them as separate
+// translation units in parallel (-DIM2WIN_PART=0..3: part 0 = 3x3 + this dispatcher, 1 = 5x5,
+// 2 = 7x7, 3 = 11x11; without the macro everything is compiled here).
+#ifndef IM2WIN_PART
+#define IM2WIN_PART -1
+#endif
+#define IM2WIN_SPEC_ARGS const void* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st, \
+                         bool may_alloc, int kind, bool out_bf16, bool bf16
+int launch_spec_3x3(IM2WIN_SPEC_ARGS);
+int launch_spec_5x5(IM2WIN_SPEC_ARGS);
+int launch_spec_7x7(IM2WIN_SPEC_ARGS);
+int launch_spec_11x11(IM2WIN_SPEC_ARGS);
+
+#if IM2WIN_PART == -1 || IM2WIN_PART == 0
+int launch_spec_3x3(IM2WIN_SPEC_ARGS) {
+  // BF16 MMAs take 16 reduction elements: sixteen channels (144 = 9 steps) leave no padding
+  if (bf16 && g.C % 16 == 0) return launch_spec<3, 3, 16, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  if (g.C >= 8) return bf16 ? launch_spec<3, 3, 8, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16)
+                            : launch_spec<3, 3, 8, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  if (g.C == 3) return bf16 ? launch_spec<3, 3, 3, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16)
+                            : launch_spec<3, 3, 3, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  return IM2WIN_EUNSUPPORTED;
+}
+#endif
+#if IM2WIN_PART == -1 || IM2WIN_PART == 1
+int launch_spec_5x5(IM2WIN_SPEC_ARGS) {
+  if (bf16 && g.C % 16 == 0) return launch_spec<5, 5, 16, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  if (g.C >= 8) return bf16 ? launch_spec<5, 5, 8, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16)
+                            : launch_spec<5, 5, 8, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  return IM2WIN_EUNSUPPORTED;
+}
+#endif
+#if IM2WIN_PART == -1 || IM2WIN_PART == 2
+int launch_spec_7x7(IM2WIN_SPEC_ARGS) {
+  if (g.C % 8 == 0) {
+    if (bf16 && g.C % 16 == 0) return launch_spec<7, 7, 16, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+    if (!bf16) return launch_spec<7, 7, 8, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  }
+  if (g.C == 3) return bf16 ? launch_spec<7, 7, 3, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16)
+                            : launch_spec<7, 7, 3, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  return IM2WIN_EUNSUPPORTED;
+}
+#endif
+#if IM2WIN_PART == -1 || IM2WIN_PART == 3
+int launch_spec_11x11(IM2WIN_SPEC_ARGS) {
+  if (g.C <= 4) return bf16 ? launch_spec<11, 11, 1, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16)
+                            : launch_spec<11, 11, 1, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  return IM2WIN_EUNSUPPORTED;
+}
+#endif
+
+#if IM2WIN_PART == -1 || IM2WIN_PART == 0
 int launch_conv_tc_persistent(const void* xhat, const float* f, float* out, const Geometry& g, int mode,
-                              cudaStream_t st, bool may_alloc, bool fused, bool src_bf16) {
+                              cudaStream_t st, bool may_alloc, bool fused, bool src_bf16, bool out_bf16) {
   const int kind = src_bf16 ? 2 : (fused ? 1 : 0);
   if (src_bf16 && (fused || mode != IM2WIN_MODE_BF16)) return IM2WIN_EUNSUPPORTED;
   const bool bf16 = mode == IM2WIN_MODE_BF16;
-  if (g.Fh == 3 && g.Fw == 3) {
-    // BF16 MMAs take 16 reduction elements: sixteen channels (144 = 9 steps) leave no padding
-    if (bf16 && g.C % 16 == 0) return launch_spec<3, 3, 16, true>(xhat, f, out, g, st, may_alloc, kind);
-    if (g.C >= 8) return bf16 ? launch_spec<3, 3, 8, true>(xhat, f, out, g, st, may_alloc, kind)
-                              : launch_spec<3, 3, 8, false>(xhat, f, out, g, st, may_alloc, kind);
-    if (g.C == 3) return bf16 ? launch_spec<3, 3, 3, true>(xhat, f, out, g, st, may_alloc, kind)
-                              : launch_spec<3, 3, 3, false>(xhat, f, out, g, st, may_alloc, kind);
-  }
-  if (g.Fh == 5 && g.Fw == 5) {
-    if (bf16 && g.C % 16 == 0) return launch_spec<5, 5, 16, true>(xhat, f, out, g, st, may_alloc, kind);
-    if (g.C >= 8) return bf16 ? launch_spec<5, 5, 8, true>(xhat, f, out, g, st, may_alloc, kind)
-                              : launch_spec<5, 5, 8, false>(xhat, f, out, g, st, may_alloc, kind);
-  }
-  if (g.Fh == 7 && g.Fw == 7 && g.C % 8 == 0) {
-    if (bf16 && g.C % 16 == 0) return launch_spec<7, 7, 16, true>(xhat, f, out, g, st, may_alloc, kind);
-    if (!bf16) return launch_spec<7, 7, 8, false>(xhat, f, out, g, st, may_alloc, kind);
-  }
-  if (g.Fh == 7 && g.Fw == 7 && g.C == 3)
-    return bf16 ? launch_spec<7, 7, 3, true>(xhat, f, out, g, st, may_alloc, kind)
-                : launch_spec<7, 7, 3, false>(xhat, f, out, g, st, may_alloc, kind);
-  if (g.Fh == 11 && g.Fw == 11 && g.C <= 4)
-    return bf16 ? launch_spec<11, 11, 1, true>(xhat, f, out, g, st, may_alloc, kind)
-                : launch_spec<11, 11, 1, false>(xhat, f, out, g, st, may_alloc, kind);
+  if (g.Fh == 3 && g.Fw == 3) return launch_spec_3x3(xhat, f, out, g, st, may_alloc, kind, out_bf16, bf16);
+  if (g.Fh == 5 && g.Fw == 5) return launch_spec_5x5(xhat, f, out, g, st, may_alloc, kind, out_bf16, bf16);
+  if (g.Fh == 7 && g.Fw == 7) return launch_spec_7x7(xhat, f, out, g, st, may_alloc, kind, out_bf16, bf16);
+  if (g.Fh == 11 && g.Fw == 11) return launch_spec_11x11(xhat, f, out, g, st, may_alloc, kind, out_bf16, bf16);
   return IM2WIN_EUNSUPPORTED;
 }
 
 #ifdef IM2WIN_PROF
+// (debug build only; with the parts compiled separately the counters cover part 0's kernels)
 extern "C" void im2win_debug_set_prof(long long* device_buf) { g_prof = device_buf; }
 #endif
+#endif  // IM2WIN_PART == -1 || IM2WIN_PART == 0
 
 }  // namespace im2win

@@ -139,3 +139,75 @@ def test_bf16_source_argument_checks():
     with pytest.raises(b.Im2winError) as e:
         b.conv(s16.view, b.SRC_IM2WIN_BF16, sf, sd, b.MODE_BF16, sout)
     assert e.value.code == b.EUNSUPPORTED
+
+
+# ------------------------------------------------------------------ bf16 OUTPUT (im2win_conv_bf16out)
+
+def _bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def gpu_conv_bf16out(x: np.ndarray, f: np.ndarray, dims, mode: int, src_kind: int) -> np.ndarray:
+    n, c, h, w, k, fh, fw, s = dims
+    ho, wo = b.out_dims(dims)
+    xd = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda()
+    fd = torch.from_numpy(np.ascontiguousarray(f, dtype=np.float32)).cuda()
+    out = Guarded16(n * k * ho * wo)
+    ws = Guarded(b.workspace_bytes(dims) // 4) if src_kind in (b.SRC_NCHW, b.SRC_NCHW_FUSED) else None
+    b.conv_bf16out(xd, src_kind, fd, dims, mode, out.view, None if ws is None else ws.view,
+                   0 if ws is None else ws.n * 4)
+    assert b.last_device_status() == 0
+    if ws is not None:
+        ws.check()
+    return out.check().reshape(n, k, ho, wo)
+
+
+# tolerance: the mode's own, plus the rounding of the result to bf16 (relative 2^-9 at most)
+TOL_OUT = {b.MODE_TF32: 5e-3 + 2.0 ** -9, b.MODE_BF16: 2e-2 + 2.0 ** -9}
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=["tf32", "bf16"])
+@pytest.mark.parametrize("src_kind", [b.SRC_NCHW, b.SRC_NCHW_FUSED], ids=["nchw", "fused"])
+@pytest.mark.parametrize("name,batch", [("tiny", 1), ("resnet3x3", 3), ("stem7x7", 1), ("deep3x3", 3), ("down3x3", 2),
+                                        ("sweep_L1", 1), ("sweep_L2", 1), ("sweep_L12", 2)])
+def test_conv_bf16_output(name, batch, src_kind, mode):
+    """Odd and even images sizes (tiny: 30x30 outputs; sweep_L1: 55x55, odd; sweep_L12: 7x7 with tiles
+    that span images), resident and streamed filters."""
+    layer = wl.CONFIGS[name].with_batch(batch)
+    dims = layer.dims()
+    x, f = wl.make_input(layer), wl.make_filter(layer)
+    got = _bf16_bits_to_f64(gpu_conv_bf16out(x, f, dims, mode, src_kind))
+    assert rel_l2(got, oracle_conv(x, f, dims)) <= TOL_OUT[mode]
+
+
+@pytest.mark.parametrize("dims", [(2, 16, 30, 30, 32, 3, 3, 1), (3, 8, 21, 23, 40, 3, 3, 2), (2, 3, 37, 35, 24, 7, 7, 2)])
+def test_conv_bf16_output_small_integers_bit_exact(dims):
+    """Exact fp32 sums (small integers): the stored words must be the oracle's Eq. (1) rounded to bf16."""
+    n, c, h, w, k, fh, fw, s = dims
+    x = wl.small_ints(21, n * c * h * w).reshape(n, c, h, w)
+    f = wl.small_ints(22, k * c * fh * fw, -2, 2).reshape(k, c, fh, fw)
+    ref = oracle_conv(x, f, dims).astype(np.float32)
+    for mode in (b.MODE_TF32, b.MODE_BF16):
+        got = gpu_conv_bf16out(x, f, dims, mode, b.SRC_NCHW)
+        assert np.array_equal(got.ravel(), bf16_rne_bits(ref))
+
+
+def test_conv_bf16_output_argument_checks():
+    layer = wl.CONFIGS["tiny"]
+    dims = layer.dims()
+    xd = torch.from_numpy(wl.make_input(layer)).cuda()
+    fd = torch.from_numpy(wl.make_filter(layer)).cuda()
+    ho, wo = b.out_dims(dims)
+    out = torch.empty(layer.N * layer.K * ho * wo, dtype=torch.int16, device="cuda")
+    ws = torch.empty(b.workspace_bytes(dims) // 4, device="cuda")
+    with pytest.raises(b.Im2winError) as e:  # the fp32 check mode has no bf16 output
+        b.conv_bf16out(xd, b.SRC_NCHW, fd, dims, b.MODE_FP32, out, ws)
+    assert e.value.code == b.EINVAL
+    odd = (1, 2, 9, 8, 3, 2, 3, 1)  # 2x3 filter: no specialised kernel, hence no bf16 epilogue
+    n, c, h, w, k, fh, fw, s = odd
+    oh, ow = b.out_dims(odd)
+    with pytest.raises(b.Im2winError) as e:
+        b.conv_bf16out(torch.zeros(n * c * h * w, device="cuda"), b.SRC_NCHW, torch.zeros(k * c * fh * fw, device="cuda"),
+                       odd, b.MODE_TF32, torch.empty(n * k * oh * ow, dtype=torch.int16, device="cuda"),
+                       torch.empty(b.workspace_bytes(odd) // 4, device="cuda"))
+    assert e.value.code == b.EUNSUPPORTED
