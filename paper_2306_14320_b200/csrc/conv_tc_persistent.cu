@@ -1066,6 +1066,20 @@ __global__ void __launch_bounds__(256) filter_to_bf16_kernel(const float* __rest
     o[i] = __float2bfloat16_rn(f[i]);
 }
 
+// The same copy with every channel group's KCG reduction elements padded with zeros to the KCGP the
+// MMA steps cover, so that a filter row is indexed by (group, step) exactly as the kernel counts them.
+__global__ void __launch_bounds__(256) filter_to_bf16_padded_kernel(const float* __restrict__ f,
+                                                                    __nv_bfloat16* __restrict__ o, int64_t n_pad,
+                                                                    int32_t Kg, int32_t KCG, int32_t KCGP, int32_t NG) {
+  const int32_t Kgp = NG * KCGP;
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n_pad; i += (int64_t)gridDim.x * 256) {
+    const int64_t j = i / Kgp;
+    const int32_t r = (int32_t)(i - j * Kgp);
+    const int32_t grp = r / KCGP, kl = r - grp * KCGP;
+    o[i] = kl < KCG ? __float2bfloat16_rn(f[j * Kg + (int64_t)grp * KCG + kl]) : __float2bfloat16_rn(0.f);
+  }
+}
+
 // ---------------------------------------------------------------------------------------------- host side
 
 #ifdef IM2WIN_PROF
@@ -1227,11 +1241,13 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   const int64_t cap = 227 * 1024 - 1024 - 1024 - ((int64_t)(P.win_span + 8) * 4 + 16);  // alignment slack, barriers, zero pad
   const int64_t b_res = (int64_t)steps_tile * P.NT * 32;  // one 32-byte-swizzled block per MMA step
   bool resident = P.n_ntiles == 1 && b_res + 2 * raw_stage <= cap;
-  // Streaming needs dense groups (padded reduction index == real index) and 16-byte aligned filter
-  // rows.  In BF16 mode the TMA source is a bf16 copy of the filter made for the duration of the call
-  // in memory from the stream-ordered pool (only where the caller allows an allocation).
-  const bool can_stream = KCG == KCGP && (g.C % CB) == 0 && (g.Kg % (BF16 ? 8 : 4)) == 0 && encode_fn() != nullptr &&
-                          (!BF16 || may_alloc);
+  // Streaming the native TF32 filter needs dense groups (padded reduction index == real index) and
+  // 16-byte aligned filter rows.  In BF16 mode the TMA source is a bf16 copy of the filter made for
+  // the duration of the call in memory from the stream-ordered pool (only where the caller allows an
+  // allocation); that copy is written with padded groups where the groups are not dense.
+  const bool pad_copy = BF16 && KCG != KCGP;
+  const bool can_stream = (g.C % CB) == 0 && encode_fn() != nullptr &&
+                          (BF16 ? may_alloc && (pad_copy || (g.Kg % 8) == 0) : KCG == KCGP && (g.Kg % 4) == 0);
   if (!resident && !can_stream) return IM2WIN_EUNSUPPORTED;
   int64_t b_bytes;
   if (resident) {
@@ -1335,20 +1351,26 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
       P.b_tma = 1;
   }
   if (!resident) {
-    const cuuint64_t gdim[2] = {(cuuint64_t)g.Kg, (cuuint64_t)g.K};
-    const cuuint64_t gstr[1] = {(cuuint64_t)g.Kg * (BF16 ? 2 : 4)};
+    const int64_t row = pad_copy ? (int64_t)P.NG * KCGP : g.Kg;  // filter row length seen by the TMA
+    const cuuint64_t gdim[2] = {(cuuint64_t)row, (cuuint64_t)g.K};
+    const cuuint64_t gstr[1] = {(cuuint64_t)row * (BF16 ? 2 : 4)};
     const cuuint32_t box[2] = {BF16 ? 64u : 32u, (cuuint32_t)P.NT};  // one 128-byte row of the swizzle
     const cuuint32_t estr[2] = {1, 1};
     void* base = const_cast<float*>(f);
     if (BF16) {
       cudaMemPool_t pool = filter_pool();
-      if (!pool || cudaMallocFromPoolAsync(&f_bf16, (size_t)g.n_flt * 2, pool, st) != cudaSuccess) {
+      const int64_t n_copy = (int64_t)g.K * row;
+      if (!pool || cudaMallocFromPoolAsync(&f_bf16, (size_t)n_copy * 2, pool, st) != cudaSuccess) {
         cudaGetLastError();
         return IM2WIN_EUNSUPPORTED;
       }
-      const int64_t blocks = (g.n_flt + 255) / 256;
-      filter_to_bf16_kernel<<<(unsigned)(blocks < 148 * 8 ? blocks : 148 * 8), 256, 0, st>>>(
-          f, static_cast<__nv_bfloat16*>(f_bf16), g.n_flt);
+      const int64_t blocks = (n_copy + 255) / 256;
+      const unsigned nb = (unsigned)(blocks < 148 * 8 ? blocks : 148 * 8);
+      if (pad_copy)
+        filter_to_bf16_padded_kernel<<<nb, 256, 0, st>>>(f, static_cast<__nv_bfloat16*>(f_bf16), n_copy, (int32_t)g.Kg,
+                                                         KCG, KCGP, P.NG);
+      else
+        filter_to_bf16_kernel<<<nb, 256, 0, st>>>(f, static_cast<__nv_bfloat16*>(f_bf16), g.n_flt);
       base = f_bf16;
     }
     if (encode_fn()(&fmap, BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, gdim,
@@ -1458,8 +1480,15 @@ int launch_spec_5x5(IM2WIN_SPEC_ARGS) {
 #if IM2WIN_PART == -1 || IM2WIN_PART == 2
 int launch_spec_7x7(IM2WIN_SPEC_ARGS) {
   if (g.C % 8 == 0) {
-    if (bf16 && g.C % 16 == 0) return launch_spec<7, 7, 16, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
-    if (!bf16) return launch_spec<7, 7, 8, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+    if (bf16) {
+      // sixteen channels per group leave no padding (784 = 49 steps); where two strip stages of
+      // sixteen channels do not fit (wide images), eight channels with a padded filter copy do
+      int rc = IM2WIN_EUNSUPPORTED;
+      if (g.C % 16 == 0) rc = launch_spec<7, 7, 16, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+      if (rc == IM2WIN_EUNSUPPORTED) rc = launch_spec<7, 7, 8, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+      return rc;
+    }
+    return launch_spec<7, 7, 8, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
   }
   if (g.C == 3) return bf16 ? launch_spec<7, 7, 3, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16)
                             : launch_spec<7, 7, 3, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);

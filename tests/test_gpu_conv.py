@@ -27,6 +27,9 @@ SMALL = [
     (1, 9, 40, 41, 300, 3, 3, 2),                                     # K > 256: two filter tiles
     (5, 7, 9, 9, 17, 3, 3, 1),                                        # 49 positions per image: tiles straddle images
     (2, 3, 37, 35, 24, 7, 7, 2), (1, 3, 51, 51, 32, 11, 11, 4), (1, 12, 14, 14, 16, 5, 5, 1),
+    (1, 24, 20, 21, 300, 3, 3, 1),       # streamed filter; in BF16 mode groups of 72 padded to 80 in the bf16 copy
+    (1, 16, 21, 230, 16, 7, 7, 2),       # wide 7x7: sixteen-channel strip stages do not fit, eight-channel groups
+    (1, 64, 21, 230, 64, 7, 7, 2),       # the same with a filter too large to be resident
 ]
 
 
