@@ -33,6 +33,9 @@
 #include "ptx_sm100.cuh"
 
 namespace im2win {
+#ifdef IM2WIN_PROF
+__attribute__((weak)) long long* g_prof = nullptr;  // debug build: one counter buffer shared by the parts
+#endif
 
 namespace {
 
@@ -384,14 +387,14 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
       ptx::mbar_init(ptx::smem_u32(&bars->raw_full[i]), 1);
       ptx::mbar_init(ptx::smem_u32(&bars->raw_empty[i]), 4);
       ptx::mbar_init(ptx::smem_u32(&bars->b_full[i]), (BRES && i == 0 && !P.b_tma) ? kThreads - 32 : 1);
-      ptx::mbar_init(ptx::smem_u32(&bars->b_empty[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->b_empty[i]), BRES ? 1 : 2);  // streamed: both issuers release a stage
     }
     for (int i = 0; i < kMaxSub; ++i) {
       ptx::mbar_init(ptx::smem_u32(&bars->a_full[i]), 4);
       ptx::mbar_init(ptx::smem_u32(&bars->a_empty[i]), 1);
     }
     for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), BRES ? P.NSETS : 1);  // one commit per MMA-issuing thread
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), BRES ? P.NSETS : 2);  // one commit per MMA-issuing thread
       ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), 4);
     }
     ptx::fence_mbar_init();
@@ -655,15 +658,18 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     // every copy issued must have landed before the CTA exits
     for (int64_t g = max(gcount - P.SR, (int64_t)0); g < gcount; ++g)
       wait_bar(P, misc, &bars->raw_full[g % P.SR], (uint32_t)(g / P.SR) & 1u, DEV_TIMEOUT_DRAIN);
-  } else if (warp == 1 || (BRES && warp >= 2 && warp <= P.NSETS)) {
+  } else if (warp == 1 || (BRES && warp >= 2 && warp <= P.NSETS) || (!BRES && warp == 3)) {
     // ================================================================ MMA ISSUER(S)
     // The loop body per MMA is kept to a handful of instructions because a single thread can only
     // issue a tcgen05.mma every few tens of cycles -- more than a narrow (N = 64) MMA takes to run.
     // With a resident filter nothing orders the groups of a tile among themselves (every MMA
     // accumulates onto an accumulator the epilogue has zeroed), so one thread per repack set, in
-    // warps 1, 2, (3), issues the groups that set produced.  With a streamed filter the stages are
-    // consumed in order by the one thread in warp 1.
-    const uint32_t me = (uint32_t)(warp - 1);
+    // warps 1, 2, (3), issues the groups that set produced.  With a streamed filter two threads (warps
+    // 1 and 3; warp 2 feeds the filter ring) share the groups by the parity of the producing set; both
+    // walk every filter stage in order -- each waits for a stage when it passes its first step and
+    // releases it when it passes its last, also across groups it does not issue, so that every stage
+    // barrier sees both of them in every phase.
+    const uint32_t me = BRES ? (uint32_t)(warp - 1) : (warp == 3 ? 1u : 0u);
     (void)me;
     if (lane == 0) {
       Ring ar0, ar1, ar2, br, dr;  // A slot (one ring per repack set), streamed filter stage, accumulator buffer
@@ -698,6 +704,27 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         for (int32_t g = g0; g < g1 && ok; ++g, gset = (gset + 1u == nsets) ? 0u : gset + 1u) {
           if constexpr (BRES) {
             if (gset != me) { st0 += S; continue; }  // another issuer's group
+          } else {
+            if ((gset & 1u) != me) {
+              // the other issuer's group: pass the filter stages that begin or end inside it
+              const uint32_t end = st0 + S;
+              uint32_t st = st0;
+              while (true) {
+                if ((st & 3u) == 0) {
+                  ok = wait_bar(P, misc, &bars->b_full[br.idx], br.phase, DEV_TIMEOUT_B_FULL, nullptr, 20);
+                  if (!ok) break;
+                }
+                const uint32_t last = st | 3u;  // last step of the stage that holds step st
+                if (last >= end) break;         // the stage runs on into the next group
+                ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u);
+                br.advance(P.SB);
+                st = last + 1u;
+                if (st >= end) break;
+              }
+              st0 = end;
+              continue;
+            }
+            b_lo = desc_lo0 + (uint32_t)br.idx * chunk16;  // (the group may begin inside a stage)
           }
           // the ring of the set that produced this group, held in registers (no indexed array)
           Ring ar = gset == 0 ? ar0 : (gset == 1 ? ar1 : ar2);
@@ -766,6 +793,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     // have landed before its first MMA)
     if constexpr (!BRES) {
       if (lane == 0) {
+        PROF_DECL(2)
         int64_t bcount = 0;
         Ring br;
         bool ok = true;
@@ -777,7 +805,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           const int32_t c0 = (g0 * S) >> 2, c1 = (g1 * S + 3) >> 2;
           for (int32_t c = c0; c < c1 && ok; ++c, ++bcount, br.advance(P.SB)) {
             const int32_t sb = br.idx;
-            ok = wait_bar(P, misc, &bars->b_empty[sb], br.phase ^ 1u, DEV_TIMEOUT_B_EMPTY);
+            ok = wait_bar(P, misc, &bars->b_empty[sb], br.phase ^ 1u, DEV_TIMEOUT_B_EMPTY, PROF_SLOT(0));
             if (!ok) break;
             const uint32_t full = ptx::smem_u32(&bars->b_full[sb]);
             ptx::mbar_expect_tx(full, b_stage_bytes);
@@ -787,6 +815,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         }
         for (int64_t c = max(bcount - P.SB, (int64_t)0); c < bcount; ++c)
           wait_bar(P, misc, &bars->b_full[c % P.SB], (uint32_t)(c / P.SB) & 1u, DEV_TIMEOUT_DRAIN);
+        PROF_DUMP(7, 1)
       }
       __syncwarp();
     }
@@ -1082,10 +1111,6 @@ __global__ void __launch_bounds__(256) filter_to_bf16_padded_kernel(const float*
 
 // ---------------------------------------------------------------------------------------------- host side
 
-#ifdef IM2WIN_PROF
-long long* g_prof = nullptr;
-#endif
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -1241,6 +1266,7 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   const int64_t cap = 227 * 1024 - 1024 - 1024 - ((int64_t)(P.win_span + 8) * 4 + 16);  // alignment slack, barriers, zero pad
   const int64_t b_res = (int64_t)steps_tile * P.NT * 32;  // one 32-byte-swizzled block per MMA step
   bool resident = P.n_ntiles == 1 && b_res + 2 * raw_stage <= cap;
+  if (getenv("IM2WIN_FORCE_STREAM") && getenv("IM2WIN_FORCE_STREAM")[0] == '1') resident = false;  // test knob
   // Streaming the native TF32 filter needs dense groups (padded reduction index == real index) and
   // 16-byte aligned filter rows.  In BF16 mode the TMA source is a bf16 copy of the filter made for
   // the duration of the call in memory from the stream-ordered pool (only where the caller allows an
@@ -1517,7 +1543,7 @@ int launch_conv_tc_persistent(const void* xhat, const float* f, float* out, cons
 }
 
 #ifdef IM2WIN_PROF
-// (debug build only; with the parts compiled separately the counters cover part 0's kernels)
+// (debug build only)
 extern "C" void im2win_debug_set_prof(long long* device_buf) { g_prof = device_buf; }
 #endif
 #endif  // IM2WIN_PART == -1 || IM2WIN_PART == 0
