@@ -77,6 +77,7 @@ struct PParams {
   uint64_t magic_TPI, magic_Wo;  // pim: ceil(2^32 / d); n / d == (n * magic) >> 32 while n * d < 2^32 (host check)
   int32_t nchunks;      // 128-byte filter chunks per tile
   int32_t l2_ahead;     // box mode: request the next tile's boxes into L2 one tile ahead
+  int32_t bslice;       // resident filter holds only this CTA's reduction slice (grid is a multiple of Z)
   int32_t b_tma;        // resident filter fetched by TMA (TF32, dense groups) instead of built by the threads
   int32_t tmem_cols;
   uint32_t idesc;
@@ -408,6 +409,19 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
+  // Slice-resident mode: the grid is a multiple of the number of reduction slices, so every unit of
+  // this CTA (t = blockIdx.x + k * gridDim.x) belongs to the same slice, and only that slice's part
+  // of the filter is kept in shared memory.
+  int32_t bs_g0 = 0, bs_ng = P.NG;
+  if constexpr (BRES) {
+    if (P.bslice) {
+      int32_t nt_b, gb0, gb1;
+      unit_range(P, (int32_t)blockIdx.x, nt_b, gb0, gb1);
+      (void)nt_b;
+      bs_g0 = gb0; bs_ng = gb1 - gb0;
+    }
+  }
+  const int32_t bs_step0 = bs_g0 * S;  // first MMA step held in the resident filter
   if constexpr (BRES) {
     // Build the whole filter operand once, one block of NT rows x 32 bytes per MMA step (padded
     // reduction indices [s*KSTEP, +KSTEP)), K-major with the 32-byte swizzle, so that the MMA thread
@@ -419,16 +433,16 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
       // (NT rows x 32 bytes, 32-byte swizzle) lays it out; the lanes of the otherwise idle warp 2
       // issue them, and no thread waits except the MMA issuers.
       if (warp == 2) {
-        const int32_t nsteps_all = P.NG * S;
+        const int32_t nsteps_all = bs_ng * S;
         const uint32_t full = ptx::smem_u32(&bars->b_full[0]);
         if (lane == 0) ptx::mbar_arrive_expect_tx(full, (uint32_t)nsteps_all * (uint32_t)P.NT * 32u);
         __syncwarp();
         for (int32_t st = lane; st < nsteps_all; st += 32)
-          tma_load_2d(ptx::smem_u32(b_smem) + (uint32_t)st * (uint32_t)P.NT * 32u, &fmap, st * KSTEP, 0, full);
+          tma_load_2d(ptx::smem_u32(b_smem) + (uint32_t)st * (uint32_t)P.NT * 32u, &fmap, (bs_step0 + st) * KSTEP, 0, full);
       }
     } else if (warp != 0) {
       constexpr int EPP = BF16 ? 8 : 4;  // elements per 16-byte piece
-      const int32_t nsteps_all = P.NG * S;
+      const int32_t nsteps_all = bs_ng * S;
       const int32_t pieces = nsteps_all * P.NT * 2;
       const uint32_t step_bytes = (uint32_t)P.NT * 32u;
       const bool vec = (KCG == KCGP) && (P.Kg % 4) == 0;  // padded index == real index, rows 16-byte aligned
@@ -450,7 +464,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
             const int32_t rest = idx >> 4;
             const int32_t jb = rest / nsteps_all;
             const int32_t sidx = rest - jb * nsteps_all, j = jb * 8 + jl;
-            const int32_t kp0 = sidx * KSTEP + c * EPP;
+            const int32_t kp0 = (bs_step0 + sidx) * KSTEP + c * EPP;
             dst[u] = sidx * (int32_t)step_bytes + (j >> 3) * 256 + (j & 7) * 32 + ((c ^ ((j >> 2) & 1)) << 4);
             if (vec && j < P.K && kp0 + EPP <= P.Kg) {
               const float4 a = __ldg(reinterpret_cast<const float4*>(P.f + (int64_t)j * P.Kg + kp0));
@@ -699,7 +713,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         int32_t nt_, g0, g1;
         unit_range(P, t, nt_, g0, g1);
         (void)nt_;
-        uint32_t st0 = (uint32_t)(g0 * S);  // steps of this tile before the current part
+        uint32_t st0 = (uint32_t)(g0 * S - (BRES ? bs_step0 : 0));  // steps before the current part (resident: of the held filter)
         uint32_t b_lo = desc_lo0;           // streamed: descriptor of the current stage
         for (int32_t g = g0; g < g1 && ok; ++g, gset = (gset + 1u == nsets) ? 0u : gset + 1u) {
           if constexpr (BRES) {
@@ -1275,9 +1289,42 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   const bool can_stream = (g.C % CB) == 0 && encode_fn() != nullptr &&
                           (BF16 ? may_alloc && (pad_copy || (g.Kg % 8) == 0) : KCG == KCGP && (g.Kg % 4) == 0);
   if (!resident && !can_stream) return IM2WIN_EUNSUPPORTED;
+  // Slice-resident mode.  A filter that does not fit whole may fit as one reduction slice per CTA:
+  // the units are (tile, slice) with the slice fastest, so with a grid that is a multiple of Z every
+  // CTA keeps to one slice, holds that slice of the filter for the whole kernel and adds its partial
+  // sums into the zeroed output.  The price is Z times the output as atomic adds, which L2 takes at
+  // about 1.4 TB/s (measured), so it pays only for long reductions onto few output channels (Table I
+  // Conv4: C = 64, 7x7, K = 64) -- estimated against the streamed mode, whose issuing threads spend
+  // about 200 cycles per MMA (measured), in microseconds at 1.9 GHz.
+  int32_t bs_z = 0, bs_gz = 0;
+  const bool bs_force = getenv("IM2WIN_BSLICE") && getenv("IM2WIN_BSLICE")[0] == '1';  // test knob
+  if ((!resident || bs_force) && P.n_ntiles == 1 && !out16 &&
+      !(getenv("IM2WIN_NO_BSLICE") && getenv("IM2WIN_NO_BSLICE")[0] == '1')) {
+    const int nsm = sm_count();
+    for (int32_t z = 2; z <= 16 && z <= P.NG && z <= nsm; ++z) {
+      const int32_t gz = (P.NG + z - 1) / z;
+      const int32_t z_eff = (P.NG + gz - 1) / gz;
+      if ((int64_t)gz * S * P.NT * 32 + 2 * raw_stage > cap) continue;
+      const double pipe = BF16 ? P.NT / 4.0 : P.NT / 2.0;  // cycles of one MMA in the tensor pipe
+      const int64_t grid_z = (int64_t)(nsm / z_eff) * z_eff;
+      const double units_cta = (double)((P.ntiles * z_eff + grid_z - 1) / grid_z);
+      const double mma_u = (double)gz * S * (pipe > 30.0 ? pipe : 30.0);
+      const double epi_u = P.NT * 31.0;
+      const bool two_acc = 2 * P.NT + 2 * 40 <= 512;
+      const double work_us = units_cta * (two_acc ? (mma_u > epi_u ? mma_u : epi_u) : mma_u + epi_u) / 1900.0;
+      const double atom_us = (double)g.n_out * 4.0 * z_eff / 1.4e6;
+      const double zero_us = 3.0 + (double)g.n_out * 4.0 / 3.0e6;
+      const double t_slice = (work_us > atom_us ? work_us : atom_us) + zero_us;
+      const double t_stream = (double)((P.ntiles + nsm - 1) / nsm) * P.NG * S * (pipe > 200.0 ? pipe : 200.0) / 1900.0;
+      if (bs_force || t_slice < 0.8 * t_stream) { bs_z = z_eff; bs_gz = gz; }
+      break;  // the smallest Z that fits
+    }
+    if (bs_z) resident = true;
+  }
   int64_t b_bytes;
   if (resident) {
-    b_bytes = b_res;
+    b_bytes = bs_z ? (int64_t)bs_gz * S * P.NT * 32 : b_res;
+    P.bslice = bs_z ? 1 : 0;
     P.SB = 1;
   } else {
     P.SB = 6;
@@ -1346,6 +1393,7 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
       if (forced >= 0 ? z == forced : c < best) { best = c; P.Z = z_eff; P.GZ = gz; }
     }
     if (forced == 0 || forced == 1) { P.Z = 1; P.GZ = P.NG; }
+    if (bs_z) { P.Z = bs_z; P.GZ = bs_gz; }
   }
   P.usub = P.n_ntiles * P.Z;
   P.ntiles *= P.Z;
@@ -1421,7 +1469,8 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
       return IM2WIN_ECUDA;
     }
   }
-  const int64_t grid = P.ntiles < sm_count() ? P.ntiles : sm_count();
+  int64_t grid = P.ntiles < sm_count() ? P.ntiles : sm_count();
+  if (P.bslice) grid = grid / P.Z * P.Z;  // every CTA keeps to one slice
   cudaError_t e;
   if (P.Z > 1 && cudaMemsetAsync(out, 0, (size_t)g.n_out * 4, st) != cudaSuccess) {  // (Z > 1 implies an fp32 output)
     cudaGetLastError();

@@ -38,17 +38,20 @@ def _built():
     ensure_built()
 
 
-@pytest.fixture(params=["auto", "nobox", "nopim", "split3", "generic"], autouse=True)
+@pytest.fixture(params=["auto", "nobox", "nopim", "split3", "bslice", "generic"], autouse=True)
 def _kernel(request, monkeypatch):
-    """Every case runs five times: with the library's own choice of tensor-core kernel (the persistent,
+    """Every case runs six times: with the library's own choice of tensor-core kernel (the persistent,
     filter-size-specialised one where it applies, tiles cut per image and strips staged by 2-D TMA
     boxes where they qualify, reduction slices where its cost model wants them), with the box staging
     switched off (per-image tiles, bulk copies), with per-image tiling switched off as well (tiles
     that span images), with three reduction slices forced wherever a layer has that many channel
-    groups (partial sums added into the zeroed output), and with the generic kernel forced."""
+    groups (partial sums added into the zeroed output), with the slice-resident filter mode forced
+    (every CTA keeps one reduction slice of the filter in shared memory), and with the generic kernel
+    forced."""
     monkeypatch.setenv("IM2WIN_FORCE_GENERIC", "1" if request.param == "generic" else "0")
     monkeypatch.setenv("IM2WIN_NO_BOX", "1" if request.param == "nobox" else "0")
     monkeypatch.setenv("IM2WIN_NO_PIM", "1" if request.param == "nopim" else "0")
+    monkeypatch.setenv("IM2WIN_BSLICE", "1" if request.param == "bslice" else "0")
     if request.param == "split3":
         monkeypatch.setenv("IM2WIN_SPLITK", "3")
     else:
