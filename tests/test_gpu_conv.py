@@ -208,6 +208,29 @@ def test_conv_full_batch_sampled(name, mode):
     assert np.isfinite(got).all()
 
 
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+def test_conv_long_reduction_few_filters_sampled(mode):
+    """Table I Conv4 (C = 64, 7x7, stride 2, K = 64: an 802 KB filter) at batch 16, where the library
+    keeps one reduction slice of the filter per CTA and adds partial sums into the zeroed output.
+    Checked at sampled output coordinates, the corners and the whole last image."""
+    layer = wl.CONFIGS["table1_Conv4"].with_batch(16)
+    dims = layer.dims()
+    n, c, h, w, k, fh, fw, s = dims
+    x, f = wl.make_input(layer), wl.make_filter(layer)
+    got = gpu_conv(x, f, dims, mode)
+    ho, wo = b.out_dims(dims)
+    rng = np.random.default_rng(4321)
+    idx = np.stack([rng.integers(0, n, 5000), rng.integers(0, k, 5000), rng.integers(0, ho, 5000),
+                    rng.integers(0, wo, 5000)], axis=1).astype(np.int32)
+    corners = np.array(list(itertools.product((0, n - 1), (0, k - 1), (0, ho - 1), (0, wo - 1))), dtype=np.int32)
+    idx = np.concatenate([idx, corners])
+    ref = oracle.conv_direct_points(x, f, oracle.Shape(*dims), idx)
+    assert rel_l2(got[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]], ref) <= TOL[mode]
+    one = layer.with_batch(1).dims()
+    assert rel_l2(got[n - 1:n], oracle_conv(x[n - 1:n], f, one)) <= TOL[mode]
+    assert np.isfinite(got).all()
+
+
 @pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16, b.MODE_FP32], ids=MODE_ID.get)
 @pytest.mark.parametrize("dims", [(19, 16, 30, 30, 32, 3, 3, 1), (3, 5, 17, 19, 7, 2, 3, 2), (1, 3, 32, 32, 16, 3, 3, 1)])
 def test_conv_host_buffers(dims, mode):
