@@ -1292,10 +1292,11 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   // Slice-resident mode.  A filter that does not fit whole may fit as one reduction slice per CTA:
   // the units are (tile, slice) with the slice fastest, so with a grid that is a multiple of Z every
   // CTA keeps to one slice, holds that slice of the filter for the whole kernel and adds its partial
-  // sums into the zeroed output.  The price is Z times the output as atomic adds, which L2 takes at
-  // about 1.4 TB/s (measured), so it pays only for long reductions onto few output channels (Table I
-  // Conv4: C = 64, 7x7, K = 64) -- estimated against the streamed mode, whose issuing threads spend
-  // about 200 cycles per MMA (measured), in microseconds at 1.9 GHz.
+  // sums into the zeroed output.  The price is Z epilogues per tile, each of atomic adds: an SM
+  // passes about one 32-bit add per cycle, so an epilogue warp spends ~85 cycles per accumulator
+  // column (measured; ~31 with plain stores).  It pays only for long reductions onto few output
+  // channels (Table I Conv4: C = 64, 7x7, K = 64) -- estimated against the streamed mode, whose
+  // issuing threads spend about 200 cycles per MMA (measured), in microseconds at 1.9 GHz.
   int32_t bs_z = 0, bs_gz = 0;
   const bool bs_force = getenv("IM2WIN_BSLICE") && getenv("IM2WIN_BSLICE")[0] == '1';  // test knob
   if ((!resident || bs_force) && P.n_ntiles == 1 && !out16 &&
@@ -1309,12 +1310,11 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
       const int64_t grid_z = (int64_t)(nsm / z_eff) * z_eff;
       const double units_cta = (double)((P.ntiles * z_eff + grid_z - 1) / grid_z);
       const double mma_u = (double)gz * S * (pipe > 30.0 ? pipe : 30.0);
-      const double epi_u = P.NT * 31.0;
+      const double epi_u = P.NT * 85.0;
       const bool two_acc = 2 * P.NT + 2 * 40 <= 512;
       const double work_us = units_cta * (two_acc ? (mma_u > epi_u ? mma_u : epi_u) : mma_u + epi_u) / 1900.0;
-      const double atom_us = (double)g.n_out * 4.0 * z_eff / 1.4e6;
       const double zero_us = 3.0 + (double)g.n_out * 4.0 / 3.0e6;
-      const double t_slice = (work_us > atom_us ? work_us : atom_us) + zero_us;
+      const double t_slice = work_us + zero_us;
       const double t_stream = (double)((P.ntiles + nsm - 1) / nsm) * P.NG * S * (pipe > 200.0 ? pipe : 200.0) / 1900.0;
       if (bs_force || t_slice < 0.8 * t_stream) { bs_z = z_eff; bs_gz = gz; }
       break;  // the smallest Z that fits
