@@ -110,7 +110,12 @@ int im2win_transform_bf16(const float* in_nchw, const im2win_shape* shape, uint1
  *            more (tiles cut per image); EUNSUPPORTED otherwise.
  * filter:    device, K*C*Fh*Fw floats, native K,C,Fh,Fw order (no repacking needed).
  * mode:      IM2WIN_MODE_*.
- * out_nchw:  device, N*K*Ho*Wo floats, every element is written.
+ * out_nchw:  device, N*K*Ho*Wo floats, every element is written.  In the tensor-core modes the
+ *            order in which the fp32 partial sums over channel groups are added is not fixed
+ *            (several threads issue the MMAs of a tile; small batches and long reductions onto
+ *            few filters add partial sums of reduction slices into the zeroed output), so two
+ *            calls on the same data agree within fp32 rounding, and bit for bit where every
+ *            product and partial sum is exactly representable.
  * workspace: device, at least im2win_workspace_bytes(shape) bytes when src_kind is NCHW
  *            (EWORKSPACE otherwise), 16-byte aligned.
  * Limits of the tensor-core modes (EUNSUPPORTED beyond them): Fh*Fw <= 1024; one output row's
