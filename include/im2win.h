@@ -5,7 +5,7 @@
  * Notation follows the paper: input I[N][C][H][W], filter F[K][C][Fh][Fw],
  * output O[N][K][Ho][Wo], one stride s for both directions, no padding, no
  * dilation, no groups, no bias, no filter flip (Section II-A, Eq. 1).  All
- * tensors are dense and row-major ("stored as a 1D array", Section I) in fp32.
+ * tensors are dense, row-major and flat in memory (Section I) in fp32.
  * The im2win tensor is Ihat[N][C][Ho][W*Fh] (Section III-A, Algorithm 1).
  *
  * Unless a function says HOST, data pointers are DEVICE pointers owned by the
@@ -14,7 +14,12 @@
  * Device work is enqueued on the CUDA stream given as `cuda_stream`
  * (a cudaStream_t cast to void*; NULL = the default stream) and the call
  * returns without synchronising.  Every function returns IM2WIN_OK (0) or a
- * negative im2win_status; nothing is launched when an error is returned.
+ * negative im2win_status.  Argument errors (EINVAL, EALIGN, EWORKSPACE,
+ * EOVERLAP, ESCRATCH) are found before anything is launched; EUNSUPPORTED
+ * and ECUDA from im2win_conv with src_kind NCHW can come after the transform
+ * has been enqueued (the workspace then holds the im2win tensor).
+ * The library allocates no device memory in any call on device pointers
+ * (im2win_conv_host, which works on host buffers, owns its device buffers).
  * There is no CPU fallback: without a CUDA device the launching calls return
  * IM2WIN_ECUDA.
  */
@@ -63,11 +68,20 @@ typedef enum {
  * (Algorithm 1, first line; Table I fixes the division as floor). */
 int im2win_out_dims(const im2win_shape* shape, int32_t* Ho, int32_t* Wo);
 
-/* Bytes of the im2win tensor, 4*N*C*Ho*Fh*W (Section III-A: "the size of the im2win tensor is
- * Ni x Ci x Hf x Wi x ((Hi-Hf)/s+1)").  This is the workspace im2win_conv needs when it is given
- * the untransformed input, and the size of im2win_transform's output.  The same tight size is
- * used when Fh <= s, where Algorithm 1 allocates the (larger or equal) input size instead. */
+/* Bytes of the im2win tensor, 4*N*C*Ho*Fh*W (the element count Section III-A gives for it: batch x
+ * channels x filter height x input width x output height).  This is the least workspace im2win_conv
+ * needs when it is given the untransformed input, and the size of im2win_transform's output.  The same
+ * tight size is used when Fh <= s, where Algorithm 1 allocates the (larger or equal) input size. */
 int im2win_workspace_bytes(const im2win_shape* shape, size_t* bytes);
+
+/* Workspace with which im2win_conv can pick its fastest kernel for (shape, src_kind, mode) (no
+ * counterpart in the paper): the im2win tensor where src_kind is NCHW (as above, rounded up to 256
+ * bytes), plus room for a re-laid-out copy of the filter that some tensor-core kernels stream by TMA
+ * (tap-major order for the strip-matrix kernel; bf16 for BF16 mode).  That copy is at most about
+ * 1.4 x the filter's own 4*K*C*Fh*Fw bytes, i.e. a few MB against an im2win tensor of tens to hundreds
+ * of MB.  A smaller workspace is legal (down to im2win_workspace_bytes, or none for the other source
+ * kinds): kernels that need no copy are used instead, some of them slower. */
+int im2win_conv_workspace_bytes(const im2win_shape* shape, int src_kind, int mode, size_t* bytes);
 
 /* Bytes an im2col matrix for the whole batch would take, 4*N*C*Fh*Fw*Ho*Wo (Section III-A).
  * Reporting only: the library never builds one. */
@@ -97,18 +111,20 @@ int im2win_transform_bf16(const float* in_nchw, const im2win_shape* shape, uint1
  * is the form consistent with Algorithm 1 otherwise.)
  * src:       device.  src_kind NCHW: the input I (N*C*H*W floats); the call first runs the
  *            transform into `workspace`, which then holds Ihat and may be reused by the caller.
- *            src_kind IM2WIN: an im2win tensor; `workspace` is ignored and may be NULL.
+ *            src_kind IM2WIN: an im2win tensor; `workspace` may be NULL, or give scratch (see below).
  *            src_kind NCHW_FUSED: the input I; the tensor-core kernel stages the input rows a tile
  *            needs and reads the windows from them, so nothing of size Ihat is written (workspace
  *            0 bytes).  Same result as the other two kinds.  Shapes without a fused specialisation
  *            (see below) fall back to transform + convolution if a sufficient `workspace` is
  *            given, else EUNSUPPORTED; IM2WIN_MODE_FP32 always takes that fallback.
  *            src_kind IM2WIN_BF16: a bf16 im2win tensor from im2win_transform_bf16; mode must be
- *            IM2WIN_MODE_BF16 (EINVAL otherwise); `workspace` is ignored.  The MMA operands are
- *            the same bf16 values as from an fp32 im2win tensor.  Implemented for layers with a
- *            filter-size specialisation whose images have roughly a thousand output positions or
- *            more (tiles cut per image); EUNSUPPORTED otherwise.
- * filter:    device, K*C*Fh*Fw floats, native K,C,Fh,Fw order (no repacking needed).
+ *            IM2WIN_MODE_BF16 (EINVAL otherwise); `workspace` optional scratch.  The MMA operands
+ *            are the same bf16 values as from an fp32 im2win tensor.  Implemented where a
+ *            tensor-core kernel with a 16-bit source applies (3x3 layers of the strip-matrix kernel
+ *            with scratch; filter-size specialisations whose images have roughly a thousand output
+ *            positions or more); EUNSUPPORTED otherwise.
+ * filter:    device, K*C*Fh*Fw floats, native K,C,Fh,Fw order (the caller repacks nothing; kernels
+ *            that want another order or bf16 write their copy into the workspace's scratch part).
  * mode:      IM2WIN_MODE_*.
  * out_nchw:  device, N*K*Ho*Wo floats, every element is written.  In the tensor-core modes the
  *            order in which the fp32 partial sums over channel groups are added is not fixed
@@ -116,8 +132,12 @@ int im2win_transform_bf16(const float* in_nchw, const im2win_shape* shape, uint1
  *            few filters add partial sums of reduction slices into the zeroed output), so two
  *            calls on the same data agree within fp32 rounding, and bit for bit where every
  *            product and partial sum is exactly representable.
- * workspace: device, at least im2win_workspace_bytes(shape) bytes when src_kind is NCHW
- *            (EWORKSPACE otherwise), 16-byte aligned.
+ * workspace: device, 16-byte aligned, caller-owned; at least im2win_workspace_bytes(shape) bytes when
+ *            src_kind is NCHW (EWORKSPACE otherwise), optional for the other kinds.  Bytes beyond
+ *            the im2win tensor (from the next 256-byte boundary) serve as scratch for the filter copy;
+ *            im2win_conv_workspace_bytes gives the size with which the fastest kernels apply.  The
+ *            whole range must not overlap src, filter or out (EOVERLAP); its contents after the
+ *            call are the im2win tensor (NCHW) followed by unspecified scratch.
  * Limits of the tensor-core modes (EUNSUPPORTED beyond them): Fh*Fw <= 1024; one output row's
  * worth of staged strips must fit in shared memory (W*Fh up to a few thousand floats).
  * IM2WIN_MODE_FP32 has no such limits. */
@@ -152,7 +172,9 @@ int im2win_host_release(void);
  * (hard-real-time loops, safety-reviewed code).  im2win_conv needs a caller-supplied workspace for
  * the im2win tensor; this variant keeps that tensor in a buffer built into the library image
  * (IM2WIN_STATIC_SCRATCH_BYTES of device memory on every GPU that loads the library, held until
- * the process exits) and itself calls no cudaMalloc, cudaFree or other allocating routine.
+ * the process exits) and itself calls no cudaMalloc, cudaFree or other allocating routine; a filter
+ * copy that a tensor-core kernel wants goes into the same buffer behind the im2win tensor when there
+ * is room, else a kernel that needs none is used.
  * Computes exactly what im2win_conv(in_nchw, IM2WIN_SRC_NCHW, ...) computes, on `cuda_stream`,
  * asynchronously.  in_nchw / filter_kcfhfw / out_nchw: device pointers as for im2win_conv.
  * Errors: IM2WIN_ESCRATCH when im2win_workspace_bytes(shape) exceeds the built-in buffer (nothing
@@ -161,15 +183,17 @@ int im2win_host_release(void);
  * with that device current); make that first call outside any stream capture.
  * All calls on a device share the one buffer: two calls whose kernels can overlap on the GPU
  * (different streams without an ordering between them) race on it and give wrong results.  The
- * buffer keeps the previous call's im2win tensor; nothing in it needs clearing, because each call
- * overwrites every element it later reads. */
+ * buffer keeps the previous call's contents; nothing in it needs clearing, because each call
+ * overwrites every element it later reads.  The cached address is an atomic per device, so first calls
+ * from several host threads are safe; the buffer itself is not. */
 #define IM2WIN_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
 int im2win_conv_static(const float* in_nchw, const float* filter_kcfhfw, const im2win_shape* shape,
                        int mode, float* out_nchw, void* cuda_stream);
 /* Kernels never trap.  A bounded wait that expires, or an internal range check that fails,
  * records a code in a device-side status word and the kernel exits early (its output is then
- * undefined).  This call synchronises `cuda_stream`, returns the word in *status (0 = clean)
- * and clears it. */
+ * undefined).  This call synchronises `cuda_stream`, stores the word in *status (0 = clean) and
+ * clears it.  Returns IM2WIN_OK when the word was clean (or holds a range-check code, 201),
+ * IM2WIN_ETIMEOUT when it names an expired wait (101..109; the code says which wait). */
 int im2win_last_device_status(void* cuda_stream, int32_t* status);
 
 /* English text for a status code; never NULL. */

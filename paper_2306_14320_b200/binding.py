@@ -14,12 +14,15 @@ from typing import Sequence
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libim2win.so")
+# The same code with settable diagnostic switches (im2win_debug_set_option); loaded by the parity tests
+# only, through use_test_library().
+TEST_LIB_PATH = os.path.join(_HERE, "libim2win_test.so")
 
 SRC_NCHW, SRC_IM2WIN, SRC_NCHW_FUSED, SRC_IM2WIN_BF16 = 0, 1, 2, 3
 MODE_TF32, MODE_BF16, MODE_FP32 = 0, 1, 2
 OK, EINVAL, EALIGN, EWORKSPACE, EOVERLAP, ECUDA, ETIMEOUT, EUNSUPPORTED, ESCRATCH = 0, -1, -2, -3, -4, -5, -6, -7, -8
 
-EXPORTS = ("im2win_out_dims", "im2win_workspace_bytes", "im2win_im2col_bytes", "im2win_transform",
+EXPORTS = ("im2win_out_dims", "im2win_workspace_bytes", "im2win_conv_workspace_bytes", "im2win_im2col_bytes", "im2win_transform",
            "im2win_workspace_bytes_bf16", "im2win_transform_bf16", "im2win_conv", "im2win_conv_bf16out", "im2win_conv_host", "im2win_host_release", "im2win_conv_static",
            "im2win_last_device_status", "im2win_strerror")
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024  # IM2WIN_STATIC_SCRATCH_BYTES of include/im2win.h
@@ -41,35 +44,64 @@ class Im2winError(RuntimeError):
 
 
 _lib = None
+_test_lib = None
+_use_test = False
+
+
+def _declare(L: ctypes.CDLL) -> ctypes.CDLL:
+    sp, vp = ctypes.POINTER(Shape), ctypes.c_void_p
+    L.im2win_out_dims.argtypes = [sp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+    L.im2win_workspace_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
+    L.im2win_conv_workspace_bytes.argtypes = [sp, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_size_t)]
+    L.im2win_im2col_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
+    L.im2win_transform.argtypes = [vp, sp, vp, vp]
+    L.im2win_workspace_bytes_bf16.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
+    L.im2win_transform_bf16.argtypes = [vp, sp, vp, vp]
+    L.im2win_conv.argtypes = [vp, ctypes.c_int, vp, sp, ctypes.c_int, vp, vp, ctypes.c_size_t, vp]
+    L.im2win_conv_bf16out.argtypes = [vp, ctypes.c_int, vp, sp, ctypes.c_int, vp, vp, ctypes.c_size_t, vp]
+    L.im2win_conv_host.argtypes = [vp, vp, sp, ctypes.c_int, vp]
+    L.im2win_host_release.argtypes = []
+    L.im2win_conv_static.argtypes = [vp, vp, sp, ctypes.c_int, vp, vp]
+    L.im2win_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
+    L.im2win_strerror.argtypes = [ctypes.c_int]
+    L.im2win_strerror.restype = ctypes.c_char_p
+    for name in EXPORTS[:-1]:
+        getattr(L, name).restype = ctypes.c_int
+    return L
 
 
 def lib() -> ctypes.CDLL:
-    """Loads libim2win.so (built in-tree by ``paper_2306_14320_b200.build``)."""
-    global _lib
-    if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2306_14320_b200.build` "
+    """Loads libim2win.so (built in-tree by ``paper_2306_14320_b200.build``), or the test build of it
+    after use_test_library(True)."""
+    global _lib, _test_lib
+    path = TEST_LIB_PATH if _use_test else LIB_PATH
+    cur = _test_lib if _use_test else _lib
+    if cur is None:
+        if not os.path.exists(path):
+            raise ImportError(f"{path} is missing: build it with `python -m paper_2306_14320_b200.build` "
                               "(there is no non-CUDA fallback)")
-        L = ctypes.CDLL(LIB_PATH)
-        sp, vp = ctypes.POINTER(Shape), ctypes.c_void_p
-        L.im2win_out_dims.argtypes = [sp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
-        L.im2win_workspace_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
-        L.im2win_im2col_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
-        L.im2win_transform.argtypes = [vp, sp, vp, vp]
-        L.im2win_workspace_bytes_bf16.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
-        L.im2win_transform_bf16.argtypes = [vp, sp, vp, vp]
-        L.im2win_conv.argtypes = [vp, ctypes.c_int, vp, sp, ctypes.c_int, vp, vp, ctypes.c_size_t, vp]
-        L.im2win_conv_bf16out.argtypes = [vp, ctypes.c_int, vp, sp, ctypes.c_int, vp, vp, ctypes.c_size_t, vp]
-        L.im2win_conv_host.argtypes = [vp, vp, sp, ctypes.c_int, vp]
-        L.im2win_host_release.argtypes = []
-        L.im2win_conv_static.argtypes = [vp, vp, sp, ctypes.c_int, vp, vp]
-        L.im2win_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
-        L.im2win_strerror.argtypes = [ctypes.c_int]
-        L.im2win_strerror.restype = ctypes.c_char_p
-        for name in EXPORTS[:-1]:
-            getattr(L, name).restype = ctypes.c_int
-        _lib = L
-    return _lib
+        cur = _declare(ctypes.CDLL(path))
+        if _use_test:
+            cur.im2win_debug_set_option.argtypes = [ctypes.c_char_p, ctypes.c_int]
+            cur.im2win_debug_set_option.restype = ctypes.c_int
+            _test_lib = cur
+        else:
+            _lib = cur
+    return cur
+
+
+def use_test_library(on: bool) -> None:
+    """Route every later call through libim2win_test.so (on) or back through the product library (off).
+    The two are separate loaded images: each has its own device status word and built-in buffers."""
+    global _use_test
+    _use_test = bool(on)
+
+
+def set_option(name: str, value: int) -> None:
+    """Test build only: set one diagnostic switch of the launchers (see Knobs in csrc/common.cuh)."""
+    if not _use_test:
+        raise RuntimeError("diagnostic switches exist in the test library only: call use_test_library(True) first")
+    _check(lib().im2win_debug_set_option(name.encode(), int(value)), f"im2win_debug_set_option({name})")
 
 
 def _check(code: int, where: str) -> None:
@@ -112,6 +144,14 @@ def out_dims(shape) -> tuple[int, int]:
 def workspace_bytes(shape) -> int:
     b = ctypes.c_size_t()
     _check(lib().im2win_workspace_bytes(ctypes.byref(Shape.of(shape)), ctypes.byref(b)), "im2win_workspace_bytes")
+    return b.value
+
+
+def conv_workspace_bytes(shape, src_kind: int, mode: int) -> int:
+    """im2win_conv_workspace_bytes: the workspace with which im2win_conv can use its fastest kernel."""
+    b = ctypes.c_size_t()
+    _check(lib().im2win_conv_workspace_bytes(ctypes.byref(Shape.of(shape)), int(src_kind), int(mode), ctypes.byref(b)),
+           "im2win_conv_workspace_bytes")
     return b.value
 
 
@@ -179,7 +219,16 @@ def host_release() -> None:
     _check(lib().im2win_host_release(), "im2win_host_release")
 
 
-def last_device_status(stream=None) -> int:
+def last_device_status_rc(stream=None) -> tuple[int, int]:
+    """im2win_last_device_status: (return code, raw status word).  The return code is ETIMEOUT when the
+    word names an expired bounded wait, OK otherwise."""
     st = ctypes.c_int32()
-    _check(lib().im2win_last_device_status(_stream(stream), ctypes.byref(st)), "im2win_last_device_status")
-    return st.value
+    rc = lib().im2win_last_device_status(_stream(stream), ctypes.byref(st))
+    if rc not in (OK, ETIMEOUT):
+        raise Im2winError(rc, "im2win_last_device_status")
+    return rc, st.value
+
+
+def last_device_status(stream=None) -> int:
+    """The raw status word (0 = clean); synchronises the stream and clears the word."""
+    return last_device_status_rc(stream)[1]

@@ -1,6 +1,6 @@
 // C-ABI entry points: argument checks, size queries and dispatch to the kernels.
+#include <atomic>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 
 #include "common.cuh"
@@ -60,16 +60,51 @@ int make_geometry(const im2win_shape* sh, Geometry* g) {
   return IM2WIN_OK;
 }
 
-int launch_conv_tc(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
-                   cudaStream_t st, bool may_alloc) {
-  // IM2WIN_FORCE_GENERIC=1 routes every shape through the generic kernel (used by the tests to
-  // cover both kernels on the same inputs).
-  const char* force = getenv("IM2WIN_FORCE_GENERIC");
-  if (!(force && force[0] == '1')) {
-    const int rc = launch_conv_tc_persistent(xhat, f, out, g, mode, st, may_alloc);
+int launch_conv_tc(const void* src, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st,
+                   Scratch scratch, int src_kind, bool out_bf16) {
+  // src_kind: 0 = fp32 im2win tensor, 1 = untransformed input consumed fused, 2 = bf16 im2win tensor.
+  // Order: the strip-matrix kernel where it is implemented and expected to win, else the persistent
+  // specialised kernel, else (fp32 im2win tensor and fp32 output only) the generic kernel.
+  int rc = IM2WIN_EUNSUPPORTED;
+  if (!knobs().force_generic) {
+    if (!knobs().no_strip) rc = launch_conv_tc_strip(src, f, out, g, mode, st, scratch, src_kind, out_bf16);
+    if (rc != IM2WIN_EUNSUPPORTED) return rc;
+    rc = launch_conv_tc_persistent(src, f, out, g, mode, st, scratch, src_kind == 1, src_kind == 2, out_bf16);
     if (rc != IM2WIN_EUNSUPPORTED) return rc;
   }
-  return launch_conv_tc_generic(xhat, f, out, g, mode, st);
+  if (src_kind != 0 || out_bf16) return IM2WIN_EUNSUPPORTED;
+  return launch_conv_tc_generic(static_cast<const float*>(src), f, out, g, mode, st);
+}
+
+size_t conv_scratch_bytes(const Geometry& g, int mode, int src_kind) {
+  if (mode != IM2WIN_MODE_TF32 && mode != IM2WIN_MODE_BF16) return 0;
+  const size_t a = strip_scratch_bytes(g, mode, src_kind), b = persistent_scratch_bytes(g, mode);
+  return a > b ? a : b;
+}
+
+#ifdef IM2WIN_TEST_KNOBS
+static Knobs g_knobs;
+const Knobs& knobs() { return g_knobs; }
+#else
+const Knobs& knobs() {
+  static const Knobs defaults;
+  return defaults;
+}
+#endif
+
+int sm_count() {
+  constexpr int kMaxDev = 64;
+  static std::atomic<int> cached[kMaxDev];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) { cudaGetLastError(); return 148; }
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    cudaGetLastError();
+    return 148;
+  }
+  cached[dev].store(n, std::memory_order_relaxed);
+  return n;
 }
 
 int32_t* device_status_word() {
@@ -146,11 +181,14 @@ int im2win_transform_bf16(const float* in_nchw, const im2win_shape* shape, uint1
   return launch_transform_bf16(in_nchw, out_im2win_bf16, g, static_cast<cudaStream_t>(cuda_stream));
 }
 
-// Shared body of im2win_conv (fp32 output) and im2win_conv_bf16out (out16: `out` holds 16-bit words;
-// tensor-core modes and the specialised kernel only).
-static int conv_impl(const void* src, int src_kind, const float* filter, const im2win_shape* shape,
-                     int mode, void* out, bool out16, void* workspace, size_t workspace_bytes,
-                     void* cuda_stream) {
+}  // extern "C"
+
+namespace im2win {
+
+// Shared body of im2win_conv (fp32 output), im2win_conv_bf16out (out16: `out` holds 16-bit words;
+// tensor-core modes, kernels with a bf16 epilogue) and im2win_conv_static.
+int conv_impl(const void* src, int src_kind, const float* filter, const im2win_shape* shape, int mode, void* out,
+              bool out16, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   float* const out_nchw = static_cast<float*>(out);
   const int64_t out_es = out16 ? 2 : 4;
   Geometry g;
@@ -169,40 +207,72 @@ static int conv_impl(const void* src, int src_kind, const float* filter, const i
                                                                 : (src_kind == IM2WIN_SRC_IM2WIN ? g.n_win : g.n_in) * 4;
   if (overlap(out_nchw, g.n_out * out_es, src, src_bytes) || overlap(out_nchw, g.n_out * out_es, filter, g.n_flt * 4))
     return IM2WIN_EOVERLAP;
+  // The workspace: first the im2win tensor (src_kind NCHW, or the fallback of NCHW_FUSED), then, from the
+  // next 256-byte boundary, whatever is left as scratch for a re-laid-out copy of the filter.
+  uint8_t* const ws = static_cast<uint8_t*>(workspace);
+  const size_t ws_bytes = ws ? workspace_bytes : 0;
+  const size_t win_bytes = (size_t)g.n_win * 4;
+  if (src_kind == IM2WIN_SRC_NCHW && ws_bytes < win_bytes) return IM2WIN_EWORKSPACE;
+  if (ws_bytes) {
+    if (!aligned16(ws)) return IM2WIN_EALIGN;
+    if (ws_bytes > (size_t)INT64_MAX || overlap(ws, (int64_t)ws_bytes, src, src_bytes) ||
+        overlap(ws, (int64_t)ws_bytes, out_nchw, g.n_out * out_es) || overlap(ws, (int64_t)ws_bytes, filter, g.n_flt * 4))
+      return IM2WIN_EOVERLAP;
+  }
+  auto scratch_from = [&](size_t offset) {
+    Scratch sc;
+    offset = (offset + 255) / 256 * 256;
+    if (ws_bytes > offset) { sc.ptr = ws + offset; sc.bytes = ws_bytes - offset; }
+    return sc;
+  };
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if (src_kind == IM2WIN_SRC_IM2WIN_BF16)  // no generic-kernel fallback for this storage variant
-    return launch_conv_tc_persistent(src, filter, out_nchw, g, mode, st, /*may_alloc=*/true, /*fused=*/false,
-                                     /*src_bf16=*/true, out16);
+  if (src_kind == IM2WIN_SRC_IM2WIN_BF16) {  // (no generic-kernel fallback for this storage variant)
+    if (knobs().force_generic) return IM2WIN_EUNSUPPORTED;
+    return launch_conv_tc(src, filter, out_nchw, g, mode, st, scratch_from(0), 2, out16);
+  }
   const float* xhat = static_cast<const float*>(src);
   if (src_kind == IM2WIN_SRC_NCHW_FUSED) {
-    if (mode != IM2WIN_MODE_FP32) {
-      const char* force = getenv("IM2WIN_FORCE_GENERIC");
-      if (!(force && force[0] == '1')) {
-        rc = launch_conv_tc_persistent(xhat, filter, out_nchw, g, mode, st, /*may_alloc=*/true, /*fused=*/true,
+    if (mode != IM2WIN_MODE_FP32 && !knobs().force_generic) {
+      rc = IM2WIN_EUNSUPPORTED;
+      if (!knobs().no_strip) rc = launch_conv_tc_strip(xhat, filter, out_nchw, g, mode, st, scratch_from(0), 1, out16);
+      if (rc == IM2WIN_EUNSUPPORTED)
+        rc = launch_conv_tc_persistent(xhat, filter, out_nchw, g, mode, st, scratch_from(0), /*fused=*/true,
                                        /*src_bf16=*/false, out16);
-        if (rc != IM2WIN_EUNSUPPORTED) return rc;
-      }
+      if (rc != IM2WIN_EUNSUPPORTED) return rc;
     }
     // no fused kernel for this shape or mode: the unfused path, if the caller supplied a workspace
-    if (!workspace || workspace_bytes < (size_t)g.n_win * 4) return IM2WIN_EUNSUPPORTED;
+    if (ws_bytes < win_bytes) return IM2WIN_EUNSUPPORTED;
     src_kind = IM2WIN_SRC_NCHW;
   }
+  Scratch scratch = scratch_from(0);
   if (src_kind == IM2WIN_SRC_NCHW) {
-    if (!workspace || workspace_bytes < (size_t)g.n_win * 4) return IM2WIN_EWORKSPACE;
-    if (!aligned16(workspace)) return IM2WIN_EALIGN;
-    if (overlap(workspace, g.n_win * 4, src, src_bytes) ||
-        overlap(workspace, g.n_win * 4, out_nchw, g.n_out * out_es) ||
-        overlap(workspace, g.n_win * 4, filter, g.n_flt * 4))
-      return IM2WIN_EOVERLAP;
-    rc = launch_transform(static_cast<const float*>(src), static_cast<float*>(workspace), g, st);
+    rc = launch_transform(static_cast<const float*>(src), reinterpret_cast<float*>(ws), g, st);
     if (rc != IM2WIN_OK) return rc;
-    xhat = static_cast<const float*>(workspace);
+    xhat = reinterpret_cast<const float*>(ws);
+    scratch = scratch_from(win_bytes);
   }
-  if (out16)  // only the specialised kernel has the bf16 epilogue
-    return launch_conv_tc_persistent(xhat, filter, out_nchw, g, mode, st, /*may_alloc=*/true, /*fused=*/false,
-                                     /*src_bf16=*/false, true);
   if (mode == IM2WIN_MODE_FP32) return launch_conv_fp32(xhat, filter, out_nchw, g, st);
-  return launch_conv_tc(xhat, filter, out_nchw, g, mode, st);
+  return launch_conv_tc(xhat, filter, out_nchw, g, mode, st, scratch, 0, out16);
+}
+
+}  // namespace im2win
+
+extern "C" {
+
+int im2win_conv_workspace_bytes(const im2win_shape* shape, int src_kind, int mode, size_t* bytes) {
+  Geometry g;
+  const int rc = make_geometry(shape, &g);
+  if (rc != IM2WIN_OK) return rc;
+  if (!bytes) return IM2WIN_EINVAL;
+  if (src_kind != IM2WIN_SRC_NCHW && src_kind != IM2WIN_SRC_IM2WIN && src_kind != IM2WIN_SRC_NCHW_FUSED &&
+      src_kind != IM2WIN_SRC_IM2WIN_BF16)
+    return IM2WIN_EINVAL;
+  if (mode != IM2WIN_MODE_TF32 && mode != IM2WIN_MODE_BF16 && mode != IM2WIN_MODE_FP32) return IM2WIN_EINVAL;
+  const size_t win = src_kind == IM2WIN_SRC_NCHW ? ((size_t)g.n_win * 4 + 255) / 256 * 256 : 0;
+  const int kind = src_kind == IM2WIN_SRC_NCHW_FUSED ? 1 : (src_kind == IM2WIN_SRC_IM2WIN_BF16 ? 2 : 0);
+  const size_t extra = conv_scratch_bytes(g, mode, kind);
+  *bytes = extra ? win + extra : (src_kind == IM2WIN_SRC_NCHW ? (size_t)g.n_win * 4 : 0);
+  return IM2WIN_OK;
 }
 
 int im2win_conv(const void* src, int src_kind, const float* filter, const im2win_shape* shape,
@@ -227,8 +297,28 @@ int im2win_last_device_status(void* cuda_stream, int32_t* status) {
   if (cudaMemcpy(&v, word, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return IM2WIN_ECUDA;
   if (v != 0 && cudaMemset(word, 0, sizeof(v)) != cudaSuccess) return IM2WIN_ECUDA;
   *status = v;
-  return IM2WIN_OK;
+  // an expired bounded wait (codes 101..199) is reported as such; the raw code stays in *status
+  return (v >= 100 && v < 200) ? IM2WIN_ETIMEOUT : IM2WIN_OK;
 }
+
+#ifdef IM2WIN_TEST_KNOBS
+// Test build only (libim2win_test.so): set one diagnostic switch by name.  Returns IM2WIN_EINVAL for
+// an unknown name.
+int im2win_debug_set_option(const char* name, int value) {
+  if (!name) return IM2WIN_EINVAL;
+  struct Entry { const char* name; int Knobs::*field; };
+  static const Entry table[] = {
+      {"force_generic", &Knobs::force_generic}, {"no_strip", &Knobs::no_strip}, {"force_strip", &Knobs::force_strip},
+      {"no_box", &Knobs::no_box}, {"no_pim", &Knobs::no_pim}, {"bslice", &Knobs::bslice},
+      {"no_bslice", &Knobs::no_bslice}, {"splitk", &Knobs::splitk}, {"force_stream", &Knobs::force_stream},
+      {"nsets", &Knobs::nsets}, {"no_l2ahead", &Knobs::no_l2ahead}, {"no_btma", &Knobs::no_btma},
+      {"ntiles", &Knobs::ntiles}, {"transform_gather", &Knobs::transform_gather},
+      {"test_skip_copy", &Knobs::test_skip_copy}, {"strip_mh", &Knobs::strip_mh}};
+  for (const Entry& e : table)
+    if (strcmp(e.name, name) == 0) { g_knobs.*(e.field) = value; return IM2WIN_OK; }
+  return IM2WIN_EINVAL;
+}
+#endif
 
 const char* im2win_strerror(int status) {
   switch (status) {
@@ -304,8 +394,19 @@ int im2win_conv_host(const float* in_host, const float* filter_host, const im2wi
   if ((rc = grow(&g_host.d_in, &g_host.b_in, (size_t)g.n_in * 4)) != IM2WIN_OK) return rc;
   if ((rc = grow(&g_host.d_f, &g_host.b_f, (size_t)g.n_flt * 4)) != IM2WIN_OK) return rc;
   if ((rc = grow(&g_host.d_out, &g_host.b_out, (size_t)g.n_out * 4)) != IM2WIN_OK) return rc;
-  // workspace for one chunk: only the shapes without a fused kernel use it
-  if ((rc = grow(&g_host.d_ws, &g_host.b_ws, (size_t)win_img * per * 4)) != IM2WIN_OK) return rc;
+  // workspace for one chunk: the im2win tensor (only the shapes without a fused kernel use it) and
+  // behind it the scratch the tensor-core kernels may want for a copy of the filter
+  size_t ws_need = ((size_t)win_img * per * 4 + 255) / 256 * 256;
+  {
+    im2win_shape shc = *shape;
+    shc.N = per;
+    Geometry gc;
+    if (make_geometry(&shc, &gc) == IM2WIN_OK) {
+      const size_t a = conv_scratch_bytes(gc, mode, 0), b = conv_scratch_bytes(gc, mode, 1);
+      ws_need += a > b ? a : b;
+    }
+  }
+  if ((rc = grow(&g_host.d_ws, &g_host.b_ws, ws_need)) != IM2WIN_OK) return rc;
   if (cudaMemcpyAsync(g_host.d_f, filter_host, (size_t)g.n_flt * 4, cudaMemcpyHostToDevice, g_host.s_in) != cudaSuccess ||
       cudaEventRecord(g_host.ev_in[kHostChunks], g_host.s_in) != cudaSuccess ||
       cudaStreamWaitEvent(g_host.s_cmp, g_host.ev_in[kHostChunks], 0) != cudaSuccess)

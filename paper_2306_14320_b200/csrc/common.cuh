@@ -45,16 +45,61 @@ int32_t* device_status_word();  // device address of the status word (nullptr if
 int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_t st);
 int launch_transform_bf16(const float* in, uint16_t* out, const Geometry& g, cudaStream_t st);
 int launch_conv_fp32(const float* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st);
-// Tensor-core convolution: the persistent specialised kernel when one applies (it returns
-// IM2WIN_EUNSUPPORTED otherwise), else the generic kernel.
+// Device memory from the caller's workspace (beyond the im2win tensor) that a tensor-core convolution
+// may use for a re-laid-out copy of the filter; ptr may be null / bytes 0 (kernels that need such a
+// copy then return IM2WIN_EUNSUPPORTED and the dispatcher moves on).  The library allocates nothing.
+struct Scratch {
+  void* ptr = nullptr;
+  size_t bytes = 0;
+};
+// Tensor-core convolution kernels.  Each returns IM2WIN_EUNSUPPORTED when it does not apply (shape,
+// scratch) before anything is enqueued; launch_conv_tc tries them in order of expected speed.
+// src_kind: 0 = fp32 im2win tensor, 1 = untransformed input consumed fused, 2 = bf16 im2win tensor.
+int launch_conv_tc_strip(const void* src, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st,
+                         Scratch scratch, int src_kind, bool out_bf16);
 int launch_conv_tc_persistent(const void* src, const float* f, float* out, const Geometry& g, int mode,
-                              cudaStream_t st, bool may_alloc, bool fused = false, bool src_bf16 = false, bool out_bf16 = false);
+                              cudaStream_t st, Scratch scratch, bool fused = false, bool src_bf16 = false,
+                              bool out_bf16 = false);
 int launch_conv_tc_generic(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
                            cudaStream_t st);
-// may_alloc = false keeps the call free of any (even stream-ordered) device allocation.
-int launch_conv_tc(const float* xhat, const float* f, float* out, const Geometry& g, int mode,
-                   cudaStream_t st, bool may_alloc = true);
+int launch_conv_tc(const void* src, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st,
+                   Scratch scratch, int src_kind, bool out_bf16);
+// Scratch bytes with which every kernel above is available for this problem (0 if none wants any).
+size_t strip_scratch_bytes(const Geometry& g, int mode, int src_kind);
+size_t persistent_scratch_bytes(const Geometry& g, int mode);
+size_t conv_scratch_bytes(const Geometry& g, int mode, int src_kind);
+// Shared body of im2win_conv / im2win_conv_bf16out / im2win_conv_static (argument checks, workspace
+// split into the im2win tensor and the filter scratch, transform, dispatch).
+int conv_impl(const void* src, int src_kind, const float* filter, const im2win_shape* shape, int mode, void* out,
+              bool out16, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? IM2WIN_OK : IM2WIN_ECUDA; }
+
+// Diagnostic switches of the launchers.  The product library answers knobs() with the constant
+// defaults below and reads no environment; only the test build of api.cu (-DIM2WIN_TEST_KNOBS,
+// linked into libim2win_test.so) keeps a mutable copy and exports im2win_debug_set_option(name, value)
+// to set a field by name, which is how the parity tests force each kernel configuration.
+struct Knobs {
+  int force_generic = 0;     // every tensor-core convolution through the generic kernel
+  int no_strip = 0;          // never use the strip-matrix kernel (conv_tc_strip.cu)
+  int force_strip = 0;       // use the strip-matrix kernel wherever it is implemented, not only where its cost model picks it
+  int no_box = 0;            // persistent kernel: strips by bulk copies instead of 2-D TMA boxes
+  int no_pim = 0;            // persistent kernel: tiles may span images
+  int bslice = 0;            // persistent kernel: force the slice-resident filter mode
+  int no_bslice = 0;         // persistent kernel: never use it
+  int splitk = -1;           // persistent kernel: force this many reduction slices (-1: cost model)
+  int force_stream = 0;      // persistent kernel: stream the filter although it would fit
+  int nsets = 0;             // persistent kernel: 2 or 3 repack sets (0: own choice)
+  int no_l2ahead = 0;        // persistent kernel: no L2 prefetch of the next tile's boxes
+  int no_btma = 0;           // persistent kernel: resident filter built by threads, not fetched by TMA
+  int ntiles = 0;            // persistent kernel: number of filter tiles (0: own choice)
+  int transform_gather = 0;  // transform: the staged-gather kernel instead of the tile kernel
+  int test_skip_copy = 0;    // transform tile kernel, single-CTA problems: announce the input copy, never issue it
+  int strip_mh = 0;          // strip-matrix kernel: 128-row halves per tile (0: own choice)
+};
+const Knobs& knobs();
+
+// Streaming multiprocessors of the current device (cached per device).
+int sm_count();
 
 }  // namespace im2win

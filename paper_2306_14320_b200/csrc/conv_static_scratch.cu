@@ -6,6 +6,8 @@
 // pool sized to the device), or a loop that runs under a "no allocation after start-up" rule, as
 // hard-real-time and safety-reviewed code does.  For them the scratch that im2win_conv takes from
 // the caller (the im2win tensor) lives here, in a file-scope device array of fixed size.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace im2win {
@@ -19,7 +21,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 // In host code `g_static_scratch` is only a handle for the runtime, not a device address.  The
 // address a kernel may use is asked for once per device (with that device current) and kept.
 constexpr int kMaxDevices = 64;
-float* g_scratch_addr[kMaxDevices] = {};
+std::atomic<float*> g_scratch_addr[kMaxDevices];  // (two first calls racing on a device both store the same address)
 
 int scratch_for_current_device(float** out) {
   int dev = -1;
@@ -27,16 +29,18 @@ int scratch_for_current_device(float** out) {
     cudaGetLastError();
     return IM2WIN_ECUDA;
   }
-  if (!g_scratch_addr[dev]) {
+  float* addr = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!addr) {
     void* p = nullptr;
     const cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
     if (e != cudaSuccess || !p) {
       cudaGetLastError();
       return IM2WIN_ECUDA;
     }
-    g_scratch_addr[dev] = static_cast<float*>(p);
+    addr = static_cast<float*>(p);
+    g_scratch_addr[dev].store(addr, std::memory_order_release);
   }
-  *out = g_scratch_addr[dev];
+  *out = addr;
   return IM2WIN_OK;
 }
 
@@ -68,13 +72,11 @@ int im2win_conv_static(const float* in_nchw, const float* filter_kcfhfw, const i
   float* scratch = nullptr;
   rc = scratch_for_current_device(&scratch);  // first call on a device: looks the address up
   if (rc != IM2WIN_OK) return rc;
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  // Nothing in the scratch has to start at zero: the transform writes every element the
-  // convolution reads, so whatever the previous call left behind is overwritten first.
-  rc = launch_transform(in_nchw, scratch, g, st);
-  if (rc != IM2WIN_OK) return rc;
-  if (mode == IM2WIN_MODE_FP32) return launch_conv_fp32(scratch, filter_kcfhfw, out_nchw, g, st);
-  return launch_conv_tc(scratch, filter_kcfhfw, out_nchw, g, mode, st, /*may_alloc=*/false);
+  // Nothing in the scratch has to start at zero: the transform writes every element of the im2win
+  // tensor the convolution reads, and what lies behind that tensor is only ever used for a copy of
+  // the filter that the same call writes first.  Whatever the previous call left behind is overwritten.
+  return conv_impl(in_nchw, IM2WIN_SRC_NCHW, filter_kcfhfw, shape, mode, out_nchw, /*out16=*/false, scratch,
+                   kStaticScratchBytes, cuda_stream);
 }
 
 }  // extern "C"

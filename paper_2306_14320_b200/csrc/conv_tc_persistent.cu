@@ -1145,44 +1145,8 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Memory pool for the temporary bf16 filter copies: the library's own, with an unlimited release
-// threshold, so that after the first call the stream-ordered allocation is served from cached
-// memory instead of going back to the driver.
-cudaMemPool_t filter_pool() {
-  static cudaMemPool_t pools[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return nullptr; }
-  if (!pools[dev]) {
-    cudaMemPoolProps props = {};
-    props.allocType = cudaMemAllocationTypePinned;
-    props.handleTypes = cudaMemHandleTypeNone;
-    props.location.type = cudaMemLocationTypeDevice;
-    props.location.id = dev;
-    cudaMemPool_t pool = nullptr;
-    if (cudaMemPoolCreate(&pool, &props) != cudaSuccess) { cudaGetLastError(); return nullptr; }
-    uint64_t keep = UINT64_MAX;
-    if (cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep) != cudaSuccess) cudaGetLastError();
-    pools[dev] = pool;
-  }
-  return pools[dev];
-}
-
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
-      cudaGetLastError();
-      n = 0;
-      return 148;
-    }
-  }
-  return n;
-}
-
 template <int FH, int FW, int CB, bool BF16, bool FUSED, bool SRC16 = false, bool OUT16 = false>
-int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc) {
+int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st, Scratch scratch) {
   constexpr bool out16 = OUT16;
   constexpr int FF = FH * FW;
   constexpr int64_t ES = SRC16 ? 2 : 4;    // bytes per source element
@@ -1218,9 +1182,9 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
     // Filter tiles stay as wide as the MMA allows (256): a unit of work costs the same number of MMA
     // instructions and window repacks whatever its width, and narrow MMAs are bound by the issuing
     // thread, so splitting K further to even out the last wave loses (measured).  Tuning aid only:
-    const char* fix = getenv("IM2WIN_NTILES");
-    if (fix && fix[0] >= '1' && fix[0] <= '8' && (g.K + (fix[0] - '0') - 1) / (fix[0] - '0') <= 256) {
-      P.n_ntiles = fix[0] - '0';
+    const int fix = knobs().ntiles;
+    if (fix >= 1 && fix <= 8 && (g.K + fix - 1) / fix <= 256) {
+      P.n_ntiles = fix;
       P.NT = ((g.K + P.n_ntiles - 1) / P.n_ntiles + 15) / 16 * 16;
     }
   }
@@ -1253,19 +1217,17 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
     while ((CB * row_align * ES) % 128 != 0) row_align *= 2;
     const int64_t boxf = (one_seg + row_align - 1) / row_align * row_align;
     const bool little_waste = tpi * 128 * 100 <= g.HoWo * 107;
-    const char* nobox = getenv("IM2WIN_NO_BOX");
-    const char* nopim = getenv("IM2WIN_NO_PIM");
     if (little_waste && tp == 128 && P.plane < ((int64_t)1 << 30) && (g.HoWo + 128) * g.Wo < ((int64_t)1 << 32) &&
-        (int64_t)g.N * tpi * tpi < ((int64_t)1 << 32) && one_seg <= (1 << 20) && !(nopim && nopim[0] == '1')) {
+        (int64_t)g.N * tpi * tpi < ((int64_t)1 << 32) && one_seg <= (1 << 20) && !knobs().no_pim) {
       P.pim = 1;
       P.TPI = (int32_t)tpi;
       P.magic_TPI = (((uint64_t)1 << 32) + (uint64_t)tpi - 1) / (uint64_t)tpi;
       P.magic_Wo = (((uint64_t)1 << 32) + (uint64_t)g.Wo - 1) / (uint64_t)g.Wo;
       pitch = (one_seg + EPC - 1) / EPC * EPC;
       if (CB >= 2 && (P.plane % EPC) == 0 && boxf * ES <= 2048 && encode_fn() != nullptr && (int64_t)g.N * g.C <= INT32_MAX &&
-          !(nobox && nobox[0] == '1')) {
+          !knobs().no_box) {
         P.box = 1;
-        P.l2_ahead = !(getenv("IM2WIN_NO_L2AHEAD") && getenv("IM2WIN_NO_L2AHEAD")[0] == '1');
+        P.l2_ahead = !knobs().no_l2ahead;
         pitch = boxf;
       }
     }
@@ -1280,14 +1242,16 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   const int64_t cap = 227 * 1024 - 1024 - 1024 - ((int64_t)(P.win_span + 8) * 4 + 16);  // alignment slack, barriers, zero pad
   const int64_t b_res = (int64_t)steps_tile * P.NT * 32;  // one 32-byte-swizzled block per MMA step
   bool resident = P.n_ntiles == 1 && b_res + 2 * raw_stage <= cap;
-  if (getenv("IM2WIN_FORCE_STREAM") && getenv("IM2WIN_FORCE_STREAM")[0] == '1') resident = false;  // test knob
+  if (knobs().force_stream) resident = false;  // test knob
   // Streaming the native TF32 filter needs dense groups (padded reduction index == real index) and
-  // 16-byte aligned filter rows.  In BF16 mode the TMA source is a bf16 copy of the filter made for
-  // the duration of the call in memory from the stream-ordered pool (only where the caller allows an
-  // allocation); that copy is written with padded groups where the groups are not dense.
+  // 16-byte aligned filter rows.  In BF16 mode the TMA source is a bf16 copy of the filter, written at
+  // the start of the call into scratch memory the caller supplied beyond the im2win tensor (without
+  // enough scratch this kernel does not apply); that copy has padded groups where the groups are not dense.
   const bool pad_copy = BF16 && KCG != KCGP;
+  const int64_t copy_row = pad_copy ? (int64_t)((g.C + CB - 1) / CB) * KCGP : g.Kg;
+  const bool have_copy_room = scratch.ptr && (int64_t)scratch.bytes >= (int64_t)g.K * copy_row * 2;
   const bool can_stream = (g.C % CB) == 0 && encode_fn() != nullptr &&
-                          (BF16 ? may_alloc && (pad_copy || (g.Kg % 8) == 0) : KCG == KCGP && (g.Kg % 4) == 0);
+                          (BF16 ? have_copy_room && (pad_copy || (g.Kg % 8) == 0) : KCG == KCGP && (g.Kg % 4) == 0);
   if (!resident && !can_stream) return IM2WIN_EUNSUPPORTED;
   // Slice-resident mode.  A filter that does not fit whole may fit as one reduction slice per CTA:
   // the units are (tile, slice) with the slice fastest, so with a grid that is a multiple of Z every
@@ -1298,9 +1262,8 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   // channels (Table I Conv4: C = 64, 7x7, K = 64) -- estimated against the streamed mode, whose
   // issuing threads spend about 200 cycles per MMA (measured), in microseconds at 1.9 GHz.
   int32_t bs_z = 0, bs_gz = 0;
-  const bool bs_force = getenv("IM2WIN_BSLICE") && getenv("IM2WIN_BSLICE")[0] == '1';  // test knob
-  if ((!resident || bs_force) && P.n_ntiles == 1 && !out16 &&
-      !(getenv("IM2WIN_NO_BSLICE") && getenv("IM2WIN_NO_BSLICE")[0] == '1')) {
+  const bool bs_force = knobs().bslice != 0;  // test knob
+  if ((!resident || bs_force) && P.n_ntiles == 1 && !out16 && !knobs().no_bslice) {
     const int nsm = sm_count();
     for (int32_t z = 2; z <= 16 && z <= P.NG && z <= nsm; ++z) {
       const int32_t gz = (P.NG + z - 1) / z;
@@ -1341,15 +1304,14 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   int32_t sr_max = (int32_t)((cap - b_bytes) / raw_stage);
   if (sr_max > kMaxStages) sr_max = kMaxStages;
   P.NSETS = (sr_max / 3 * 3 >= 6 || sr_max == 3) ? 3 : 2;
-  if (const char* fix = getenv("IM2WIN_NSETS")) {
-    if (fix[0] == '2' || fix[0] == '3') P.NSETS = fix[0] - '0';
-  }
+  const bool nsets_fixed = knobs().nsets == 2 || knobs().nsets == 3;
+  if (nsets_fixed) P.NSETS = knobs().nsets;
   // TMEM: accumulators first, then the rings of A slots, one ring of NSS slots per set (a barrier
   // must be waited on by one party that sees every one of its phases, so the sets cannot share slots)
   P.ND = (2 * P.NT + P.NSETS * SLOT_COLS <= 512) ? 2 : 1;
   // a third set only pays where every set still owns at least two slots (a set with one slot waits
   // for the MMAs of each part before it can store the next)
-  if ((512 - P.ND * P.NT) / SLOT_COLS / P.NSETS < 2 && !getenv("IM2WIN_NSETS")) P.NSETS = 2;
+  if ((512 - P.ND * P.NT) / SLOT_COLS / P.NSETS < 2 && !nsets_fixed) P.NSETS = 2;
   P.ND = (2 * P.NT + P.NSETS * SLOT_COLS <= 512) ? 2 : 1;
   if (P.ND * P.NT + P.NSETS * SLOT_COLS > 512) P.NSETS = 2;
   P.SR = sr_max / P.NSETS * P.NSETS;
@@ -1381,8 +1343,7 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
     int32_t gmul = 1;
     if (!resident) while ((gmul * S) % 4 != 0) ++gmul;
     double best = cost(1, P.NG) * 0.92;  // a split must win clearly
-    int forced = -1;
-    if (const char* fix = getenv("IM2WIN_SPLITK")) forced = atoi(fix);
+    int forced = knobs().splitk;
     if (out16) forced = 1;  // partial sums cannot be added into a bf16 output
     for (int32_t z = 2; z <= 16 && z <= P.NG; ++z) {
       int32_t gz = (P.NG + z - 1) / z;
@@ -1411,9 +1372,9 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
 
   CUtensorMap fmap;
   memset(&fmap, 0, sizeof(fmap));
-  void* f_bf16 = nullptr;  // BF16 streamed mode: temporary bf16 copy of the filter
+  void* f_bf16 = nullptr;  // BF16 streamed mode: bf16 copy of the filter in the caller's scratch
   if (resident && !BF16 && KCG == KCGP && (g.C % CB) == 0 && (g.Kg % 4) == 0 && encode_fn() != nullptr &&
-      !(getenv("IM2WIN_NO_BTMA") && getenv("IM2WIN_NO_BTMA")[0] == '1')) {
+      !knobs().no_btma) {
     // the native filter as a K x Kg matrix, fetched one MMA step (8 reduction elements) at a time
     const cuuint64_t gdim[2] = {(cuuint64_t)g.Kg, (cuuint64_t)g.K};
     const cuuint64_t gstr[1] = {(cuuint64_t)g.Kg * 4};
@@ -1432,12 +1393,8 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
     const cuuint32_t estr[2] = {1, 1};
     void* base = const_cast<float*>(f);
     if (BF16) {
-      cudaMemPool_t pool = filter_pool();
       const int64_t n_copy = (int64_t)g.K * row;
-      if (!pool || cudaMallocFromPoolAsync(&f_bf16, (size_t)n_copy * 2, pool, st) != cudaSuccess) {
-        cudaGetLastError();
-        return IM2WIN_EUNSUPPORTED;
-      }
+      f_bf16 = scratch.ptr;
       const int64_t blocks = (n_copy + 255) / 256;
       const unsigned nb = (unsigned)(blocks < 148 * 8 ? blocks : 148 * 8);
       if (pad_copy)
@@ -1450,7 +1407,6 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
     if (encode_fn()(&fmap, BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, gdim,
                     gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
-      if (f_bf16) cudaFreeAsync(f_bf16, st);
       return IM2WIN_EUNSUPPORTED;
     }
   }
@@ -1465,7 +1421,6 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
     if (encode_fn()(&xmap, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(xhat), gdim, gstr, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
-      if (f_bf16) cudaFreeAsync(f_bf16, st);
       return IM2WIN_ECUDA;
     }
   }
@@ -1474,7 +1429,6 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   cudaError_t e;
   if (P.Z > 1 && cudaMemsetAsync(out, 0, (size_t)g.n_out * 4, st) != cudaSuccess) {  // (Z > 1 implies an fp32 output)
     cudaGetLastError();
-    if (f_bf16) cudaFreeAsync(f_bf16, st);
     return IM2WIN_ECUDA;
   }
   if (resident) {
@@ -1485,39 +1439,37 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   } else {
     auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, false, FUSED, SRC16, OUT16>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-    if (e != cudaSuccess) { cudaGetLastError(); if (f_bf16) cudaFreeAsync(f_bf16, st); return IM2WIN_ECUDA; }
+    if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
     kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
   }
-  const int rc = cuda_status(cudaGetLastError());
-  if (f_bf16) cudaFreeAsync(f_bf16, st);  // stream-ordered: released after the kernel has run
-  return rc;
+  return cuda_status(cudaGetLastError());
 }
 
 // src_kind: 0 = im2win tensor (fp32), 1 = untransformed input consumed fused, 2 = im2win tensor stored as bf16
 template <int FH, int FW, int CB, bool BF16>
-int launch_spec(const void* src, const float* f, float* out, const Geometry& g, cudaStream_t st, bool may_alloc,
+int launch_spec(const void* src, const float* f, float* out, const Geometry& g, cudaStream_t st, Scratch scratch,
                 int src_kind, bool out16) {
   if (out16) {  // the bf16 epilogue exists for the unfused sources
     if (src_kind == 1) return IM2WIN_EUNSUPPORTED;
     if (src_kind == 2) {
-      if constexpr (BF16) return launch_spec_impl<FH, FW, CB, true, false, true, true>(src, f, out, g, st, may_alloc);
+      if constexpr (BF16) return launch_spec_impl<FH, FW, CB, true, false, true, true>(src, f, out, g, st, scratch);
       else return IM2WIN_EUNSUPPORTED;
     }
-    return launch_spec_impl<FH, FW, CB, BF16, false, false, true>(src, f, out, g, st, may_alloc);
+    return launch_spec_impl<FH, FW, CB, BF16, false, false, true>(src, f, out, g, st, scratch);
   }
   if (src_kind == 2) {
-    if constexpr (BF16) return launch_spec_impl<FH, FW, CB, true, false, true>(src, f, out, g, st, may_alloc);
+    if constexpr (BF16) return launch_spec_impl<FH, FW, CB, true, false, true>(src, f, out, g, st, scratch);
     else return IM2WIN_EUNSUPPORTED;
   }
-  return src_kind == 1 ? launch_spec_impl<FH, FW, CB, BF16, true>(src, f, out, g, st, may_alloc)
-                       : launch_spec_impl<FH, FW, CB, BF16, false>(src, f, out, g, st, may_alloc);
+  return src_kind == 1 ? launch_spec_impl<FH, FW, CB, BF16, true>(src, f, out, g, st, scratch)
+                       : launch_spec_impl<FH, FW, CB, BF16, false>(src, f, out, g, st, scratch);
 }
 
 }  // namespace
 
 // Returns IM2WIN_EUNSUPPORTED when no specialisation applies (the caller then uses the generic kernel).
-// may_alloc: whether the call may take temporary device memory from the stream-ordered pool (the
-// BF16 copy of a filter that is too large to stay in shared memory).
+// scratch: device memory of the caller's (beyond the im2win tensor) for the bf16 copy of a filter that
+// is too large to stay in shared memory (BF16 mode); without it those shapes are declined.
 // fused: `xhat` is the untransformed NCHW input and the windows are built from staged input rows
 // (no im2win tensor exists in global memory).
 // The filter-size families are separate functions so that the build can compile them as separate
@@ -1527,7 +1479,7 @@ int launch_spec(const void* src, const float* f, float* out, const Geometry& g, 
 #define IM2WIN_PART -1
 #endif
 #define IM2WIN_SPEC_ARGS const void* xhat, const float* f, float* out, const Geometry& g, cudaStream_t st, \
-                         bool may_alloc, int kind, bool out_bf16, bool bf16
+                         Scratch scratch, int kind, bool out_bf16, bool bf16
 int launch_spec_3x3(IM2WIN_SPEC_ARGS);
 int launch_spec_5x5(IM2WIN_SPEC_ARGS);
 int launch_spec_7x7(IM2WIN_SPEC_ARGS);
@@ -1536,19 +1488,19 @@ int launch_spec_11x11(IM2WIN_SPEC_ARGS);
 #if IM2WIN_PART == -1 || IM2WIN_PART == 0
 int launch_spec_3x3(IM2WIN_SPEC_ARGS) {
   // BF16 MMAs take 16 reduction elements: sixteen channels (144 = 9 steps) leave no padding
-  if (bf16 && g.C % 16 == 0) return launch_spec<3, 3, 16, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
-  if (g.C >= 8) return bf16 ? launch_spec<3, 3, 8, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16)
-                            : launch_spec<3, 3, 8, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
-  if (g.C == 3) return bf16 ? launch_spec<3, 3, 3, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16)
-                            : launch_spec<3, 3, 3, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  if (bf16 && g.C % 16 == 0) return launch_spec<3, 3, 16, true>(xhat, f, out, g, st, scratch, kind, out_bf16);
+  if (g.C >= 8) return bf16 ? launch_spec<3, 3, 8, true>(xhat, f, out, g, st, scratch, kind, out_bf16)
+                            : launch_spec<3, 3, 8, false>(xhat, f, out, g, st, scratch, kind, out_bf16);
+  if (g.C == 3) return bf16 ? launch_spec<3, 3, 3, true>(xhat, f, out, g, st, scratch, kind, out_bf16)
+                            : launch_spec<3, 3, 3, false>(xhat, f, out, g, st, scratch, kind, out_bf16);
   return IM2WIN_EUNSUPPORTED;
 }
 #endif
 #if IM2WIN_PART == -1 || IM2WIN_PART == 1
 int launch_spec_5x5(IM2WIN_SPEC_ARGS) {
-  if (bf16 && g.C % 16 == 0) return launch_spec<5, 5, 16, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
-  if (g.C >= 8) return bf16 ? launch_spec<5, 5, 8, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16)
-                            : launch_spec<5, 5, 8, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  if (bf16 && g.C % 16 == 0) return launch_spec<5, 5, 16, true>(xhat, f, out, g, st, scratch, kind, out_bf16);
+  if (g.C >= 8) return bf16 ? launch_spec<5, 5, 8, true>(xhat, f, out, g, st, scratch, kind, out_bf16)
+                            : launch_spec<5, 5, 8, false>(xhat, f, out, g, st, scratch, kind, out_bf16);
   return IM2WIN_EUNSUPPORTED;
 }
 #endif
@@ -1559,36 +1511,45 @@ int launch_spec_7x7(IM2WIN_SPEC_ARGS) {
       // sixteen channels per group leave no padding (784 = 49 steps); where two strip stages of
       // sixteen channels do not fit (wide images), eight channels with a padded filter copy do
       int rc = IM2WIN_EUNSUPPORTED;
-      if (g.C % 16 == 0) rc = launch_spec<7, 7, 16, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
-      if (rc == IM2WIN_EUNSUPPORTED) rc = launch_spec<7, 7, 8, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+      if (g.C % 16 == 0) rc = launch_spec<7, 7, 16, true>(xhat, f, out, g, st, scratch, kind, out_bf16);
+      if (rc == IM2WIN_EUNSUPPORTED) rc = launch_spec<7, 7, 8, true>(xhat, f, out, g, st, scratch, kind, out_bf16);
       return rc;
     }
-    return launch_spec<7, 7, 8, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+    return launch_spec<7, 7, 8, false>(xhat, f, out, g, st, scratch, kind, out_bf16);
   }
-  if (g.C == 3) return bf16 ? launch_spec<7, 7, 3, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16)
-                            : launch_spec<7, 7, 3, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  if (g.C == 3) return bf16 ? launch_spec<7, 7, 3, true>(xhat, f, out, g, st, scratch, kind, out_bf16)
+                            : launch_spec<7, 7, 3, false>(xhat, f, out, g, st, scratch, kind, out_bf16);
   return IM2WIN_EUNSUPPORTED;
 }
 #endif
 #if IM2WIN_PART == -1 || IM2WIN_PART == 3
 int launch_spec_11x11(IM2WIN_SPEC_ARGS) {
-  if (g.C <= 4) return bf16 ? launch_spec<11, 11, 1, true>(xhat, f, out, g, st, may_alloc, kind, out_bf16)
-                            : launch_spec<11, 11, 1, false>(xhat, f, out, g, st, may_alloc, kind, out_bf16);
+  if (g.C <= 4) return bf16 ? launch_spec<11, 11, 1, true>(xhat, f, out, g, st, scratch, kind, out_bf16)
+                            : launch_spec<11, 11, 1, false>(xhat, f, out, g, st, scratch, kind, out_bf16);
   return IM2WIN_EUNSUPPORTED;
 }
 #endif
 
 #if IM2WIN_PART == -1 || IM2WIN_PART == 0
 int launch_conv_tc_persistent(const void* xhat, const float* f, float* out, const Geometry& g, int mode,
-                              cudaStream_t st, bool may_alloc, bool fused, bool src_bf16, bool out_bf16) {
+                              cudaStream_t st, Scratch scratch, bool fused, bool src_bf16, bool out_bf16) {
   const int kind = src_bf16 ? 2 : (fused ? 1 : 0);
   if (src_bf16 && (fused || mode != IM2WIN_MODE_BF16)) return IM2WIN_EUNSUPPORTED;
   const bool bf16 = mode == IM2WIN_MODE_BF16;
-  if (g.Fh == 3 && g.Fw == 3) return launch_spec_3x3(xhat, f, out, g, st, may_alloc, kind, out_bf16, bf16);
-  if (g.Fh == 5 && g.Fw == 5) return launch_spec_5x5(xhat, f, out, g, st, may_alloc, kind, out_bf16, bf16);
-  if (g.Fh == 7 && g.Fw == 7) return launch_spec_7x7(xhat, f, out, g, st, may_alloc, kind, out_bf16, bf16);
-  if (g.Fh == 11 && g.Fw == 11) return launch_spec_11x11(xhat, f, out, g, st, may_alloc, kind, out_bf16, bf16);
+  if (g.Fh == 3 && g.Fw == 3) return launch_spec_3x3(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh == 5 && g.Fw == 5) return launch_spec_5x5(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh == 7 && g.Fw == 7) return launch_spec_7x7(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh == 11 && g.Fw == 11) return launch_spec_11x11(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
   return IM2WIN_EUNSUPPORTED;
+}
+
+// Upper bound of the scratch bytes any BF16 specialisation asks for: a bf16 copy of the filter whose
+// channel groups (8 or 16 channels, or fewer for tiny C) are padded to whole MMA steps of 16.
+size_t persistent_scratch_bytes(const Geometry& g, int mode) {
+  if (mode != IM2WIN_MODE_BF16) return 0;
+  const int64_t ff = g.FF;
+  const int64_t row = g.C >= 8 ? (int64_t)((g.C + 7) / 8) * ((8 * ff + 15) / 16 * 16) : (int64_t)g.C * ((ff + 15) / 16 * 16);
+  return (size_t)((int64_t)g.K * row * 2 + 255) / 256 * 256;
 }
 
 #ifdef IM2WIN_PROF

@@ -500,8 +500,7 @@ int launch_transform_tile(const float* in, void* out, bool out16, const Geometry
   P.QW = (g.W + 3) / 4;
   {
     // honoured for single-CTA problems only: every CTA would wait out its own second otherwise
-    const char* hook = getenv("IM2WIN_TEST_SKIP_COPY");
-    P.test_skip_copy = (hook && hook[0] == '1' && ctas == 1) ? 1 : 0;
+    P.test_skip_copy = (knobs().test_skip_copy && ctas == 1) ? 1 : 0;
   }
   P.planes = planes; P.HW = hw; P.HoL = g.HoL; P.n_in_total = g.n_in;
   const int64_t units_plane = (int64_t)(nblk == 1 ? g.Ho : MB) * P.QW;
@@ -589,8 +588,7 @@ static int launch_transform_staged(const float* in, float* out, uint16_t* out16,
 
 int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_t st) {
   {
-    const char* old = getenv("IM2WIN_TRANSFORM_GATHER");
-    if (!(old && old[0] == '1')) {
+    if (!knobs().transform_gather) {
       const int rc = launch_transform_tile(in, out, false, g, st);
       if (rc != IM2WIN_EUNSUPPORTED) return rc;
     }
@@ -600,8 +598,7 @@ int launch_transform(const float* in, float* out, const Geometry& g, cudaStream_
 
 int launch_transform_bf16(const float* in, uint16_t* out, const Geometry& g, cudaStream_t st) {
   {
-    const char* old = getenv("IM2WIN_TRANSFORM_GATHER");
-    if (!(old && old[0] == '1')) {
+    if (!knobs().transform_gather) {
       const int rc = launch_transform_tile(in, out, true, g, st);
       if (rc != IM2WIN_EUNSUPPORTED) return rc;
     }

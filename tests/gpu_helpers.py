@@ -17,6 +17,51 @@ def ensure_built():
     build.build_library()
 
 
+# Kernel configurations of the convolution parity tests.  "auto" and "minws" run the PRODUCT library
+# (its own choice of kernel; "minws" with the smallest legal workspace, i.e. without scratch for a
+# filter copy); every other one runs the test build of the same code with one diagnostic switch set.
+CONV_CONFIGS = {
+    "auto": {}, "minws": {}, "strip": {"force_strip": 1}, "strip2": {"force_strip": 1, "strip_mh": 2},
+    "nostrip": {"no_strip": 1},
+    "nobox": {"no_strip": 1, "no_box": 1}, "nopim": {"no_strip": 1, "no_pim": 1},
+    "split3": {"no_strip": 1, "splitk": 3}, "bslice": {"no_strip": 1, "bslice": 1}, "generic": {"force_generic": 1},
+}
+_KNOB_DEFAULTS = {"force_generic": 0, "no_strip": 0, "force_strip": 0, "no_box": 0, "no_pim": 0, "bslice": 0,
+                  "no_bslice": 0, "splitk": -1, "force_stream": 0, "nsets": 0, "no_l2ahead": 0, "no_btma": 0,
+                  "ntiles": 0, "transform_gather": 0, "test_skip_copy": 0, "strip_mh": 0}
+_min_workspace = False
+
+
+def apply_config(name: str = "auto", **extra) -> None:
+    """Selects the library (product or test build) and sets the switches of configuration `name`."""
+    global _min_workspace
+    knobs = dict(CONV_CONFIGS.get(name, {}), **extra)
+    _min_workspace = name == "minws"
+    b.use_test_library(bool(knobs))
+    if knobs:
+        for k, v in _KNOB_DEFAULTS.items():
+            b.set_option(k, knobs.get(k, v))
+
+
+def reset_config() -> None:
+    global _min_workspace
+    _min_workspace = False
+    b.use_test_library(True)
+    for k, v in _KNOB_DEFAULTS.items():
+        b.set_option(k, v)
+    b.use_test_library(False)
+
+
+def conv_workspace_floats(dims, src_kind: int, mode: int) -> int:
+    """Workspace the tests hand to im2win_conv: what im2win_conv_workspace_bytes asks for (room for
+    the im2win tensor in every case, so that the documented fallbacks can run), or in the "minws"
+    configuration only the im2win tensor."""
+    least = b.workspace_bytes(dims)
+    if _min_workspace:
+        return least // 4
+    return max(least, b.conv_workspace_bytes(dims, b.SRC_NCHW, mode), b.conv_workspace_bytes(dims, src_kind, mode)) // 4
+
+
 class Guarded:
     """A device buffer of n floats with sentinel-filled guard bands on both sides; the payload is
     pre-filled with the sentinel too, so elements a kernel forgets to write are seen."""
@@ -50,9 +95,8 @@ def gpu_conv(x: np.ndarray, f: np.ndarray, dims, mode: int, src_kind: int = b.SR
     xd = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda()
     fd = torch.from_numpy(np.ascontiguousarray(f, dtype=np.float32)).cuda()
     out = Guarded(n * k * ho * wo)
-    ws = Guarded(b.workspace_bytes(dims) // 4) if src_kind in (b.SRC_NCHW, b.SRC_NCHW_FUSED) else None
-    b.conv(xd, src_kind, fd, dims, mode, out.view, None if ws is None else ws.view,
-           0 if ws is None else ws.n * 4)
+    ws = Guarded(conv_workspace_floats(dims, src_kind, mode))
+    b.conv(xd, src_kind, fd, dims, mode, out.view, ws.view, ws.n * 4)
     status = b.last_device_status()
     assert status == 0, f"device status {status}"
     if ws is not None:

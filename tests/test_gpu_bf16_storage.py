@@ -9,7 +9,7 @@ import torch
 import oracle
 from paper_2306_14320_b200 import binding as b
 from paper_2306_14320_b200 import workloads as wl
-from gpu_helpers import GUARD, TOL, Guarded, ensure_built, oracle_conv, rel_l2
+from gpu_helpers import GUARD, TOL, Guarded, apply_config, conv_workspace_floats, ensure_built, oracle_conv, rel_l2, reset_config
 
 pytestmark = pytest.mark.gpu
 
@@ -29,10 +29,12 @@ def _built():
 
 
 @pytest.fixture(params=["auto", "gather"], autouse=True)
-def _kernel(request, monkeypatch):
-    """Every case runs with the library's own choice of transform kernel (the TMA tile kernel where it
-    applies) and with the staged-gather kernel forced."""
-    monkeypatch.setenv("IM2WIN_TRANSFORM_GATHER", "1" if request.param == "gather" else "0")
+def _kernel(request):
+    """Every case runs with the product library's own choice of transform kernel (the TMA tile kernel
+    where it applies) and with the staged-gather kernel forced (a switch of the test build)."""
+    apply_config("gather" if request.param == "gather" else "auto", **({"transform_gather": 1} if request.param == "gather" else {}))
+    yield request.param
+    reset_config()
 
 
 def bf16_rne_bits(a: np.ndarray) -> np.ndarray:
@@ -71,8 +73,10 @@ def gpu_conv_from_bf16(ihat16: Guarded16, f: np.ndarray, dims) -> np.ndarray:
     ho, wo = b.out_dims(dims)
     fd = torch.from_numpy(np.ascontiguousarray(f, dtype=np.float32)).cuda()
     out = Guarded(n * k * ho * wo)
-    b.conv(ihat16.view, b.SRC_IM2WIN_BF16, fd, dims, b.MODE_BF16, out.view)
+    ws = Guarded(max(64, b.conv_workspace_bytes(dims, b.SRC_IM2WIN_BF16, b.MODE_BF16) // 4))  # scratch for a filter copy
+    b.conv(ihat16.view, b.SRC_IM2WIN_BF16, fd, dims, b.MODE_BF16, out.view, ws.view, ws.n * 4)
     assert b.last_device_status() == 0
+    ws.check()
     return out.check().reshape(n, k, ho, wo)
 
 
@@ -93,10 +97,13 @@ def test_transform_bf16_bit_exact_layer_shapes(name, batch):
     assert np.array_equal(gpu_transform_bf16(x, layer.dims()).check(), ref)
 
 
-@pytest.mark.parametrize("staging", ["box", "bulk"])
+@pytest.mark.parametrize("staging", ["auto", "box", "bulk"])
 @pytest.mark.parametrize("name,batch", LAYERS)
-def test_conv_from_bf16_im2win_tensor(name, batch, staging, monkeypatch):
-    monkeypatch.setenv("IM2WIN_NO_BOX", "1" if staging == "bulk" else "0")
+def test_conv_from_bf16_im2win_tensor(name, batch, staging, _kernel):
+    """staging: the library's own choice of kernel; the persistent kernel with 2-D TMA boxes; the same
+    with bulk copies."""
+    if staging != "auto":
+        apply_config(staging, no_strip=1, no_box=1 if staging == "bulk" else 0, transform_gather=1 if _kernel == "gather" else 0)
     layer = wl.CONFIGS[name].with_batch(batch)
     dims = layer.dims()
     x, f = wl.make_input(layer), wl.make_filter(layer)
@@ -153,12 +160,10 @@ def gpu_conv_bf16out(x: np.ndarray, f: np.ndarray, dims, mode: int, src_kind: in
     xd = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda()
     fd = torch.from_numpy(np.ascontiguousarray(f, dtype=np.float32)).cuda()
     out = Guarded16(n * k * ho * wo)
-    ws = Guarded(b.workspace_bytes(dims) // 4) if src_kind in (b.SRC_NCHW, b.SRC_NCHW_FUSED) else None
-    b.conv_bf16out(xd, src_kind, fd, dims, mode, out.view, None if ws is None else ws.view,
-                   0 if ws is None else ws.n * 4)
+    ws = Guarded(conv_workspace_floats(dims, src_kind, mode))
+    b.conv_bf16out(xd, src_kind, fd, dims, mode, out.view, ws.view, ws.n * 4)
     assert b.last_device_status() == 0
-    if ws is not None:
-        ws.check()
+    ws.check()
     return out.check().reshape(n, k, ho, wo)
 
 

@@ -12,7 +12,7 @@ import pytest
 import oracle
 from paper_2306_14320_b200 import binding as b
 from paper_2306_14320_b200 import workloads as wl
-from gpu_helpers import TOL, ensure_built, gpu_conv, oracle_conv, rel_l2
+from gpu_helpers import CONV_CONFIGS, TOL, apply_config, ensure_built, gpu_conv, oracle_conv, rel_l2, reset_config
 
 pytestmark = pytest.mark.gpu
 
@@ -38,24 +38,18 @@ def _built():
     ensure_built()
 
 
-@pytest.fixture(params=["auto", "nobox", "nopim", "split3", "bslice", "generic"], autouse=True)
-def _kernel(request, monkeypatch):
-    """Every case runs six times: with the library's own choice of tensor-core kernel (the persistent,
-    filter-size-specialised one where it applies, tiles cut per image and strips staged by 2-D TMA
-    boxes where they qualify, reduction slices where its cost model wants them), with the box staging
-    switched off (per-image tiles, bulk copies), with per-image tiling switched off as well (tiles
-    that span images), with three reduction slices forced wherever a layer has that many channel
-    groups (partial sums added into the zeroed output), with the slice-resident filter mode forced
-    (every CTA keeps one reduction slice of the filter in shared memory), and with the generic kernel
-    forced."""
-    monkeypatch.setenv("IM2WIN_FORCE_GENERIC", "1" if request.param == "generic" else "0")
-    monkeypatch.setenv("IM2WIN_NO_BOX", "1" if request.param == "nobox" else "0")
-    monkeypatch.setenv("IM2WIN_NO_PIM", "1" if request.param == "nopim" else "0")
-    monkeypatch.setenv("IM2WIN_BSLICE", "1" if request.param == "bslice" else "0")
-    if request.param == "split3":
-        monkeypatch.setenv("IM2WIN_SPLITK", "3")
-    else:
-        monkeypatch.delenv("IM2WIN_SPLITK", raising=False)
+@pytest.fixture(params=list(CONV_CONFIGS), autouse=True)
+def _kernel(request):
+    """Every case runs once per kernel configuration: the product library's own choice ("auto"; the
+    same with the smallest legal workspace, "minws"), and the test build with one switch set -- the
+    strip-matrix kernel forced wherever it is implemented (one and two 128-row halves per tile), the
+    strip-matrix kernel off (the persistent, filter-size-specialised kernel's own choice), that kernel
+    with box staging off (per-image tiles, bulk copies), with per-image tiling off as well (tiles that
+    span images), with three reduction slices forced, with the slice-resident filter mode forced, and
+    the generic kernel forced."""
+    apply_config(request.param)
+    yield request.param
+    reset_config()
 
 
 def _data(dims, seed, ints=False):
@@ -182,30 +176,139 @@ def test_conv_table1_layers_batch1(layer, mode):
     assert rel_l2(gpu_conv(x, f, layer.dims(), mode), oracle_conv(x, f, layer.dims())) <= TOL[mode]
 
 
+# Inputs and oracle results of the full-size cases, computed once per module (every case runs in
+# several kernel configurations, and the oracle takes seconds per layer at batch 128).
+_CACHE: dict = {}
+
+
+def _cached(key, make):
+    if key not in _CACHE:
+        _CACHE[key] = make()
+    return _CACHE[key]
+
+
+def _layer_ints(layer):
+    n, c, h, w, k, fh, fw, s = layer.dims()
+    x = wl.small_ints(9000 + layer.seed, n * c * h * w).reshape(n, c, h, w)
+    f = wl.small_ints(9500 + layer.seed, k * c * fh * fw, -2, 2).reshape(k, c, fh, fw)
+    return x, f
+
+
+def _exact_f32(ref64):
+    """The oracle's fp64 result as fp32, after checking that the conversion loses nothing."""
+    assert np.abs(ref64).max() < 2 ** 24 and np.array_equal(ref64, np.rint(ref64))
+    return ref64.astype(np.float32)
+
+
+FULL = ["resnet3x3", "stem7x7", "deep3x3", "down3x3"]
+
+
 @pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
-@pytest.mark.parametrize("name", ["resnet3x3", "stem7x7", "deep3x3", "down3x3"])
-def test_conv_full_batch_sampled(name, mode):
-    """Batch 128, the launch configuration the benchmark times.  The oracle evaluates Eq. (1) at 20000
-    sampled output coordinates (plus every corner of the output tensor) and at the whole first and
-    last image."""
+@pytest.mark.parametrize("src", ["nchw", "fused"])
+@pytest.mark.parametrize("name", FULL)
+def test_conv_full_batch_small_integers_whole_tensor_bit_exact(name, src, mode, _kernel):
+    """Batch 128, the launch configuration the benchmark times (ring phases wrapping over ~170 tiles
+    per CTA, the look-ahead of the next tile, the last partial wave): on small-integer data every one
+    of the 6 to 103 million outputs must equal the oracle's Eq. (1) exactly."""
+    if src == "fused" and _kernel not in ("auto", "strip", "nostrip"):
+        pytest.skip("the fused source kind is covered in the library's own, the strip-matrix and the persistent configuration")
     layer = wl.CONFIGS[name]
     dims = layer.dims()
-    n, c, h, w, k, fh, fw, s = dims
-    x, f = wl.make_input(layer), wl.make_filter(layer)
+    x, f = _cached(("ints", name), lambda: _layer_ints(layer))
+    ref = _cached(("ints_ref", name), lambda: _exact_f32(oracle_conv(x, f, dims)))
+    got = gpu_conv(x, f, dims, mode, src_kind=b.SRC_NCHW_FUSED if src == "fused" else b.SRC_NCHW)
+    assert np.array_equal(got, ref)
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("name", FULL)
+def test_conv_full_batch_whole_tensor(name, mode):
+    """Batch 128 on the benchmark's data: relative L2 over the WHOLE output against the oracle's Eq. (1),
+    plus a bound on the largest single error (a wrong accumulator column in one tile of one image would
+    move the norm by nothing, but is off by the size of an output, hundreds of times this bound)."""
+    layer = wl.CONFIGS[name]
+    dims = layer.dims()
+    x, f = _cached(("real", name), lambda: (wl.make_input(layer), wl.make_filter(layer)))
+    ref = _cached(("real_ref", name), lambda: oracle_conv(x, f, dims))
     got = gpu_conv(x, f, dims, mode)
-    ho, wo = b.out_dims(dims)
-    rng = np.random.default_rng(1234)
-    idx = np.stack([rng.integers(0, n, 20000), rng.integers(0, k, 20000), rng.integers(0, ho, 20000),
-                    rng.integers(0, wo, 20000)], axis=1).astype(np.int32)
-    corners = np.array(list(itertools.product((0, n - 1), (0, k - 1), (0, ho - 1), (0, wo - 1))), dtype=np.int32)
-    idx = np.concatenate([idx, corners])
-    ref = oracle.conv_direct_points(x, f, oracle.Shape(*dims), idx)
-    sample = got[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]]
-    assert rel_l2(sample, ref) <= TOL[mode]
-    for img in (0, n - 1):
-        one = layer.with_batch(1).dims()
-        assert rel_l2(got[img:img + 1], oracle_conv(x[img:img + 1], f, one)) <= TOL[mode]
     assert np.isfinite(got).all()
+    assert rel_l2(got, ref) <= TOL[mode]
+    rms = float(np.sqrt(np.mean(ref * ref)))
+    assert float(np.abs(got - ref).max()) <= 8.0 * TOL[mode] * rms
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("batch", [32, 128])
+@pytest.mark.parametrize("layer", wl.SWEEP, ids=lambda l: l.name)
+def test_conv_sweep_layers_batch_32_and_128(layer, batch, mode, _kernel):
+    """The twelve-layer sweep at the batch sizes the benchmark times, with the library's own choice of
+    path at each (reduction slices at 32, streamed filters and multi-wave persistent loops at 128): Eq. (1)
+    at 20 000 sampled coordinates and every corner, and the whole first and last image."""
+    if _kernel not in ("auto", "minws", "strip", "nostrip"):
+        pytest.skip("forced persistent-kernel variants are covered at small sizes")
+    layer = layer.with_batch(batch)
+    dims = layer.dims()
+    n, c, h, w, k, fh, fw, s = dims
+    ho, wo = b.out_dims(dims)
+
+    def make():
+        x, f = wl.make_input(layer), wl.make_filter(layer)
+        rng = np.random.default_rng(77 + batch)
+        idx = np.stack([rng.integers(0, n, 20000), rng.integers(0, k, 20000), rng.integers(0, ho, 20000),
+                        rng.integers(0, wo, 20000)], axis=1).astype(np.int32)
+        corners = np.array(list(itertools.product((0, n - 1), (0, k - 1), (0, ho - 1), (0, wo - 1))), dtype=np.int32)
+        idx = np.concatenate([idx, corners])
+        pts = oracle.conv_direct_points(x, f, oracle.Shape(*dims), idx)
+        one = layer.with_batch(1).dims()
+        ends = {img: oracle_conv(x[img:img + 1], f, one) for img in (0, n - 1)}
+        return x, f, idx, pts, ends
+
+    x, f, idx, pts, ends = _cached(("sweep", layer.name, batch), make)
+    got = gpu_conv(x, f, dims, mode)
+    assert np.isfinite(got).all()
+    sample = got[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]]
+    assert rel_l2(sample, pts) <= TOL[mode]
+    rms = float(np.sqrt(np.mean(pts * pts)))
+    assert float(np.abs(sample - pts).max()) <= 8.0 * TOL[mode] * rms
+    for img, ref in ends.items():
+        assert rel_l2(got[img:img + 1], ref) <= TOL[mode]
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("layer", wl.SWEEP, ids=lambda l: l.name)
+def test_conv_sweep_layers_batch32_small_integers_bit_exact(layer, mode, _kernel):
+    if _kernel not in ("auto", "minws", "strip", "nostrip"):
+        pytest.skip("forced persistent-kernel variants are covered at small sizes")
+    layer = layer.with_batch(32)
+    dims = layer.dims()
+    x, f = _cached(("ints", layer.name, 32), lambda: _layer_ints(layer))
+    ref = _cached(("ints_ref", layer.name, 32), lambda: _exact_f32(oracle_conv(x, f, dims)))
+    assert np.array_equal(gpu_conv(x, f, dims, mode), ref)
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("name", ["resnet3x3", "deep3x3"])
+def test_conv_fifty_repeats_are_bit_identical_on_exact_data(name, mode, _kernel):
+    """Several threads may issue the MMAs of one tile onto the same accumulator; a lost update would
+    show as a run that differs.  Fifty runs at batch 128 on small-integer data, compared on the device."""
+    import torch
+    if _kernel not in ("auto", "nostrip", "split3"):
+        pytest.skip("one configuration per kernel family")
+    layer = wl.CONFIGS[name]
+    dims = layer.dims()
+    x, f = _cached(("ints", name), lambda: _layer_ints(layer))
+    ho, wo = b.out_dims(dims)
+    xd, fd = torch.from_numpy(x).cuda(), torch.from_numpy(f).cuda()
+    ws = torch.empty(b.conv_workspace_bytes(dims, b.SRC_NCHW, mode) // 4, dtype=torch.float32, device="cuda")
+    outs = [torch.empty((layer.N, layer.K, ho, wo), dtype=torch.float32, device="cuda") for _ in range(2)]
+    b.conv(xd, b.SRC_NCHW, fd, dims, mode, outs[0], ws)
+    for _ in range(50):
+        outs[1].fill_(float("nan"))
+        b.conv(ws, b.SRC_IM2WIN, fd, dims, mode, outs[1], ws[b.workspace_bytes(dims) // 4:] if ws.numel() > b.workspace_bytes(dims) // 4 + 64 else None)
+        assert torch.equal(outs[0], outs[1])
+    assert b.last_device_status() == 0
+    ref = _cached(("ints_ref", name), lambda: _exact_f32(oracle_conv(x, f, dims)))
+    assert np.array_equal(outs[0].cpu().numpy(), ref)
 
 
 @pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)

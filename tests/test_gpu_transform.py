@@ -4,7 +4,7 @@ import pytest
 
 import oracle
 from paper_2306_14320_b200 import workloads as wl
-from gpu_helpers import ensure_built, gpu_transform
+from gpu_helpers import apply_config, ensure_built, gpu_transform, reset_config
 
 pytestmark = pytest.mark.gpu
 
@@ -26,10 +26,13 @@ def _built():
 
 
 @pytest.fixture(params=["auto", "gather"], autouse=True)
-def _kernel(request, monkeypatch):
-    """Every case runs twice: with the library's own choice of kernel (the TMA tile kernel where a job's
-    input and output ranges fit its shared-memory budget), and with the staged-gather kernel forced."""
-    monkeypatch.setenv("IM2WIN_TRANSFORM_GATHER", "1" if request.param == "gather" else "0")
+def _kernel(request):
+    """Every case runs twice: with the product library's own choice of kernel (the TMA tile kernel where
+    a job's input and output ranges fit its shared-memory budget), and with the staged-gather kernel
+    forced (a switch of the test build of the library)."""
+    apply_config("gather" if request.param == "gather" else "auto", **({"transform_gather": 1} if request.param == "gather" else {}))
+    yield
+    reset_config()
 
 
 def _bits(a):
@@ -69,10 +72,23 @@ def test_transform_bit_exact_full_batch(name):
     assert np.array_equal(_bits(got), _bits(ref))
 
 
-def test_bounded_wait_expiry_is_reported_and_the_context_survives(monkeypatch, request):
-    """Failure detection without a fault: a test hook makes the tile kernel announce its input copy but
-    never issue it (single-CTA problem), so the bounded wait runs out after about a second.  The kernel
-    must return by itself, the status word must name the wait, and the next call must work."""
+@pytest.mark.parametrize("batch", [32, 128])
+@pytest.mark.parametrize("layer", wl.SWEEP, ids=lambda l: l.name)
+def test_transform_bit_exact_sweep_layers_batch_32_and_128(layer, batch):
+    """The twelve-layer sweep at the batch sizes the benchmark times, every element compared."""
+    layer = layer.with_batch(batch)
+    x = wl.make_input(layer)
+    ref = oracle.im2win(x, oracle.Shape(*layer.dims()))
+    got = gpu_transform(x, layer.dims())
+    assert got.size == ref.size
+    assert np.array_equal(_bits(got), _bits(ref))
+
+
+def test_bounded_wait_expiry_is_reported_and_the_context_survives(request):
+    """Failure detection without a fault: a switch of the test build makes the tile kernel announce its
+    input copy but never issue it (single-CTA problem), so the bounded wait runs out after about a
+    second.  The kernel must return by itself, the status call must return ETIMEOUT and name the wait,
+    and the next call must work."""
     if "gather" in request.node.name:
         pytest.skip("the hook belongs to the tile kernel")
     import time
@@ -83,13 +99,13 @@ def test_bounded_wait_expiry_is_reported_and_the_context_survives(monkeypatch, r
     x = wl.normal01(77, 64).reshape(1, 1, 8, 8)
     xd = torch.from_numpy(x).cuda()
     out = Guarded(b.workspace_bytes(dims) // 4)
-    monkeypatch.setenv("IM2WIN_TEST_SKIP_COPY", "1")
+    apply_config("hook", test_skip_copy=1)
     t0 = time.perf_counter()
     b.transform(xd, dims, out.view)
-    status = b.last_device_status()  # synchronises the stream
+    rc, status = b.last_device_status_rc()  # synchronises the stream
     waited = time.perf_counter() - t0
-    monkeypatch.setenv("IM2WIN_TEST_SKIP_COPY", "0")
-    assert status == 109, status  # DEV_TIMEOUT_COPY
+    b.set_option("test_skip_copy", 0)
+    assert rc == b.ETIMEOUT and status == 109, (rc, status)  # DEV_TIMEOUT_COPY
     assert 0.5 < waited < 20.0, waited
     assert b.last_device_status() == 0  # reading the word cleared it
     ref = oracle.im2win(x, oracle.Shape(*dims))
