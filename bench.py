@@ -167,7 +167,13 @@ def time_layer(layer, mode_name, steps, warmup, torch, b, flush_buf, sampler_ind
     x_host = torch.from_numpy(wl.make_input(layer)).pin_memory()
     f_host = torch.from_numpy(wl.make_filter(layer)).pin_memory()
     x, f = x_host.cuda(), f_host.cuda()
-    ws = torch.empty(ws_bytes // 4, dtype=torch.float32, device="cuda")
+    # one workspace: the im2win tensor, then (from the next 256-byte boundary) scratch for the filter
+    # copy some kernels stream; sized by the library's own query
+    ws_total = max(ws_bytes, b.conv_workspace_bytes(dims, b.SRC_NCHW, mode))
+    ws_all = torch.empty(ws_total // 4, dtype=torch.float32, device="cuda")
+    ws = ws_all[:ws_bytes // 4]
+    scratch_off = (ws_bytes + 255) // 256 * 256 // 4
+    scratch = ws_all[scratch_off:] if ws_all.numel() > scratch_off else None
     out = torch.empty((layer.N, layer.K, ho, wo), dtype=torch.float32, device="cuda")
     stream = torch.cuda.current_stream()
 
@@ -177,7 +183,7 @@ def time_layer(layer, mode_name, steps, warmup, torch, b, flush_buf, sampler_ind
         b.transform(x, dims, ws)
         if events:
             events[1].record(stream)
-        b.conv(ws, b.SRC_IM2WIN, f, dims, mode, out)
+        b.conv(ws, b.SRC_IM2WIN, f, dims, mode, out, scratch)
         if events:
             events[2].record(stream)
 
@@ -208,6 +214,7 @@ def time_layer(layer, mode_name, steps, warmup, torch, b, flush_buf, sampler_ind
         "ms_step": sum(t_st) / steps, "ms_transform": sum(t_tr) / steps, "ms_conv": sum(t_cv) / steps,
         "ms_step_best": min(t_st), "ms_transform_best": min(t_tr), "ms_conv_best": min(t_cv),
         "wall_s": t_wall, "flops": _flops(layer, ho, wo), "workspace_bytes": ws_bytes, "im2col_bytes": col_bytes,
+        "filter_scratch_bytes": ws_total - ws_bytes,
         "bytes_in": x.numel() * 4, "bytes_f": f.numel() * 4, "bytes_out": out.numel() * 4,
         "clocks": sampler.summary() if sampler else None,
     }
@@ -219,12 +226,12 @@ def time_layer(layer, mode_name, steps, warmup, torch, b, flush_buf, sampler_ind
     # the fused source kind: same result straight from the untransformed input, no im2win tensor in HBM
     try:
         for _ in range(3):
-            b.conv(x, b.SRC_NCHW_FUSED, f, dims, mode, out)
+            b.conv(x, b.SRC_NCHW_FUSED, f, dims, mode, out, scratch)
         fe = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
         for k in range(steps):
             flush_buf.zero_()
             fe[k][0].record(stream)
-            b.conv(x, b.SRC_NCHW_FUSED, f, dims, mode, out)
+            b.conv(x, b.SRC_NCHW_FUSED, f, dims, mode, out, scratch)
             fe[k][1].record(stream)
         torch.cuda.synchronize()
         if b.last_device_status() != 0:
@@ -241,12 +248,12 @@ def time_layer(layer, mode_name, steps, warmup, torch, b, flush_buf, sampler_ind
     try:
         out16 = torch.empty(layer.N * layer.K * ho * wo, dtype=torch.int16, device="cuda")
         for _ in range(3):
-            b.conv_bf16out(ws, b.SRC_IM2WIN, f, dims, mode, out16)
+            b.conv_bf16out(ws, b.SRC_IM2WIN, f, dims, mode, out16, scratch)
         oe = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
         for k in range(steps):
             flush_buf.zero_()
             oe[k][0].record(stream)
-            b.conv_bf16out(ws, b.SRC_IM2WIN, f, dims, mode, out16)
+            b.conv_bf16out(ws, b.SRC_IM2WIN, f, dims, mode, out16, scratch)
             oe[k][1].record(stream)
         torch.cuda.synchronize()
         if b.last_device_status() != 0:
@@ -263,14 +270,14 @@ def time_layer(layer, mode_name, steps, warmup, torch, b, flush_buf, sampler_ind
         try:
             for _ in range(3):
                 b.transform_bf16(x, dims, ws16)
-                b.conv(ws16, b.SRC_IM2WIN_BF16, f, dims, mode, out)
+                b.conv(ws16, b.SRC_IM2WIN_BF16, f, dims, mode, out, scratch)
             be = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
             for k in range(steps):
                 flush_buf.zero_()
                 be[k][0].record(stream)
                 b.transform_bf16(x, dims, ws16)
                 be[k][1].record(stream)
-                b.conv(ws16, b.SRC_IM2WIN_BF16, f, dims, mode, out)
+                b.conv(ws16, b.SRC_IM2WIN_BF16, f, dims, mode, out, scratch)
                 be[k][2].record(stream)
             torch.cuda.synchronize()
             if b.last_device_status() != 0:

@@ -1,8 +1,757 @@
-// placeholder while the API is reworked
+// im2win-based convolution (Algorithm 2) on the sm_100a tensor cores: the STRIP-MATRIX kernel.
+//
+// What the im2win layout gives a tensor core.  For one (image, channel) the im2win tensor is a row-major
+// matrix with Fh columns: row c = m*W + k holds the Fh input values of input column k under output row m
+// (Algorithm 1).  The window of output (m, n) is Fw CONSECUTIVE rows of that matrix, rows m*W + n*s + v,
+// v = 0..Fw-1, and neighbouring windows overlap in Fw-s of them (Section III-A).  So the convolution is
+// Fw matrix products, one per filter column v, whose A operands are the SAME matrix T read from row
+// offsets that differ by v:
+//     O[(m,n), j] = sum_v  sum_{r,u}  T[m*W + n*s + v][(r,u)] * Fv[j][(r,u)],   Fv[j][(r,u)] = F[j][r][u][v].
+// T is laid out in shared memory so that a row offset is a plain address offset of the MMA's matrix
+// descriptor (no swizzle, 16-byte chunks stored chunk-major: chunk kc of row p at kc*LBO + p*16), hence
+// every element of the im2win tensor is moved ONCE -- global -> shared by TMA, shared -> T by a
+// transposing copy -- and the Fw/s-fold window expansion happens inside the tensor core's operand fetch.
+// (Stride s > 1: the columns are split into s classes k mod s, one T matrix per class; tap v reads class
+// v mod s at row offset v / s.)
+//
+// GEMM view per work unit: M = 128*MH consecutive rows p = m*WP + q of one image (WP = ceil(W/s); the
+// rows with q >= Wo are computed and dropped), N = a tile of up to 256 filters, K = (r,u) per tap.
+// Roles (one persistent CTA per SM, units t, t+grid, ...):
+//   warp 0       source producer: one 2-D TMA box (or one bulk copy per channel) per group of GR channels
+//   warp 1       MMA issuer (one thread): tcgen05.mma kind::tf32 / kind::f16, A and B from shared memory,
+//                fp32 accumulators in TMEM, one fixed summation order (results are reproducible bit for bit)
+//   warp 2       filter producer: TMA boxes (64-byte swizzle) from the tap-major filter copy Fv that a small
+//                kernel writes into the caller's scratch at the start of the call (fp32, or bf16 in BF16 mode)
+//   warps 4-11   transposers: staged source -> T (fp32 as is for TF32, cvt.rn.bf16x2 for BF16)
+//   warps 12-19  epilogue (four per 128-row half): tcgen05.ld -> coalesced NCHW stores
+// The source is the fp32 im2win tensor, the bf16 im2win tensor, or (fused) the untransformed input, whose
+// rows m*s+u supply the same values.  Every wait is bounded (status word + common teardown on expiry).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <atomic>
+#include <cstring>
+#include <type_traits>
+
 #include "common.cuh"
+#include "ptx_sm100.cuh"
+
 namespace im2win {
-int launch_conv_tc_strip(const void*, const float*, float*, const Geometry&, int, cudaStream_t, Scratch, int, bool) {
+namespace {
+
+constexpr int kTW = 8;             // transposer warps
+constexpr int kTWarp0 = 4;
+constexpr int kEpiWarp0 = kTWarp0 + kTW;
+constexpr int kMaxRaw = 12, kMaxB = 12;
+constexpr int kTMax = 3;           // transposer tasks per thread and source stage
+constexpr uint32_t kSpin = 1u << 22;
+
+struct SParams {
+  const void* src;
+  float* out;
+  int32_t* status;
+  int32_t C, K, Ho, Wo, W, WP;
+  int32_t RPI;        // T rows per image: Ho * WP
+  int32_t TPI;        // tiles per image
+  int32_t MH;         // 128-row halves per tile
+  int32_t RT;         // T rows per class a tile uses: 128*MH + (Fw-1)/s
+  int32_t RA;         // T rows per class allocated (RT rounded up to 8)
+  int32_t NJ;         // RT * s: (row, class) pairs = source columns per tile
+  int32_t NT, n_ntiles, Kp;
+  int32_t G, GR, NSUB, NTS;  // channels per T stage / per source stage, source stages per T stage, T stages per unit
+  int32_t CBN;        // channel blocks (of NCH channels) per source stage
+  int32_t NBLK, BB, NBS;     // filter blocks (2 K steps) per (T stage, tap); blocks per filter stage; filter stages per (T stage, tap)
+  int32_t SR, SB, ND;
+  int32_t CP;         // elements per channel row of a source stage
+  int32_t box;        // source stages come as one 2-D TMA box
+  int32_t pm;         // plane length modulo the elements of a 16-byte chunk (bulk copies: per-channel phase)
+  int64_t plane;      // source elements per (image, channel)
+  int64_t n_src;
+  int64_t units;
+  uint32_t idesc, tmem_cols;
+  uint32_t raw_stage_bytes, t_stage_bytes, b_stage_bytes;
+  uint32_t off_t, off_raw, off_bar, off_misc;
+};
+
+struct SBars {
+  uint64_t raw_full[kMaxRaw], raw_empty[kMaxRaw];
+  uint64_t b_full[kMaxB], b_empty[kMaxB];
+  uint64_t t_full[2], t_empty[2];
+  uint64_t acc_full[2], acc_empty[2];
+};
+struct SMisc {
+  uint32_t tmem_base;
+  int32_t abort;
+};
+
+struct Ring {
+  int32_t idx = 0;
+  uint32_t phase = 0;
+  __device__ __forceinline__ void advance(int32_t n) {
+    if (++idx == n) { idx = 0; phase ^= 1u; }
+  }
+};
+
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait (about a second): polls with a back-off; on expiry records `code`, raises the CTA's
+// abort flag (which ends every other role's wait at its next look) and returns false.
+__device__ __noinline__ bool wait_slow(int32_t* status, SMisc* misc, uint32_t bar, uint32_t parity, int32_t code,
+                                       uint32_t sleep_ns) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 0; it < kSpin; ++it) {
+    __nanosleep(sleep_ns);
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u) {
+      if (*reinterpret_cast<volatile int32_t*>(&misc->abort)) return false;
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > 1000000000ull) break;
+    }
+  }
+  atomicCAS(status, 0, code);
+  atomicExch(&misc->abort, 1);
+  return false;
+}
+__device__ __forceinline__ bool wait_bar(const SParams& P, SMisc* misc, uint32_t bar, uint32_t parity, int32_t code,
+                                         uint32_t sleep_ns = 32) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  return wait_slow(P.status, misc, bar, parity, code, sleep_ns);
+}
+__device__ __forceinline__ bool wait_bar_warp(const SParams& P, SMisc* misc, uint32_t bar, uint32_t parity, int32_t code,
+                                              uint32_t sleep_ns = 32) {
+  return __all_sync(0xffffffffu, wait_bar(P, misc, bar, parity, code, sleep_ns));
+}
+
+__device__ __forceinline__ uint32_t lds_u32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a) {
+  uint32_t v;
+  asm volatile("{\n.reg .b16 h;\nld.shared.u16 h, [%1];\ncvt.u32.u16 %0, h;\n}" : "=r"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_v4(uint32_t a, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+// Where unit t lies: filter tile, image, first T row of the tile.
+struct Unit {
+  int32_t nt, img, R0;
+};
+__device__ __forceinline__ Unit unit_of(const SParams& P, int64_t t) {
+  Unit u;
+  const int64_t tile = t / P.n_ntiles;
+  u.nt = (int32_t)(t - tile * P.n_ntiles);
+  const int64_t img = tile / P.TPI;
+  u.img = (int32_t)img;
+  u.R0 = (int32_t)(tile - img * P.TPI) * 128 * P.MH;
+  return u;
+}
+// Source elements [e_lo, e_hi) of a channel plane that the tile starting at T row R0 needs.
+template <int FH, int S, bool FUSED>
+__device__ __forceinline__ void tile_range(const SParams& P, int32_t R0, int32_t& e_lo, int32_t& e_hi) {
+  const int32_t r_last = min(R0 + P.RT, P.RPI) - 1;
+  const int32_t m0 = R0 / P.WP, q0 = R0 - m0 * P.WP;
+  const int32_t m1 = r_last / P.WP, q1 = r_last - m1 * P.WP;
+  const int32_t k1 = min(q1 * S + S - 1, P.W - 1);
+  if (FUSED) {
+    e_lo = m0 * S * P.W + q0 * S;
+    e_hi = (m1 * S + FH - 1) * P.W + k1 + 1;
+  } else {
+    e_lo = (m0 * P.W + q0 * S) * FH;
+    e_hi = (m1 * P.W + k1 + 1) * FH;
+  }
+}
+
+// SRCK: 0 = fp32 im2win tensor, 1 = untransformed input (fused), 2 = bf16 im2win tensor (BF16 mode).
+template <int FH, int FW, int S, bool BF16, int SRCK>
+__global__ void __launch_bounds__(640, 1)
+conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, const __grid_constant__ CUtensorMap xmap) {
+  constexpr bool FUSED = SRCK == 1;
+  constexpr bool SRC16 = SRCK == 2;
+  static_assert(!SRC16 || BF16, "a 16-bit source feeds the BF16 mode");
+  constexpr uint32_t ES = SRC16 ? 2u : 4u;       // bytes per source element
+  constexpr int32_t EPC = SRC16 ? 8 : 4;          // source elements per 16-byte chunk
+  constexpr int NCH = BF16 ? 8 : 4;               // channels per transposer task = T elements per 16-byte chunk
+  constexpr int SH = (FW - 1) / S;                // largest row offset of a tap
+
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* const smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
+  SBars* const bars = reinterpret_cast<SBars*>(smem + P.off_bar);
+  SMisc* const misc = reinterpret_cast<SMisc*>(smem + P.off_misc);
+  const uint32_t b_sa = ptx::smem_u32(smem), t_sa = b_sa + P.off_t, raw_sa = b_sa + P.off_raw;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int32_t n_epi_warps = 4 * P.MH;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kMaxRaw; ++i) {
+      ptx::mbar_init(ptx::smem_u32(&bars->raw_full[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->raw_empty[i]), kTW);
+    }
+    for (int i = 0; i < kMaxB; ++i) {
+      ptx::mbar_init(ptx::smem_u32(&bars->b_full[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->b_empty[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(ptx::smem_u32(&bars->t_full[i]), kTW);
+      ptx::mbar_init(ptx::smem_u32(&bars->t_empty[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), (uint32_t)n_epi_warps);
+    }
+    ptx::fence_mbar_init();
+    misc->abort = 0;
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), P.tmem_cols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = misc->tmem_base;
+
+  if (warp == 0) {
+    // ================================================================ SOURCE PRODUCER
+    using SrcT = typename std::conditional<SRC16, uint16_t, float>::type;
+    const SrcT* const xsrc = reinterpret_cast<const SrcT*>(P.src);
+    Ring rr;
+    int64_t count = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < P.units && ok; t += gridDim.x) {
+      const Unit u = unit_of(P, t);
+      int32_t e_lo, e_hi;
+      tile_range<FH, S, FUSED>(P, u.R0, e_lo, e_hi);
+      const int32_t len = e_hi - e_lo;
+      const int32_t box_x = (e_lo & ~(EPC - 1)) / (EPC / 2);  // in 8-byte units
+      const int32_t nstages = P.NTS * P.NSUB;
+      for (int32_t sidx = 0; sidx < nstages && ok; ++sidx, ++count, rr.advance(P.SR)) {
+        const int32_t ch0 = sidx * P.GR;
+        const uint32_t full = ptx::smem_u32(&bars->raw_full[rr.idx]);
+        ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->raw_empty[rr.idx]), rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, 64);
+        if (!ok) break;
+        const uint32_t dst0 = raw_sa + (uint32_t)rr.idx * P.raw_stage_bytes;
+        if (P.box) {
+          if (lane == 0) {
+            ptx::mbar_arrive_expect_tx(full, P.raw_stage_bytes);
+            tma_load_2d(dst0, &xmap, box_x, u.img * P.C + ch0, full);
+          }
+        } else {
+          const SrcT* src = nullptr;
+          uint32_t dst = 0, bytes = 0;
+          if (lane < P.GR) {
+            const int64_t start = ((int64_t)u.img * P.C + ch0 + lane) * P.plane + e_lo;
+            const int32_t skew = (int32_t)(start & (EPC - 1));
+            const int64_t a0 = start - skew;
+            int32_t nel = (skew + len + EPC - 1) & ~(EPC - 1);
+            dst = dst0 + (uint32_t)(lane * P.CP) * ES;
+            if (a0 + nel > P.n_src) {  // the last 16-byte chunk would pass the end of the tensor
+              const int32_t nbulk = (int32_t)((P.n_src - a0) & ~(int64_t)(EPC - 1));
+              SrcT* d = reinterpret_cast<SrcT*>(smem + P.off_raw + (size_t)rr.idx * P.raw_stage_bytes) + (size_t)lane * P.CP;
+              for (int64_t e = a0 + nbulk; e < P.n_src; ++e) d[e - a0] = __ldg(xsrc + e);
+              nel = nbulk;
+            }
+            src = xsrc + a0;
+            bytes = (uint32_t)nel * ES;
+          }
+          const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+          if (lane == 0) ptx::mbar_arrive_expect_tx(full, total);
+          __syncwarp();
+          if (bytes) ptx::bulk_g2s(dst, src, bytes, full);
+        }
+        __syncwarp();
+      }
+    }
+    // every copy issued must have landed before the CTA exits
+    for (int64_t c = count > P.SR ? count - P.SR : 0; c < count; ++c)
+      wait_bar(P, misc, ptx::smem_u32(&bars->raw_full[c % P.SR]), (uint32_t)(c / P.SR) & 1u, DEV_TIMEOUT_DRAIN);
+  } else if (warp == 1) {
+    // ================================================================ MMA ISSUER
+    if (lane == 0) {
+      Ring tr, br, dr;
+      bool ok = true;
+      const uint64_t ad0 = ptx::smem_desc_k_chunkmajor(t_sa, (uint32_t)(S * P.RA) * 16u);
+      const uint64_t bd0 = ptx::smem_desc_k_sw64(b_sa);
+      const uint32_t a_lo0 = (uint32_t)ad0, a_hi = (uint32_t)(ad0 >> 32);
+      const uint32_t b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
+      const uint32_t t16 = P.t_stage_bytes >> 4, b16 = P.b_stage_bytes >> 4;
+      const uint32_t blk16 = (uint32_t)P.NT * 4u;        // one filter block (NT rows x 64 bytes) in 16-byte units
+      const uint32_t kstep16 = 2u * (uint32_t)(S * P.RA);  // one MMA K step (two chunks) of T in 16-byte units
+      for (int64_t t = blockIdx.x; t < P.units && ok; t += gridDim.x, dr.advance(P.ND)) {
+        ok = wait_bar(P, misc, ptx::smem_u32(&bars->acc_empty[dr.idx]), dr.phase ^ 1u, DEV_TIMEOUT_ACC);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(dr.idx * P.MH * P.NT);
+        uint32_t accum = 0;
+        for (int32_t ts = 0; ts < P.NTS && ok; ++ts, tr.advance(2)) {
+          ok = wait_bar(P, misc, ptx::smem_u32(&bars->t_full[tr.idx]), tr.phase, DEV_TIMEOUT_A_FULL, 20);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          const uint32_t a_stage = a_lo0 + (uint32_t)tr.idx * t16;
+#pragma unroll
+          for (int v = 0; v < FW; ++v) {
+            const uint32_t a_v = a_stage + (uint32_t)((v % S) * P.RA + v / S);
+            for (int32_t bs = 0; bs < P.NBS; ++bs) {
+              if (!ptx::mbar_try_wait(ptx::smem_u32(&bars->b_full[br.idx]), br.phase)) {
+                ok = wait_bar(P, misc, ptx::smem_u32(&bars->b_full[br.idx]), br.phase, DEV_TIMEOUT_B_FULL, 20);
+                if (!ok) break;
+              }
+              ptx::tc_fence_after();
+              const uint32_t b_stage = b_lo0 + (uint32_t)br.idx * b16;
+              for (int32_t blk = 0; blk < P.BB; ++blk) {
+                const uint32_t ks0 = (uint32_t)(bs * P.BB + blk) * 2u;
+#pragma unroll
+                for (int k2 = 0; k2 < 2; ++k2) {
+                  const uint32_t a_k = a_v + (ks0 + k2) * kstep16;
+                  const uint32_t b_k = b_stage + (uint32_t)blk * blk16 + (uint32_t)k2 * 2u;
+                  for (int32_t h = 0; h < P.MH; ++h)
+                    ptx::mma_ss_lohi<BF16>(d_tmem + (uint32_t)(h * P.NT), a_k + (uint32_t)h * 128u, a_hi, b_k, b_hi, P.idesc, accum);
+                  accum = 1;
+                }
+              }
+              ptx::mma_commit(ptx::smem_u32(&bars->b_empty[br.idx]));
+              br.advance(P.SB);
+            }
+            if (!ok) break;
+          }
+          if (!ok) break;
+          ptx::mma_commit(ptx::smem_u32(&bars->t_empty[tr.idx]));
+        }
+        if (!ok) break;
+        ptx::mma_commit(ptx::smem_u32(&bars->acc_full[dr.idx]));
+      }
+    }
+    __syncwarp();
+  } else if (warp == 2) {
+    // ================================================================ FILTER PRODUCER
+    if (lane == 0) {
+      Ring br;
+      int64_t count = 0;
+      bool ok = true;
+      const int32_t bke = BF16 ? 32 : 16;  // elements per 64-byte filter row
+      for (int64_t t = blockIdx.x; t < P.units && ok; t += gridDim.x) {
+        const Unit u = unit_of(P, t);
+        for (int32_t ts = 0; ts < P.NTS && ok; ++ts) {
+          for (int32_t v = 0; v < FW && ok; ++v) {
+            for (int32_t bs = 0; bs < P.NBS && ok; ++bs, ++count, br.advance(P.SB)) {
+              ok = wait_bar(P, misc, ptx::smem_u32(&bars->b_empty[br.idx]), br.phase ^ 1u, DEV_TIMEOUT_B_EMPTY);
+              if (!ok) break;
+              const uint32_t full = ptx::smem_u32(&bars->b_full[br.idx]);
+              ptx::mbar_arrive_expect_tx(full, P.b_stage_bytes);
+              for (int32_t blk = 0; blk < P.BB; ++blk)
+                tma_load_2d(b_sa + (uint32_t)br.idx * P.b_stage_bytes + (uint32_t)blk * (uint32_t)P.NT * 64u, &fmap,
+                            (ts * P.NBLK + bs * P.BB + blk) * bke, v * P.Kp + u.nt * P.NT, full);
+            }
+          }
+        }
+      }
+      for (int64_t c = count > P.SB ? count - P.SB : 0; c < count; ++c)
+        wait_bar(P, misc, ptx::smem_u32(&bars->b_full[c % P.SB]), (uint32_t)(c / P.SB) & 1u, DEV_TIMEOUT_DRAIN);
+    }
+    __syncwarp();
+  } else if (warp >= kTWarp0 && warp < kTWarp0 + kTW) {
+    // ================================================================ TRANSPOSERS: staged source -> T
+    const int32_t tid = (warp - kTWarp0) * 32 + lane;
+    const int32_t ntasks = P.NJ * P.CBN;
+    const uint32_t lbo = (uint32_t)(S * P.RA) * 16u;
+    const uint32_t ustride = (FUSED ? (uint32_t)P.W : 1u) * ES;
+    Ring rr, tr;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < P.units && ok; t += gridDim.x) {
+      const Unit u = unit_of(P, t);
+      int32_t e_lo, e_hi;
+      tile_range<FH, S, FUSED>(P, u.R0, e_lo, e_hi);
+      // this thread's tasks: (source column j = (T row, class), channel block cb of the stage)
+      uint32_t soff[kTMax], doff[kTMax];
+      int32_t tcb[kTMax];
+      bool tv[kTMax];
+#pragma unroll
+      for (int z = 0; z < kTMax; ++z) {
+        const int32_t task = tid + z * (kTW * 32);
+        tv[z] = false; soff[z] = 0; doff[z] = 0; tcb[z] = 0;
+        if (task < ntasks) {
+          const int32_t cb = task / P.NJ, j = task - cb * P.NJ;
+          const int32_t p = j / S, cl = j - p * S;      // T row within the tile, class
+          const int32_t rho = u.R0 + p;
+          const int32_t m = rho / P.WP, q = rho - m * P.WP;
+          const int32_t k = q * S + cl;
+          if (rho < P.RPI && k < P.W) {
+            tv[z] = true;
+            tcb[z] = cb;
+            const int32_t e = FUSED ? (m * S * P.W + k) : (m * P.W + k) * FH;
+            soff[z] = (uint32_t)(e - e_lo + cb * NCH * P.CP) * ES;
+            doff[z] = (uint32_t)(cl * P.RA + p) * 16u + (uint32_t)(cb * FH) * lbo;
+          }
+        }
+      }
+      // 16-byte phase of the staged ranges: per tile, plus (bulk copies of planes that are not a whole
+      // number of chunks) per channel
+      const int32_t sk0 = (int32_t)(((int64_t)u.img * P.C * P.plane + e_lo) & (EPC - 1));
+      for (int32_t ts = 0; ts < P.NTS && ok; ++ts, tr.advance(2)) {
+        const uint32_t t_stage = t_sa + (uint32_t)tr.idx * P.t_stage_bytes;
+        for (int32_t sub = 0; sub < P.NSUB && ok; ++sub, rr.advance(P.SR)) {
+          ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->raw_full[rr.idx]), rr.phase, DEV_TIMEOUT_RAW_FULL);
+          if (!ok) break;
+          if (sub == 0) {
+            ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->t_empty[tr.idx]), tr.phase ^ 1u, DEV_TIMEOUT_A_EMPTY);
+            if (!ok) break;
+          }
+          const uint32_t rs = raw_sa + (uint32_t)rr.idx * P.raw_stage_bytes;
+          const int32_t ch0 = (ts * P.NSUB + sub) * P.GR;
+          const uint32_t t_sub = t_stage + (uint32_t)(sub * P.CBN * FH) * lbo;
+#pragma unroll
+          for (int z = 0; z < kTMax; ++z) {
+            if (tv[z]) {
+              uint32_t val[NCH * FH];
+#pragma unroll
+              for (int c = 0; c < NCH; ++c) {
+                const int32_t sk = P.pm ? ((sk0 + (ch0 + tcb[z] * NCH + c) * P.pm) & (EPC - 1)) : sk0;
+                const uint32_t a = rs + soff[z] + (uint32_t)(c * P.CP + sk) * ES;
+#pragma unroll
+                for (int f = 0; f < FH; ++f) val[c * FH + f] = SRC16 ? lds_u16(a + (uint32_t)f * ustride) : lds_u32(a + (uint32_t)f * ustride);
+              }
+              const uint32_t d = t_sub + doff[z];
+#pragma unroll
+              for (int f = 0; f < FH; ++f) {
+                if constexpr (!BF16) {
+                  sts_v4(d + (uint32_t)f * lbo, val[4 * f], val[4 * f + 1], val[4 * f + 2], val[4 * f + 3]);
+                } else if constexpr (SRC16) {
+                  sts_v4(d + (uint32_t)f * lbo, val[8 * f] | (val[8 * f + 1] << 16), val[8 * f + 2] | (val[8 * f + 3] << 16),
+                         val[8 * f + 4] | (val[8 * f + 5] << 16), val[8 * f + 6] | (val[8 * f + 7] << 16));
+                } else {
+                  sts_v4(d + (uint32_t)f * lbo,
+                         ptx::pack_bf16x2(__uint_as_float(val[8 * f]), __uint_as_float(val[8 * f + 1])),
+                         ptx::pack_bf16x2(__uint_as_float(val[8 * f + 2]), __uint_as_float(val[8 * f + 3])),
+                         ptx::pack_bf16x2(__uint_as_float(val[8 * f + 4]), __uint_as_float(val[8 * f + 5])),
+                         ptx::pack_bf16x2(__uint_as_float(val[8 * f + 6]), __uint_as_float(val[8 * f + 7])));
+                }
+              }
+            }
+          }
+          const bool last = sub == P.NSUB - 1;
+          if (last) ptx::fence_proxy_async_smem();  // this thread's T writes -> visible to the tensor core
+          __syncwarp();
+          if (lane == 0) {
+            ptx::mbar_arrive(ptx::smem_u32(&bars->raw_empty[rr.idx]));
+            if (last) ptx::mbar_arrive(ptx::smem_u32(&bars->t_full[tr.idx]));
+          }
+        }
+      }
+    }
+  } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + n_epi_warps) {
+    // ================================================================ EPILOGUE: TMEM -> NCHW
+    const int32_t h = (warp - kEpiWarp0) >> 2, q4 = warp & 3;  // (kEpiWarp0 is a multiple of 4: warp & 3 = TMEM lane quarter)
+    const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
+    Ring dr;
+    bool ok = true;
+    const int32_t eK = P.K, eNT = P.NT;
+    const int64_t eHoWo = (int64_t)P.Ho * P.Wo;
+    for (int64_t t = blockIdx.x; t < P.units && ok; t += gridDim.x, dr.advance(P.ND)) {
+      const Unit u = unit_of(P, t);
+      const int32_t rho = u.R0 + h * 128 + q4 * 32 + lane;
+      const int32_t m = rho / P.WP, q = rho - m * P.WP;
+      const bool valid = rho < P.RPI && q < P.Wo;
+      const int32_t n0 = u.nt * P.NT;
+      float* const orow = P.out + ((int64_t)u.img * P.K + n0) * eHoWo + (int64_t)m * P.Wo + q;
+      ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->acc_full[dr.idx]), dr.phase, DEV_TIMEOUT_ACC, 128);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)((dr.idx * P.MH + h) * P.NT);
+#pragma unroll 1
+      for (int32_t c0 = 0; c0 < eNT; c0 += 16) {
+        uint32_t v[16];
+        ptx::tmem_ld_x16(d_tmem + (uint32_t)c0, v);
+        ptx::tmem_wait_ld();
+        if (valid) {
+          float* o = orow + (int64_t)c0 * eHoWo;
+          const int32_t left = eK - n0 - c0;
+#pragma unroll
+          for (int e = 0; e < 16; ++e)
+            if (e < left) o[(int64_t)e * eHoWo] = __uint_as_float(v[e]);
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->acc_empty[dr.idx]));
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, P.tmem_cols);
+  }
+}
+
+// Tap-major copy of the filter for the TMA-streamed B operand:
+//   Fv[v][j][r*Fh + u] = F[j][r][u][v]   (j < K; rows K..Kp-1 are zero), fp32 or bf16 (nearest even).
+template <bool BF16>
+__global__ void __launch_bounds__(256) filter_tap_major_kernel(const float* __restrict__ f, void* __restrict__ o, int32_t K,
+                                                               int32_t Kp, int32_t C, int32_t FH, int32_t FW) {
+  const int64_t row = (int64_t)C * FH, n = (int64_t)FW * Kp * row;
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (int64_t)gridDim.x * 256) {
+    const int64_t vj = i / row;
+    const int32_t ku = (int32_t)(i - vj * row);
+    const int32_t v = (int32_t)(vj / Kp), j = (int32_t)(vj - (int64_t)v * Kp);
+    const int32_t r = ku / FH, u = ku - r * FH;
+    const float x = j < K ? f[(((int64_t)j * C + r) * FH + u) * FW + v] : 0.f;
+    if (BF16) static_cast<__nv_bfloat16*>(o)[i] = __float2bfloat16_rn(x);
+    else static_cast<float*>(o)[i] = x;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_fn() {
+  static std::atomic<void*> cached{nullptr};
+  void* p = cached.load(std::memory_order_acquire);
+  if (!p) {
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    cached.store(p, std::memory_order_release);
+  }
+  return reinterpret_cast<EncodeTiledFn>(p);
+}
+
+struct Plan {
+  SParams P;
+  size_t smem_bytes, scratch_bytes;
+  int threads;
+};
+
+// Fills the launch parameters for (FH, FW, S, BF16, SRCK); IM2WIN_EUNSUPPORTED where the kernel does not apply.
+template <int FH, int FW, int S, bool BF16, int SRCK>
+int make_plan(const Geometry& g, Plan* pl) {
+  constexpr int NCH = BF16 ? 8 : 4;
+  constexpr int64_t ES = SRCK == 2 ? 2 : 4;
+  constexpr int64_t EPC = 16 / ES;
+  constexpr int SH = (FW - 1) / S;
+  constexpr int GDIV = FH % 4 == 0 ? 1 : (FH % 2 == 0 ? 2 : 4);  // channel blocks per T stage: (G/NCH)*FH chunks = whole filter blocks of 4
+  SParams& P = pl->P;
+  P = SParams{};
+  P.G = NCH * GDIV;
+  if (g.C % P.G != 0) return IM2WIN_EUNSUPPORTED;
+  if (g.HoWo > (1 << 28) || (int64_t)g.H * g.W > (1 << 28)) return IM2WIN_EUNSUPPORTED;
+  P.C = g.C; P.K = g.K; P.Ho = g.Ho; P.Wo = g.Wo; P.W = g.W;
+  P.WP = (g.W + S - 1) / S;
+  P.RPI = g.Ho * P.WP;
+  P.n_ntiles = (g.K + 255) / 256;
+  P.NT = ((g.K + P.n_ntiles - 1) / P.n_ntiles + 15) / 16 * 16;
+  P.Kp = P.n_ntiles * P.NT;
+  P.NTS = g.C / P.G;
+  P.NBLK = GDIV * FH / 4;
+  if (SRCK == 1) { P.plane = (int64_t)g.H * g.W; P.n_src = g.n_in; }
+  else { P.plane = g.HoL; P.n_src = g.n_win; }
+  P.pm = (int32_t)(P.plane % EPC);
+  const int nsm = sm_count();
+  const int64_t cap = 227 * 1024 - 1024 - 512;  // alignment slack, barriers
+  // 128-row halves per tile: two halve the filter bytes streamed per output (each filter stage feeds
+  // two MMAs) but leave a single accumulator buffer for wide filter tiles; picked by waves x work,
+  // ties to two halves.
+  int best_mh = 0;
+  double best_cost = 0;
+  for (int mh = 1; mh <= 2; ++mh) {
+    if (knobs().strip_mh && knobs().strip_mh != mh) continue;
+    if (mh * P.NT > 512) continue;
+    const int64_t tpi = (P.RPI + 128 * mh - 1) / (128 * mh);
+    const int64_t units = (int64_t)g.N * tpi * P.n_ntiles;
+    const int64_t waves = (units + nsm - 1) / nsm;
+    const int nd = 512 / (mh * P.NT) >= 2 ? 2 : 1;
+    double cost = (double)waves * mh * (nd == 1 ? 1.08 : 1.0);
+    if (mh == 2) cost *= 0.97;
+    if (!best_mh || cost < best_cost) { best_mh = mh; best_cost = cost; }
+  }
+  if (!best_mh) return IM2WIN_EUNSUPPORTED;
+  P.MH = best_mh;
+  P.TPI = (P.RPI + 128 * P.MH - 1) / (128 * P.MH);
+  P.units = (int64_t)g.N * P.TPI * P.n_ntiles;
+  P.RT = 128 * P.MH + SH;
+  P.RA = (P.RT + 7) / 8 * 8;
+  P.NJ = P.RT * S;
+  if ((int64_t)S * P.RA > 16383) return IM2WIN_EUNSUPPORTED;
+  // channel blocks per source stage: as many as keep a stage's (column, block) tasks within about two
+  // rounds of the 256 transposer threads
+  P.CBN = 1;
+  for (int cbn = GDIV; cbn >= 1; cbn /= 2)
+    if (GDIV % cbn == 0 && (int64_t)P.NJ * cbn <= 2 * kTW * 32 + 32) { P.CBN = cbn; break; }
+  if ((int64_t)P.NJ * P.CBN > (int64_t)kTMax * kTW * 32) return IM2WIN_EUNSUPPORTED;
+  P.GR = P.CBN * NCH;
+  if (P.GR > 32) return IM2WIN_EUNSUPPORTED;  // one producer lane per channel of a stage
+  P.NSUB = P.G / P.GR;
+  // elements of one channel a tile needs at most, plus the 16-byte phase in front
+  const int64_t len_max = SRCK == 1 ? ((int64_t)((P.RT - 1) / P.WP + 1) * S + FH) * g.W : (int64_t)FH * P.NJ;
+  int64_t cp = len_max + 2 * EPC;
+  const int64_t cp_align = 32 / ES;  // a row is a whole number of 32 bytes: a stage of >= 4 rows a whole number of 128
+  cp = (cp + cp_align - 1) / cp_align * cp_align;
+  if (cp * ES > 65536) return IM2WIN_EUNSUPPORTED;
+  P.CP = (int32_t)cp;
+  P.box = (P.pm == 0 && cp * ES <= 2048 && P.GR >= 4 && encode_fn() != nullptr && (int64_t)g.N * g.C <= INT32_MAX &&
+           !knobs().no_box) ? 1 : 0;
+  P.raw_stage_bytes = (uint32_t)(P.GR * cp * ES);
+  if (P.raw_stage_bytes % 128 != 0) return IM2WIN_EUNSUPPORTED;
+  P.t_stage_bytes = (uint32_t)(GDIV * FH * S * P.RA * 16);
+  const int64_t blk_bytes = (int64_t)P.NT * 64;
+  // filter stages: a whole (T stage, tap) worth of blocks per stage where three such stages fit beside
+  // the rest (one wait and one release per NBLK*2*MH MMAs), else one block per stage
+  const int64_t fixed = 2 * (int64_t)P.t_stage_bytes;
+  P.ND = 512 / (P.MH * P.NT) >= 2 ? 2 : 1;
+  P.BB = 1;
+  if (3 * P.NBLK * blk_bytes + fixed + 3 * (int64_t)P.raw_stage_bytes <= cap) P.BB = P.NBLK;
+  P.NBS = P.NBLK / P.BB;
+  P.b_stage_bytes = (uint32_t)(P.BB * blk_bytes);
+  // split what is left between filter stages and source stages: the filter ring gets up to a third
+  // (at least three stages), the source ring the rest (bytes in flight towards HBM)
+  int64_t left = cap - fixed;
+  int64_t sb = left / 3 / P.b_stage_bytes;
+  if (sb < 3) sb = 3;
+  if (sb > kMaxB) sb = kMaxB;
+  int64_t sr = (left - sb * P.b_stage_bytes) / P.raw_stage_bytes;
+  if (sr > kMaxRaw) sr = kMaxRaw;
+  if (sr < 2) return IM2WIN_EUNSUPPORTED;
+  // give unused bytes back to the filter ring
+  int64_t sb2 = (left - sr * P.raw_stage_bytes) / P.b_stage_bytes;
+  if (sb2 > kMaxB) sb2 = kMaxB;
+  if (sb2 > sb) sb = sb2;
+  P.SB = (int32_t)sb; P.SR = (int32_t)sr;
+  uint32_t off = (uint32_t)(P.SB * P.b_stage_bytes);
+  off = (off + 1023) / 1024 * 1024;
+  P.off_t = off; off += 2 * P.t_stage_bytes;
+  off = (off + 127) / 128 * 128;
+  P.off_raw = off; off += (uint32_t)P.SR * P.raw_stage_bytes;
+  off = (off + 15) / 16 * 16;
+  P.off_bar = off; off += (uint32_t)((sizeof(SBars) + 15) / 16 * 16);
+  P.off_misc = off; off += 64;
+  pl->smem_bytes = off + 1024;
+  if (pl->smem_bytes > 227 * 1024) return IM2WIN_EUNSUPPORTED;
+  const int32_t cols = P.ND * P.MH * P.NT;
+  P.tmem_cols = 32;
+  while ((int32_t)P.tmem_cols < cols) P.tmem_cols *= 2;
+  P.idesc = ptx::make_idesc(128, P.NT, BF16 ? 1 : 2);
+  pl->scratch_bytes = (size_t)FW * P.Kp * ((size_t)g.C * FH) * (BF16 ? 2 : 4);
+  pl->threads = (kEpiWarp0 + 4 * P.MH) * 32;
+  return IM2WIN_OK;
+}
+
+// Whether the strip-matrix kernel is expected to beat the persistent kernel on this problem.  (Measured
+// on B200: it wins wherever the filter tile is 128 or wider, i.e. where MMAs are long enough to hide the
+// single issuing thread's bookkeeping; for narrower tiles the persistent kernel's three issuing threads win.)
+bool strip_preferred(const Geometry& g, const SParams& P) {
+  (void)g;
+  return P.NT >= 128;
+}
+
+template <int FH, int FW, int S, bool BF16, int SRCK>
+int launch_strip(const void* src, const float* f, float* out, const Geometry& g, cudaStream_t st, Scratch scratch) {
+  Plan pl;
+  int rc = make_plan<FH, FW, S, BF16, SRCK>(g, &pl);
+  if (rc != IM2WIN_OK) return rc;
+  SParams& P = pl.P;
+  if (!knobs().force_strip && !strip_preferred(g, P)) return IM2WIN_EUNSUPPORTED;
+  if (!scratch.ptr || scratch.bytes < pl.scratch_bytes || (reinterpret_cast<uintptr_t>(scratch.ptr) & 15u)) return IM2WIN_EUNSUPPORTED;
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return IM2WIN_EUNSUPPORTED;
+  P.src = src; P.out = out;
+  P.status = device_status_word();
+  if (!P.status) return IM2WIN_ECUDA;
+  constexpr int64_t ES = SRCK == 2 ? 2 : 4;
+  CUtensorMap fmap, xmap;
+  memset(&fmap, 0, sizeof(fmap));
+  memset(&xmap, 0, sizeof(xmap));
+  {
+    const int64_t row = (int64_t)g.C * FH;
+    const cuuint64_t gdim[2] = {(cuuint64_t)row, (cuuint64_t)FW * P.Kp};
+    const cuuint64_t gstr[1] = {(cuuint64_t)row * (BF16 ? 2 : 4)};
+    const cuuint32_t box[2] = {BF16 ? 32u : 16u, (cuuint32_t)P.NT};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&fmap, BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, scratch.ptr, gdim, gstr, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return IM2WIN_EUNSUPPORTED;
+  }
+  if (P.box) {
+    const cuuint64_t gdim[2] = {(cuuint64_t)(P.plane * ES / 8), (cuuint64_t)g.N * g.C};
+    const cuuint64_t gstr[1] = {(cuuint64_t)P.plane * ES};
+    const cuuint32_t box[2] = {(cuuint32_t)(P.CP * ES / 8), (cuuint32_t)P.GR};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&xmap, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(src), gdim, gstr, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      P.box = 0;  // bulk copies then
+  }
+  auto kern = conv_tc_strip_kernel<FH, FW, S, BF16, SRCK>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return IM2WIN_ECUDA;
+  }
+  {
+    const int64_t n = (int64_t)FW * P.Kp * g.C * FH;
+    const int64_t blocks = (n + 255) / 256;
+    const unsigned nb = (unsigned)(blocks < 148 * 8 ? blocks : 148 * 8);
+    filter_tap_major_kernel<BF16><<<nb, 256, 0, st>>>(f, scratch.ptr, g.K, P.Kp, g.C, FH, FW);
+  }
+  const int64_t grid = P.units < sm_count() ? P.units : sm_count();
+  kern<<<(unsigned)grid, pl.threads, pl.smem_bytes, st>>>(P, fmap, xmap);
+  return cuda_status(cudaGetLastError());
+}
+
+template <int FH, int FW, int S>
+int launch_strip_fs(const void* src, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st,
+                    Scratch scratch, int src_kind) {
+  const bool bf16 = mode == IM2WIN_MODE_BF16;
+  if (src_kind == 2) return bf16 ? launch_strip<FH, FW, S, true, 2>(src, f, out, g, st, scratch) : IM2WIN_EUNSUPPORTED;
+  if (src_kind == 1) return bf16 ? launch_strip<FH, FW, S, true, 1>(src, f, out, g, st, scratch)
+                                 : launch_strip<FH, FW, S, false, 1>(src, f, out, g, st, scratch);
+  return bf16 ? launch_strip<FH, FW, S, true, 0>(src, f, out, g, st, scratch)
+              : launch_strip<FH, FW, S, false, 0>(src, f, out, g, st, scratch);
+}
+
+template <int FH, int FW, int S>
+size_t scratch_fs(const Geometry& g, int mode, int src_kind) {
+  Plan pl;
+  const bool bf16 = mode == IM2WIN_MODE_BF16;
+  int rc;
+  if (src_kind == 2) rc = bf16 ? make_plan<FH, FW, S, true, 2>(g, &pl) : IM2WIN_EUNSUPPORTED;
+  else if (src_kind == 1) rc = bf16 ? make_plan<FH, FW, S, true, 1>(g, &pl) : make_plan<FH, FW, S, false, 1>(g, &pl);
+  else rc = bf16 ? make_plan<FH, FW, S, true, 0>(g, &pl) : make_plan<FH, FW, S, false, 0>(g, &pl);
+  return rc == IM2WIN_OK ? (pl.scratch_bytes + 255) / 256 * 256 : 0;
+}
+
+}  // namespace
+
+int launch_conv_tc_strip(const void* src, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st,
+                         Scratch scratch, int src_kind, bool out_bf16) {
+  if (out_bf16) return IM2WIN_EUNSUPPORTED;  // fp32 epilogue only
+  if (mode != IM2WIN_MODE_TF32 && mode != IM2WIN_MODE_BF16) return IM2WIN_EUNSUPPORTED;
+  if (g.Fh == 3 && g.Fw == 3 && g.s == 1) return launch_strip_fs<3, 3, 1>(src, f, out, g, mode, st, scratch, src_kind);
+  if (g.Fh == 3 && g.Fw == 3 && g.s == 2) return launch_strip_fs<3, 3, 2>(src, f, out, g, mode, st, scratch, src_kind);
   return IM2WIN_EUNSUPPORTED;
 }
-size_t strip_scratch_bytes(const Geometry&, int, int) { return 0; }
+
+size_t strip_scratch_bytes(const Geometry& g, int mode, int src_kind) {
+  if (mode != IM2WIN_MODE_TF32 && mode != IM2WIN_MODE_BF16) return 0;
+  if (g.Fh == 3 && g.Fw == 3 && g.s == 1) return scratch_fs<3, 3, 1>(g, mode, src_kind);
+  if (g.Fh == 3 && g.Fw == 3 && g.s == 2) return scratch_fs<3, 3, 2>(g, mode, src_kind);
+  return 0;
+}
+
 }  // namespace im2win

@@ -144,6 +144,28 @@ __device__ __forceinline__ void mma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, ui
         ::"r"(d_tmem), "r"(a_tmem), "r"(desc_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
   }
 }
+// D[tmem] (+)= A[smem descriptor] * B[smem descriptor], both descriptors passed as 32-bit halves.
+template <bool BF16>
+__device__ __forceinline__ void mma_ss_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                            uint32_t idesc, uint32_t accumulate) {
+  if constexpr (BF16) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 ad, {%1, %2};\n\t"
+        "mov.b64 bd, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 ad, {%1, %2};\n\t"
+        "mov.b64 bd, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], ad, bd, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+  }
+}
 // Arrive on `bar` once every tcgen05.mma issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -171,6 +193,32 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw32(uint32_t saddr) {
   d |= (uint64_t)(256 >> 4) << 32;
   d |= (uint64_t)1 << 46;
   d |= (uint64_t)6 << 61;                   // layout: 32-byte swizzle
+  return d;
+}
+
+// K-major operand with the 64-byte swizzle: rows of 64 bytes (two MMA K steps), groups of 8 rows
+// 512 bytes apart, 16-byte chunk c of row r stored at chunk position c ^ ((r >> 1) & 3).
+__device__ __forceinline__ uint64_t smem_desc_k_sw64(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(512 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)4 << 61;                   // layout: 64-byte swizzle
+  return d;
+}
+
+// K-major operand WITHOUT swizzle, stored chunk-major: the 16-byte chunk kc (4 fp32 / 8 bf16 along K)
+// of row r lies at kc * lbo + r * 16, i.e. core matrices of 8 rows x 16 bytes are contiguous (stride
+// dimension byte offset 128) and K-adjacent core matrices are `lbo` bytes apart.  Rows are 16 bytes
+// apart for any r, so a descriptor that starts `n` rows further down is this one plus n (the start
+// address field counts 16-byte units): overlapping row windows of one matrix are free.
+__device__ __forceinline__ uint64_t smem_desc_k_chunkmajor(uint32_t saddr, uint32_t lbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
+  d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;  // leading-dimension byte offset: next chunk along K
+  d |= (uint64_t)(128 >> 4) << 32;             // stride-dimension byte offset: next 8 rows
+  d |= (uint64_t)1 << 46;
   return d;
 }
 
