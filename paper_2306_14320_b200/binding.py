@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
         if _use_test:
             cur.im2win_debug_set_option.argtypes = [ctypes.c_char_p, ctypes.c_int]
             cur.im2win_debug_set_option.restype = ctypes.c_int
+            cur.im2win_debug_last_kernel.argtypes = []
+            cur.im2win_debug_last_kernel.restype = ctypes.c_int
             _test_lib = cur
         else:
             _lib = cur
@@ -145,6 +147,16 @@ def workspace_bytes(shape) -> int:
     b = ctypes.c_size_t()
     _check(lib().im2win_workspace_bytes(ctypes.byref(Shape.of(shape)), ctypes.byref(b)), "im2win_workspace_bytes")
     return b.value
+
+
+KERNEL_STRIP, KERNEL_PERSISTENT, KERNEL_GENERIC, KERNEL_FP32 = 1, 2, 3, 4
+
+
+def last_kernel() -> int:
+    """Test build only: which convolution kernel the last call launched (KERNEL_*)."""
+    if not _use_test:
+        raise RuntimeError("the test library only: call use_test_library(True) first")
+    return lib().im2win_debug_last_kernel()
 
 
 def conv_workspace_bytes(shape, src_kind: int, mode: int) -> int:

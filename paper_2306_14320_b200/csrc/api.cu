@@ -92,6 +92,9 @@ const Knobs& knobs() {
 }
 #endif
 
+static std::atomic<int> g_last_kernel{KERNEL_NONE};
+void note_kernel(int which) { g_last_kernel.store(which, std::memory_order_relaxed); }
+
 int sm_count() {
   constexpr int kMaxDev = 64;
   static std::atomic<int> cached[kMaxDev];
@@ -302,6 +305,9 @@ int im2win_last_device_status(void* cuda_stream, int32_t* status) {
 }
 
 #ifdef IM2WIN_TEST_KNOBS
+// Test build only: which convolution kernel the last call launched (KERNEL_* of common.cuh).
+int im2win_debug_last_kernel(void) { return g_last_kernel.load(std::memory_order_relaxed); }
+
 // Test build only (libim2win_test.so): set one diagnostic switch by name.  Returns IM2WIN_EINVAL for
 // an unknown name.
 int im2win_debug_set_option(const char* name, int value) {
@@ -313,7 +319,7 @@ int im2win_debug_set_option(const char* name, int value) {
       {"no_bslice", &Knobs::no_bslice}, {"splitk", &Knobs::splitk}, {"force_stream", &Knobs::force_stream},
       {"nsets", &Knobs::nsets}, {"no_l2ahead", &Knobs::no_l2ahead}, {"no_btma", &Knobs::no_btma},
       {"ntiles", &Knobs::ntiles}, {"transform_gather", &Knobs::transform_gather},
-      {"test_skip_copy", &Knobs::test_skip_copy}, {"strip_mh", &Knobs::strip_mh}};
+      {"test_skip_copy", &Knobs::test_skip_copy}, {"strip_mh", &Knobs::strip_mh}, {"strip_pair", &Knobs::strip_pair}};
   for (const Entry& e : table)
     if (strcmp(e.name, name) == 0) { g_knobs.*(e.field) = value; return IM2WIN_OK; }
   return IM2WIN_EINVAL;

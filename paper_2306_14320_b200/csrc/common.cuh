@@ -96,8 +96,14 @@ struct Knobs {
   int transform_gather = 0;  // transform: the staged-gather kernel instead of the tile kernel
   int test_skip_copy = 0;    // transform tile kernel, single-CTA problems: announce the input copy, never issue it
   int strip_mh = 0;          // strip-matrix kernel: 128-row halves per tile (0: own choice)
+  int strip_pair = 0;        // strip-matrix kernel: 1 = CTA pairs (cta_group::2) forced, 2 = single CTAs forced, 0 = own choice
 };
 const Knobs& knobs();
+
+// Which convolution kernel the last launch on this host thread's library image used (a diagnostic the
+// test build exposes as im2win_debug_last_kernel; the product library only writes it).
+enum : int { KERNEL_NONE = 0, KERNEL_STRIP = 1, KERNEL_PERSISTENT = 2, KERNEL_GENERIC = 3, KERNEL_FP32 = 4 };
+void note_kernel(int which);
 
 // Streaming multiprocessors of the current device (cached per device).
 int sm_count();

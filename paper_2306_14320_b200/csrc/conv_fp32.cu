@@ -42,6 +42,7 @@ int launch_conv_fp32(const float* xhat, const float* f, float* out, const Geomet
   const int64_t blocks = (g.n_out + 255) / 256;
   const int grid = (int)(blocks < 148 * 32 ? blocks : 148 * 32);
   conv_fp32_kernel<<<grid, 256, 0, st>>>(xhat, f, out, g);
+  note_kernel(KERNEL_FP32);
   return cuda_status(cudaGetLastError());
 }
 

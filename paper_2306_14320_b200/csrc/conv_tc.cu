@@ -488,6 +488,7 @@ int launch_conv_tc_generic(const float* xhat, const float* f, float* out, const 
                                        (int)smem_bytes);
   if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
   conv_tc_kernel<<<(unsigned)nblocks, kThreads, smem_bytes, st>>>(P);
+  note_kernel(KERNEL_GENERIC);
   return cuda_status(cudaGetLastError());
 }
 

@@ -1442,6 +1442,7 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
     if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
     kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
   }
+  note_kernel(KERNEL_PERSISTENT);
   return cuda_status(cudaGetLastError());
 }
 

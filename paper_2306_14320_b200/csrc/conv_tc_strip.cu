@@ -37,6 +37,16 @@
 #include "ptx_sm100.cuh"
 
 namespace im2win {
+#ifdef IM2WIN_PROF
+extern long long* g_prof;  // debug build: counter buffer (defined in conv_tc_persistent.cu)
+#define SPROF_DECL long long pw[7] = {}; const long long pt0 = clock64();
+#define SPROF_W(k, ...) { const long long c0_ = clock64(); __VA_ARGS__; pw[k] += clock64() - c0_; }
+#define SPROF_DUMP(role) if (P.prof && blockIdx.x < 8 && lane == 0) { long long* o_ = P.prof + ((long long)blockIdx.x * 8 + (role)) * 8; o_[0] = clock64() - pt0; for (int z_ = 0; z_ < 7; ++z_) o_[1 + z_] = pw[z_]; }
+#else
+#define SPROF_DECL
+#define SPROF_W(k, ...) { __VA_ARGS__; }
+#define SPROF_DUMP(role)
+#endif
 namespace {
 
 constexpr int kTW = 8;             // transposer warps
@@ -58,10 +68,15 @@ struct SParams {
   int32_t RA;         // T rows per class allocated (RT rounded up to 8)
   int32_t NJ;         // RT * s: (row, class) pairs = source columns per tile
   int32_t NT, n_ntiles, Kp;
+  int32_t NTB;        // filter rows one CTA holds per block: NT, or NT/2 when two CTAs share an MMA
+  int32_t pair;       // two CTAs (a cluster) work as one: tcgen05.mma.cta_group::2, M = 256, each CTA its own rows and half the filter tile
+  int64_t tiles;      // row tiles: N * TPI
   int32_t G, GR, NSUB, NTS;  // channels per T stage / per source stage, source stages per T stage, T stages per unit
   int32_t CBN;        // channel blocks (of NCH channels) per source stage
   int32_t NBLK, BB, NBS;     // filter blocks (2 K steps) per (T stage, tap); blocks per filter stage; filter stages per (T stage, tap)
   int32_t SR, SB, ND;
+  int32_t epi_split;  // the epilogue warps store columns [0, epi_split); with one accumulator buffer the (then idle)
+                      // transposer warps store [epi_split, NT); epi_split == NT: no help
   int32_t CP;         // elements per channel row of a source stage
   int32_t box;        // source stages come as one 2-D TMA box
   int32_t pm;         // plane length modulo the elements of a 16-byte chunk (bulk copies: per-channel phase)
@@ -71,6 +86,9 @@ struct SParams {
   uint32_t idesc, tmem_cols;
   uint32_t raw_stage_bytes, t_stage_bytes, b_stage_bytes;
   uint32_t off_t, off_raw, off_bar, off_misc;
+#ifdef IM2WIN_PROF
+  long long* prof;
+#endif
 };
 
 struct SBars {
@@ -146,18 +164,89 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
 
-// Where unit t lies: filter tile, image, first T row of the tile.
+// Cluster helpers (pair mode: a cluster of two CTAs).
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA box whose completion is signalled on a barrier of the pair's leader CTA (a shared::cluster address)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+// D[tmem of both CTAs] (+)= A[each CTA's own rows] * B[each CTA holds half the N rows]; M = 256.
+template <bool BF16>
+__device__ __forceinline__ void mma_ss_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                            uint32_t idesc, uint32_t accumulate) {
+  if constexpr (BF16) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 ad, {%1, %2};\n\t"
+        "mov.b64 bd, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], ad, bd, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 ad, {%1, %2};\n\t"
+        "mov.b64 bd, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], ad, bd, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+  }
+}
+// Arrive on the barrier at the same shared-memory offset in both CTAs of the pair once every MMA issued so far is done.
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
+// Work of iteration `it` of this CTA: filter tile, image, first T row of the row tile, and whether its
+// results are stored.  Single-CTA mode: units t = blockIdx.x + it*grid, the filter tile fastest.  Pair
+// mode: the pair (cluster) takes two consecutive row tiles of one filter tile, one per CTA; where the
+// number of row tiles is odd the last pair's second CTA repeats the last tile without storing.
 struct Unit {
   int32_t nt, img, R0;
+  bool store;
 };
-__device__ __forceinline__ Unit unit_of(const SParams& P, int64_t t) {
-  Unit u;
-  const int64_t tile = t / P.n_ntiles;
-  u.nt = (int32_t)(t - tile * P.n_ntiles);
+template <bool PAIR>
+__device__ __forceinline__ bool unit_at(const SParams& P, int64_t it, uint32_t rank, Unit& u) {
+  int64_t tile;
+  if (PAIR) {
+    const int64_t pu = (int64_t)(blockIdx.x >> 1) + it * (int64_t)(gridDim.x >> 1);
+    if (pu >= P.units) return false;
+    const int64_t half = (P.tiles + 1) >> 1;
+    const int64_t nt = pu / half;
+    tile = 2 * (pu - nt * half) + rank;
+    u.store = tile < P.tiles;
+    if (!u.store) tile = P.tiles - 1;
+    u.nt = (int32_t)nt;
+  } else {
+    const int64_t t = (int64_t)blockIdx.x + it * (int64_t)gridDim.x;
+    if (t >= P.units) return false;
+    tile = t / P.n_ntiles;
+    u.nt = (int32_t)(t - tile * P.n_ntiles);
+    u.store = true;
+  }
   const int64_t img = tile / P.TPI;
   u.img = (int32_t)img;
   u.R0 = (int32_t)(tile - img * P.TPI) * 128 * P.MH;
-  return u;
+  return true;
 }
 // Source elements [e_lo, e_hi) of a channel plane that the tile starting at T row R0 needs.
 template <int FH, int S, bool FUSED>
@@ -175,8 +264,111 @@ __device__ __forceinline__ void tile_range(const SParams& P, int32_t R0, int32_t
   }
 }
 
+// Stores columns [c_begin, c_end) (multiples of 16) of one warp's 32 accumulator rows: TMEM -> registers
+// -> NCHW.  The TMEM load of the next 16 columns is in flight while the current 16 are stored.
+__device__ __forceinline__ void store_columns(uint32_t d_tmem, float* orow, int64_t HoWo, int32_t c_begin, int32_t c_end,
+                                              int32_t k_left, bool valid) {
+  uint32_t va[16], vb[16];
+  if (c_begin >= c_end) return;
+  ptx::tmem_ld_x16(d_tmem + (uint32_t)c_begin, va);
+#pragma unroll 1
+  for (int32_t c0 = c_begin; c0 < c_end; c0 += 32) {
+    ptx::tmem_wait_ld();
+    const bool more = c0 + 16 < c_end;
+    if (more) ptx::tmem_ld_x16(d_tmem + (uint32_t)(c0 + 16), vb);
+    if (valid) {
+      float* o = orow + (int64_t)c0 * HoWo;
+      const int32_t left = k_left - c0;
+#pragma unroll
+      for (int e = 0; e < 16; ++e)
+        if (e < left) o[(int64_t)e * HoWo] = __uint_as_float(va[e]);
+    }
+    if (more) {
+      ptx::tmem_wait_ld();
+      if (c0 + 32 < c_end) ptx::tmem_ld_x16(d_tmem + (uint32_t)(c0 + 32), va);
+      if (valid) {
+        float* o = orow + (int64_t)(c0 + 16) * HoWo;
+        const int32_t left = k_left - c0 - 16;
+#pragma unroll
+        for (int e = 0; e < 16; ++e)
+          if (e < left) o[(int64_t)e * HoWo] = __uint_as_float(vb[e]);
+      }
+    }
+  }
+}
+
+// The MMA-issuing thread's whole life.  A filter stage holds the NBLK blocks of one (T stage, tap),
+// so there is one wait and one release per NBLK*2*MH MMAs.
+template <int FW, int S, bool BF16, int MH, int NBLK, bool PAIR>
+__device__ __forceinline__ void mma_role(const SParams& P, SBars* bars, SMisc* misc, uint32_t tmem_base, uint32_t t_sa,
+                                         uint32_t b_sa) {
+  Ring tr, br, dr;
+  bool ok = true;
+  SPROF_DECL
+  const uint64_t ad0 = ptx::smem_desc_k_chunkmajor(t_sa, (uint32_t)(S * P.RA) * 16u);
+  const uint64_t bd0 = ptx::smem_desc_k_sw64(b_sa);
+  const uint32_t a_lo0 = (uint32_t)ad0, a_hi = (uint32_t)(ad0 >> 32);
+  const uint32_t b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
+  const uint32_t t16 = P.t_stage_bytes >> 4, b16 = P.b_stage_bytes >> 4;
+  const uint32_t blk16 = (uint32_t)P.NTB * 4u;         // one filter block (NTB rows x 64 bytes) in 16-byte units
+  const uint32_t kstep16 = 2u * (uint32_t)(S * P.RA);  // one MMA K step (two chunks) of T in 16-byte units
+  const uint32_t RA = (uint32_t)P.RA, NT = (uint32_t)P.NT, idesc = P.idesc;
+  const uint32_t t_full0 = ptx::smem_u32(&bars->t_full[0]), t_empty0 = ptx::smem_u32(&bars->t_empty[0]);
+  const uint32_t b_full0 = ptx::smem_u32(&bars->b_full[0]), b_empty0 = ptx::smem_u32(&bars->b_empty[0]);
+  const int32_t lane = 0;
+  (void)lane;
+  for (int64_t it = 0; ok; ++it, dr.advance(P.ND)) {
+    Unit u;
+    if (!unit_at<PAIR>(P, it, 0, u)) break;
+    SPROF_W(0, ok = wait_bar(P, misc, ptx::smem_u32(&bars->acc_empty[dr.idx]), dr.phase ^ 1u, DEV_TIMEOUT_ACC))
+    if (!ok) break;
+    ptx::tc_fence_after();
+    const uint32_t d_tmem = tmem_base + (uint32_t)(dr.idx * MH) * NT;
+    uint32_t accum = 0;
+    for (int32_t ts = 0; ts < P.NTS && ok; ++ts, tr.advance(2)) {
+      SPROF_W(1, ok = wait_bar(P, misc, t_full0 + (uint32_t)tr.idx * 8u, tr.phase, DEV_TIMEOUT_A_FULL, 20))
+      if (!ok) break;
+      const uint32_t a_stage = a_lo0 + (uint32_t)tr.idx * t16;
+#pragma unroll
+      for (int v = 0; v < FW; ++v) {
+        SPROF_W(2, ok = wait_bar(P, misc, b_full0 + (uint32_t)br.idx * 8u, br.phase, DEV_TIMEOUT_B_FULL, 20))
+        if (!ok) break;
+        ptx::tc_fence_after();
+        uint32_t a_k = a_stage + (uint32_t)(v % S) * RA + (uint32_t)(v / S);
+        uint32_t b_k = b_lo0 + (uint32_t)br.idx * b16;
+#pragma unroll
+        for (int blk = 0; blk < NBLK; ++blk) {
+#pragma unroll
+          for (int k2 = 0; k2 < 2; ++k2) {
+            if constexpr (PAIR) {
+              mma_ss_pair<BF16>(d_tmem, a_k, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, accum);
+              if (MH == 2) mma_ss_pair<BF16>(d_tmem + NT, a_k + 128u, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, accum);
+            } else {
+              ptx::mma_ss_lohi<BF16>(d_tmem, a_k, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, accum);
+              if (MH == 2) ptx::mma_ss_lohi<BF16>(d_tmem + NT, a_k + 128u, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, accum);
+            }
+            accum = 1;
+            a_k += kstep16;
+          }
+          b_k += blk16;
+        }
+        if constexpr (PAIR) mma_commit_pair(b_empty0 + (uint32_t)br.idx * 8u);
+        else ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u);
+        br.advance(P.SB);
+      }
+      if (!ok) break;
+      if constexpr (PAIR) mma_commit_pair(t_empty0 + (uint32_t)tr.idx * 8u);
+      else ptx::mma_commit(t_empty0 + (uint32_t)tr.idx * 8u);
+    }
+    if (!ok) break;
+    if constexpr (PAIR) mma_commit_pair(ptx::smem_u32(&bars->acc_full[dr.idx]));
+    else ptx::mma_commit(ptx::smem_u32(&bars->acc_full[dr.idx]));
+  }
+  SPROF_DUMP(1)
+}
+
 // SRCK: 0 = fp32 im2win tensor, 1 = untransformed input (fused), 2 = bf16 im2win tensor (BF16 mode).
-template <int FH, int FW, int S, bool BF16, int SRCK>
+template <int FH, int FW, int S, bool BF16, int SRCK, bool PAIR>
 __global__ void __launch_bounds__(640, 1)
 conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, const __grid_constant__ CUtensorMap xmap) {
   constexpr bool FUSED = SRCK == 1;
@@ -185,7 +377,8 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
   constexpr uint32_t ES = SRC16 ? 2u : 4u;       // bytes per source element
   constexpr int32_t EPC = SRC16 ? 8 : 4;          // source elements per 16-byte chunk
   constexpr int NCH = BF16 ? 8 : 4;               // channels per transposer task = T elements per 16-byte chunk
-  constexpr int SH = (FW - 1) / S;                // largest row offset of a tap
+  constexpr int GDIV = FH % 4 == 0 ? 1 : (FH % 2 == 0 ? 2 : 4);
+  constexpr int NBLK = GDIV * FH / 4;             // filter blocks (two K steps each) per (T stage, tap)
 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* const smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -194,6 +387,8 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
   const uint32_t b_sa = ptx::smem_u32(smem), t_sa = b_sa + P.off_t, raw_sa = b_sa + P.off_raw;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int32_t n_epi_warps = 4 * P.MH;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // pair mode: 0 = the leader, whose thread issues the MMAs of both
+  constexpr uint32_t kShare = PAIR ? 2u : 1u;            // CTAs that arrive on the leader's "full"-side barriers
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxRaw; ++i) {
@@ -205,20 +400,26 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
       ptx::mbar_init(ptx::smem_u32(&bars->b_empty[i]), 1);
     }
     for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(ptx::smem_u32(&bars->t_full[i]), kTW);
+      ptx::mbar_init(ptx::smem_u32(&bars->t_full[i]), kTW * kShare);
       ptx::mbar_init(ptx::smem_u32(&bars->t_empty[i]), 1);
       ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), 1);
-      ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), (uint32_t)n_epi_warps);
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), (uint32_t)n_epi_warps * kShare * (P.epi_split < P.NT ? 2u : 1u));
     }
     ptx::fence_mbar_init();
     misc->abort = 0;
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), P.tmem_cols);
-    ptx::tmem_relinquish();
+    if constexpr (PAIR) {  // (the same warp of both CTAs)
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(ptx::smem_u32(&misc->tmem_base)), "r"(P.tmem_cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), P.tmem_cols);
+      ptx::tmem_relinquish();
+    }
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();  // both CTAs' barriers exist before either signals the other's
   ptx::tc_fence_after();
   const uint32_t tmem_base = misc->tmem_base;
 
@@ -229,8 +430,10 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
     Ring rr;
     int64_t count = 0;
     bool ok = true;
-    for (int64_t t = blockIdx.x; t < P.units && ok; t += gridDim.x) {
-      const Unit u = unit_of(P, t);
+    SPROF_DECL
+    for (int64_t it = 0; ok; ++it) {
+      Unit u;
+      if (!unit_at<PAIR>(P, it, rank, u)) break;
       int32_t e_lo, e_hi;
       tile_range<FH, S, FUSED>(P, u.R0, e_lo, e_hi);
       const int32_t len = e_hi - e_lo;
@@ -239,7 +442,7 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
       for (int32_t sidx = 0; sidx < nstages && ok; ++sidx, ++count, rr.advance(P.SR)) {
         const int32_t ch0 = sidx * P.GR;
         const uint32_t full = ptx::smem_u32(&bars->raw_full[rr.idx]);
-        ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->raw_empty[rr.idx]), rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, 64);
+        SPROF_W(0, ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->raw_empty[rr.idx]), rr.phase ^ 1u, DEV_TIMEOUT_RAW_EMPTY, 64))
         if (!ok) break;
         const uint32_t dst0 = raw_sa + (uint32_t)rr.idx * P.raw_stage_bytes;
         if (P.box) {
@@ -273,64 +476,18 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
         __syncwarp();
       }
     }
+    SPROF_DUMP(0)
     // every copy issued must have landed before the CTA exits
     for (int64_t c = count > P.SR ? count - P.SR : 0; c < count; ++c)
       wait_bar(P, misc, ptx::smem_u32(&bars->raw_full[c % P.SR]), (uint32_t)(c / P.SR) & 1u, DEV_TIMEOUT_DRAIN);
   } else if (warp == 1) {
     // ================================================================ MMA ISSUER
-    if (lane == 0) {
-      Ring tr, br, dr;
-      bool ok = true;
-      const uint64_t ad0 = ptx::smem_desc_k_chunkmajor(t_sa, (uint32_t)(S * P.RA) * 16u);
-      const uint64_t bd0 = ptx::smem_desc_k_sw64(b_sa);
-      const uint32_t a_lo0 = (uint32_t)ad0, a_hi = (uint32_t)(ad0 >> 32);
-      const uint32_t b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
-      const uint32_t t16 = P.t_stage_bytes >> 4, b16 = P.b_stage_bytes >> 4;
-      const uint32_t blk16 = (uint32_t)P.NT * 4u;        // one filter block (NT rows x 64 bytes) in 16-byte units
-      const uint32_t kstep16 = 2u * (uint32_t)(S * P.RA);  // one MMA K step (two chunks) of T in 16-byte units
-      for (int64_t t = blockIdx.x; t < P.units && ok; t += gridDim.x, dr.advance(P.ND)) {
-        ok = wait_bar(P, misc, ptx::smem_u32(&bars->acc_empty[dr.idx]), dr.phase ^ 1u, DEV_TIMEOUT_ACC);
-        if (!ok) break;
-        ptx::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(dr.idx * P.MH * P.NT);
-        uint32_t accum = 0;
-        for (int32_t ts = 0; ts < P.NTS && ok; ++ts, tr.advance(2)) {
-          ok = wait_bar(P, misc, ptx::smem_u32(&bars->t_full[tr.idx]), tr.phase, DEV_TIMEOUT_A_FULL, 20);
-          if (!ok) break;
-          ptx::tc_fence_after();
-          const uint32_t a_stage = a_lo0 + (uint32_t)tr.idx * t16;
-#pragma unroll
-          for (int v = 0; v < FW; ++v) {
-            const uint32_t a_v = a_stage + (uint32_t)((v % S) * P.RA + v / S);
-            for (int32_t bs = 0; bs < P.NBS; ++bs) {
-              if (!ptx::mbar_try_wait(ptx::smem_u32(&bars->b_full[br.idx]), br.phase)) {
-                ok = wait_bar(P, misc, ptx::smem_u32(&bars->b_full[br.idx]), br.phase, DEV_TIMEOUT_B_FULL, 20);
-                if (!ok) break;
-              }
-              ptx::tc_fence_after();
-              const uint32_t b_stage = b_lo0 + (uint32_t)br.idx * b16;
-              for (int32_t blk = 0; blk < P.BB; ++blk) {
-                const uint32_t ks0 = (uint32_t)(bs * P.BB + blk) * 2u;
-#pragma unroll
-                for (int k2 = 0; k2 < 2; ++k2) {
-                  const uint32_t a_k = a_v + (ks0 + k2) * kstep16;
-                  const uint32_t b_k = b_stage + (uint32_t)blk * blk16 + (uint32_t)k2 * 2u;
-                  for (int32_t h = 0; h < P.MH; ++h)
-                    ptx::mma_ss_lohi<BF16>(d_tmem + (uint32_t)(h * P.NT), a_k + (uint32_t)h * 128u, a_hi, b_k, b_hi, P.idesc, accum);
-                  accum = 1;
-                }
-              }
-              ptx::mma_commit(ptx::smem_u32(&bars->b_empty[br.idx]));
-              br.advance(P.SB);
-            }
-            if (!ok) break;
-          }
-          if (!ok) break;
-          ptx::mma_commit(ptx::smem_u32(&bars->t_empty[tr.idx]));
-        }
-        if (!ok) break;
-        ptx::mma_commit(ptx::smem_u32(&bars->acc_full[dr.idx]));
-      }
+    // One thread.  Its instruction stream is what bounds narrow filter tiles, so the loop over one
+    // T stage is fully unrolled for the compile-time (taps, filter blocks, halves) and steps the
+    // descriptors by additions of registers computed once.
+    if (lane == 0 && rank == 0) {
+      if (P.MH == 1) mma_role<FW, S, BF16, 1, NBLK, PAIR>(P, bars, misc, tmem_base, t_sa, b_sa);
+      else mma_role<FW, S, BF16, 2, NBLK, PAIR>(P, bars, misc, tmem_base, t_sa, b_sa);
     }
     __syncwarp();
   } else if (warp == 2) {
@@ -339,25 +496,39 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
       Ring br;
       int64_t count = 0;
       bool ok = true;
+      SPROF_DECL
       const int32_t bke = BF16 ? 32 : 16;  // elements per 64-byte filter row
-      for (int64_t t = blockIdx.x; t < P.units && ok; t += gridDim.x) {
-        const Unit u = unit_of(P, t);
+      // Pair mode: this CTA fetches its half of every block's rows, and the bytes of both CTAs are counted
+      // on the leader's barrier: the leader announces both halves with its one arrival (its own copies go
+      // through the ordinary local form), the other CTA only issues its copies.  (Its bytes may land
+      // before the announcement: the phase cannot complete before the leader's arrival, and the other
+      // CTA cannot run a phase ahead, because it needs the stage's release, which follows the phase.)
+      asm volatile("griddepcontrol.wait;" ::: "memory");  // the filter copy is written by the kernel launched just before
+      const bool remote = PAIR && rank != 0;
+      const uint32_t b_full_lead0 = remote ? mapa(ptx::smem_u32(&bars->b_full[0]), 0) : ptx::smem_u32(&bars->b_full[0]);
+      for (int64_t it = 0; ok; ++it) {
+        Unit u;
+        if (!unit_at<PAIR>(P, it, rank, u)) break;
+        const int32_t row0 = u.nt * P.NT + (int32_t)rank * P.NTB;
         for (int32_t ts = 0; ts < P.NTS && ok; ++ts) {
-          for (int32_t v = 0; v < FW && ok; ++v) {
-            for (int32_t bs = 0; bs < P.NBS && ok; ++bs, ++count, br.advance(P.SB)) {
-              ok = wait_bar(P, misc, ptx::smem_u32(&bars->b_empty[br.idx]), br.phase ^ 1u, DEV_TIMEOUT_B_EMPTY);
-              if (!ok) break;
-              const uint32_t full = ptx::smem_u32(&bars->b_full[br.idx]);
-              ptx::mbar_arrive_expect_tx(full, P.b_stage_bytes);
-              for (int32_t blk = 0; blk < P.BB; ++blk)
-                tma_load_2d(b_sa + (uint32_t)br.idx * P.b_stage_bytes + (uint32_t)blk * (uint32_t)P.NT * 64u, &fmap,
-                            (ts * P.NBLK + bs * P.BB + blk) * bke, v * P.Kp + u.nt * P.NT, full);
+          for (int32_t v = 0; v < FW && ok; ++v, ++count, br.advance(P.SB)) {
+            SPROF_W(0, ok = wait_bar(P, misc, ptx::smem_u32(&bars->b_empty[br.idx]), br.phase ^ 1u, DEV_TIMEOUT_B_EMPTY))
+            if (!ok) break;
+            const uint32_t full = b_full_lead0 + (uint32_t)br.idx * 8u;
+            if (!remote) ptx::mbar_arrive_expect_tx(full, P.b_stage_bytes * kShare);
+            for (int32_t blk = 0; blk < P.BB; ++blk) {
+              const uint32_t dst = b_sa + (uint32_t)br.idx * P.b_stage_bytes + (uint32_t)blk * (uint32_t)P.NTB * 64u;
+              if (remote) tma_load_2d_pair(dst, &fmap, (ts * P.NBLK + blk) * bke, v * P.Kp + row0, full);
+              else tma_load_2d(dst, &fmap, (ts * P.NBLK + blk) * bke, v * P.Kp + row0, full);
             }
           }
         }
       }
+      SPROF_DUMP(7)
+      // every copy issued must have landed before the CTA exits: the stage's release by the MMAs that
+      // read it says so (in pair mode the bytes are counted on the leader's barrier, not here)
       for (int64_t c = count > P.SB ? count - P.SB : 0; c < count; ++c)
-        wait_bar(P, misc, ptx::smem_u32(&bars->b_full[c % P.SB]), (uint32_t)(c / P.SB) & 1u, DEV_TIMEOUT_DRAIN);
+        wait_bar(P, misc, ptx::smem_u32(&bars->b_empty[c % P.SB]), (uint32_t)(c / P.SB) & 1u, DEV_TIMEOUT_DRAIN);
     }
     __syncwarp();
   } else if (warp >= kTWarp0 && warp < kTWarp0 + kTW) {
@@ -368,8 +539,13 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
     const uint32_t ustride = (FUSED ? (uint32_t)P.W : 1u) * ES;
     Ring rr, tr;
     bool ok = true;
-    for (int64_t t = blockIdx.x; t < P.units && ok; t += gridDim.x) {
-      const Unit u = unit_of(P, t);
+    SPROF_DECL
+    uint32_t hphase = 0;  // (epilogue help) phase of the single accumulator buffer's "full" barrier
+    const bool remote = PAIR && rank != 0;
+    const uint32_t t_full_lead0 = remote ? mapa(ptx::smem_u32(&bars->t_full[0]), 0) : ptx::smem_u32(&bars->t_full[0]);
+    for (int64_t it = 0; ok; ++it) {
+      Unit u;
+      if (!unit_at<PAIR>(P, it, rank, u)) break;
       int32_t e_lo, e_hi;
       tile_range<FH, S, FUSED>(P, u.R0, e_lo, e_hi);
       // this thread's tasks: (source column j = (T row, class), channel block cb of the stage)
@@ -401,12 +577,15 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
       for (int32_t ts = 0; ts < P.NTS && ok; ++ts, tr.advance(2)) {
         const uint32_t t_stage = t_sa + (uint32_t)tr.idx * P.t_stage_bytes;
         for (int32_t sub = 0; sub < P.NSUB && ok; ++sub, rr.advance(P.SR)) {
-          ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->raw_full[rr.idx]), rr.phase, DEV_TIMEOUT_RAW_FULL);
+          SPROF_W(0, ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->raw_full[rr.idx]), rr.phase, DEV_TIMEOUT_RAW_FULL))
           if (!ok) break;
           if (sub == 0) {
-            ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->t_empty[tr.idx]), tr.phase ^ 1u, DEV_TIMEOUT_A_EMPTY);
+            SPROF_W(1, ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->t_empty[tr.idx]), tr.phase ^ 1u, DEV_TIMEOUT_A_EMPTY))
             if (!ok) break;
           }
+#ifdef IM2WIN_PROF
+          const long long cw0 = clock64();
+#endif
           const uint32_t rs = raw_sa + (uint32_t)rr.idx * P.raw_stage_bytes;
           const int32_t ch0 = (ts * P.NSUB + sub) * P.GR;
           const uint32_t t_sub = t_stage + (uint32_t)(sub * P.CBN * FH) * lbo;
@@ -442,74 +621,107 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
           const bool last = sub == P.NSUB - 1;
           if (last) ptx::fence_proxy_async_smem();  // this thread's T writes -> visible to the tensor core
           __syncwarp();
+#ifdef IM2WIN_PROF
+          pw[2] += clock64() - cw0;
+#endif
           if (lane == 0) {
             ptx::mbar_arrive(ptx::smem_u32(&bars->raw_empty[rr.idx]));
-            if (last) ptx::mbar_arrive(ptx::smem_u32(&bars->t_full[tr.idx]));
+            if (last) {
+              if (remote) arrive_cluster(t_full_lead0 + (uint32_t)tr.idx * 8u);
+              else ptx::mbar_arrive(t_full_lead0 + (uint32_t)tr.idx * 8u);
+            }
+          }
+        }
+      }
+      // One accumulator buffer: nothing can be transposed for the next unit before this unit's MMAs are
+      // done, so this warp stores the upper columns of its TMEM lane quarter meanwhile.
+      if (ok && P.epi_split < P.NT) {
+        const int32_t hh = (warp - kTWarp0) >> 2, q4 = warp & 3;
+        ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->acc_full[0]), hphase, DEV_TIMEOUT_ACC, 128);
+        if (!ok) break;
+        hphase ^= 1u;
+        ptx::tc_fence_after();
+        if (hh < P.MH) {
+          const int32_t rho = u.R0 + hh * 128 + q4 * 32 + lane;
+          const int32_t m = rho / P.WP, q = rho - m * P.WP;
+          const bool valid = u.store && rho < P.RPI && q < P.Wo;
+          const int32_t n0 = u.nt * P.NT;
+          const int64_t HoWo = (int64_t)P.Ho * P.Wo;
+          float* const orow = P.out + ((int64_t)u.img * P.K + n0) * HoWo + (int64_t)m * P.Wo + q;
+          store_columns(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(hh * P.NT), orow, HoWo, P.epi_split, P.NT, P.K - n0, valid);
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            const uint32_t ae = ptx::smem_u32(&bars->acc_empty[0]);
+            if (remote) arrive_cluster(mapa(ae, 0));
+            else ptx::mbar_arrive(ae);
           }
         }
       }
     }
+    if (warp == kTWarp0) { SPROF_DUMP(2) }
   } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + n_epi_warps) {
     // ================================================================ EPILOGUE: TMEM -> NCHW
     const int32_t h = (warp - kEpiWarp0) >> 2, q4 = warp & 3;  // (kEpiWarp0 is a multiple of 4: warp & 3 = TMEM lane quarter)
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
     Ring dr;
     bool ok = true;
-    const int32_t eK = P.K, eNT = P.NT;
+    SPROF_DECL
+    const int32_t eK = P.K;
     const int64_t eHoWo = (int64_t)P.Ho * P.Wo;
-    for (int64_t t = blockIdx.x; t < P.units && ok; t += gridDim.x, dr.advance(P.ND)) {
-      const Unit u = unit_of(P, t);
+    const bool remote = PAIR && rank != 0;
+    const uint32_t acc_empty_lead0 = remote ? mapa(ptx::smem_u32(&bars->acc_empty[0]), 0) : ptx::smem_u32(&bars->acc_empty[0]);
+    for (int64_t it = 0; ok; ++it, dr.advance(P.ND)) {
+      Unit u;
+      if (!unit_at<PAIR>(P, it, rank, u)) break;
       const int32_t rho = u.R0 + h * 128 + q4 * 32 + lane;
       const int32_t m = rho / P.WP, q = rho - m * P.WP;
-      const bool valid = rho < P.RPI && q < P.Wo;
+      const bool valid = u.store && rho < P.RPI && q < P.Wo;
       const int32_t n0 = u.nt * P.NT;
       float* const orow = P.out + ((int64_t)u.img * P.K + n0) * eHoWo + (int64_t)m * P.Wo + q;
-      ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->acc_full[dr.idx]), dr.phase, DEV_TIMEOUT_ACC, 128);
+      SPROF_W(0, ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->acc_full[dr.idx]), dr.phase, DEV_TIMEOUT_ACC, 128))
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)((dr.idx * P.MH + h) * P.NT);
-#pragma unroll 1
-      for (int32_t c0 = 0; c0 < eNT; c0 += 16) {
-        uint32_t v[16];
-        ptx::tmem_ld_x16(d_tmem + (uint32_t)c0, v);
-        ptx::tmem_wait_ld();
-        if (valid) {
-          float* o = orow + (int64_t)c0 * eHoWo;
-          const int32_t left = eK - n0 - c0;
-#pragma unroll
-          for (int e = 0; e < 16; ++e)
-            if (e < left) o[(int64_t)e * eHoWo] = __uint_as_float(v[e]);
-        }
-      }
+      store_columns(d_tmem, orow, eHoWo, 0, P.epi_split, eK - n0, valid);
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->acc_empty[dr.idx]));
+      if (lane == 0) {
+        if (remote) arrive_cluster(acc_empty_lead0 + (uint32_t)dr.idx * 8u);
+        else ptx::mbar_arrive(acc_empty_lead0 + (uint32_t)dr.idx * 8u);
+      }
     }
+    if (warp == kEpiWarp0) { SPROF_DUMP(6) }
   }
 
   // ------------------------------------------------------------------ teardown
   ptx::tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();  // neither CTA leaves while the other may still signal its barriers
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, P.tmem_cols);
+    if constexpr (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(P.tmem_cols) : "memory");
+    else ptx::tmem_dealloc(tmem_base, P.tmem_cols);
   }
 }
 
 // Tap-major copy of the filter for the TMA-streamed B operand:
 //   Fv[v][j][r*Fh + u] = F[j][r][u][v]   (j < K; rows K..Kp-1 are zero), fp32 or bf16 (nearest even).
+// One block row per (v, j): no division but the one by the (small) filter height.
 template <bool BF16>
 __global__ void __launch_bounds__(256) filter_tap_major_kernel(const float* __restrict__ f, void* __restrict__ o, int32_t K,
-                                                               int32_t Kp, int32_t C, int32_t FH, int32_t FW) {
-  const int64_t row = (int64_t)C * FH, n = (int64_t)FW * Kp * row;
-  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (int64_t)gridDim.x * 256) {
-    const int64_t vj = i / row;
-    const int32_t ku = (int32_t)(i - vj * row);
-    const int32_t v = (int32_t)(vj / Kp), j = (int32_t)(vj - (int64_t)v * Kp);
-    const int32_t r = ku / FH, u = ku - r * FH;
-    const float x = j < K ? f[(((int64_t)j * C + r) * FH + u) * FW + v] : 0.f;
-    if (BF16) static_cast<__nv_bfloat16*>(o)[i] = __float2bfloat16_rn(x);
-    else static_cast<float*>(o)[i] = x;
+                                                               int32_t Kp, int32_t row, int32_t FH, int32_t FW) {
+  // the convolution kernel that follows may start its prologue now (it waits for this grid's completion
+  // before it reads the copy)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int32_t vj = (int32_t)blockIdx.y;
+  const int32_t v = vj / Kp, j = vj - v * Kp;
+  const float* fj = f + (int64_t)j * row * FW + v;
+  const int64_t obase = (int64_t)vj * row;
+  for (int32_t ku = (int32_t)(blockIdx.x * 256 + threadIdx.x); ku < row; ku += (int32_t)gridDim.x * 256) {
+    const float x = j < K ? __ldg(fj + (int64_t)ku * FW) : 0.f;   // (r*Fh + u)*Fw + v = ku*Fw + v
+    if (BF16) static_cast<__nv_bfloat16*>(o)[obase + ku] = __float2bfloat16_rn(x);
+    else static_cast<float*>(o)[obase + ku] = x;
   }
 }
 
@@ -541,7 +753,7 @@ struct Plan {
 
 // Fills the launch parameters for (FH, FW, S, BF16, SRCK); IM2WIN_EUNSUPPORTED where the kernel does not apply.
 template <int FH, int FW, int S, bool BF16, int SRCK>
-int make_plan(const Geometry& g, Plan* pl) {
+int make_plan(const Geometry& g, Plan* pl, int pair, int mh_fixed) {
   constexpr int NCH = BF16 ? 8 : 4;
   constexpr int64_t ES = SRCK == 2 ? 2 : 4;
   constexpr int64_t EPC = 16 / ES;
@@ -558,46 +770,24 @@ int make_plan(const Geometry& g, Plan* pl) {
   P.n_ntiles = (g.K + 255) / 256;
   P.NT = ((g.K + P.n_ntiles - 1) / P.n_ntiles + 15) / 16 * 16;
   P.Kp = P.n_ntiles * P.NT;
+  if ((int64_t)FW * P.Kp > 65535) return IM2WIN_EUNSUPPORTED;  // (grid of the filter-copy kernel)
+  P.pair = pair;
+  P.NTB = pair ? P.NT / 2 : P.NT;
   P.NTS = g.C / P.G;
   P.NBLK = GDIV * FH / 4;
   if (SRCK == 1) { P.plane = (int64_t)g.H * g.W; P.n_src = g.n_in; }
   else { P.plane = g.HoL; P.n_src = g.n_win; }
   P.pm = (int32_t)(P.plane % EPC);
-  const int nsm = sm_count();
   const int64_t cap = 227 * 1024 - 1024 - 512;  // alignment slack, barriers
-  // 128-row halves per tile: two halve the filter bytes streamed per output (each filter stage feeds
-  // two MMAs) but leave a single accumulator buffer for wide filter tiles; picked by waves x work,
-  // ties to two halves.
-  int best_mh = 0;
-  double best_cost = 0;
-  for (int mh = 1; mh <= 2; ++mh) {
-    if (knobs().strip_mh && knobs().strip_mh != mh) continue;
-    if (mh * P.NT > 512) continue;
-    const int64_t tpi = (P.RPI + 128 * mh - 1) / (128 * mh);
-    const int64_t units = (int64_t)g.N * tpi * P.n_ntiles;
-    const int64_t waves = (units + nsm - 1) / nsm;
-    const int nd = 512 / (mh * P.NT) >= 2 ? 2 : 1;
-    double cost = (double)waves * mh * (nd == 1 ? 1.08 : 1.0);
-    if (mh == 2) cost *= 0.97;
-    if (!best_mh || cost < best_cost) { best_mh = mh; best_cost = cost; }
-  }
-  if (!best_mh) return IM2WIN_EUNSUPPORTED;
-  P.MH = best_mh;
+  P.MH = mh_fixed;
+  if (P.MH * P.NT > 512) return IM2WIN_EUNSUPPORTED;
   P.TPI = (P.RPI + 128 * P.MH - 1) / (128 * P.MH);
-  P.units = (int64_t)g.N * P.TPI * P.n_ntiles;
+  P.tiles = (int64_t)g.N * P.TPI;
+  P.units = pair ? ((P.tiles + 1) / 2) * P.n_ntiles : P.tiles * P.n_ntiles;
   P.RT = 128 * P.MH + SH;
   P.RA = (P.RT + 7) / 8 * 8;
   P.NJ = P.RT * S;
   if ((int64_t)S * P.RA > 16383) return IM2WIN_EUNSUPPORTED;
-  // channel blocks per source stage: as many as keep a stage's (column, block) tasks within about two
-  // rounds of the 256 transposer threads
-  P.CBN = 1;
-  for (int cbn = GDIV; cbn >= 1; cbn /= 2)
-    if (GDIV % cbn == 0 && (int64_t)P.NJ * cbn <= 2 * kTW * 32 + 32) { P.CBN = cbn; break; }
-  if ((int64_t)P.NJ * P.CBN > (int64_t)kTMax * kTW * 32) return IM2WIN_EUNSUPPORTED;
-  P.GR = P.CBN * NCH;
-  if (P.GR > 32) return IM2WIN_EUNSUPPORTED;  // one producer lane per channel of a stage
-  P.NSUB = P.G / P.GR;
   // elements of one channel a tile needs at most, plus the 16-byte phase in front
   const int64_t len_max = SRCK == 1 ? ((int64_t)((P.RT - 1) / P.WP + 1) * S + FH) * g.W : (int64_t)FH * P.NJ;
   int64_t cp = len_max + 2 * EPC;
@@ -605,33 +795,40 @@ int make_plan(const Geometry& g, Plan* pl) {
   cp = (cp + cp_align - 1) / cp_align * cp_align;
   if (cp * ES > 65536) return IM2WIN_EUNSUPPORTED;
   P.CP = (int32_t)cp;
-  P.box = (P.pm == 0 && cp * ES <= 2048 && P.GR >= 4 && encode_fn() != nullptr && (int64_t)g.N * g.C <= INT32_MAX &&
-           !knobs().no_box) ? 1 : 0;
-  P.raw_stage_bytes = (uint32_t)(P.GR * cp * ES);
-  if (P.raw_stage_bytes % 128 != 0) return IM2WIN_EUNSUPPORTED;
   P.t_stage_bytes = (uint32_t)(GDIV * FH * S * P.RA * 16);
-  const int64_t blk_bytes = (int64_t)P.NT * 64;
-  // filter stages: a whole (T stage, tap) worth of blocks per stage where three such stages fit beside
-  // the rest (one wait and one release per NBLK*2*MH MMAs), else one block per stage
+  const int64_t blk_bytes = (int64_t)P.NTB * 64;
   const int64_t fixed = 2 * (int64_t)P.t_stage_bytes;
   P.ND = 512 / (P.MH * P.NT) >= 2 ? 2 : 1;
-  P.BB = 1;
-  if (3 * P.NBLK * blk_bytes + fixed + 3 * (int64_t)P.raw_stage_bytes <= cap) P.BB = P.NBLK;
-  P.NBS = P.NBLK / P.BB;
+  P.BB = P.NBLK;  // a filter stage = the blocks of one (T stage, tap): one wait and one release per NBLK*2*MH MMAs
+  P.NBS = 1;
   P.b_stage_bytes = (uint32_t)(P.BB * blk_bytes);
-  // split what is left between filter stages and source stages: the filter ring gets up to a third
-  // (at least three stages), the source ring the rest (bytes in flight towards HBM)
-  int64_t left = cap - fixed;
-  int64_t sb = left / 3 / P.b_stage_bytes;
-  if (sb < 3) sb = 3;
-  if (sb > kMaxB) sb = kMaxB;
-  int64_t sr = (left - sb * P.b_stage_bytes) / P.raw_stage_bytes;
-  if (sr > kMaxRaw) sr = kMaxRaw;
-  if (sr < 2) return IM2WIN_EUNSUPPORTED;
-  // give unused bytes back to the filter ring
-  int64_t sb2 = (left - sr * P.raw_stage_bytes) / P.b_stage_bytes;
-  if (sb2 > kMaxB) sb2 = kMaxB;
-  if (sb2 > sb) sb = sb2;
+  // Channel blocks per source stage: as many as keep a stage's (column, block) tasks within about two
+  // rounds of the 256 transposer threads, fewer if the rings do not fit otherwise.  What is left beside
+  // the two T stages goes to the rings: at least two stages each, then filter stages up to four (the
+  // filter stream is the larger one wherever the filter tile is wide), then source stages.
+  int64_t sb = 0, sr = 0;
+  const int64_t left = cap - fixed;
+  for (int cbn = GDIV; cbn >= 1; cbn /= 2) {
+    if (GDIV % cbn != 0 || (int64_t)P.NJ * cbn > 2 * kTW * 32 + 32) {
+      if (cbn > 1) continue;
+    }
+    if ((int64_t)P.NJ * cbn > (int64_t)kTMax * kTW * 32) return IM2WIN_EUNSUPPORTED;
+    const int64_t raw_bytes = (int64_t)cbn * NCH * cp * ES;
+    if (cbn * NCH > 32 || raw_bytes % 128 != 0) continue;
+    if (2 * (int64_t)P.b_stage_bytes + 2 * raw_bytes > left) continue;
+    P.CBN = cbn;
+    P.GR = cbn * NCH;
+    P.raw_stage_bytes = (uint32_t)raw_bytes;
+    sb = 2; sr = 2;
+    while (sb < 4 && (sb + 1) * P.b_stage_bytes + sr * raw_bytes <= left) ++sb;
+    while (sr < kMaxRaw && sb * P.b_stage_bytes + (sr + 1) * raw_bytes <= left) ++sr;
+    while (sb < kMaxB && (sb + 1) * P.b_stage_bytes + sr * raw_bytes <= left) ++sb;
+    break;
+  }
+  if (!sb) return IM2WIN_EUNSUPPORTED;
+  P.NSUB = P.G / P.GR;
+  P.box = (P.pm == 0 && cp * ES <= 2048 && P.GR >= 4 && encode_fn() != nullptr && (int64_t)g.N * g.C <= INT32_MAX &&
+           !knobs().no_box) ? 1 : 0;
   P.SB = (int32_t)sb; P.SR = (int32_t)sr;
   uint32_t off = (uint32_t)(P.SB * P.b_stage_bytes);
   off = (off + 1023) / 1024 * 1024;
@@ -643,10 +840,13 @@ int make_plan(const Geometry& g, Plan* pl) {
   P.off_misc = off; off += 64;
   pl->smem_bytes = off + 1024;
   if (pl->smem_bytes > 227 * 1024) return IM2WIN_EUNSUPPORTED;
+  // one accumulator buffer: the transposer warps (two sets of four, one per half) store the upper half of
+  // the columns; with one half per tile only the first set helps, so the epilogue warps keep all columns
+  P.epi_split = (P.ND == 1 && P.MH == 2 && P.NT >= 64) ? (P.NT / 2 + 15) / 16 * 16 : P.NT;
   const int32_t cols = P.ND * P.MH * P.NT;
   P.tmem_cols = 32;
   while ((int32_t)P.tmem_cols < cols) P.tmem_cols *= 2;
-  P.idesc = ptx::make_idesc(128, P.NT, BF16 ? 1 : 2);
+  P.idesc = ptx::make_idesc(pair ? 256 : 128, P.NT, BF16 ? 1 : 2);
   pl->scratch_bytes = (size_t)FW * P.Kp * ((size_t)g.C * FH) * (BF16 ? 2 : 4);
   pl->threads = (kEpiWarp0 + 4 * P.MH) * 32;
   return IM2WIN_OK;
@@ -660,10 +860,91 @@ bool strip_preferred(const Geometry& g, const SParams& P) {
   return P.NT >= 128;
 }
 
+// Cost of a plan in units of one 128-row MMA pass over the whole reduction, per SM (smaller is better):
+// waves of units over the SMs (or SM pairs) x halves per unit, with what was measured on B200 folded in:
+// a single CTA that streams a wide filter tile is bound by shared-memory bandwidth (operand fetch of the
+// MMAs plus the TMA writes of the filter stages), which two halves per tile (each filter stage feeds two
+// MMAs) and CTA pairs (each CTA holds and fetches half the filter rows) relieve; a single accumulator
+// buffer leaves the epilogue of every unit exposed.
+double plan_cost(const SParams& P, int nsm) {
+  const int64_t slots = P.pair ? nsm / 2 : nsm;
+  const int64_t waves = (P.units + slots - 1) / slots;
+  double per_unit = P.MH;
+  const double wide = P.NT >= 192 ? 1.0 : (P.NT >= 96 ? 0.5 : 0.0);
+  if (!P.pair) per_unit *= 1.0 + wide * (P.MH == 1 ? 0.6 : 0.3);
+  else per_unit *= 1.0 + wide * (P.MH == 1 ? 0.1 : 0.0);
+  if (P.ND == 1) per_unit += 0.12 * P.MH;
+  return (double)waves * per_unit + 0.05;
+}
+
+template <int FH, int FW, int S, bool BF16, int SRCK>
+int choose_plan(const Geometry& g, Plan* best) {
+  const int nsm = sm_count();
+  bool have = false;
+  double best_cost = 0;
+  for (int pair = 1; pair >= 0; --pair) {
+    if (knobs().strip_pair == 1 && !pair) continue;
+    if (knobs().strip_pair == 2 && pair) continue;
+    for (int mh = 1; mh <= 2; ++mh) {
+      if (knobs().strip_mh && knobs().strip_mh != mh) continue;
+      Plan pl;
+      if (make_plan<FH, FW, S, BF16, SRCK>(g, &pl, pair, mh) != IM2WIN_OK) continue;
+      const double c = plan_cost(pl.P, nsm);
+      if (!have || c < best_cost) { *best = pl; best_cost = c; have = true; }
+    }
+  }
+  return have ? IM2WIN_OK : IM2WIN_EUNSUPPORTED;
+}
+
+template <int FH, int FW, int S, bool BF16, int SRCK, bool PAIR>
+int launch_kernel(const SParams& P, const Plan& pl, const CUtensorMap& fmap, const CUtensorMap& xmap, cudaStream_t st) {
+  auto kern = conv_tc_strip_kernel<FH, FW, S, BF16, SRCK, PAIR>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return IM2WIN_ECUDA;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3((unsigned)pl.threads);
+  cfg.dynamicSmemBytes = pl.smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  // programmatic dependent launch: the prologue (barriers, TMEM, first source copies) overlaps the
+  // filter-copy kernel launched just before; the filter producer waits for that kernel (griddepcontrol.wait)
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int64_t grid;
+  if (PAIR) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+    cfg.gridDim = dim3((unsigned)(sm_count() / 2 * 2));
+    int max_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg) != cudaSuccess || max_clusters < 1) {
+      cudaGetLastError();
+      return IM2WIN_EUNSUPPORTED;
+    }
+    int64_t pairs = sm_count() / 2;
+    if (pairs > max_clusters) pairs = max_clusters;
+    if (pairs > P.units) pairs = P.units;
+    grid = 2 * pairs;
+  } else {
+    grid = P.units < sm_count() ? P.units : sm_count();
+  }
+  cfg.gridDim = dim3((unsigned)grid);
+  if (cudaLaunchKernelEx(&cfg, kern, P, fmap, xmap) != cudaSuccess) {
+    cudaGetLastError();
+    return IM2WIN_ECUDA;
+  }
+  note_kernel(KERNEL_STRIP);
+  return IM2WIN_OK;
+}
+
 template <int FH, int FW, int S, bool BF16, int SRCK>
 int launch_strip(const void* src, const float* f, float* out, const Geometry& g, cudaStream_t st, Scratch scratch) {
   Plan pl;
-  int rc = make_plan<FH, FW, S, BF16, SRCK>(g, &pl);
+  int rc = choose_plan<FH, FW, S, BF16, SRCK>(g, &pl);
   if (rc != IM2WIN_OK) return rc;
   SParams& P = pl.P;
   if (!knobs().force_strip && !strip_preferred(g, P)) return IM2WIN_EUNSUPPORTED;
@@ -671,6 +952,9 @@ int launch_strip(const void* src, const float* f, float* out, const Geometry& g,
   EncodeTiledFn enc = encode_fn();
   if (!enc) return IM2WIN_EUNSUPPORTED;
   P.src = src; P.out = out;
+#ifdef IM2WIN_PROF
+  P.prof = g_prof;
+#endif
   P.status = device_status_word();
   if (!P.status) return IM2WIN_ECUDA;
   constexpr int64_t ES = SRCK == 2 ? 2 : 4;
@@ -681,7 +965,7 @@ int launch_strip(const void* src, const float* f, float* out, const Geometry& g,
     const int64_t row = (int64_t)g.C * FH;
     const cuuint64_t gdim[2] = {(cuuint64_t)row, (cuuint64_t)FW * P.Kp};
     const cuuint64_t gstr[1] = {(cuuint64_t)row * (BF16 ? 2 : 4)};
-    const cuuint32_t box[2] = {BF16 ? 32u : 16u, (cuuint32_t)P.NT};
+    const cuuint32_t box[2] = {BF16 ? 32u : 16u, (cuuint32_t)P.NTB};
     const cuuint32_t estr[2] = {1, 1};
     if (enc(&fmap, BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, scratch.ptr, gdim, gstr, box,
             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -698,20 +982,13 @@ int launch_strip(const void* src, const float* f, float* out, const Geometry& g,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       P.box = 0;  // bulk copies then
   }
-  auto kern = conv_tc_strip_kernel<FH, FW, S, BF16, SRCK>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes) != cudaSuccess) {
-    cudaGetLastError();
-    return IM2WIN_ECUDA;
-  }
   {
-    const int64_t n = (int64_t)FW * P.Kp * g.C * FH;
-    const int64_t blocks = (n + 255) / 256;
-    const unsigned nb = (unsigned)(blocks < 148 * 8 ? blocks : 148 * 8);
-    filter_tap_major_kernel<BF16><<<nb, 256, 0, st>>>(f, scratch.ptr, g.K, P.Kp, g.C, FH, FW);
+    const int32_t row = g.C * FH;
+    const dim3 pg((unsigned)((row + 255) / 256 < 4 ? (row + 255) / 256 : 4), (unsigned)(FW * P.Kp));
+    filter_tap_major_kernel<BF16><<<pg, 256, 0, st>>>(f, scratch.ptr, g.K, P.Kp, row, FH, FW);
   }
-  const int64_t grid = P.units < sm_count() ? P.units : sm_count();
-  kern<<<(unsigned)grid, pl.threads, pl.smem_bytes, st>>>(P, fmap, xmap);
-  return cuda_status(cudaGetLastError());
+  return P.pair ? launch_kernel<FH, FW, S, BF16, SRCK, true>(P, pl, fmap, xmap, st)
+                : launch_kernel<FH, FW, S, BF16, SRCK, false>(P, pl, fmap, xmap, st);
 }
 
 template <int FH, int FW, int S>
@@ -730,9 +1007,9 @@ size_t scratch_fs(const Geometry& g, int mode, int src_kind) {
   Plan pl;
   const bool bf16 = mode == IM2WIN_MODE_BF16;
   int rc;
-  if (src_kind == 2) rc = bf16 ? make_plan<FH, FW, S, true, 2>(g, &pl) : IM2WIN_EUNSUPPORTED;
-  else if (src_kind == 1) rc = bf16 ? make_plan<FH, FW, S, true, 1>(g, &pl) : make_plan<FH, FW, S, false, 1>(g, &pl);
-  else rc = bf16 ? make_plan<FH, FW, S, true, 0>(g, &pl) : make_plan<FH, FW, S, false, 0>(g, &pl);
+  if (src_kind == 2) rc = bf16 ? choose_plan<FH, FW, S, true, 2>(g, &pl) : IM2WIN_EUNSUPPORTED;
+  else if (src_kind == 1) rc = bf16 ? choose_plan<FH, FW, S, true, 1>(g, &pl) : choose_plan<FH, FW, S, false, 1>(g, &pl);
+  else rc = bf16 ? choose_plan<FH, FW, S, true, 0>(g, &pl) : choose_plan<FH, FW, S, false, 0>(g, &pl);
   return rc == IM2WIN_OK ? (pl.scratch_bytes + 255) / 256 * 256 : 0;
 }
 
