@@ -1233,6 +1233,10 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
     }
   }
   if (SRC16 && !P.pim) return IM2WIN_EUNSUPPORTED;  // the 16-bit source is implemented for per-image tiling only
+  // Tiles that span images: each of the strip producer's 32 lanes owns at most two (channel, image
+  // segment) pairs of a group, so a group holds at most 64 of them.  (Sixteen-channel groups on images
+  // of fewer than ~40 positions exceed that; the dispatcher then takes the eight-channel variant.)
+  if (!P.pim && (int64_t)CB * nseg_max > 64) return IM2WIN_EUNSUPPORTED;
   P.chan_pitch = (int32_t)pitch;
   const int64_t tiles_m = P.pim ? (int64_t)g.N * P.TPI : (g.Mtot + P.TP - 1) / P.TP;
   P.ntiles = tiles_m * P.n_ntiles;
@@ -1489,7 +1493,10 @@ int launch_spec_11x11(IM2WIN_SPEC_ARGS);
 #if IM2WIN_PART == -1 || IM2WIN_PART == 0
 int launch_spec_3x3(IM2WIN_SPEC_ARGS) {
   // BF16 MMAs take 16 reduction elements: sixteen channels (144 = 9 steps) leave no padding
-  if (bf16 && g.C % 16 == 0) return launch_spec<3, 3, 16, true>(xhat, f, out, g, st, scratch, kind, out_bf16);
+  if (bf16 && g.C % 16 == 0) {
+    const int rc = launch_spec<3, 3, 16, true>(xhat, f, out, g, st, scratch, kind, out_bf16);
+    if (rc != IM2WIN_EUNSUPPORTED) return rc;
+  }
   if (g.C >= 8) return bf16 ? launch_spec<3, 3, 8, true>(xhat, f, out, g, st, scratch, kind, out_bf16)
                             : launch_spec<3, 3, 8, false>(xhat, f, out, g, st, scratch, kind, out_bf16);
   if (g.C == 3) return bf16 ? launch_spec<3, 3, 3, true>(xhat, f, out, g, st, scratch, kind, out_bf16)
@@ -1499,7 +1506,10 @@ int launch_spec_3x3(IM2WIN_SPEC_ARGS) {
 #endif
 #if IM2WIN_PART == -1 || IM2WIN_PART == 1
 int launch_spec_5x5(IM2WIN_SPEC_ARGS) {
-  if (bf16 && g.C % 16 == 0) return launch_spec<5, 5, 16, true>(xhat, f, out, g, st, scratch, kind, out_bf16);
+  if (bf16 && g.C % 16 == 0) {
+    const int rc = launch_spec<5, 5, 16, true>(xhat, f, out, g, st, scratch, kind, out_bf16);
+    if (rc != IM2WIN_EUNSUPPORTED) return rc;
+  }
   if (g.C >= 8) return bf16 ? launch_spec<5, 5, 8, true>(xhat, f, out, g, st, scratch, kind, out_bf16)
                             : launch_spec<5, 5, 8, false>(xhat, f, out, g, st, scratch, kind, out_bf16);
   return IM2WIN_EUNSUPPORTED;

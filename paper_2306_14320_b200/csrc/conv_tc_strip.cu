@@ -852,48 +852,58 @@ int make_plan(const Geometry& g, Plan* pl, int pair, int mh_fixed) {
   return IM2WIN_OK;
 }
 
-// Whether the strip-matrix kernel is expected to beat the persistent kernel on this problem.  (Measured
-// on B200: it wins wherever the filter tile is 128 or wider, i.e. where MMAs are long enough to hide the
-// single issuing thread's bookkeeping; for narrower tiles the persistent kernel's three issuing threads win.)
-bool strip_preferred(const Geometry& g, const SParams& P) {
-  (void)g;
-  return P.NT >= 128;
-}
-
-// Cost of a plan in units of one 128-row MMA pass over the whole reduction, per SM (smaller is better):
-// waves of units over the SMs (or SM pairs) x halves per unit, with what was measured on B200 folded in:
-// a single CTA that streams a wide filter tile is bound by shared-memory bandwidth (operand fetch of the
-// MMAs plus the TMA writes of the filter stages), which two halves per tile (each filter stage feeds two
-// MMAs) and CTA pairs (each CTA holds and fetches half the filter rows) relieve; a single accumulator
-// buffer leaves the epilogue of every unit exposed.
-double plan_cost(const SParams& P, int nsm) {
-  const int64_t slots = P.pair ? nsm / 2 : nsm;
-  const int64_t waves = (P.units + slots - 1) / slots;
-  double per_unit = P.MH;
-  const double wide = P.NT >= 192 ? 1.0 : (P.NT >= 96 ? 0.5 : 0.0);
-  if (!P.pair) per_unit *= 1.0 + wide * (P.MH == 1 ? 0.6 : 0.3);
-  else per_unit *= 1.0 + wide * (P.MH == 1 ? 0.1 : 0.0);
-  if (P.ND == 1) per_unit += 0.12 * P.MH;
-  return (double)waves * per_unit + 0.05;
-}
-
+// Which variant of the kernel a problem gets (knobs override; rules from measurements on B200, batch 128):
+//  * filter tiles of 192 columns or more run as CTA pairs (each CTA fetches half the filter rows: a single
+//    CTA streaming a wide tile is bound by shared-memory bandwidth -- operand fetch of the MMAs plus the
+//    TMA writes of the filter stages -- and by the filter stream's L2 rate); narrower tiles run on single
+//    CTAs (a pair's MMAs cost the issuing thread about twice as long, which short MMAs cannot hide);
+//  * two 128-row halves per tile (each filter stage feeds two MMAs, half the filter bytes per output) for
+//    pairs in TF32 mode when an image has more than 128 T rows, and for single CTAs whose units would
+//    otherwise be short (few channels); one half otherwise: it keeps two accumulator buffers, so that
+//    the epilogue overlaps the next unit, and in BF16 mode it leaves room for the fp32 strip ring.
 template <int FH, int FW, int S, bool BF16, int SRCK>
 int choose_plan(const Geometry& g, Plan* best) {
-  const int nsm = sm_count();
-  bool have = false;
-  double best_cost = 0;
-  for (int pair = 1; pair >= 0; --pair) {
-    if (knobs().strip_pair == 1 && !pair) continue;
-    if (knobs().strip_pair == 2 && pair) continue;
-    for (int mh = 1; mh <= 2; ++mh) {
-      if (knobs().strip_mh && knobs().strip_mh != mh) continue;
-      Plan pl;
-      if (make_plan<FH, FW, S, BF16, SRCK>(g, &pl, pair, mh) != IM2WIN_OK) continue;
-      const double c = plan_cost(pl.P, nsm);
-      if (!have || c < best_cost) { *best = pl; best_cost = c; have = true; }
-    }
+  const int nt = (((g.K + (g.K + 255) / 256 - 1) / ((g.K + 255) / 256)) + 15) / 16 * 16;
+  const int wp = (g.W + S - 1) / S;
+  int pair = nt >= 192 ? 1 : 0;
+  int mh;
+  if (pair) mh = (!BF16 && (int64_t)g.Ho * wp > 128) ? 2 : 1;
+  else mh = ((int64_t)g.C * FH * FW / 8 < 100) ? 2 : 1;
+  if (knobs().strip_pair == 1) pair = 1;
+  if (knobs().strip_pair == 2) pair = 0;
+  if (knobs().strip_mh) mh = knobs().strip_mh;
+  // the preferred variant, then the others (a variant may not fit shared or tensor memory)
+  const int order[4][2] = {{pair, mh}, {pair, 3 - mh}, {1 - pair, mh}, {1 - pair, 3 - mh}};
+  for (const auto& o : order) {
+    if (knobs().strip_pair == 1 && !o[0]) continue;
+    if (knobs().strip_pair == 2 && o[0]) continue;
+    if (knobs().strip_mh && knobs().strip_mh != o[1]) continue;
+    if (make_plan<FH, FW, S, BF16, SRCK>(g, best, o[0], o[1]) == IM2WIN_OK) return IM2WIN_OK;
   }
-  return have ? IM2WIN_OK : IM2WIN_EUNSUPPORTED;
+  return IM2WIN_EUNSUPPORTED;
+}
+
+// Whether the strip-matrix kernel is expected to beat the persistent kernel (conv_tc_persistent.cu) on
+// this problem.  Measured on B200 (batch 128, the 3x3 layers of the benchmark lists): per wave of
+// 128-row passes it takes about 0.8 (TF32) / 0.75 (BF16) of the persistent kernel's time where the
+// filter tile is 96 or wider (narrower MMAs are bound by its single issuing thread, where the persistent
+// kernel's three win) and the stride is 1 (with two column classes its T stages leave the rings too
+// little shared memory).  The persistent kernel's tiles may span images, this kernel's do not, so the
+// comparison is between the two kernels' waves: small images whose tiles just fill one wave there stay
+// there.  In BF16 mode a filter small enough to stay resident in the persistent kernel's shared memory
+// also stays there.
+template <int FH, int FW, int S, bool BF16>
+bool strip_preferred(const Geometry& g, const SParams& P) {
+  if (S != 1 || P.NT < 96) return false;
+  if (BF16 && (int64_t)g.K * g.Kg * 2 <= 160 * 1024) return false;
+  const int nsm = sm_count();
+  const int64_t slots = P.pair ? nsm / 2 : nsm;
+  const double strip_passes = (double)((P.units + slots - 1) / slots) * P.MH;
+  const int64_t tpi = (g.HoWo + 127) / 128;
+  const bool pim = tpi * 128 * 100 <= g.HoWo * 107;
+  const int64_t tiles = pim ? (int64_t)g.N * tpi : (g.Mtot + 127) / 128;
+  const double persistent_passes = (double)((tiles * P.n_ntiles + nsm - 1) / nsm);
+  return BF16 ? strip_passes * 0.75 < persistent_passes : strip_passes * 0.8 <= persistent_passes;
 }
 
 template <int FH, int FW, int S, bool BF16, int SRCK, bool PAIR>
@@ -947,7 +957,7 @@ int launch_strip(const void* src, const float* f, float* out, const Geometry& g,
   int rc = choose_plan<FH, FW, S, BF16, SRCK>(g, &pl);
   if (rc != IM2WIN_OK) return rc;
   SParams& P = pl.P;
-  if (!knobs().force_strip && !strip_preferred(g, P)) return IM2WIN_EUNSUPPORTED;
+  if (!knobs().force_strip && !strip_preferred<FH, FW, S, BF16>(g, P)) return IM2WIN_EUNSUPPORTED;
   if (!scratch.ptr || scratch.bytes < pl.scratch_bytes || (reinterpret_cast<uintptr_t>(scratch.ptr) & 15u)) return IM2WIN_EUNSUPPORTED;
   EncodeTiledFn enc = encode_fn();
   if (!enc) return IM2WIN_EUNSUPPORTED;

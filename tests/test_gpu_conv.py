@@ -275,6 +275,41 @@ def test_conv_sweep_layers_batch_32_and_128(layer, batch, mode, _kernel):
 
 
 @pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("layer", [l for l in wl.TABLE_I_LAYERS if l.name != "table1_Conv4"], ids=lambda l: l.name)
+def test_conv_table1_layers_batch128(layer, mode, _kernel):
+    """The paper's own workload: Table I's unpadded layers at batch 128 (Conv4, whose tensors take
+    gigabytes, is covered at batch 16 below).  Eq. (1) at 20 000 sampled coordinates and every corner,
+    the whole first and last image, and no element that is not finite."""
+    if _kernel not in ("auto", "minws", "strip", "pair2", "nostrip"):
+        pytest.skip("forced persistent-kernel variants are covered at small sizes")
+    dims = layer.dims()
+    n, c, h, w, k, fh, fw, s = dims
+    ho, wo = b.out_dims(dims)
+
+    def make():
+        x, f = wl.make_input(layer), wl.make_filter(layer)
+        rng = np.random.default_rng(99)
+        idx = np.stack([rng.integers(0, n, 20000), rng.integers(0, k, 20000), rng.integers(0, ho, 20000),
+                        rng.integers(0, wo, 20000)], axis=1).astype(np.int32)
+        corners = np.array(list(itertools.product((0, n - 1), (0, k - 1), (0, ho - 1), (0, wo - 1))), dtype=np.int32)
+        idx = np.concatenate([idx, corners])
+        pts = oracle.conv_direct_points(x, f, oracle.Shape(*dims), idx)
+        one = layer.with_batch(1).dims()
+        ends = {img: oracle_conv(x[img:img + 1], f, one) for img in (0, n - 1)}
+        return x, f, idx, pts, ends
+
+    x, f, idx, pts, ends = _cached(("table1", layer.name), make)
+    got = gpu_conv(x, f, dims, mode)
+    assert np.isfinite(got).all()
+    sample = got[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]]
+    assert rel_l2(sample, pts) <= TOL[mode]
+    rms = float(np.sqrt(np.mean(pts * pts)))
+    assert float(np.abs(sample - pts).max()) <= 8.0 * TOL[mode] * rms
+    for img, ref in ends.items():
+        assert rel_l2(got[img:img + 1], ref) <= TOL[mode]
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
 @pytest.mark.parametrize("layer", wl.SWEEP, ids=lambda l: l.name)
 def test_conv_sweep_layers_batch32_small_integers_bit_exact(layer, mode, _kernel):
     if _kernel not in ("auto", "minws", "strip", "nostrip"):
