@@ -71,6 +71,11 @@ int launch_conv_tc(const void* src, const float* f, float* out, const Geometry& 
     if (rc != IM2WIN_EUNSUPPORTED) return rc;
     rc = launch_conv_tc_persistent(src, f, out, g, mode, st, scratch, src_kind == 1, src_kind == 2, out_bf16);
     if (rc != IM2WIN_EUNSUPPORTED) return rc;
+    // sources the generic kernel does not read (bf16 im2win tensor, fused): the strip-matrix kernel wherever it applies
+    if (src_kind != 0 && !knobs().no_strip) {
+      rc = launch_conv_tc_strip(src, f, out, g, mode, st, scratch, src_kind, out_bf16, /*even_if_slower=*/true);
+      if (rc != IM2WIN_EUNSUPPORTED) return rc;
+    }
   }
   if (src_kind != 0 || out_bf16) return IM2WIN_EUNSUPPORTED;
   return launch_conv_tc_generic(static_cast<const float*>(src), f, out, g, mode, st);
@@ -241,6 +246,8 @@ int conv_impl(const void* src, int src_kind, const float* filter, const im2win_s
       if (rc == IM2WIN_EUNSUPPORTED)
         rc = launch_conv_tc_persistent(xhat, filter, out_nchw, g, mode, st, scratch_from(0), /*fused=*/true,
                                        /*src_bf16=*/false, out16);
+      if (rc == IM2WIN_EUNSUPPORTED && !knobs().no_strip)
+        rc = launch_conv_tc_strip(xhat, filter, out_nchw, g, mode, st, scratch_from(0), 1, out16, /*even_if_slower=*/true);
       if (rc != IM2WIN_EUNSUPPORTED) return rc;
     }
     // no fused kernel for this shape or mode: the unfused path, if the caller supplied a workspace

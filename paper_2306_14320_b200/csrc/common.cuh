@@ -55,8 +55,10 @@ struct Scratch {
 // Tensor-core convolution kernels.  Each returns IM2WIN_EUNSUPPORTED when it does not apply (shape,
 // scratch) before anything is enqueued; launch_conv_tc tries them in order of expected speed.
 // src_kind: 0 = fp32 im2win tensor, 1 = untransformed input consumed fused, 2 = bf16 im2win tensor.
+// (even_if_slower: take the problem wherever the kernel is implemented, not only where it is expected to
+// be the fastest -- for sources no other kernel accepts)
 int launch_conv_tc_strip(const void* src, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st,
-                         Scratch scratch, int src_kind, bool out_bf16);
+                         Scratch scratch, int src_kind, bool out_bf16, bool even_if_slower = false);
 int launch_conv_tc_persistent(const void* src, const float* f, float* out, const Geometry& g, int mode,
                               cudaStream_t st, Scratch scratch, bool fused = false, bool src_bf16 = false,
                               bool out_bf16 = false);

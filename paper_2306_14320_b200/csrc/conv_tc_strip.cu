@@ -804,8 +804,7 @@ int make_plan(const Geometry& g, Plan* pl, int pair, int mh_fixed) {
   P.b_stage_bytes = (uint32_t)(P.BB * blk_bytes);
   // Channel blocks per source stage: as many as keep a stage's (column, block) tasks within about two
   // rounds of the 256 transposer threads, fewer if the rings do not fit otherwise.  What is left beside
-  // the two T stages goes to the rings: at least two stages each, then filter stages up to four (the
-  // filter stream is the larger one wherever the filter tile is wide), then source stages.
+  // the two T stages goes to the two rings stage by stage, in proportion to what each needs in flight.
   int64_t sb = 0, sr = 0;
   const int64_t left = cap - fixed;
   for (int cbn = GDIV; cbn >= 1; cbn /= 2) {
@@ -819,10 +818,21 @@ int make_plan(const Geometry& g, Plan* pl, int pair, int mh_fixed) {
     P.CBN = cbn;
     P.GR = cbn * NCH;
     P.raw_stage_bytes = (uint32_t)raw_bytes;
+    // stages each ring wants: the bytes it must keep in flight to cover the memory latency (about 2500
+    // cycles under load) at its consumption rate, plus the stage being consumed
+    const double mma_cyc = P.NT / 2.0 > 50.0 ? P.NT / 2.0 : 50.0;
+    const double b_stage_cyc = (double)P.NBLK * 2 * P.MH * mma_cyc;
+    const double raw_stage_cyc = b_stage_cyc * FW * cbn / GDIV;
+    const int64_t want_b = (int64_t)(2500.0 / b_stage_cyc + 0.999) + 1, want_r = (int64_t)(2500.0 / raw_stage_cyc + 0.999) + 1;
     sb = 2; sr = 2;
-    while (sb < 4 && (sb + 1) * P.b_stage_bytes + sr * raw_bytes <= left) ++sb;
-    while (sr < kMaxRaw && sb * P.b_stage_bytes + (sr + 1) * raw_bytes <= left) ++sr;
-    while (sb < kMaxB && (sb + 1) * P.b_stage_bytes + sr * raw_bytes <= left) ++sb;
+    while (true) {  // one more stage for the ring that is further below what it wants, while it fits
+      const bool can_b = sb < kMaxB && (sb + 1) * P.b_stage_bytes + sr * raw_bytes <= left;
+      const bool can_r = sr < kMaxRaw && sb * P.b_stage_bytes + (sr + 1) * raw_bytes <= left;
+      if (!can_b && !can_r) break;
+      const double fill_b = (double)sb / (double)want_b, fill_r = (double)sr / (double)want_r;
+      if (can_b && (!can_r || fill_b <= fill_r)) ++sb;
+      else ++sr;
+    }
     break;
   }
   if (!sb) return IM2WIN_EUNSUPPORTED;
@@ -952,12 +962,13 @@ int launch_kernel(const SParams& P, const Plan& pl, const CUtensorMap& fmap, con
 }
 
 template <int FH, int FW, int S, bool BF16, int SRCK>
-int launch_strip(const void* src, const float* f, float* out, const Geometry& g, cudaStream_t st, Scratch scratch) {
+int launch_strip(const void* src, const float* f, float* out, const Geometry& g, cudaStream_t st, Scratch scratch,
+                 bool even_if_slower) {
   Plan pl;
   int rc = choose_plan<FH, FW, S, BF16, SRCK>(g, &pl);
   if (rc != IM2WIN_OK) return rc;
   SParams& P = pl.P;
-  if (!knobs().force_strip && !strip_preferred<FH, FW, S, BF16>(g, P)) return IM2WIN_EUNSUPPORTED;
+  if (!even_if_slower && !knobs().force_strip && !strip_preferred<FH, FW, S, BF16>(g, P)) return IM2WIN_EUNSUPPORTED;
   if (!scratch.ptr || scratch.bytes < pl.scratch_bytes || (reinterpret_cast<uintptr_t>(scratch.ptr) & 15u)) return IM2WIN_EUNSUPPORTED;
   EncodeTiledFn enc = encode_fn();
   if (!enc) return IM2WIN_EUNSUPPORTED;
@@ -1003,13 +1014,13 @@ int launch_strip(const void* src, const float* f, float* out, const Geometry& g,
 
 template <int FH, int FW, int S>
 int launch_strip_fs(const void* src, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st,
-                    Scratch scratch, int src_kind) {
+                    Scratch scratch, int src_kind, bool slow_ok) {
   const bool bf16 = mode == IM2WIN_MODE_BF16;
-  if (src_kind == 2) return bf16 ? launch_strip<FH, FW, S, true, 2>(src, f, out, g, st, scratch) : IM2WIN_EUNSUPPORTED;
-  if (src_kind == 1) return bf16 ? launch_strip<FH, FW, S, true, 1>(src, f, out, g, st, scratch)
-                                 : launch_strip<FH, FW, S, false, 1>(src, f, out, g, st, scratch);
-  return bf16 ? launch_strip<FH, FW, S, true, 0>(src, f, out, g, st, scratch)
-              : launch_strip<FH, FW, S, false, 0>(src, f, out, g, st, scratch);
+  if (src_kind == 2) return bf16 ? launch_strip<FH, FW, S, true, 2>(src, f, out, g, st, scratch, slow_ok) : IM2WIN_EUNSUPPORTED;
+  if (src_kind == 1) return bf16 ? launch_strip<FH, FW, S, true, 1>(src, f, out, g, st, scratch, slow_ok)
+                                 : launch_strip<FH, FW, S, false, 1>(src, f, out, g, st, scratch, slow_ok);
+  return bf16 ? launch_strip<FH, FW, S, true, 0>(src, f, out, g, st, scratch, slow_ok)
+              : launch_strip<FH, FW, S, false, 0>(src, f, out, g, st, scratch, slow_ok);
 }
 
 template <int FH, int FW, int S>
@@ -1026,11 +1037,11 @@ size_t scratch_fs(const Geometry& g, int mode, int src_kind) {
 }  // namespace
 
 int launch_conv_tc_strip(const void* src, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st,
-                         Scratch scratch, int src_kind, bool out_bf16) {
+                         Scratch scratch, int src_kind, bool out_bf16, bool even_if_slower) {
   if (out_bf16) return IM2WIN_EUNSUPPORTED;  // fp32 epilogue only
   if (mode != IM2WIN_MODE_TF32 && mode != IM2WIN_MODE_BF16) return IM2WIN_EUNSUPPORTED;
-  if (g.Fh == 3 && g.Fw == 3 && g.s == 1) return launch_strip_fs<3, 3, 1>(src, f, out, g, mode, st, scratch, src_kind);
-  if (g.Fh == 3 && g.Fw == 3 && g.s == 2) return launch_strip_fs<3, 3, 2>(src, f, out, g, mode, st, scratch, src_kind);
+  if (g.Fh == 3 && g.Fw == 3 && g.s == 1) return launch_strip_fs<3, 3, 1>(src, f, out, g, mode, st, scratch, src_kind, even_if_slower);
+  if (g.Fh == 3 && g.Fw == 3 && g.s == 2) return launch_strip_fs<3, 3, 2>(src, f, out, g, mode, st, scratch, src_kind, even_if_slower);
   return IM2WIN_EUNSUPPORTED;
 }
 

@@ -30,7 +30,13 @@ SMALL = [
     (1, 24, 20, 21, 300, 3, 3, 1),       # streamed filter; in BF16 mode groups of 72 padded to 80 in the bf16 copy
     (1, 16, 21, 230, 16, 7, 7, 2),       # wide 7x7: sixteen-channel strip stages do not fit, eight-channel groups
     (1, 64, 21, 230, 64, 7, 7, 2),       # the same with a filter too large to be resident
+    # shapes the strip-matrix kernel takes (3x3, channels in multiples of 16 / 32): odd widths, filter counts
+    # that are no multiple of 16, two filter tiles, stride 2 with odd and even widths, images smaller than a
+    # tile and of a single output, several tiles per image
+    (2, 16, 11, 13, 24, 3, 3, 1), (3, 32, 9, 10, 40, 3, 3, 2), (1, 64, 17, 19, 300, 3, 3, 1), (2, 32, 20, 33, 17, 3, 3, 2),
+    (2, 64, 5, 5, 16, 3, 3, 1), (3, 32, 3, 3, 8, 3, 3, 1), (1, 32, 40, 37, 48, 3, 3, 1), (1, 32, 45, 44, 130, 3, 3, 2),
 ]
+STRIP_SHAPES = [d for d in SMALL if d[5] == 3 and d[6] == 3 and d[1] % 32 == 0 and d[7] in (1, 2)]
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -118,6 +124,20 @@ def test_conv_small_integers_bit_exact(dims, mode):
     assert np.abs(ref).max() < 2 ** 24
     got = gpu_conv(x, f, dims, mode)
     assert np.array_equal(got.astype(np.float64), ref)
+
+
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("dims", STRIP_SHAPES)
+def test_forced_strip_configurations_run_the_strip_kernel(dims, mode, _kernel):
+    """The configurations that force the strip-matrix kernel must really run it on the shapes it
+    implements (a silent fall-through to another kernel would leave it untested)."""
+    if _kernel not in ("strip", "strip2", "pair", "pair2"):
+        pytest.skip("only for the configurations that force the strip-matrix kernel")
+    x, f = _data(dims, 800, ints=True)
+    got = gpu_conv(x, f, dims, mode)
+    if dims[7] == 1 or _kernel in ("strip", "pair"):  # (two halves per tile and stride 2 together exceed shared memory)
+        assert b.last_kernel() == b.KERNEL_STRIP
+    assert np.array_equal(got.astype(np.float64), oracle_conv(x, f, dims))
 
 
 @pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
