@@ -778,7 +778,9 @@ int make_plan(const Geometry& g, Plan* pl, int pair, int mh_fixed) {
   if (SRCK == 1) { P.plane = (int64_t)g.H * g.W; P.n_src = g.n_in; }
   else { P.plane = g.HoL; P.n_src = g.n_win; }
   P.pm = (int32_t)(P.plane % EPC);
-  const int64_t cap = 227 * 1024 - 1024 - 512;  // alignment slack, barriers
+  // dynamic shared memory for the three areas: the limit less the base alignment (1024), the round-ups
+  // between the areas (1024 + 128 + 16), the barriers and the small state block
+  const int64_t cap = 227 * 1024 - 1024 - (1024 + 128 + 16) - (int64_t)((sizeof(SBars) + 15) / 16 * 16) - 64;
   P.MH = mh_fixed;
   if (P.MH * P.NT > 512) return IM2WIN_EUNSUPPORTED;
   P.TPI = (P.RPI + 128 * P.MH - 1) / (128 * P.MH);
