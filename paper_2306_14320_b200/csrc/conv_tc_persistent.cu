@@ -1362,6 +1362,8 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   }
   P.usub = P.n_ntiles * P.Z;
   P.ntiles *= P.Z;
+  // the roles count work units in 32 bits (t, t + grid, ...): decline what does not fit, instead of wrapping
+  if (P.ntiles > (int64_t)INT32_MAX - sm_count()) return IM2WIN_EUNSUPPORTED;
   const int32_t cols = P.ND * P.NT + P.NSETS * P.NSS * SLOT_COLS;
   P.tmem_cols = 32;
   while (P.tmem_cols < cols) P.tmem_cols *= 2;

@@ -870,16 +870,16 @@ int make_plan(const Geometry& g, Plan* pl, int pair, int mh_fixed) {
 //    TMA writes of the filter stages -- and by the filter stream's L2 rate); narrower tiles run on single
 //    CTAs (a pair's MMAs cost the issuing thread about twice as long, which short MMAs cannot hide);
 //  * two 128-row halves per tile (each filter stage feeds two MMAs, half the filter bytes per output) for
-//    pairs in TF32 mode when an image has more than 128 T rows, and for single CTAs whose units would
-//    otherwise be short (few channels); one half otherwise: it keeps two accumulator buffers, so that
-//    the epilogue overlaps the next unit, and in BF16 mode it leaves room for the fp32 strip ring.
+//    pairs when an image has more than 128 T rows, and for single CTAs whose units would otherwise be
+//    short (few channels); one half otherwise: it keeps two accumulator buffers, so that the epilogue
+//    overlaps the next unit.
 template <int FH, int FW, int S, bool BF16, int SRCK>
 int choose_plan(const Geometry& g, Plan* best) {
   const int nt = (((g.K + (g.K + 255) / 256 - 1) / ((g.K + 255) / 256)) + 15) / 16 * 16;
   const int wp = (g.W + S - 1) / S;
   int pair = nt >= 192 ? 1 : 0;
   int mh;
-  if (pair) mh = (!BF16 && (int64_t)g.Ho * wp > 128) ? 2 : 1;
+  if (pair) mh = ((int64_t)g.Ho * wp > 128) ? 2 : 1;
   else mh = ((int64_t)g.C * FH * FW / 8 < 100) ? 2 : 1;
   if (knobs().strip_pair == 1) pair = 1;
   if (knobs().strip_pair == 2) pair = 0;
