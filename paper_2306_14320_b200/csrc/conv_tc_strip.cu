@@ -903,7 +903,7 @@ int choose_plan(const Geometry& g, Plan* best) {
 // little shared memory).  The persistent kernel's tiles may span images, this kernel's do not, so the
 // comparison is between the two kernels' waves: small images whose tiles just fill one wave there stay
 // there.  In BF16 mode a filter small enough to stay resident in the persistent kernel's shared memory
-// also stays there.
+// also stays there.  Launches that fill less than half the SMs stay there too (reduction slices).
 template <int FH, int FW, int S, bool BF16>
 bool strip_preferred(const Geometry& g, const SParams& P) {
   if (S != 1 || P.NT < 96) return false;
@@ -914,6 +914,9 @@ bool strip_preferred(const Geometry& g, const SParams& P) {
   const int64_t tpi = (g.HoWo + 127) / 128;
   const bool pim = tpi * 128 * 100 <= g.HoWo * 107;
   const int64_t tiles = pim ? (int64_t)g.N * tpi : (g.Mtot + 127) / 128;
+  // an under-filled launch: the persistent kernel cuts the reduction into slices there and wins
+  // (measured at batch 1 and 32 on the deepest layers)
+  if (tiles * P.n_ntiles * 2 <= nsm) return false;
   const double persistent_passes = (double)((tiles * P.n_ntiles + nsm - 1) / nsm);
   return BF16 ? strip_passes * 0.75 < persistent_passes : strip_passes * 0.8 <= persistent_passes;
 }
