@@ -37,7 +37,11 @@ UNIT = "TFLOP/s"
 NOMINAL_TF32_OVER_BF16 = 1.1 / 2.25
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (conv_tc_persistent__*.md)
-NCU_TRAFFIC_BYTES = {("resnet3x3", "tf32"): 319.57e6 + 81.23e6, ("deep3x3", "bf16"): 89.40e6 + 4.28e6, ("stem7x7", "tf32"): 277.09e6 + 352.88e6, ("down3x3", "tf32"): 322.88e6 + 73.69e6}
+# (conv_tc_persistent__*.md, conv_tc_strip__*.md): the kernel the library chooses for that workload
+NCU_TRAFFIC_BYTES = {("resnet3x3", "tf32"): 319.57e6 + 81.23e6, ("stem7x7", "tf32"): 277.09e6 + 352.88e6,
+                     ("down3x3", "tf32"): 322.35e6 + 74.64e6,
+                     ("deep3x3", "tf32"): 90.54e6 + 4.44e6, ("deep3x3", "bf16"): 89.36e6 + 3.78e6}
+KERNEL_NAMES = {1: "conv_tc_strip_kernel", 2: "conv_tc_persistent_kernel", 3: "conv_tc_kernel", 4: "conv_fp32_kernel"}
 
 
 def _peaks():
@@ -112,6 +116,27 @@ def time_conv_only(layer, mode_name, steps, torch, b, flush_buf):
     if b.last_device_status() != 0:
         raise RuntimeError("device status word set")
     return {"ms": sum(ts) / len(ts), "ms_best_of_5": min(ts[:5]), "tflops": _flops(layer, ho, wo) / (sum(ts) / len(ts)) / 1e9}
+
+
+def kernel_used(layer, mode_name, torch, b):
+    """Name of the convolution kernel the library chooses for this workload: one untimed call through the
+    test build of the same object files (the only build that records its choice), default switches."""
+    mode = {"tf32": b.MODE_TF32, "bf16": b.MODE_BF16}[mode_name]
+    dims = layer.dims()
+    ho, wo = b.out_dims(dims)
+    try:
+        b.use_test_library(True)
+        ws = torch.zeros(b.conv_workspace_bytes(dims, b.SRC_NCHW, mode) // 4 + 64, dtype=torch.float32, device="cuda")
+        x = torch.zeros((layer.N, layer.C, layer.H, layer.W), dtype=torch.float32, device="cuda")
+        f = torch.zeros((layer.K, layer.C, layer.Fh, layer.Fw), dtype=torch.float32, device="cuda")
+        out = torch.empty((layer.N, layer.K, ho, wo), dtype=torch.float32, device="cuda")
+        b.conv(x, b.SRC_NCHW, f, dims, mode, out, ws)
+        torch.cuda.synchronize()
+        return KERNEL_NAMES.get(b.last_kernel(), "unknown")
+    except (ImportError, OSError, RuntimeError, AttributeError):
+        return "unknown"
+    finally:
+        b.use_test_library(False)
 
 
 def _flops(layer, ho, wo):
@@ -331,21 +356,23 @@ def time_layer(layer, mode_name, steps, warmup, torch, b, flush_buf, sampler_ind
     except b.Im2winError as exc:
         if exc.code != b.EUNSUPPORTED:
             raise
-    # the bf16 storage variant of the im2win tensor (BF16 mode only; layers with per-image tiling)
+    # the bf16 storage variant of the im2win tensor: always a BF16-mode convolution, whatever the line's mode
     res["ms_transform_bf16"] = res["ms_conv_bf16src"] = None
-    if mode == b.MODE_BF16:
+    if True:
         ws16 = torch.empty(b.workspace_bytes_bf16(dims) // 2, dtype=torch.int16, device="cuda")
+        n16 = b.conv_workspace_bytes(dims, b.SRC_IM2WIN_BF16, b.MODE_BF16)
+        scratch16 = torch.empty(n16 // 4 + 64, dtype=torch.float32, device="cuda") if n16 else None
         try:
             for _ in range(3):
                 b.transform_bf16(x, dims, ws16)
-                b.conv(ws16, b.SRC_IM2WIN_BF16, f, dims, mode, out, scratch)
+                b.conv(ws16, b.SRC_IM2WIN_BF16, f, dims, b.MODE_BF16, out, scratch16)
             be = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
             for k in range(steps):
                 flush_buf.zero_()
                 be[k][0].record(stream)
                 b.transform_bf16(x, dims, ws16)
                 be[k][1].record(stream)
-                b.conv(ws16, b.SRC_IM2WIN_BF16, f, dims, mode, out, scratch)
+                b.conv(ws16, b.SRC_IM2WIN_BF16, f, dims, b.MODE_BF16, out, scratch16)
                 be[k][2].record(stream)
             torch.cuda.synchronize()
             if b.last_device_status() != 0:
@@ -460,7 +487,7 @@ def run_gpu(args):
         roof = {"bound": "tensor", "achieved": flops / ms_conv / 1e9, "peak": tensor_peak, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = args.traffic if args.traffic is not None else NCU_TRAFFIC_BYTES.get((layer.name, args.mode))
-    roof["kernel"] = "conv_tc_persistent_kernel"
+    roof["kernel"] = kernel_used(layer, args.mode, torch, b)
     roof["peak_source"] = f"of {peaks['source']}" + (" (bf16 burst x nominal tf32/bf16 ratio)" if roof["bound"] == "tensor" and args.mode == "tf32" else "")
     roof["algorithmic_bytes_per_launch"] = r["conv_bytes"]
     roof["kernel_ms"] = ms_conv
@@ -481,6 +508,7 @@ def run_gpu(args):
                 r2["frac_tensor_peak"] = r2["tflops"] / pk
                 if matmul_peaks:
                     r2["frac_measured_matmul"] = r2["tflops"] / matmul_peaks[f"{m}_tflops"]
+                r2["kernel"] = kernel_used(wl.CONFIGS[name], m, torch, b)
                 extra[name][m] = r2
     cpu = _cpu_baseline(layer) if world == 1 and not args.no_cpu_baseline else None
     line = {
@@ -508,7 +536,7 @@ def run_gpu(args):
                    "frac_hbm": r["fused_bytes"] / r["ms_fused"] / 1e6 / peaks["hbm_gbs"]} if r.get("ms_fused") else None),
         "bf16_storage": ({"ms_transform": r["ms_transform_bf16"], "ms_conv": r["ms_conv_bf16src"],
                           "what": "the im2win tensor stored as bf16 (im2win_transform_bf16, src_kind IM2WIN_BF16): "
-                                  "half the workspace; BF16 mode only; not part of `value`"}
+                                  "half the workspace; a BF16-mode convolution whatever this line's mode; not part of `value`"}
                          if r.get("ms_conv_bf16src") else None),
         "bf16_output": ({"ms_conv": r["ms_conv_bf16out"],
                          "what": "im2win_conv_bf16out: the same convolution with the result stored as bf16 "

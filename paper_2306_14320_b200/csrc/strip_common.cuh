@@ -1,0 +1,203 @@
+// Shared pieces of the shared-memory-operand tensor-core kernels (conv_tc_strip.cu, conv_tc_window.cu):
+// barrier block, bounded waits, TMA / cluster / tcgen05 pair helpers, the pipelined TMEM -> NCHW store.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <atomic>
+#include <cstdint>
+
+#include "common.cuh"
+#include "ptx_sm100.cuh"
+
+namespace im2win {
+namespace stripc {
+
+constexpr int kTW = 8;             // transposer warps
+constexpr int kTWarp0 = 4;
+constexpr int kEpiWarp0 = kTWarp0 + kTW;
+constexpr int kMaxRaw = 12, kMaxB = 12;
+constexpr int kTMax = 3;           // transposer tasks per thread and source stage
+constexpr uint32_t kSpin = 1u << 22;
+
+struct SBars {
+  uint64_t raw_full[kMaxRaw], raw_empty[kMaxRaw];
+  uint64_t b_full[kMaxB], b_empty[kMaxB];
+  uint64_t t_full[2], t_empty[2];
+  uint64_t acc_full[2], acc_empty[2];
+};
+struct SMisc {
+  uint32_t tmem_base;
+  int32_t abort;
+};
+
+struct Ring {
+  int32_t idx = 0;
+  uint32_t phase = 0;
+  __device__ __forceinline__ void advance(int32_t n) {
+    if (++idx == n) { idx = 0; phase ^= 1u; }
+  }
+};
+
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait (about a second): polls with a back-off; on expiry records `code`, raises the CTA's
+// abort flag (which ends every other role's wait at its next look) and returns false.
+static __device__ __noinline__ bool wait_slow(int32_t* status, SMisc* misc, uint32_t bar, uint32_t parity, int32_t code,
+                                       uint32_t sleep_ns) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 0; it < kSpin; ++it) {
+    __nanosleep(sleep_ns);
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u) {
+      if (*reinterpret_cast<volatile int32_t*>(&misc->abort)) return false;
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > 1000000000ull) break;
+    }
+  }
+  atomicCAS(status, 0, code);
+  atomicExch(&misc->abort, 1);
+  return false;
+}
+template <class PT>
+__device__ __forceinline__ bool wait_bar(const PT& P, SMisc* misc, uint32_t bar, uint32_t parity, int32_t code,
+                                         uint32_t sleep_ns = 32) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  return wait_slow(P.status, misc, bar, parity, code, sleep_ns);
+}
+template <class PT>
+__device__ __forceinline__ bool wait_bar_warp(const PT& P, SMisc* misc, uint32_t bar, uint32_t parity, int32_t code,
+                                              uint32_t sleep_ns = 32) {
+  return __all_sync(0xffffffffu, wait_bar(P, misc, bar, parity, code, sleep_ns));
+}
+
+__device__ __forceinline__ uint32_t lds_u32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a) {
+  uint32_t v;
+  asm volatile("{\n.reg .b16 h;\nld.shared.u16 h, [%1];\ncvt.u32.u16 %0, h;\n}" : "=r"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_v4(uint32_t a, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+// Cluster helpers (pair mode: a cluster of two CTAs).
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA box whose completion is signalled on a barrier of the pair's leader CTA (a shared::cluster address)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+// D[tmem of both CTAs] (+)= A[each CTA's own rows] * B[each CTA holds half the N rows]; M = 256.
+template <bool BF16>
+__device__ __forceinline__ void mma_ss_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                            uint32_t idesc, uint32_t accumulate) {
+  if constexpr (BF16) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 ad, {%1, %2};\n\t"
+        "mov.b64 bd, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], ad, bd, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 ad, {%1, %2};\n\t"
+        "mov.b64 bd, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], ad, bd, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+  }
+}
+// Arrive on the barrier at the same shared-memory offset in both CTAs of the pair once every MMA issued so far is done.
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
+// Stores columns [c_begin, c_end) (multiples of 16) of one warp's 32 accumulator rows: TMEM -> registers
+// -> NCHW.  The TMEM load of the next 16 columns is in flight while the current 16 are stored.
+__device__ __forceinline__ void store_columns(uint32_t d_tmem, float* orow, int64_t HoWo, int32_t c_begin, int32_t c_end,
+                                              int32_t k_left, bool valid) {
+  uint32_t va[16], vb[16];
+  if (c_begin >= c_end) return;
+  ptx::tmem_ld_x16(d_tmem + (uint32_t)c_begin, va);
+#pragma unroll 1
+  for (int32_t c0 = c_begin; c0 < c_end; c0 += 32) {
+    ptx::tmem_wait_ld();
+    const bool more = c0 + 16 < c_end;
+    if (more) ptx::tmem_ld_x16(d_tmem + (uint32_t)(c0 + 16), vb);
+    if (valid) {
+      float* o = orow + (int64_t)c0 * HoWo;
+      const int32_t left = k_left - c0;
+#pragma unroll
+      for (int e = 0; e < 16; ++e)
+        if (e < left) o[(int64_t)e * HoWo] = __uint_as_float(va[e]);
+    }
+    if (more) {
+      ptx::tmem_wait_ld();
+      if (c0 + 32 < c_end) ptx::tmem_ld_x16(d_tmem + (uint32_t)(c0 + 32), va);
+      if (valid) {
+        float* o = orow + (int64_t)(c0 + 16) * HoWo;
+        const int32_t left = k_left - c0 - 16;
+#pragma unroll
+        for (int e = 0; e < 16; ++e)
+          if (e < left) o[(int64_t)e * HoWo] = __uint_as_float(vb[e]);
+      }
+    }
+  }
+}
+
+// ---- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+inline EncodeTiledFn encode_fn() {
+  static std::atomic<void*> cached{nullptr};
+  void* p = cached.load(std::memory_order_acquire);
+  if (!p) {
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    cached.store(p, std::memory_order_release);
+  }
+  return reinterpret_cast<EncodeTiledFn>(p);
+}
+
+}  // namespace stripc
+}  // namespace im2win
