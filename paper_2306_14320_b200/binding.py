@@ -149,7 +149,7 @@ def workspace_bytes(shape) -> int:
     return b.value
 
 
-KERNEL_STRIP, KERNEL_PERSISTENT, KERNEL_GENERIC, KERNEL_FP32 = 1, 2, 3, 4
+KERNEL_STRIP, KERNEL_PERSISTENT, KERNEL_GENERIC, KERNEL_FP32, KERNEL_WINDOW = 1, 2, 3, 4, 5
 
 
 def last_kernel() -> int:

@@ -63,17 +63,24 @@ int make_geometry(const im2win_shape* sh, Geometry* g) {
 int launch_conv_tc(const void* src, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st,
                    Scratch scratch, int src_kind, bool out_bf16) {
   // src_kind: 0 = fp32 im2win tensor, 1 = untransformed input consumed fused, 2 = bf16 im2win tensor.
-  // Order: the strip-matrix kernel where it is implemented and expected to win, else the persistent
-  // specialised kernel, else (fp32 im2win tensor and fp32 output only) the generic kernel.
+  // Order: the window-offset and the strip-matrix kernel where each is implemented and expected to win, else
+  // the persistent specialised kernel, else (fp32 im2win tensor and fp32 output only) the generic kernel.
   int rc = IM2WIN_EUNSUPPORTED;
   if (!knobs().force_generic) {
+    rc = launch_conv_tc_window(src, f, out, g, mode, st, scratch, src_kind, out_bf16);
+    if (rc != IM2WIN_EUNSUPPORTED) return rc;
     if (!knobs().no_strip) rc = launch_conv_tc_strip(src, f, out, g, mode, st, scratch, src_kind, out_bf16);
     if (rc != IM2WIN_EUNSUPPORTED) return rc;
     rc = launch_conv_tc_persistent(src, f, out, g, mode, st, scratch, src_kind == 1, src_kind == 2, out_bf16);
     if (rc != IM2WIN_EUNSUPPORTED) return rc;
-    // sources the generic kernel does not read (bf16 im2win tensor, fused): the strip-matrix kernel wherever it applies
+    // sources the generic kernel does not read (bf16 im2win tensor, fused): the strip-matrix or the
+    // window-offset kernel wherever one applies
     if (src_kind != 0 && !knobs().no_strip) {
       rc = launch_conv_tc_strip(src, f, out, g, mode, st, scratch, src_kind, out_bf16, /*even_if_slower=*/true);
+      if (rc != IM2WIN_EUNSUPPORTED) return rc;
+    }
+    if (src_kind != 0) {
+      rc = launch_conv_tc_window(src, f, out, g, mode, st, scratch, src_kind, out_bf16, /*even_if_slower=*/true);
       if (rc != IM2WIN_EUNSUPPORTED) return rc;
     }
   }
@@ -84,7 +91,8 @@ int launch_conv_tc(const void* src, const float* f, float* out, const Geometry& 
 size_t conv_scratch_bytes(const Geometry& g, int mode, int src_kind) {
   if (mode != IM2WIN_MODE_TF32 && mode != IM2WIN_MODE_BF16) return 0;
   const size_t a = strip_scratch_bytes(g, mode, src_kind), b = persistent_scratch_bytes(g, mode);
-  return a > b ? a : b;
+  const size_t c = knobs().no_window ? 0 : window_scratch_bytes(g, mode, src_kind);
+  return a > b ? (a > c ? a : c) : (b > c ? b : c);
 }
 
 #ifdef IM2WIN_TEST_KNOBS
@@ -241,13 +249,16 @@ int conv_impl(const void* src, int src_kind, const float* filter, const im2win_s
   const float* xhat = static_cast<const float*>(src);
   if (src_kind == IM2WIN_SRC_NCHW_FUSED) {
     if (mode != IM2WIN_MODE_FP32 && !knobs().force_generic) {
-      rc = IM2WIN_EUNSUPPORTED;
-      if (!knobs().no_strip) rc = launch_conv_tc_strip(xhat, filter, out_nchw, g, mode, st, scratch_from(0), 1, out16);
+      rc = launch_conv_tc_window(xhat, filter, out_nchw, g, mode, st, scratch_from(0), 1, out16);
+      if (rc == IM2WIN_EUNSUPPORTED && !knobs().no_strip)
+        rc = launch_conv_tc_strip(xhat, filter, out_nchw, g, mode, st, scratch_from(0), 1, out16);
       if (rc == IM2WIN_EUNSUPPORTED)
         rc = launch_conv_tc_persistent(xhat, filter, out_nchw, g, mode, st, scratch_from(0), /*fused=*/true,
                                        /*src_bf16=*/false, out16);
       if (rc == IM2WIN_EUNSUPPORTED && !knobs().no_strip)
         rc = launch_conv_tc_strip(xhat, filter, out_nchw, g, mode, st, scratch_from(0), 1, out16, /*even_if_slower=*/true);
+      if (rc == IM2WIN_EUNSUPPORTED)
+        rc = launch_conv_tc_window(xhat, filter, out_nchw, g, mode, st, scratch_from(0), 1, out16, /*even_if_slower=*/true);
       if (rc != IM2WIN_EUNSUPPORTED) return rc;
     }
     // no fused kernel for this shape or mode: the unfused path, if the caller supplied a workspace
@@ -326,7 +337,8 @@ int im2win_debug_set_option(const char* name, int value) {
       {"no_bslice", &Knobs::no_bslice}, {"splitk", &Knobs::splitk}, {"force_stream", &Knobs::force_stream},
       {"nsets", &Knobs::nsets}, {"no_l2ahead", &Knobs::no_l2ahead}, {"no_btma", &Knobs::no_btma},
       {"ntiles", &Knobs::ntiles}, {"transform_gather", &Knobs::transform_gather},
-      {"test_skip_copy", &Knobs::test_skip_copy}, {"strip_mh", &Knobs::strip_mh}, {"strip_pair", &Knobs::strip_pair}};
+      {"test_skip_copy", &Knobs::test_skip_copy}, {"strip_mh", &Knobs::strip_mh}, {"strip_pair", &Knobs::strip_pair},
+      {"force_window", &Knobs::force_window}, {"no_window", &Knobs::no_window}, {"window_mh", &Knobs::window_mh}};
   for (const Entry& e : table)
     if (strcmp(e.name, name) == 0) { g_knobs.*(e.field) = value; return IM2WIN_OK; }
   return IM2WIN_EINVAL;

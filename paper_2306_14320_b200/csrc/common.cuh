@@ -68,6 +68,10 @@ int launch_conv_tc(const void* src, const float* f, float* out, const Geometry& 
                    Scratch scratch, int src_kind, bool out_bf16);
 // Scratch bytes with which every kernel above is available for this problem (0 if none wants any).
 size_t strip_scratch_bytes(const Geometry& g, int mode, int src_kind);
+// The window-offset kernel (conv_tc_window.cu; stride 1, 3x3 and 5x5): same source kinds and scratch rules.
+int launch_conv_tc_window(const void* src, const float* f, float* out, const Geometry& g, int mode, cudaStream_t st,
+                          Scratch scratch, int src_kind, bool out_bf16, bool even_if_slower = false);
+size_t window_scratch_bytes(const Geometry& g, int mode, int src_kind);
 size_t persistent_scratch_bytes(const Geometry& g, int mode);
 size_t conv_scratch_bytes(const Geometry& g, int mode, int src_kind);
 // Shared body of im2win_conv / im2win_conv_bf16out / im2win_conv_static (argument checks, workspace
@@ -99,12 +103,15 @@ struct Knobs {
   int test_skip_copy = 0;    // transform tile kernel, single-CTA problems: announce the input copy, never issue it
   int strip_mh = 0;          // strip-matrix kernel: 128-row halves per tile (0: own choice)
   int strip_pair = 0;        // strip-matrix kernel: 1 = CTA pairs (cta_group::2) forced, 2 = single CTAs forced, 0 = own choice
+  int force_window = 0;      // use the window-offset kernel (conv_tc_window.cu) wherever it is implemented
+  int no_window = 0;         // never use it
+  int window_mh = 0;         // window-offset kernel: 128-row blocks per tile (0: own choice)
 };
 const Knobs& knobs();
 
 // Which convolution kernel the last launch on this host thread's library image used (a diagnostic the
 // test build exposes as im2win_debug_last_kernel; the product library only writes it).
-enum : int { KERNEL_NONE = 0, KERNEL_STRIP = 1, KERNEL_PERSISTENT = 2, KERNEL_GENERIC = 3, KERNEL_FP32 = 4 };
+enum : int { KERNEL_NONE = 0, KERNEL_STRIP = 1, KERNEL_PERSISTENT = 2, KERNEL_GENERIC = 3, KERNEL_FP32 = 4, KERNEL_WINDOW = 5 };
 void note_kernel(int which);
 
 // Streaming multiprocessors of the current device (cached per device).

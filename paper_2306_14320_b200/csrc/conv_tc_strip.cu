@@ -38,16 +38,6 @@
 #include "strip_common.cuh"
 
 namespace im2win {
-#ifdef IM2WIN_PROF
-extern long long* g_prof;  // debug build: counter buffer (defined in conv_tc_persistent.cu)
-#define SPROF_DECL long long pw[7] = {}; const long long pt0 = clock64();
-#define SPROF_W(k, ...) { const long long c0_ = clock64(); __VA_ARGS__; pw[k] += clock64() - c0_; }
-#define SPROF_DUMP(role) if (P.prof && blockIdx.x < 8 && lane == 0) { long long* o_ = P.prof + ((long long)blockIdx.x * 8 + (role)) * 8; o_[0] = clock64() - pt0; for (int z_ = 0; z_ < 7; ++z_) o_[1 + z_] = pw[z_]; }
-#else
-#define SPROF_DECL
-#define SPROF_W(k, ...) { __VA_ARGS__; }
-#define SPROF_DUMP(role)
-#endif
 namespace {
 
 using namespace stripc;

@@ -104,7 +104,7 @@ def test_conv_from_bf16_im2win_tensor(name, batch, staging, _kernel):
     """staging: the library's own choice of kernel; the persistent kernel with 2-D TMA boxes; the same
     with bulk copies."""
     if staging != "auto":
-        apply_config(staging, no_strip=1, no_box=1 if staging == "bulk" else 0, transform_gather=1 if _kernel == "gather" else 0)
+        apply_config(staging, no_strip=1, no_window=1, no_box=1 if staging == "bulk" else 0, transform_gather=1 if _kernel == "gather" else 0)
     layer = wl.CONFIGS[name].with_batch(batch)
     dims = layer.dims()
     x, f = wl.make_input(layer), wl.make_filter(layer)

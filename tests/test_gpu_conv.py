@@ -35,8 +35,12 @@ SMALL = [
     # tile and of a single output, several tiles per image
     (2, 16, 11, 13, 24, 3, 3, 1), (3, 32, 9, 10, 40, 3, 3, 2), (1, 64, 17, 19, 300, 3, 3, 1), (2, 32, 20, 33, 17, 3, 3, 2),
     (2, 64, 5, 5, 16, 3, 3, 1), (3, 32, 3, 3, 8, 3, 3, 1), (1, 32, 40, 37, 48, 3, 3, 1), (1, 32, 45, 44, 130, 3, 3, 2),
+    # shapes for the window-offset kernel (stride 1, 3x3 and 5x5): a 5x5 filter, source ranges of several TMA
+    # boxes, four 128-row blocks per tile with a ragged last tile
+    (1, 32, 14, 15, 24, 5, 5, 1), (2, 64, 30, 28, 64, 3, 3, 1), (1, 32, 70, 66, 32, 3, 3, 1),
 ]
 STRIP_SHAPES = [d for d in SMALL if d[5] == 3 and d[6] == 3 and d[1] % 32 == 0 and d[7] in (1, 2)]
+WINDOW_SHAPES = [d for d in SMALL if (d[5], d[6]) in ((3, 3), (5, 5)) and d[1] % 32 == 0 and d[7] == 1]
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -49,6 +53,7 @@ def _kernel(request):
     """Every case runs once per kernel configuration: the product library's own choice ("auto"; the
     same with the smallest legal workspace, "minws"), and the test build with one switch set -- the
     strip-matrix kernel forced wherever it is implemented (one and two 128-row halves per tile), the
+    window-offset kernel forced wherever it is implemented (its own tile height, one and two 128-row blocks), the
     strip-matrix kernel off (the persistent, filter-size-specialised kernel's own choice), that kernel
     with box staging off (per-image tiles, bulk copies), with per-image tiling off as well (tiles that
     span images), with three reduction slices forced, with the slice-resident filter mode forced, and
@@ -137,6 +142,19 @@ def test_forced_strip_configurations_run_the_strip_kernel(dims, mode, _kernel):
     got = gpu_conv(x, f, dims, mode)
     if dims[7] == 1 or _kernel in ("strip", "pair"):  # (two halves per tile and stride 2 together exceed shared memory)
         assert b.last_kernel() == b.KERNEL_STRIP
+    assert np.array_equal(got.astype(np.float64), oracle_conv(x, f, dims))
+
+
+@pytest.mark.parametrize("src_kind", [b.SRC_NCHW, b.SRC_NCHW_FUSED], ids=["im2win", "fused"])
+@pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
+@pytest.mark.parametrize("dims", WINDOW_SHAPES)
+def test_forced_window_configurations_run_the_window_kernel(dims, mode, src_kind, _kernel):
+    """The same for the window-offset kernel, from the im2win tensor and fused."""
+    if _kernel not in ("window", "window1", "window2"):
+        pytest.skip("only for the configurations that force the window-offset kernel")
+    x, f = _data(dims, 810, ints=True)
+    got = gpu_conv(x, f, dims, mode, src_kind=src_kind)
+    assert b.last_kernel() == b.KERNEL_WINDOW
     assert np.array_equal(got.astype(np.float64), oracle_conv(x, f, dims))
 
 
@@ -230,8 +248,8 @@ def test_conv_full_batch_small_integers_whole_tensor_bit_exact(name, src, mode, 
     """Batch 128, the launch configuration the benchmark times (ring phases wrapping over ~170 tiles
     per CTA, the look-ahead of the next tile, the last partial wave): on small-integer data every one
     of the 6 to 103 million outputs must equal the oracle's Eq. (1) exactly."""
-    if src == "fused" and _kernel not in ("auto", "strip", "nostrip"):
-        pytest.skip("the fused source kind is covered in the library's own, the strip-matrix and the persistent configuration")
+    if src == "fused" and _kernel not in ("auto", "strip", "window", "nostrip"):
+        pytest.skip("the fused source kind is covered in the library's own, the strip-matrix, the window-offset and the persistent configuration")
     layer = wl.CONFIGS[name]
     dims = layer.dims()
     x, f = _cached(("ints", name), lambda: _layer_ints(layer))
@@ -264,7 +282,7 @@ def test_conv_sweep_layers_batch_32_and_128(layer, batch, mode, _kernel):
     """The twelve-layer sweep at the batch sizes the benchmark times, with the library's own choice of
     path at each (reduction slices at 32, streamed filters and multi-wave persistent loops at 128): Eq. (1)
     at 20 000 sampled coordinates and every corner, and the whole first and last image."""
-    if _kernel not in ("auto", "minws", "strip", "nostrip"):
+    if _kernel not in ("auto", "minws", "strip", "window", "nostrip"):
         pytest.skip("forced persistent-kernel variants are covered at small sizes")
     layer = layer.with_batch(batch)
     dims = layer.dims()
@@ -300,7 +318,7 @@ def test_conv_table1_layers_batch128(layer, mode, _kernel):
     """The paper's own workload: Table I's unpadded layers at batch 128 (Conv4, whose tensors take
     gigabytes, is covered at batch 16 below).  Eq. (1) at 20 000 sampled coordinates and every corner,
     the whole first and last image, and no element that is not finite."""
-    if _kernel not in ("auto", "minws", "strip", "pair2", "nostrip"):
+    if _kernel not in ("auto", "minws", "strip", "pair2", "window", "nostrip"):
         pytest.skip("forced persistent-kernel variants are covered at small sizes")
     dims = layer.dims()
     n, c, h, w, k, fh, fw, s = dims
@@ -332,7 +350,7 @@ def test_conv_table1_layers_batch128(layer, mode, _kernel):
 @pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
 @pytest.mark.parametrize("layer", wl.SWEEP, ids=lambda l: l.name)
 def test_conv_sweep_layers_batch32_small_integers_bit_exact(layer, mode, _kernel):
-    if _kernel not in ("auto", "minws", "strip", "nostrip"):
+    if _kernel not in ("auto", "minws", "strip", "window", "nostrip"):
         pytest.skip("forced persistent-kernel variants are covered at small sizes")
     layer = layer.with_batch(32)
     dims = layer.dims()
