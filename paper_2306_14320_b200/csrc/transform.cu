@@ -50,8 +50,11 @@ struct Cursor {  // position of an output element inside the CTA's range
 
 // One CTA: either PB whole consecutive planes (small planes), or one block of MB output rows of one
 // plane.  In both cases the input it needs and the output it writes are one contiguous range each.
+// FHT: the filter height as a compile-time constant (division by it is then a multiplication), or 0.
+template <int FHT>
 __global__ void __launch_bounds__(kThreads) transform_smem_kernel(const TransformParams P) {
   extern __shared__ __align__(16) float smem[];
+  const int32_t Fh = FHT ? FHT : P.Fh;
   const int64_t job = blockIdx.x;
   const int64_t pg = job / P.nblk;
   const int32_t b = (int32_t)(job - pg * P.nblk);
@@ -60,7 +63,7 @@ __global__ void __launch_bounds__(kThreads) transform_smem_kernel(const Transfor
   const int32_t npl = whole ? (int32_t)min((int64_t)P.PB, P.planes - plane0) : 1;
   const int32_t m0 = b * P.MB;
   const int32_t mb = whole ? P.Ho : min(P.MB, P.Ho - m0);
-  const int32_t rows_in = whole ? P.H : (mb - 1) * P.s + P.Fh;
+  const int32_t rows_in = whole ? P.H : (mb - 1) * P.s + Fh;
   const int32_t plane_floats = rows_in * P.W;  // staged floats per plane
   const int32_t n_in = npl * plane_floats;
 
@@ -102,13 +105,13 @@ __global__ void __launch_bounds__(kThreads) transform_smem_kernel(const Transfor
     Cursor c;
     c.mm = mm;
     c.k = (int32_t)(((uint64_t)(uint32_t)r2 * P.magic_Fh) >> 32);
-    c.u = r2 - c.k * P.Fh;
+    c.u = r2 - c.k * Fh;
     c.base = pl * plane_floats + mm * sW;
     return c;
   };
   auto fetch = [&](const Cursor& c) { return tile[c.base + c.u * P.W + c.k]; };
   auto advance = [&](Cursor c) -> Cursor {
-    if (++c.u == P.Fh) {
+    if (++c.u == Fh) {
       c.u = 0;
       if (++c.k == P.W) {  // next strip: next output row, or the first row of the next plane
         c.k = 0;
@@ -124,14 +127,52 @@ __global__ void __launch_bounds__(kThreads) transform_smem_kernel(const Transfor
 
   if ((int32_t)threadIdx.x < head) dst[threadIdx.x] = fetch(locate(threadIdx.x));
   float4* dst4 = reinterpret_cast<float4*>(dst + head);
-  for (int32_t i = threadIdx.x; i < nvec; i += kThreads) {
-    Cursor c = locate(head + (i << 2));
-    float4 v;
-    v.x = fetch(c); c = advance(c);
-    v.y = fetch(c); c = advance(c);
-    v.z = fetch(c); c = advance(c);
-    v.w = fetch(c);
-    dst4[i] = v;
+  static_assert(FHT == 0 || FHT >= 4, "a 16-byte chunk must not wrap the filter height twice");
+  if (FHT != 0 && P.L >= 4 * kThreads) {
+    // Long strips (the stems): the thread's position (strip, offset in the strip) is stepped from one
+    // 16-byte chunk to its next, 4*kThreads elements on, instead of being located anew, and the four
+    // gathers of a chunk that lies inside one strip walk (u, k) with compile-time Fh.  The kernel is
+    // bound by its instruction count: this path issues about a third of the general one's.
+    constexpr int FD = FHT ? FHT : 1;
+    const int32_t L = P.L, W = P.W;
+    Cursor c0 = locate(head + ((int32_t)threadIdx.x << 2));
+    int32_t r2 = c0.k * FD + c0.u, mm = c0.mm, base = c0.base;
+    for (int32_t i = threadIdx.x; i < nvec; i += kThreads) {
+      float4 v;
+      if (r2 + 3 < L) {
+        int32_t k = r2 / FD, u = r2 - k * FD;
+        const float* t = tile + base + k;
+        int32_t idx = u * W;
+        v.x = t[idx]; if (++u == FD) { u = 0; idx = idx - (FD - 1) * W + 1; } else idx += W;
+        v.y = t[idx]; if (++u == FD) { u = 0; idx = idx - (FD - 1) * W + 1; } else idx += W;
+        v.z = t[idx]; if (++u == FD) { u = 0; idx = idx - (FD - 1) * W + 1; } else idx += W;
+        v.w = t[idx];
+      } else {  // the chunk straddles two strips
+        Cursor c;
+        c.base = base; c.mm = mm; c.k = r2 / FD; c.u = r2 - c.k * FD;
+        v.x = fetch(c); c = advance(c);
+        v.y = fetch(c); c = advance(c);
+        v.z = fetch(c); c = advance(c);
+        v.w = fetch(c);
+      }
+      dst4[i] = v;
+      r2 += 4 * kThreads;
+      while (r2 >= L) {  // (at most once per step: L >= 4*kThreads)
+        r2 -= L;
+        base += sW;
+        if (++mm == mb) { mm = 0; base += plane_floats - mb * sW; }
+      }
+    }
+  } else {
+    for (int32_t i = threadIdx.x; i < nvec; i += kThreads) {
+      Cursor c = locate(head + (i << 2));
+      float4 v;
+      v.x = fetch(c); c = advance(c);
+      v.y = fetch(c); c = advance(c);
+      v.z = fetch(c); c = advance(c);
+      v.w = fetch(c);
+      dst4[i] = v;
+    }
   }
   if ((int32_t)threadIdx.x < n_out - tail0) dst[tail0 + threadIdx.x] = fetch(locate(tail0 + threadIdx.x));
 }
@@ -570,7 +611,9 @@ static int launch_transform_staged(const float* in, float* out, uint16_t* out16,
   }
   if (smem > 48 * 1024) {
     cudaError_t e = out16 ? cudaFuncSetAttribute(transform_smem_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                          : cudaFuncSetAttribute(transform_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                          : (g.Fh == 7 ? cudaFuncSetAttribute(transform_smem_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                             : g.Fh == 11 ? cudaFuncSetAttribute(transform_smem_kernel<11>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                                          : cudaFuncSetAttribute(transform_smem_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     if (e != cudaSuccess) return IM2WIN_ECUDA;
   }
   TransformParams P;
@@ -582,7 +625,9 @@ static int launch_transform_staged(const float* in, float* out, uint16_t* out16,
   P.magic_Fh = magic_for((uint32_t)g.Fh);
   P.magic_HoL = magic_for((uint32_t)g.HoL);
   if (out16) transform_smem_bf16_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(P, out16);
-  else transform_smem_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(P);
+  else if (g.Fh == 7) transform_smem_kernel<7><<<(unsigned)ctas, kThreads, smem, st>>>(P);
+  else if (g.Fh == 11) transform_smem_kernel<11><<<(unsigned)ctas, kThreads, smem, st>>>(P);
+  else transform_smem_kernel<0><<<(unsigned)ctas, kThreads, smem, st>>>(P);
   return cuda_status(cudaGetLastError());
 }
 
