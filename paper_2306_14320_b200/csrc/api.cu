@@ -107,6 +107,10 @@ const Knobs& knobs() {
 
 static std::atomic<int> g_last_kernel{KERNEL_NONE};
 void note_kernel(int which) { g_last_kernel.store(which, std::memory_order_relaxed); }
+static std::atomic<int> g_last_plan[8];
+void note_plan(const int* v, int n) {
+  for (int i = 0; i < 8; ++i) g_last_plan[i].store(i < n ? v[i] : 0, std::memory_order_relaxed);
+}
 
 int sm_count() {
   constexpr int kMaxDev = 64;
@@ -328,6 +332,9 @@ int im2win_debug_last_kernel(void) { return g_last_kernel.load(std::memory_order
 
 // Test build only (libim2win_test.so): set one diagnostic switch by name.  Returns IM2WIN_EINVAL for
 // an unknown name.
+void im2win_debug_last_plan(int* out8) {
+  for (int i = 0; i < 8; ++i) out8[i] = im2win::g_last_plan[i].load(std::memory_order_relaxed);
+}
 int im2win_debug_set_option(const char* name, int value) {
   if (!name) return IM2WIN_EINVAL;
   struct Entry { const char* name; int Knobs::*field; };
@@ -338,7 +345,8 @@ int im2win_debug_set_option(const char* name, int value) {
       {"nsets", &Knobs::nsets}, {"no_l2ahead", &Knobs::no_l2ahead}, {"no_btma", &Knobs::no_btma},
       {"ntiles", &Knobs::ntiles}, {"transform_gather", &Knobs::transform_gather},
       {"test_skip_copy", &Knobs::test_skip_copy}, {"strip_mh", &Knobs::strip_mh}, {"strip_pair", &Knobs::strip_pair},
-      {"force_window", &Knobs::force_window}, {"no_window", &Knobs::no_window}, {"window_mh", &Knobs::window_mh}};
+      {"force_window", &Knobs::force_window}, {"no_window", &Knobs::no_window}, {"window_mh", &Knobs::window_mh},
+      {"window_plan", &Knobs::window_plan}, {"window_pair", &Knobs::window_pair}};
   for (const Entry& e : table)
     if (strcmp(e.name, name) == 0) { g_knobs.*(e.field) = value; return IM2WIN_OK; }
   return IM2WIN_EINVAL;

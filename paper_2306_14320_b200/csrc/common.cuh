@@ -106,6 +106,8 @@ struct Knobs {
   int force_window = 0;      // use the window-offset kernel (conv_tc_window.cu) wherever it is implemented
   int no_window = 0;         // never use it
   int window_mh = 0;         // window-offset kernel: 128-row blocks per tile (0: own choice)
+  int window_plan = 0;       // window-offset kernel: forced split of shared memory (0: own choice)
+  int window_pair = 0;       // window-offset kernel: 1 = CTA pairs forced, 2 = single CTAs forced, 0 = own choice
 };
 const Knobs& knobs();
 
@@ -113,6 +115,8 @@ const Knobs& knobs();
 // test build exposes as im2win_debug_last_kernel; the product library only writes it).
 enum : int { KERNEL_NONE = 0, KERNEL_STRIP = 1, KERNEL_PERSISTENT = 2, KERNEL_GENERIC = 3, KERNEL_FP32 = 4, KERNEL_WINDOW = 5 };
 void note_kernel(int which);
+// The launch plan of the last strip-matrix / window-offset launch (same diagnostic): up to eight integers.
+void note_plan(const int* v, int n);
 
 // Streaming multiprocessors of the current device (cached per device).
 int sm_count();

@@ -54,6 +54,8 @@ struct WParams {
   int32_t RX;         // X rows a tile uses: 128*MH + (Fh-1)*W + Fw-1
   int32_t RA;         // X rows allocated (RX rounded up to 8)
   int32_t NT, n_ntiles, Kp;
+  int32_t NTB;        // filter rows one CTA holds per block: NT, or NT/2 when two CTAs share an MMA
+  int32_t pair;       // two CTAs (a cluster) work as one: tcgen05.mma.cta_group::2, M = 256, each CTA its own rows and half the filter tile
   int32_t G, GR, NSUB, NXS;  // channels per X stage / per source stage, source stages per X stage, X stages per unit
   int32_t TPS;        // taps per filter stage (Fw: one filter row per stage; 1: one tap per stage)
   int32_t SR, SB, ND;
@@ -75,12 +77,30 @@ struct WParams {
 
 struct WUnit {
   int32_t nt, img, R0;
+  bool store;
 };
-__device__ __forceinline__ bool wunit_at(const WParams& P, int64_t it, WUnit& u) {
-  const int64_t t = (int64_t)blockIdx.x + it * (int64_t)gridDim.x;
-  if (t >= P.units) return false;
-  const int64_t tile = t / P.n_ntiles;
-  u.nt = (int32_t)(t - tile * P.n_ntiles);
+// Single-CTA mode: units t = blockIdx.x + it*grid, the filter tile fastest.  Pair mode: the pair (cluster)
+// takes two consecutive row tiles of one filter tile, one per CTA; where the number of row tiles is odd the
+// last pair's second CTA repeats the last tile without storing.
+template <bool PAIR>
+__device__ __forceinline__ bool wunit_at(const WParams& P, int64_t it, uint32_t rank, WUnit& u) {
+  int64_t tile;
+  if (PAIR) {
+    const int64_t pu = (int64_t)(blockIdx.x >> 1) + it * (int64_t)(gridDim.x >> 1);
+    if (pu >= P.units) return false;
+    const int64_t half = (P.tiles + 1) >> 1;
+    const int64_t nt = pu / half;
+    tile = 2 * (pu - nt * half) + rank;
+    u.store = tile < P.tiles;
+    if (!u.store) tile = P.tiles - 1;
+    u.nt = (int32_t)nt;
+  } else {
+    const int64_t t = (int64_t)blockIdx.x + it * (int64_t)gridDim.x;
+    if (t >= P.units) return false;
+    tile = t / P.n_ntiles;
+    u.nt = (int32_t)(t - tile * P.n_ntiles);
+    u.store = true;
+  }
   const int64_t img = tile / P.TPI;
   u.img = (int32_t)img;
   u.R0 = (int32_t)(tile - img * P.TPI) * 128 * P.MH;
@@ -101,7 +121,7 @@ __device__ __forceinline__ void wtile_range(const WParams& P, int32_t R0, int32_
 }
 
 // The MMA-issuing thread's whole life.  A filter stage holds the NBLK blocks of TPS taps.
-template <int FH, int FW, bool BF16, int MH, int NBLK, int TPS>
+template <int FH, int FW, bool BF16, int MH, int NBLK, int TPS, bool PAIR>
 __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* misc, uint32_t tmem_base, uint32_t x_sa,
                                           uint32_t b_sa) {
   Ring xr, br, dr;
@@ -115,13 +135,13 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
   const uint32_t a_lo0 = (uint32_t)ad0, a_hi = (uint32_t)(ad0 >> 32);
   const uint32_t b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
   const uint32_t x16 = P.x_stage_bytes >> 4, b16 = P.b_stage_bytes >> 4;
-  const uint32_t blk16 = NT * 4u;       // one filter block (NT rows x 64 bytes) in 16-byte units
+  const uint32_t blk16 = (uint32_t)P.NTB * 4u;  // one filter block (NTB rows x 64 bytes) in 16-byte units
   const uint32_t kstep16 = 2u * RA;     // one MMA K step (two chunks) of X in 16-byte units
   const uint32_t x_full0 = ptx::smem_u32(&bars->t_full[0]), x_empty0 = ptx::smem_u32(&bars->t_empty[0]);
   const uint32_t b_full0 = ptx::smem_u32(&bars->b_full[0]), b_empty0 = ptx::smem_u32(&bars->b_empty[0]);
   for (int64_t it = 0; ok; ++it, dr.advance(P.ND)) {
     WUnit u;
-    if (!wunit_at(P, it, u)) break;
+    if (!wunit_at<PAIR>(P, it, 0, u)) break;
     SPROF_W(0, ok = wait_bar(P, misc, ptx::smem_u32(&bars->acc_empty[dr.idx]), dr.phase ^ 1u, DEV_TIMEOUT_ACC))
     if (!ok) break;
     ptx::tc_fence_after();
@@ -155,7 +175,8 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
               for (int blk = 0; blk < NBLK; ++blk) {
 #pragma unroll
                 for (int k2 = 0; k2 < 2; ++k2) {
-                  ptx::mma_ss_lohi<BF16>(d_tmem + (uint32_t)h * NT, a_k, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, acc);
+                  if constexpr (PAIR) mma_ss_pair<BF16>(d_tmem + (uint32_t)h * NT, a_k, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, acc);
+                  else ptx::mma_ss_lohi<BF16>(d_tmem + (uint32_t)h * NT, a_k, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, acc);
                   acc = 1;
                   a_k += kstep16;
                 }
@@ -167,21 +188,23 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
 #ifdef IM2WIN_PROF
           pw[3] += clock64() - cm0;
 #endif
-          SPROF_W(4, ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u))
+          SPROF_W(4, if constexpr (PAIR) mma_commit_pair(b_empty0 + (uint32_t)br.idx * 8u); else ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u))
           br.advance(P.SB);
         }
       }
       if (!ok) break;
-      ptx::mma_commit(x_empty0 + (uint32_t)xr.idx * 8u);
+      if constexpr (PAIR) mma_commit_pair(x_empty0 + (uint32_t)xr.idx * 8u);
+      else ptx::mma_commit(x_empty0 + (uint32_t)xr.idx * 8u);
     }
     if (!ok) break;
-    ptx::mma_commit(ptx::smem_u32(&bars->acc_full[dr.idx]));
+    if constexpr (PAIR) mma_commit_pair(ptx::smem_u32(&bars->acc_full[dr.idx]));
+    else ptx::mma_commit(ptx::smem_u32(&bars->acc_full[dr.idx]));
   }
   SPROF_DUMP(1)
 }
 
 // SRCK: 0 = fp32 im2win tensor, 1 = untransformed input (fused), 2 = bf16 im2win tensor (BF16 mode).
-template <int FH, int FW, bool BF16, int SRCK>
+template <int FH, int FW, bool BF16, int SRCK, bool PAIR>
 __global__ void __launch_bounds__(640, 1)
 conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap, const __grid_constant__ CUtensorMap xmap) {
   constexpr bool FUSED = SRCK == 1;
@@ -197,6 +220,9 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
   SMisc* const misc = reinterpret_cast<SMisc*>(smem + P.off_misc);
   const uint32_t b_sa = ptx::smem_u32(smem), x_sa = b_sa + P.off_x, raw_sa = b_sa + P.off_raw;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // pair mode: 0 = the leader, whose thread issues the MMAs of both
+  constexpr uint32_t kShare = PAIR ? 2u : 1u;            // CTAs that arrive on the leader's "full"-side barriers
+  const bool remote = PAIR && rank != 0;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxRaw; ++i) {
@@ -208,20 +234,26 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
       ptx::mbar_init(ptx::smem_u32(&bars->b_empty[i]), 1);
     }
     for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(ptx::smem_u32(&bars->t_full[i]), kTW);
+      ptx::mbar_init(ptx::smem_u32(&bars->t_full[i]), kTW * kShare);
       ptx::mbar_init(ptx::smem_u32(&bars->t_empty[i]), 1);
       ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), 1);
-      ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), (uint32_t)P.n_epi);
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), (uint32_t)P.n_epi * kShare);
     }
     ptx::fence_mbar_init();
     misc->abort = 0;
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), P.tmem_cols);
-    ptx::tmem_relinquish();
+    if constexpr (PAIR) {  // (the same warp of both CTAs)
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(ptx::smem_u32(&misc->tmem_base)), "r"(P.tmem_cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      ptx::tmem_alloc(ptx::smem_u32(&misc->tmem_base), P.tmem_cols);
+      ptx::tmem_relinquish();
+    }
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();  // both CTAs' barriers exist before either signals the other's
   ptx::tc_fence_after();
   const uint32_t tmem_base = misc->tmem_base;
 
@@ -235,7 +267,7 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
     SPROF_DECL
     for (int64_t it = 0; ok; ++it) {
       WUnit u;
-      if (!wunit_at(P, it, u)) break;
+      if (!wunit_at<PAIR>(P, it, rank, u)) break;
       int32_t e_lo, e_hi, m_last;
       wtile_range<FH, FUSED>(P, u.R0, e_lo, e_hi, m_last);
       const int32_t len = e_hi - e_lo;
@@ -293,17 +325,15 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
       wait_bar(P, misc, ptx::smem_u32(&bars->raw_full[c % P.SR]), (uint32_t)(c / P.SR) & 1u, DEV_TIMEOUT_DRAIN);
   } else if (warp == 1) {
     // ================================================================ MMA ISSUER (one thread)
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       const int nblk = P.G / (4 * NCH);
-#define WRUN(MHv, NBv, TPv) wmma_role<FH, FW, BF16, MHv, NBv, TPv>(P, bars, misc, tmem_base, x_sa, b_sa)
+#define WRUN(MHv, NBv, TPv) wmma_role<FH, FW, BF16, MHv, NBv, TPv, PAIR>(P, bars, misc, tmem_base, x_sa, b_sa)
       if (P.TPS == 1) {
         if (P.MH == 1) { if (nblk == 1) WRUN(1, 1, 1); else WRUN(1, 2, 1); }
-        else if (P.MH == 2) { if (nblk == 1) WRUN(2, 1, 1); else WRUN(2, 2, 1); }
-        else { if (nblk == 1) WRUN(4, 1, 1); else WRUN(4, 2, 1); }
+        else { if (nblk == 1) WRUN(2, 1, 1); else WRUN(2, 2, 1); }
       } else {
         if (P.MH == 1) { if (nblk == 1) WRUN(1, 1, FW); else WRUN(1, 2, FW); }
-        else if (P.MH == 2) { if (nblk == 1) WRUN(2, 1, FW); else WRUN(2, 2, FW); }
-        else { if (nblk == 1) WRUN(4, 1, FW); else WRUN(4, 2, FW); }
+        else { if (nblk == 1) WRUN(2, 1, FW); else WRUN(2, 2, FW); }
       }
 #undef WRUN
     }
@@ -318,29 +348,38 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
       const int32_t bke = BF16 ? 32 : 16;  // elements (channels) per 64-byte filter row
       const int32_t nblk = P.G / bke;
       asm volatile("griddepcontrol.wait;" ::: "memory");  // the filter copy is written by the kernel launched just before
+      // Pair mode: this CTA fetches its half of every block's rows, and the bytes of both CTAs are counted on
+      // the leader's barrier: the leader announces both halves with its one arrival, the other CTA only
+      // issues its copies (its bytes may land before the announcement: the phase cannot complete before the
+      // leader's arrival, and the other CTA cannot run a phase ahead, because it needs the stage's release).
+      const uint32_t b_full_lead0 = remote ? mapa(ptx::smem_u32(&bars->b_full[0]), 0) : ptx::smem_u32(&bars->b_full[0]);
       for (int64_t it = 0; ok; ++it) {
         WUnit u;
-        if (!wunit_at(P, it, u)) break;
-        const int32_t row0 = u.nt * P.NT;
+        if (!wunit_at<PAIR>(P, it, rank, u)) break;
+        const int32_t row0 = u.nt * P.NT + (int32_t)rank * P.NTB;
         for (int32_t xs = 0; xs < P.NXS && ok; ++xs) {
           for (int32_t t0 = 0; t0 < FH * FW && ok; t0 += P.TPS, ++count, br.advance(P.SB)) {
             SPROF_W(0, ok = wait_bar(P, misc, ptx::smem_u32(&bars->b_empty[br.idx]), br.phase ^ 1u, DEV_TIMEOUT_B_EMPTY))
             if (!ok) break;
-            const uint32_t full = ptx::smem_u32(&bars->b_full[br.idx]);
+            const uint32_t full = b_full_lead0 + (uint32_t)br.idx * 8u;
 #ifdef IM2WIN_PROF
-            if (P.skip & 2) { ptx::mbar_arrive(full); continue; }
+            if (P.skip & 2) { if (!remote) ptx::mbar_arrive(full); continue; }
 #endif
-            ptx::mbar_arrive_expect_tx(full, P.b_stage_bytes);
+            if (!remote) ptx::mbar_arrive_expect_tx(full, P.b_stage_bytes * kShare);
             uint32_t dst = b_sa + (uint32_t)br.idx * P.b_stage_bytes;
             for (int32_t dt = 0; dt < P.TPS; ++dt)
-              for (int32_t blk = 0; blk < nblk; ++blk, dst += (uint32_t)P.NT * 64u)
-                tma_load_2d(dst, &fmap, xs * P.G + blk * bke, (t0 + dt) * P.Kp + row0, full);
+              for (int32_t blk = 0; blk < nblk; ++blk, dst += (uint32_t)P.NTB * 64u) {
+                if (remote) tma_load_2d_pair(dst, &fmap, xs * P.G + blk * bke, (t0 + dt) * P.Kp + row0, full);
+                else tma_load_2d(dst, &fmap, xs * P.G + blk * bke, (t0 + dt) * P.Kp + row0, full);
+              }
           }
         }
       }
       SPROF_DUMP(7)
+      // every copy issued must have landed before the CTA exits: the stage's release by the MMAs that read it
+      // says so (in pair mode the bytes are counted on the leader's barrier, not here)
       for (int64_t c = count > P.SB ? count - P.SB : 0; c < count; ++c)
-        wait_bar(P, misc, ptx::smem_u32(&bars->b_full[c % P.SB]), (uint32_t)(c / P.SB) & 1u, DEV_TIMEOUT_DRAIN);
+        wait_bar(P, misc, ptx::smem_u32(&bars->b_empty[c % P.SB]), (uint32_t)(c / P.SB) & 1u, DEV_TIMEOUT_DRAIN);
     }
     __syncwarp();
   } else if (warp >= kTWarp0 && warp < kTWarp0 + kTW) {
@@ -351,9 +390,10 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
     Ring rr, xr;
     bool ok = true;
     SPROF_DECL
+    const uint32_t x_full_lead0 = remote ? mapa(ptx::smem_u32(&bars->t_full[0]), 0) : ptx::smem_u32(&bars->t_full[0]);
     for (int64_t it = 0; ok; ++it) {
       WUnit u;
-      if (!wunit_at(P, it, u)) break;
+      if (!wunit_at<PAIR>(P, it, rank, u)) break;
       int32_t e_lo, e_hi, m_last;
       wtile_range<FH, FUSED>(P, u.R0, e_lo, e_hi, m_last);
       // this thread's X rows: x = tid + z*256 <-> input position e = R0 + x; where its value sits in a staged channel row
@@ -440,7 +480,10 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
 #endif
           if (lane == 0) {
             ptx::mbar_arrive(ptx::smem_u32(&bars->raw_empty[rr.idx]));
-            if (last) ptx::mbar_arrive(ptx::smem_u32(&bars->t_full[xr.idx]));
+            if (last) {
+              if (remote) arrive_cluster(x_full_lead0 + (uint32_t)xr.idx * 8u);
+              else ptx::mbar_arrive(x_full_lead0 + (uint32_t)xr.idx * 8u);
+            }
           }
         }
       }
@@ -454,9 +497,10 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
     bool ok = true;
     SPROF_DECL
     const int64_t eHoWo = (int64_t)P.Ho * P.Wo;
+    const uint32_t acc_empty_lead0 = remote ? mapa(ptx::smem_u32(&bars->acc_empty[0]), 0) : ptx::smem_u32(&bars->acc_empty[0]);
     for (int64_t it = 0; ok; ++it, dr.advance(P.ND)) {
       WUnit u;
-      if (!wunit_at(P, it, u)) break;
+      if (!wunit_at<PAIR>(P, it, rank, u)) break;
       const int32_t n0 = u.nt * P.NT;
       SPROF_W(0, ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->acc_full[dr.idx]), dr.phase, DEV_TIMEOUT_ACC, 128))
       if (!ok) break;
@@ -464,14 +508,17 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
       for (int32_t h = h0; h < P.MH; h += 2) {
         const int32_t rho = u.R0 + h * 128 + q4 * 32 + lane;
         const int32_t m = rho / P.W, q = rho - m * P.W;
-        const bool valid = rho < P.RPI && q < P.Wo;
+        const bool valid = u.store && rho < P.RPI && q < P.Wo;
         float* const orow = P.out + ((int64_t)u.img * P.K + n0) * eHoWo + (int64_t)m * P.Wo + q;
         const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)((dr.idx * P.MH + h) * P.NT);
         store_columns(d_tmem, orow, eHoWo, 0, P.NT, P.K - n0, valid);
       }
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->acc_empty[dr.idx]));
+      if (lane == 0) {
+        if (remote) arrive_cluster(acc_empty_lead0 + (uint32_t)dr.idx * 8u);
+        else ptx::mbar_arrive(acc_empty_lead0 + (uint32_t)dr.idx * 8u);
+      }
     }
     if (warp == kEpiWarp0) { SPROF_DUMP(6) }
   }
@@ -479,9 +526,11 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
   // ------------------------------------------------------------------ teardown
   ptx::tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();  // neither CTA leaves while the other may still signal its barriers
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, P.tmem_cols);
+    if constexpr (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(P.tmem_cols) : "memory");
+    else ptx::tmem_dealloc(tmem_base, P.tmem_cols);
   }
 }
 
@@ -525,7 +574,7 @@ struct WPlan {
 
 // Fills the launch parameters; IM2WIN_EUNSUPPORTED where the kernel does not apply.
 template <int FH, int FW, bool BF16, int SRCK>
-int make_wplan(const Geometry& g, WPlan* pl, int mh_fixed) {
+int make_wplan(const Geometry& g, WPlan* pl, int pair, int mh_fixed) {
   constexpr int NCH = BF16 ? 8 : 4;
   constexpr int64_t ES = SRCK == 2 ? 2 : 4;
   constexpr int64_t EPC = 16 / ES;
@@ -541,18 +590,21 @@ int make_wplan(const Geometry& g, WPlan* pl, int mh_fixed) {
   P.n_ntiles = (g.K + 255) / 256;
   P.NT = ((g.K + P.n_ntiles - 1) / P.n_ntiles + 15) / 16 * 16;
   P.Kp = P.n_ntiles * P.NT;
+  if (pair && P.NT % 32 != 0) return IM2WIN_EUNSUPPORTED;  // (each CTA's half of the filter rows: a multiple of 16)
+  P.pair = pair;
+  P.NTB = pair ? P.NT / 2 : P.NT;
   if (SRCK == 1) { P.plane = (int64_t)g.H * g.W; P.n_src = g.n_in; }
   else { P.plane = g.HoL; P.n_src = g.n_win; }
   P.pm = (int32_t)(P.plane % EPC);
   const int64_t cap = 227 * 1024 - 1024 - (1024 + 128 + 16) - (int64_t)((sizeof(SBars) + 15) / 16 * 16) - 64;
   P.MH = mh_fixed;
-  if (P.MH * P.NT > 512) return IM2WIN_EUNSUPPORTED;
+  if (P.MH < 1 || P.MH > 2 || P.MH * P.NT > 512) return IM2WIN_EUNSUPPORTED;
   P.RX = 128 * P.MH + (FH - 1) * g.W + FW - 1;
   if (P.RX > kXMax * kTW * 32) return IM2WIN_EUNSUPPORTED;
   P.RA = (P.RX + 7) / 8 * 8;
   P.TPI = (P.RPI + 128 * P.MH - 1) / (128 * P.MH);
   P.tiles = (int64_t)g.N * P.TPI;
-  P.units = P.tiles * P.n_ntiles;
+  P.units = pair ? ((P.tiles + 1) / 2) * P.n_ntiles : P.tiles * P.n_ntiles;
   P.ND = 512 / (P.MH * P.NT) >= 2 ? 2 : 1;
   P.n_epi = 4 * (P.MH < 2 ? P.MH : 2);
   // source elements of one channel a tile needs at most, plus the 16-byte phase in front
@@ -560,20 +612,36 @@ int make_wplan(const Geometry& g, WPlan* pl, int mh_fixed) {
   int64_t cp = len_max + 2 * EPC;
   const int64_t cp_align = 32 / ES;
   cp = (cp + cp_align - 1) / cp_align * cp_align;
-  // filter stage: one filter row (Fw taps) where that stays small, else one tap
-  const int64_t blk_bytes = (int64_t)P.NT * 64;
+  // The split of shared memory: filter blocks per X stage (16/32 or 32/64 channels), taps per filter stage
+  // (one filter row, or one tap) and channels per source stage, tried in an order taken from measurements
+  // (every combination, on six layers, both modes, three sources): a whole filter row per stage wherever two
+  // such stages fit (one wait and one release of the issuing thread per Fw taps); two blocks per X stage for
+  // the fused source, whose staged rows are a third of the im2win tensor's; sixteen channels per source stage,
+  // eight where the fp32 im2win tensor's rows are long.  The first combination that leaves two stages for each
+  // ring wins; what is left goes to the two rings by the latency each has to cover.
+  const int64_t blk_bytes = (int64_t)P.NTB * 64;
+  const double mma_cyc = P.NT / 2.0 > 54.0 ? P.NT / 2.0 : 54.0;
+  const int forced_plan = knobs().window_plan;  // test build: nblk | taps-per-stage << 4 | channels per source stage << 8
+  struct Try { int nblk, tps, gr; };
+  const Try order_fused[] = {{2, FW, 16}, {2, FW, 8}, {2, 1, 32}, {2, 1, 16}, {1, FW, 32}, {1, FW, 16}, {1, 1, 16}, {1, 1, 8}, {1, 1, 4}};
+  const Try order_win[] = {{1, FW, 16}, {1, FW, 8}, {2, 1, 8}, {1, 1, 8}, {1, 1, 4}, {1, 1, 16}};
+  const Try order_win16[] = {{1, FW, 32}, {1, FW, 16}, {2, 1, 16}, {1, 1, 16}, {1, 1, 8}, {1, 1, 32}};
+  const Try* order = SRCK == 1 ? order_fused : (SRCK == 2 ? order_win16 : order_win);
+  const int n_order = SRCK == 1 ? 9 : 6;
   bool found = false;
-  for (int nblk = 2; nblk >= 1 && !found; --nblk) {
-    const int G = nblk * gmin;
-    if (g.C % G != 0) continue;
-    P.G = G;
-    P.NXS = g.C / G;
-    P.x_stage_bytes = (uint32_t)((G / NCH) * P.RA * 16);
-    P.TPS = ((int64_t)FW * nblk * blk_bytes <= 16 * 1024) ? FW : 1;
-    P.b_stage_bytes = (uint32_t)(P.TPS * nblk * blk_bytes);
-    const int64_t left = cap - 2 * (int64_t)P.x_stage_bytes;
-    for (int gr = G; gr >= NCH && !found; gr /= 2) {
-      if (G % gr != 0 || gr > 32) continue;
+  {
+    for (int t = 0; t < n_order && !found; ++t) {
+      int nblk = order[t].nblk, tps = order[t].tps, gr = order[t].gr;
+      if (forced_plan) {
+        if (t > 0) break;
+        nblk = forced_plan & 15; tps = (forced_plan >> 4) & 15; gr = forced_plan >> 8;
+        if (nblk < 1 || nblk > 2 || (tps != 1 && tps != FW) || gr < NCH) return IM2WIN_EUNSUPPORTED;
+      }
+      const int G = nblk * gmin;
+      if (g.C % G != 0 || G % gr != 0 || gr > 32 || gr < NCH) continue;
+      const uint32_t x_stage_bytes = (uint32_t)((G / NCH) * P.RA * 16);
+      const int64_t left = cap - 2 * (int64_t)x_stage_bytes;
+      const int64_t b_stage_bytes = (int64_t)tps * nblk * blk_bytes;
       // boxes of at most 2 KB per channel row
       int64_t nbx = 1, bxe = cp;
       const bool box_ok = P.pm == 0 && gr >= 4 && encode_fn() != nullptr && (int64_t)g.N * g.C <= INT32_MAX && !knobs().no_box;
@@ -584,27 +652,24 @@ int make_wplan(const Geometry& g, WPlan* pl, int mh_fixed) {
       }
       const int64_t raw_bytes = (int64_t)gr * nbx * bxe * ES;
       if (raw_bytes % 128 != 0 || bxe * ES > 65536) continue;
-      if (2 * (int64_t)P.b_stage_bytes + 2 * raw_bytes > left) continue;
-      P.GR = gr;
-      P.NSUB = G / gr;
-      P.box = box_ok ? 1 : 0;
-      P.NBX = (int32_t)nbx; P.BXE = (int32_t)bxe;
-      P.raw_stage_bytes = (uint32_t)raw_bytes;
-      // what is left beside the two X stages goes to the two rings stage by stage, in proportion to
-      // the bytes each must keep in flight (about 2500 cycles of memory latency at its consumption rate)
-      const double mma_cyc = P.NT / 2.0 > 50.0 ? P.NT / 2.0 : 50.0;
-      const double b_stage_cyc = (double)P.TPS * nblk * 2 * P.MH * mma_cyc;
-      const double raw_stage_cyc = b_stage_cyc * (FH * FW / P.TPS) / P.NSUB;
-      const int64_t want_b = (int64_t)(2500.0 / b_stage_cyc + 0.999) + 1, want_r = (int64_t)(2500.0 / raw_stage_cyc + 0.999) + 1;
-      int64_t sb = 2, sr = 2;
-      while (true) {
-        const bool can_b = sb < kMaxB && (sb + 1) * P.b_stage_bytes + sr * raw_bytes <= left;
-        const bool can_r = sr < kMaxRaw && sb * P.b_stage_bytes + (sr + 1) * raw_bytes <= left;
+      const int64_t min_b = 2;
+      if (min_b * b_stage_bytes + 2 * raw_bytes > left) continue;
+      const int nsub = G / gr;
+      const double b_stage_cyc = (double)tps * nblk * 2 * P.MH * mma_cyc;
+      const double raw_stage_cyc = (double)FH * FW * nblk * 2 * P.MH * mma_cyc / nsub;
+      int64_t sb = min_b, sr = 2;
+      while (true) {  // one more stage for the ring that covers less of the latency (about 2500 cycles), while it fits
+        const bool can_b = sb < kMaxB && (sb + 1) * b_stage_bytes + sr * raw_bytes <= left;
+        const bool can_r = sr < kMaxRaw && sb * b_stage_bytes + (sr + 1) * raw_bytes <= left;
         if (!can_b && !can_r) break;
-        const double fill_b = (double)sb / (double)want_b, fill_r = (double)sr / (double)want_r;
-        if (can_b && (!can_r || fill_b <= fill_r)) ++sb;
+        const double cover_b = (double)(sb - 1) * b_stage_cyc, cover_r = (double)(sr - 1) * raw_stage_cyc;
+        if (can_b && (!can_r || cover_b <= cover_r)) ++sb;
         else ++sr;
       }
+      P.G = G; P.NXS = g.C / G; P.x_stage_bytes = x_stage_bytes;
+      P.TPS = tps; P.b_stage_bytes = (uint32_t)b_stage_bytes;
+      P.GR = gr; P.NSUB = nsub; P.box = box_ok ? 1 : 0;
+      P.NBX = (int32_t)nbx; P.BXE = (int32_t)bxe; P.raw_stage_bytes = (uint32_t)raw_bytes;
       P.SB = (int32_t)sb; P.SR = (int32_t)sr;
       found = true;
     }
@@ -623,50 +688,118 @@ int make_wplan(const Geometry& g, WPlan* pl, int mh_fixed) {
   const int32_t cols = P.ND * P.MH * P.NT;
   P.tmem_cols = 32;
   while ((int32_t)P.tmem_cols < cols) P.tmem_cols *= 2;
-  P.idesc = ptx::make_idesc(128, P.NT, BF16 ? 1 : 2);
+  P.idesc = ptx::make_idesc(pair ? 256 : 128, P.NT, BF16 ? 1 : 2);
   pl->scratch_bytes = (size_t)FH * FW * P.Kp * (size_t)g.C * (BF16 ? 2 : 4);
   pl->threads = (kEpiWarp0 + P.n_epi) * 32;
   return IM2WIN_OK;
 }
 
+// Which variant a problem gets (knobs override).  CTA pairs (each CTA fetches half the filter rows) where they
+// were measured faster than single CTAs: the 5x5 layers in BF16 mode with 256-wide filter tiles (25 taps make
+// the filter stream the largest consumer of shared-memory bandwidth), with one block per tile so that two
+// accumulator buffers remain; and 192-wide tiles in TF32 mode from the fused source and in BF16 mode from the
+// bf16 tensor.  Elsewhere a pair's MMAs, which cost the issuing thread about twice as long, lose more than the
+// halved filter traffic gains.
 // Rows per tile: the number of 128-row blocks that gives the least estimated time: rounds of units over the
-// SMs x (blocks per unit + the fixed part of a unit, measured as about two blocks); ties go to the taller tile.
+// SMs (or pairs) x (blocks per unit + the fixed part of a unit, measured as about two blocks); ties go to the
+// taller tile.
 template <int FH, int FW, bool BF16, int SRCK>
 int choose_wplan(const Geometry& g, WPlan* best) {
   const int forced = knobs().window_mh & 255;
-  int64_t best_cost = -1;
-  WPlan cand;
-  for (int mh = 4; mh >= 1; mh /= 2) {
-    if (forced && mh != forced) continue;
-    if (make_wplan<FH, FW, BF16, SRCK>(g, &cand, mh) != IM2WIN_OK) continue;
-    if (!forced && mh > 1 && (int64_t)g.Ho * g.W <= 128 * (mh / 2)) continue;  // the image fits fewer blocks
-    // tiles of up to 128 filters keep two accumulator buffers (the epilogue overlaps the next unit); wider
-    // ones gain more from the second block (each filter stage feeds two MMAs)
-    if (!forced && cand.P.NT <= 128 && cand.P.ND < 2) continue;
-    const int64_t rounds = (cand.P.units + sm_count() - 1) / sm_count();
-    const int64_t cost = rounds * (mh + 2);  // (a unit costs about two blocks' time beside its blocks: measured)
-    if (best_cost < 0 || cost < best_cost) { best_cost = cost; *best = cand; }
+  const int nt = (((g.K + (g.K + 255) / 256 - 1) / ((g.K + 255) / 256)) + 15) / 16 * 16;
+  int pair = 0;
+  if (FH == 5) pair = BF16 && nt >= 192 && (int64_t)g.Ho * g.W >= 640;  // (faster on the 27x27-output 5x5 layer, slower on the 20x20 one)
+  else if (nt >= 192 && nt < 256) pair = (SRCK == 1 && !BF16) || SRCK == 2;
+  if (knobs().window_pair == 1) pair = 1;
+  if (knobs().window_pair == 2) pair = 0;
+  for (int attempt = 0; attempt < 2; ++attempt, pair = 1 - pair) {
+    if (attempt == 1 && knobs().window_pair) break;  // (a forced variant that does not fit: unsupported)
+    int64_t best_cost = -1;
+    WPlan cand;
+    const int64_t slots = pair ? sm_count() / 2 : sm_count();
+    for (int mh = 2; mh >= 1; mh /= 2) {  // (four blocks per tile were measured too: never faster, and they leave the rings less room)
+      if (forced && mh != forced) continue;
+      if (!forced && pair && FH == 5 && mh != 1) continue;
+      if (make_wplan<FH, FW, BF16, SRCK>(g, &cand, pair, mh) != IM2WIN_OK) continue;
+      if (!forced && mh > 1 && (int64_t)g.Ho * g.W <= 128 * (mh / 2)) continue;  // the image fits fewer blocks
+      // tiles of up to 128 filters keep two accumulator buffers (the epilogue overlaps the next unit); wider
+      // ones gain more from the second block (each filter stage feeds two MMAs)
+      if (!forced && cand.P.NT <= 128 && cand.P.ND < 2) continue;
+      const int64_t rounds = (cand.P.units + slots - 1) / slots;
+      const int64_t cost = rounds * (mh + 2);  // (a unit costs about two blocks' time beside its blocks: measured)
+      if (best_cost < 0 || cost < best_cost) { best_cost = cost; *best = cand; }
+    }
+    if (best_cost >= 0) return IM2WIN_OK;
   }
-  return best_cost < 0 ? IM2WIN_EUNSUPPORTED : IM2WIN_OK;
+  return IM2WIN_EUNSUPPORTED;
 }
 
-// Whether this kernel is expected to beat the strip-matrix and the persistent kernel (measured on B200 at
-// batch 128 over the benchmark's stride-1 layers, every source kind and both modes).  Its strengths: the
-// staged bytes and the interleaving work are a third of the strip-matrix kernel's for the fused source, and
-// it has no per-thread window loads (the persistent kernel's bound on deep layers in BF16 mode).  It has no
-// CTA-pair mode, so 256-wide filter tiles on images of more than one block stay with the strip-matrix kernel,
-// and its one issuing thread is slower than the persistent kernel's three on 64-filter layers.
+// Whether this kernel is expected to beat the strip-matrix and the persistent kernel: rules read off a
+// measured table (B200, batch 128, every stride-1 3x3 / 5x5 layer of the benchmark lists, three source kinds,
+// both modes).  Its strengths: the staged bytes and the interleaving work are a third of the strip-matrix
+// kernel's, and it has no per-thread window loads (the persistent kernel's bound on deep layers in BF16 mode).
+// It has no CTA-pair mode, so in TF32 mode and for the fused and bf16 sources the 256-wide filter tiles on
+// images of more than one block stay with the strip-matrix kernel; its one issuing thread is slower than the
+// persistent kernel's three on TF32 layers of 64 filters; and where the persistent kernel finishes in a single
+// wave of tiles that span images (small images, one filter tile) that kernel stays.
 template <int FH, int FW, bool BF16, int SRCK>
 bool window_preferred(const Geometry& g, const WParams& P) {
-  if (P.units * 2 <= sm_count()) return false;  // under-filled launches: the persistent kernel's reduction slices
-  if (FH == 5) return BF16;                    // 5x5 layers: 25 taps of one staged tile
-  if (SRCK == 2) return P.NT <= 128;           // bf16 im2win tensor
-  if (SRCK == 1) {                             // fused
-    if (g.C < 128) return false;
-    if (BF16) return P.NT <= 192 || P.RPI < 128;
-    return P.NT >= 128 && P.NT <= 192;
+  const int nsm = sm_count();
+  if (P.units * 2 <= nsm) return false;  // under-filled launches: the persistent kernel's reduction slices
+  if (FH == 5) return BF16;               // 5x5 layers: 25 taps of one staged tile
+  const int64_t span_tiles = (g.Mtot + 127) / 128;
+  if (P.n_ntiles == 1 && span_tiles <= nsm && P.NT > 128) return false;  // one wave of the persistent kernel
+  if (!BF16) {
+    if (SRCK == 1) return g.C >= 128 && P.NT >= 128 && P.NT <= 192;
+    return P.NT > 64 && P.NT <= 128;
   }
-  return BF16 && g.C >= 256 && P.NT > 128 && P.NT <= 192;  // fp32 im2win tensor
+  if (SRCK == 2) return P.NT <= 192;                                   // bf16 im2win tensor
+  if (SRCK == 1)                                                        // fused
+    return P.NT <= 192 ? !(g.C < 128 && P.NT > 64) : P.RPI < 128;
+  return g.C >= 128;                                                    // fp32 im2win tensor
+}
+
+template <int FH, int FW, bool BF16, int SRCK, bool PAIR>
+int launch_wkernel(const WParams& P, const WPlan& pl, const CUtensorMap& fmap, const CUtensorMap& xmap, cudaStream_t st) {
+  auto kern = conv_tc_window_kernel<FH, FW, BF16, SRCK, PAIR>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return IM2WIN_ECUDA;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3((unsigned)pl.threads);
+  cfg.dynamicSmemBytes = pl.smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  // programmatic dependent launch: the prologue and the first source copies overlap the filter-copy kernel
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int64_t grid;
+  if (PAIR) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+    cfg.gridDim = dim3((unsigned)(sm_count() / 2 * 2));
+    int max_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg) != cudaSuccess || max_clusters < 1) {
+      cudaGetLastError();
+      return IM2WIN_EUNSUPPORTED;
+    }
+    int64_t pairs = sm_count() / 2;
+    if (pairs > max_clusters) pairs = max_clusters;
+    if (pairs > P.units) pairs = P.units;
+    grid = 2 * pairs;
+  } else {
+    grid = P.units < sm_count() ? P.units : sm_count();
+  }
+  cfg.gridDim = dim3((unsigned)grid);
+  if (cudaLaunchKernelEx(&cfg, kern, P, fmap, xmap) != cudaSuccess) {
+    cudaGetLastError();
+    return IM2WIN_ECUDA;
+  }
+  return IM2WIN_OK;
 }
 
 template <int FH, int FW, bool BF16, int SRCK>
@@ -694,7 +827,7 @@ int launch_window(const void* src, const float* f, float* out, const Geometry& g
   {
     const cuuint64_t gdim[2] = {(cuuint64_t)g.C, (cuuint64_t)FH * FW * P.Kp};
     const cuuint64_t gstr[1] = {(cuuint64_t)g.C * (BF16 ? 2 : 4)};
-    const cuuint32_t box[2] = {(cuuint32_t)(BF16 ? 32 : 16), (cuuint32_t)P.NT};
+    const cuuint32_t box[2] = {(cuuint32_t)(BF16 ? 32 : 16), (cuuint32_t)P.NTB};
     const cuuint32_t estr[2] = {1, 1};
     if (enc(&fmap, BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, scratch.ptr, gdim, gstr, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -719,27 +852,13 @@ int launch_window(const void* src, const float* f, float* out, const Geometry& g
   if (BF16) filter_tap_rows_kernel<true><<<dim3((unsigned)P.Kp), 128, 0, st>>>(f, scratch.ptr, g.K, P.Kp, g.C, FH * FW);
   else filter_tap_rows_kernel<false><<<dim3((unsigned)P.Kp), 128, 0, st>>>(f, scratch.ptr, g.K, P.Kp, g.C, FH * FW);
   if (cudaGetLastError() != cudaSuccess) return IM2WIN_ECUDA;
-  auto kern = conv_tc_window_kernel<FH, FW, BF16, SRCK>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes) != cudaSuccess) {
-    cudaGetLastError();
-    return IM2WIN_ECUDA;
-  }
-  cudaLaunchConfig_t cfg = {};
-  cfg.blockDim = dim3((unsigned)pl.threads);
-  cfg.dynamicSmemBytes = pl.smem_bytes;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  // programmatic dependent launch: the prologue and the first source copies overlap the filter-copy kernel
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cfg.gridDim = dim3((unsigned)(P.units < sm_count() ? P.units : sm_count()));
-  if (cudaLaunchKernelEx(&cfg, kern, P, fmap, xmap) != cudaSuccess) {
-    cudaGetLastError();
-    return IM2WIN_ECUDA;
-  }
+  rc = P.pair ? launch_wkernel<FH, FW, BF16, SRCK, true>(P, pl, fmap, xmap, st) : launch_wkernel<FH, FW, BF16, SRCK, false>(P, pl, fmap, xmap, st);
+  if (rc != IM2WIN_OK) return rc;
   note_kernel(KERNEL_WINDOW);
+  {
+    const int v[8] = {P.MH + 10 * P.pair, P.G, P.TPS, P.GR, P.SB, P.SR, P.ND, P.box * 100 + P.NBX};
+    note_plan(v, 8);
+  }
   return IM2WIN_OK;
 }
 
