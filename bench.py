@@ -41,7 +41,8 @@ NOMINAL_TF32_OVER_BF16 = 1.1 / 2.25
 NCU_TRAFFIC_BYTES = {("resnet3x3", "tf32"): 319.57e6 + 81.23e6, ("stem7x7", "tf32"): 277.09e6 + 352.88e6,
                      ("down3x3", "tf32"): 322.35e6 + 74.64e6,
                      ("deep3x3", "tf32"): 90.54e6 + 4.44e6, ("deep3x3", "bf16"): 89.36e6 + 3.78e6}
-KERNEL_NAMES = {1: "conv_tc_strip_kernel", 2: "conv_tc_persistent_kernel", 3: "conv_tc_kernel", 4: "conv_fp32_kernel"}
+KERNEL_NAMES = {1: "conv_tc_strip_kernel", 2: "conv_tc_persistent_kernel", 3: "conv_tc_kernel", 4: "conv_fp32_kernel",
+                5: "conv_tc_window_kernel"}
 
 
 def _peaks():
@@ -500,7 +501,7 @@ def run_gpu(args):
     # the tensor-bound layers of the benchmark definition, convolution only (not part of `value`)
     extra = {}
     if world == 1 and not args.no_extra_layers:
-        for name in ("deep3x3", "sweep_L5", "sweep_L10"):
+        for name in ("deep3x3", "sweep_L5", "sweep_L10", "sweep_L4", "sweep_L2"):
             extra[name] = {}
             for m in ("tf32", "bf16"):
                 r2 = time_conv_only(wl.CONFIGS[name], m, 10, torch, b, flush_buf)

@@ -77,8 +77,8 @@ int im2win_workspace_bytes(const im2win_shape* shape, size_t* bytes);
 /* Workspace with which im2win_conv can pick its fastest kernel for (shape, src_kind, mode) (no
  * counterpart in the paper): the im2win tensor where src_kind is NCHW (as above, rounded up to 256
  * bytes), plus room for a re-laid-out copy of the filter that some tensor-core kernels stream by TMA
- * (tap-major order for the strip-matrix kernel; bf16 for BF16 mode).  That copy is at most about
- * 1.4 x the filter's own 4*K*C*Fh*Fw bytes, i.e. a few MB against an im2win tensor of tens to hundreds
+ * (tap-major orders for the strip-matrix and window-offset kernels; bf16 for BF16 mode).  That copy is at
+ * most about 1.4 x the filter's own 4*K*C*Fh*Fw bytes, i.e. a few MB against an im2win tensor of tens to hundreds
  * of MB.  A smaller workspace is legal (down to im2win_workspace_bytes, or none for the other source
  * kinds): kernels that need no copy are used instead, some of them slower. */
 int im2win_conv_workspace_bytes(const im2win_shape* shape, int src_kind, int mode, size_t* bytes);
@@ -121,8 +121,9 @@ int im2win_transform_bf16(const float* in_nchw, const im2win_shape* shape, uint1
  *            IM2WIN_MODE_BF16 (EINVAL otherwise); `workspace` optional scratch.  The MMA operands
  *            are the same bf16 values as from an fp32 im2win tensor.  Implemented where a
  *            tensor-core kernel with a 16-bit source applies (3x3 layers of the strip-matrix kernel
- *            with scratch; filter-size specialisations whose images have roughly a thousand output
- *            positions or more); EUNSUPPORTED otherwise.
+ *            and stride-1 3x3 / 5x5 layers of the window-offset kernel, both with scratch;
+ *            filter-size specialisations whose images have roughly a thousand output positions or
+ *            more); EUNSUPPORTED otherwise.
  * filter:    device, K*C*Fh*Fw floats, native K,C,Fh,Fw order (the caller repacks nothing; kernels
  *            that want another order or bf16 write their copy into the workspace's scratch part).
  * mode:      IM2WIN_MODE_*.

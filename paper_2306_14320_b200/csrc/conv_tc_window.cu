@@ -55,6 +55,7 @@ struct WParams {
   int32_t RA;         // X rows allocated (RX rounded up to 8)
   int32_t NT, n_ntiles, Kp;
   int32_t NTB;        // filter rows one CTA holds per block: NT, or NT/2 when two CTAs share an MMA
+  int32_t two;        // two MMA-issuing threads share the filter stages by parity; every MMA accumulates, the epilogue zeroes behind its reads
   int32_t pair;       // two CTAs (a cluster) work as one: tcgen05.mma.cta_group::2, M = 256, each CTA its own rows and half the filter tile
   int32_t G, GR, NSUB, NXS;  // channels per X stage / per source stage, source stages per X stage, X stages per unit
   int32_t TPS;        // taps per filter stage (Fw: one filter row per stage; 1: one tap per stage)
@@ -123,9 +124,11 @@ __device__ __forceinline__ void wtile_range(const WParams& P, int32_t R0, int32_
 // The MMA-issuing thread's whole life.  A filter stage holds the NBLK blocks of TPS taps.
 template <int FH, int FW, bool BF16, int MH, int NBLK, int TPS, bool PAIR>
 __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* misc, uint32_t tmem_base, uint32_t x_sa,
-                                          uint32_t b_sa) {
+                                          uint32_t b_sa, uint32_t which) {
   Ring xr, br, dr;
   bool ok = true;
+  const bool two = P.two != 0;
+  uint32_t bc = 0;  // filter stages so far: with two issuing threads, thread `which` takes those of its parity
   SPROF_DECL
   const int32_t lane = 0;
   (void)lane;
@@ -146,7 +149,7 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
     if (!ok) break;
     ptx::tc_fence_after();
     const uint32_t d_tmem = tmem_base + (uint32_t)(dr.idx * MH) * NT;
-    uint32_t accum = 0;
+    uint32_t accum = two ? 1u : 0u;
     for (int32_t xs = 0; xs < P.NXS && ok; ++xs, xr.advance(2)) {
       SPROF_W(1, ok = wait_bar(P, misc, x_full0 + (uint32_t)xr.idx * 8u, xr.phase, DEV_TIMEOUT_A_FULL, 20))
       if (!ok) break;
@@ -155,6 +158,7 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
       for (int uu = 0; uu < FH && ok; ++uu, a_u += W) {
 #pragma unroll
         for (int v0 = 0; v0 < FW; v0 += TPS) {
+          if (two && ((bc++ & 1u) != which)) { br.advance(P.SB); continue; }
           SPROF_W(2, ok = wait_bar(P, misc, b_full0 + (uint32_t)br.idx * 8u, br.phase, DEV_TIMEOUT_B_FULL, 20))
           if (!ok) break;
           ptx::tc_fence_after();
@@ -235,8 +239,8 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
     }
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(ptx::smem_u32(&bars->t_full[i]), kTW * kShare);
-      ptx::mbar_init(ptx::smem_u32(&bars->t_empty[i]), 1);
-      ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&bars->t_empty[i]), 1u + (uint32_t)P.two);
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), 1u + (uint32_t)P.two);
       ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), (uint32_t)P.n_epi * kShare);
     }
     ptx::fence_mbar_init();
@@ -256,6 +260,16 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
   if constexpr (PAIR) cluster_sync_all();  // both CTAs' barriers exist before either signals the other's
   ptx::tc_fence_after();
   const uint32_t tmem_base = misc->tmem_base;
+  if (P.two) {  // every MMA accumulates: the accumulators start as zeros (one warp per TMEM lane quarter)
+    if (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4) {
+      const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+      for (uint32_t c = 0; c < P.tmem_cols; c += 16) ptx::tmem_zero_x16(tmem_base + lane_base + c);
+      ptx::tmem_wait_st();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+  }
 
   if (warp == 0) {
     // ================================================================ SOURCE PRODUCER
@@ -323,11 +337,12 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
     // every copy issued must have landed before the CTA exits
     for (int64_t c = count > P.SR ? count - P.SR : 0; c < count; ++c)
       wait_bar(P, misc, ptx::smem_u32(&bars->raw_full[c % P.SR]), (uint32_t)(c / P.SR) & 1u, DEV_TIMEOUT_DRAIN);
-  } else if (warp == 1) {
-    // ================================================================ MMA ISSUER (one thread)
+  } else if (warp == 1 || (warp == 3 && P.two)) {
+    // ================================================================ MMA ISSUER (one thread, or one each of warps 1 and 3)
     if (lane == 0 && rank == 0) {
+      const uint32_t which = warp == 1 ? 0u : 1u;
       const int nblk = P.G / (4 * NCH);
-#define WRUN(MHv, NBv, TPv) wmma_role<FH, FW, BF16, MHv, NBv, TPv, PAIR>(P, bars, misc, tmem_base, x_sa, b_sa)
+#define WRUN(MHv, NBv, TPv) wmma_role<FH, FW, BF16, MHv, NBv, TPv, PAIR>(P, bars, misc, tmem_base, x_sa, b_sa, which)
       if (P.TPS == 1) {
         if (P.MH == 1) { if (nblk == 1) WRUN(1, 1, 1); else WRUN(1, 2, 1); }
         else { if (nblk == 1) WRUN(2, 1, 1); else WRUN(2, 2, 1); }
@@ -511,7 +526,7 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
         const bool valid = u.store && rho < P.RPI && q < P.Wo;
         float* const orow = P.out + ((int64_t)u.img * P.K + n0) * eHoWo + (int64_t)m * P.Wo + q;
         const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)((dr.idx * P.MH + h) * P.NT);
-        store_columns(d_tmem, orow, eHoWo, 0, P.NT, P.K - n0, valid);
+        store_columns(d_tmem, orow, eHoWo, 0, P.NT, P.K - n0, valid, P.two != 0);
       }
       ptx::tc_fence_before();
       __syncwarp();
@@ -592,6 +607,10 @@ int make_wplan(const Geometry& g, WPlan* pl, int pair, int mh_fixed) {
   P.Kp = P.n_ntiles * P.NT;
   if (pair && P.NT % 32 != 0) return IM2WIN_EUNSUPPORTED;  // (each CTA's half of the filter rows: a multiple of 16)
   P.pair = pair;
+  // Two issuing threads where one is the bound: 64-column MMAs take the tensor pipe 54 cycles (their 128-row A
+  // operand is fetched for only 64 columns) but one thread 64 or more to issue; measured: 64-filter layers gain
+  // 10-20 %, wider tiles nothing.
+  P.two = (!pair && (knobs().window_two == 1 || (knobs().window_two == 0 && P.NT <= 64))) ? 1 : 0;
   P.NTB = pair ? P.NT / 2 : P.NT;
   if (SRCK == 1) { P.plane = (int64_t)g.H * g.W; P.n_src = g.n_in; }
   else { P.plane = g.HoL; P.n_src = g.n_win; }
@@ -750,7 +769,7 @@ bool window_preferred(const Geometry& g, const WParams& P) {
   const int64_t span_tiles = (g.Mtot + 127) / 128;
   if (P.n_ntiles == 1 && span_tiles <= nsm && P.NT > 128) return false;  // one wave of the persistent kernel
   if (!BF16) {
-    if (SRCK == 1) return g.C >= 128 && P.NT >= 128 && P.NT <= 192;
+    if (SRCK == 1) return (g.C >= 128 && P.NT >= 128 && P.NT <= 192) || P.NT == 64;
     return P.NT > 64 && P.NT <= 128;
   }
   if (SRCK == 2) return P.NT <= 192;                                   // bf16 im2win tensor

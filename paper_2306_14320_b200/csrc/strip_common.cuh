@@ -158,9 +158,10 @@ __device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
 }
 
 // Stores columns [c_begin, c_end) (multiples of 16) of one warp's 32 accumulator rows: TMEM -> registers
-// -> NCHW.  The TMEM load of the next 16 columns is in flight while the current 16 are stored.
+// -> NCHW.  The TMEM load of the next 16 columns is in flight while the current 16 are stored.  With
+// zero_behind the columns are zeroed once read (kernels whose MMAs all accumulate).
 __device__ __forceinline__ void store_columns(uint32_t d_tmem, float* orow, int64_t HoWo, int32_t c_begin, int32_t c_end,
-                                              int32_t k_left, bool valid) {
+                                              int32_t k_left, bool valid, bool zero_behind = false) {
   uint32_t va[16], vb[16];
   if (c_begin >= c_end) return;
   ptx::tmem_ld_x16(d_tmem + (uint32_t)c_begin, va);
@@ -169,6 +170,7 @@ __device__ __forceinline__ void store_columns(uint32_t d_tmem, float* orow, int6
     ptx::tmem_wait_ld();
     const bool more = c0 + 16 < c_end;
     if (more) ptx::tmem_ld_x16(d_tmem + (uint32_t)(c0 + 16), vb);
+    if (zero_behind) ptx::tmem_zero_x16(d_tmem + (uint32_t)c0);  // (the columns just read: the next unit accumulates onto zeros)
     if (valid) {
       float* o = orow + (int64_t)c0 * HoWo;
       const int32_t left = k_left - c0;
@@ -179,6 +181,7 @@ __device__ __forceinline__ void store_columns(uint32_t d_tmem, float* orow, int6
     if (more) {
       ptx::tmem_wait_ld();
       if (c0 + 32 < c_end) ptx::tmem_ld_x16(d_tmem + (uint32_t)(c0 + 32), va);
+      if (zero_behind) ptx::tmem_zero_x16(d_tmem + (uint32_t)(c0 + 16));
       if (valid) {
         float* o = orow + (int64_t)(c0 + 16) * HoWo;
         const int32_t left = k_left - c0 - 16;
@@ -188,6 +191,7 @@ __device__ __forceinline__ void store_columns(uint32_t d_tmem, float* orow, int6
       }
     }
   }
+  if (zero_behind) ptx::tmem_wait_st();
 }
 
 // ---- host side
