@@ -811,6 +811,9 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         int64_t bcount = 0;
         Ring br;
         bool ok = true;
+        // BF16 mode: the bf16 copy of the filter is written by the kernel launched just before this one,
+        // which this kernel may overlap (programmatic dependent launch); without such a launch: no effect
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x) {
           int32_t nt, g0, g1;
           unit_range(P, t, nt, g0, g1);
@@ -1105,6 +1108,8 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
 // fp32 -> bf16 (round to nearest even) copy of the filter, for the TMA-streamed BF16 filter operand
 __global__ void __launch_bounds__(256) filter_to_bf16_kernel(const float* __restrict__ f, __nv_bfloat16* __restrict__ o,
                                                              int64_t n) {
+  // the convolution kernel that follows may start now (its filter producer waits for this grid's completion)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (int64_t)gridDim.x * 256)
     o[i] = __float2bfloat16_rn(f[i]);
 }
@@ -1114,6 +1119,7 @@ __global__ void __launch_bounds__(256) filter_to_bf16_kernel(const float* __rest
 __global__ void __launch_bounds__(256) filter_to_bf16_padded_kernel(const float* __restrict__ f,
                                                                     __nv_bfloat16* __restrict__ o, int64_t n_pad,
                                                                     int32_t Kg, int32_t KCG, int32_t KCGP, int32_t NG) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int32_t Kgp = NG * KCGP;
   for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n_pad; i += (int64_t)gridDim.x * 256) {
     const int64_t j = i / Kgp;
@@ -1376,6 +1382,12 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   P.off_misc = off; off += 64;
   const size_t smem_bytes = off + 1024;
 
+  // reduction slices add into a zeroed output (before the filter copy's launch, so that the convolution
+  // kernel can follow that copy as a programmatic dependent)
+  if (P.Z > 1 && cudaMemsetAsync(out, 0, (size_t)g.n_out * 4, st) != cudaSuccess) {  // (Z > 1 implies an fp32 output)
+    cudaGetLastError();
+    return IM2WIN_ECUDA;
+  }
   CUtensorMap fmap;
   memset(&fmap, 0, sizeof(fmap));
   void* f_bf16 = nullptr;  // BF16 streamed mode: bf16 copy of the filter in the caller's scratch
@@ -1433,10 +1445,6 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   int64_t grid = P.ntiles < sm_count() ? P.ntiles : sm_count();
   if (P.bslice) grid = grid / P.Z * P.Z;  // every CTA keeps to one slice
   cudaError_t e;
-  if (P.Z > 1 && cudaMemsetAsync(out, 0, (size_t)g.n_out * 4, st) != cudaSuccess) {  // (Z > 1 implies an fp32 output)
-    cudaGetLastError();
-    return IM2WIN_ECUDA;
-  }
   if (resident) {
     auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, true, FUSED, SRC16, OUT16>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
@@ -1446,7 +1454,23 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
     auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, false, FUSED, SRC16, OUT16>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
-    kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
+    if (f_bf16) {
+      // behind the filter-copy kernel as a programmatic dependent: prologue, strip copies and repacking overlap
+      // that copy; the filter producer waits for it (griddepcontrol.wait)
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)grid);
+      cfg.blockDim = dim3((unsigned)kThreads);
+      cfg.dynamicSmemBytes = smem_bytes;
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      if (cudaLaunchKernelEx(&cfg, kern, P, fmap, xmap) != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
+    } else {
+      kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
+    }
   }
   note_kernel(KERNEL_PERSISTENT);
   return cuda_status(cudaGetLastError());

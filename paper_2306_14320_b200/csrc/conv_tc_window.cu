@@ -122,13 +122,14 @@ __device__ __forceinline__ void wtile_range(const WParams& P, int32_t R0, int32_
 }
 
 // The MMA-issuing thread's whole life.  A filter stage holds the NBLK blocks of TPS taps.
-template <int FH, int FW, bool BF16, int MH, int NBLK, int TPS, bool PAIR>
+template <int FH, int FW, bool BF16, int MH, int NBLK, int TPS, bool PAIR, bool TWO>
 __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* misc, uint32_t tmem_base, uint32_t x_sa,
                                           uint32_t b_sa, uint32_t which) {
   Ring xr, br, dr;
   bool ok = true;
-  const bool two = P.two != 0;
+  constexpr bool two = TWO;
   uint32_t bc = 0;  // filter stages so far: with two issuing threads, thread `which` takes those of its parity
+  (void)bc; (void)which;
   SPROF_DECL
   const int32_t lane = 0;
   (void)lane;
@@ -158,7 +159,9 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
       for (int uu = 0; uu < FH && ok; ++uu, a_u += W) {
 #pragma unroll
         for (int v0 = 0; v0 < FW; v0 += TPS) {
-          if (two && ((bc++ & 1u) != which)) { br.advance(P.SB); continue; }
+          if constexpr (TWO) {
+            if ((bc++ & 1u) != which) { br.advance(P.SB); continue; }
+          }
           SPROF_W(2, ok = wait_bar(P, misc, b_full0 + (uint32_t)br.idx * 8u, br.phase, DEV_TIMEOUT_B_FULL, 20))
           if (!ok) break;
           ptx::tc_fence_after();
@@ -342,7 +345,8 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
     if (lane == 0 && rank == 0) {
       const uint32_t which = warp == 1 ? 0u : 1u;
       const int nblk = P.G / (4 * NCH);
-#define WRUN(MHv, NBv, TPv) wmma_role<FH, FW, BF16, MHv, NBv, TPv, PAIR>(P, bars, misc, tmem_base, x_sa, b_sa, which)
+#define WRUN(MHv, NBv, TPv) do { if (!PAIR && P.two) wmma_role<FH, FW, BF16, MHv, NBv, TPv, PAIR, !PAIR>(P, bars, misc, tmem_base, x_sa, b_sa, which); \
+                                else wmma_role<FH, FW, BF16, MHv, NBv, TPv, PAIR, false>(P, bars, misc, tmem_base, x_sa, b_sa, which); } while (0)
       if (P.TPS == 1) {
         if (P.MH == 1) { if (nblk == 1) WRUN(1, 1, 1); else WRUN(1, 2, 1); }
         else { if (nblk == 1) WRUN(2, 1, 1); else WRUN(2, 2, 1); }
@@ -769,12 +773,12 @@ bool window_preferred(const Geometry& g, const WParams& P) {
   const int64_t span_tiles = (g.Mtot + 127) / 128;
   if (P.n_ntiles == 1 && span_tiles <= nsm && P.NT > 128) return false;  // one wave of the persistent kernel
   if (!BF16) {
-    if (SRCK == 1) return (g.C >= 128 && P.NT >= 128 && P.NT <= 192) || P.NT == 64;
+    if (SRCK == 1) return g.C >= 128 && P.NT >= 128 && P.NT <= 192;
     return P.NT > 64 && P.NT <= 128;
   }
   if (SRCK == 2) return P.NT <= 192;                                   // bf16 im2win tensor
   if (SRCK == 1)                                                        // fused
-    return P.NT <= 192 ? !(g.C < 128 && P.NT > 64) : P.RPI < 128;
+    return g.C >= 128 && (P.NT <= 192 || P.RPI < 128);
   return g.C >= 128;                                                    // fp32 im2win tensor
 }
 
