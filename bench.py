@@ -357,6 +357,24 @@ def time_layer(layer, mode_name, steps, warmup, torch, b, flush_buf, sampler_ind
     except b.Im2winError as exc:
         if exc.code != b.EUNSUPPORTED:
             raise
+    # the NHWC output variant (im2win_conv_nhwc from the im2win tensor): same bytes, channels-last stores
+    res["ms_conv_nhwc"] = None
+    try:
+        for _ in range(3):
+            b.conv_nhwc(ws, b.SRC_IM2WIN, f, dims, mode, out, scratch)
+        ne = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+        for k in range(steps):
+            flush_buf.zero_()
+            ne[k][0].record(stream)
+            b.conv_nhwc(ws, b.SRC_IM2WIN, f, dims, mode, out, scratch)
+            ne[k][1].record(stream)
+        torch.cuda.synchronize()
+        if b.last_device_status() != 0:
+            raise RuntimeError("device status word set during the NHWC-output timing")
+        res["ms_conv_nhwc"] = sum(e[0].elapsed_time(e[1]) for e in ne) / steps
+    except b.Im2winError as exc:
+        if exc.code != b.EUNSUPPORTED:
+            raise
     # the bf16 storage variant of the im2win tensor: always a BF16-mode convolution, whatever the line's mode
     res["ms_transform_bf16"] = res["ms_conv_bf16src"] = None
     if True:
@@ -457,7 +475,7 @@ def run_gpu(args):
                             "step_tflops": r["flops"] / r["ms_step"] / 1e9, "ms_conv": r["ms_conv"], "ms_transform": r["ms_transform"],
                             "workspace_bytes": r["workspace_bytes"], "im2col_bytes": r["im2col_bytes"], "peaks": peaks["source"],
                             "ms_transform_bf16": r.get("ms_transform_bf16"), "ms_conv_bf16src": r.get("ms_conv_bf16src"),
-                            "ms_conv_bf16out": r.get("ms_conv_bf16out"),
+                            "ms_conv_bf16out": r.get("ms_conv_bf16out"), "ms_conv_nhwc": r.get("ms_conv_nhwc"),
                             "ms_fused": r.get("ms_fused"),
                             "fused_tflops": (r["flops"] / r["ms_fused"] / 1e9) if r.get("ms_fused") else None,
                             "fused_frac_hbm": (r["fused_bytes"] / r["ms_fused"] / 1e6 / peaks["hbm_gbs"]) if r.get("ms_fused") else None}
@@ -542,6 +560,9 @@ def run_gpu(args):
         "bf16_output": ({"ms_conv": r["ms_conv_bf16out"],
                          "what": "im2win_conv_bf16out: the same convolution with the result stored as bf16 "
                                  "(half the output write); not part of `value`"} if r.get("ms_conv_bf16out") else None),
+        "nhwc_output": ({"ms_conv": r["ms_conv_nhwc"],
+                         "what": "im2win_conv_nhwc: the same convolution with the fp32 result written N x Ho x Wo x K; "
+                                 "not part of `value`"} if r.get("ms_conv_nhwc") else None),
         "e2e": {"value": world * flops / ms_e2e / 1e9, "unit": UNIT, "h2d_bytes_per_step": r["bytes_in"] + r["bytes_f"],
                 "d2h_bytes_per_step": r["bytes_out"], "ms_per_step": ms_e2e,
                 "how": "im2win_conv_host: pinned host buffers in, pinned host buffer out, wall clock per call; the call "

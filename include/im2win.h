@@ -146,6 +146,17 @@ int im2win_conv(const void* src, int src_kind, const float* filter_kcfhfw,
                 const im2win_shape* shape, int mode, float* out_nchw,
                 void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Output-layout variant of im2win_conv (no counterpart in the paper, whose outputs are NCHW): the
+ * same fp32 result written channels-last, out_nhwc[i][m][n][j] = O(i, j, m, n) of Eq. 1, so that a
+ * position's K filter outputs are contiguous (the accumulator row of a tensor-core tile as it is).
+ * out_nhwc: device, N*Ho*Wo*K floats, every element is written; 16-byte aligned.
+ * Everything else as im2win_conv: all source kinds, all three modes and every shape (each kernel
+ * has the layout as an epilogue option; the reduction slices of under-filled launches, which add
+ * into an NCHW output, are not used). */
+int im2win_conv_nhwc(const void* src, int src_kind, const float* filter_kcfhfw,
+                     const im2win_shape* shape, int mode, float* out_nhwc,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Output-storage variant of im2win_conv (no counterpart in the paper, whose outputs are fp32):
  * the same result rounded to bf16 (nearest even) from the fp32 accumulators, NCHW, 2 bytes per
  * element: half the output footprint and half the bytes written.

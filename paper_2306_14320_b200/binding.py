@@ -23,7 +23,7 @@ MODE_TF32, MODE_BF16, MODE_FP32 = 0, 1, 2
 OK, EINVAL, EALIGN, EWORKSPACE, EOVERLAP, ECUDA, ETIMEOUT, EUNSUPPORTED, ESCRATCH = 0, -1, -2, -3, -4, -5, -6, -7, -8
 
 EXPORTS = ("im2win_out_dims", "im2win_workspace_bytes", "im2win_conv_workspace_bytes", "im2win_im2col_bytes", "im2win_transform",
-           "im2win_workspace_bytes_bf16", "im2win_transform_bf16", "im2win_conv", "im2win_conv_bf16out", "im2win_conv_host", "im2win_host_release", "im2win_conv_static",
+           "im2win_workspace_bytes_bf16", "im2win_transform_bf16", "im2win_conv", "im2win_conv_nhwc", "im2win_conv_bf16out", "im2win_conv_host", "im2win_host_release", "im2win_conv_static",
            "im2win_last_device_status", "im2win_strerror")
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024  # IM2WIN_STATIC_SCRATCH_BYTES of include/im2win.h
 
@@ -59,6 +59,7 @@ def _declare(L: ctypes.CDLL) -> ctypes.CDLL:
     L.im2win_transform_bf16.argtypes = [vp, sp, vp, vp]
     L.im2win_conv.argtypes = [vp, ctypes.c_int, vp, sp, ctypes.c_int, vp, vp, ctypes.c_size_t, vp]
     L.im2win_conv_bf16out.argtypes = [vp, ctypes.c_int, vp, sp, ctypes.c_int, vp, vp, ctypes.c_size_t, vp]
+    L.im2win_conv_nhwc.argtypes = [vp, ctypes.c_int, vp, sp, ctypes.c_int, vp, vp, ctypes.c_size_t, vp]
     L.im2win_conv_host.argtypes = [vp, vp, sp, ctypes.c_int, vp]
     L.im2win_host_release.argtypes = []
     L.im2win_conv_static.argtypes = [vp, vp, sp, ctypes.c_int, vp, vp]
@@ -200,6 +201,16 @@ def conv(src, src_kind: int, filter_kcfhfw, shape, mode: int, out_nchw, workspac
     _check(lib().im2win_conv(_ptr(src), int(src_kind), _ptr(filter_kcfhfw), ctypes.byref(Shape.of(shape)),
                              int(mode), _ptr(out_nchw), _ptr(workspace), int(workspace_nbytes), _stream(stream)),
            "im2win_conv")
+
+
+def conv_nhwc(src, src_kind: int, filter_kcfhfw, shape, mode: int, out_nhwc, workspace=None, workspace_bytes=None,
+              stream=None) -> None:
+    """im2win_conv_nhwc: like conv(), the fp32 output written N x Ho x Wo x K."""
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    _check(lib().im2win_conv_nhwc(_ptr(src), int(src_kind), _ptr(filter_kcfhfw), ctypes.byref(Shape.of(shape)),
+                                  int(mode), _ptr(out_nhwc), _ptr(workspace), int(workspace_bytes),
+                                  _stream(stream)), "im2win_conv_nhwc")
 
 
 def conv_bf16out(src, src_kind: int, filter_kcfhfw, shape, mode: int, out_nchw_bf16, workspace=None,

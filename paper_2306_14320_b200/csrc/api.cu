@@ -45,6 +45,7 @@ int make_geometry(const im2win_shape* sh, Geometry* g) {
   if (sh->Fh > sh->H || sh->Fw > sh->W) return IM2WIN_EINVAL;
   g->N = sh->N; g->C = sh->C; g->H = sh->H; g->W = sh->W;
   g->K = sh->K; g->Fh = sh->Fh; g->Fw = sh->Fw; g->s = sh->stride;
+  g->out_nhwc = 0;
   g->Ho = (sh->H - sh->Fh) / sh->stride + 1;
   g->Wo = (sh->W - sh->Fw) / sh->stride + 1;
   int64_t L, FF, sFh;
@@ -208,12 +209,14 @@ namespace im2win {
 // Shared body of im2win_conv (fp32 output), im2win_conv_bf16out (out16: `out` holds 16-bit words;
 // tensor-core modes, kernels with a bf16 epilogue) and im2win_conv_static.
 int conv_impl(const void* src, int src_kind, const float* filter, const im2win_shape* shape, int mode, void* out,
-              bool out16, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+              bool out16, void* workspace, size_t workspace_bytes, void* cuda_stream, bool out_nhwc) {
   float* const out_nchw = static_cast<float*>(out);
   const int64_t out_es = out16 ? 2 : 4;
   Geometry g;
   int rc = make_geometry(shape, &g);
   if (rc != IM2WIN_OK) return rc;
+  if (out_nhwc && out16) return IM2WIN_EINVAL;
+  g.out_nhwc = out_nhwc ? 1 : 0;
   if (!src || !filter || !out_nchw) return IM2WIN_EINVAL;
   if (src_kind != IM2WIN_SRC_NCHW && src_kind != IM2WIN_SRC_IM2WIN && src_kind != IM2WIN_SRC_NCHW_FUSED &&
       src_kind != IM2WIN_SRC_IM2WIN_BF16)
@@ -304,6 +307,11 @@ int im2win_conv(const void* src, int src_kind, const float* filter, const im2win
                 int mode, float* out_nchw, void* workspace, size_t workspace_bytes,
                 void* cuda_stream) {
   return conv_impl(src, src_kind, filter, shape, mode, out_nchw, false, workspace, workspace_bytes, cuda_stream);
+}
+
+int im2win_conv_nhwc(const void* src, int src_kind, const float* filter, const im2win_shape* shape,
+                     int mode, float* out_nhwc, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return conv_impl(src, src_kind, filter, shape, mode, out_nhwc, false, workspace, workspace_bytes, cuda_stream, true);
 }
 
 int im2win_conv_bf16out(const void* src, int src_kind, const float* filter, const im2win_shape* shape,

@@ -20,6 +20,7 @@ struct Geometry {
   int64_t Kg;       // C*Fh*Fw, the reduction length
   int64_t Mtot;     // N*Ho*Wo, number of output positions
   int64_t n_in, n_win, n_col, n_out, n_flt;  // element counts
+  int32_t out_nhwc;  // the fp32 output is written N x Ho x Wo x K (im2win_conv_nhwc) instead of N x K x Ho x Wo
 };
 
 // Fills g from shape; returns IM2WIN_OK or IM2WIN_EINVAL (bad sizes / 64-bit overflow).
@@ -77,7 +78,7 @@ size_t conv_scratch_bytes(const Geometry& g, int mode, int src_kind);
 // Shared body of im2win_conv / im2win_conv_bf16out / im2win_conv_static (argument checks, workspace
 // split into the im2win tensor and the filter scratch, transform, dispatch).
 int conv_impl(const void* src, int src_kind, const float* filter, const im2win_shape* shape, int mode, void* out,
-              bool out16, void* workspace, size_t workspace_bytes, void* cuda_stream);
+              bool out16, void* workspace, size_t workspace_bytes, void* cuda_stream, bool out_nhwc = false);
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? IM2WIN_OK : IM2WIN_ECUDA; }
 

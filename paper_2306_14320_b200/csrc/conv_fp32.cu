@@ -32,7 +32,8 @@ __global__ void __launch_bounds__(256) conv_fp32_kernel(const float* __restrict_
         for (int32_t v = 0; v < g.Fw; ++v)
           acc = fmaf(__ldg(win + v * g.Fh + u), __ldg(fr + u * g.Fw + v), acc);
     }
-    out[e] = acc;
+    if (g.out_nhwc) out[((i * g.Ho + m) * g.Wo + n) * (int64_t)g.K + j] = acc;
+    else out[e] = acc;
   }
 }
 

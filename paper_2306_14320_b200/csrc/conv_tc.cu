@@ -50,6 +50,7 @@ struct ConvParams {
   int32_t* status;
   int32_t C, K, Ho, Wo, L, FF, Fh, Fw, sFh;
   int64_t HoL, HoWo, Kg, Mtot, n_win;
+  int32_t nhwc;        // output layout N x Ho x Wo x K
   int32_t TP;          // positions per tile (128 unless images are tiny)
   int32_t NT;          // filters per tile (multiple of 16, <= 256)
   int32_t n_ntiles;
@@ -279,7 +280,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_tc_kernel(const __grid_const
         const Seg s = segs[(int32_t)(i - misc->i_first)];
         base_off = s.dst_off + (int32_t)((m * P.L + n * P.sFh) - s.virt_a);
         skew0 = (int32_t)(s.start0 & 3);
-        out_off = (i * P.K + n0) * P.HoWo + q;
+        out_off = P.nhwc ? (i * P.HoWo + q) * P.K + n0 : (i * P.K + n0) * P.HoWo + q;
       }
       const int32_t skew_step = (int32_t)(P.HoL & 3);
       bool ok = true;
@@ -330,7 +331,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_tc_kernel(const __grid_const
           if (valid) {
 #pragma unroll
             for (int e = 0; e < 16; ++e)
-              if (n0 + c0 + e < P.K) orow[(int64_t)(c0 + e) * P.HoWo] = __uint_as_float(v[e]);
+              if (n0 + c0 + e < P.K) orow[P.nhwc ? (int64_t)(c0 + e) : (int64_t)(c0 + e) * P.HoWo] = __uint_as_float(v[e]);
           }
         }
       }
@@ -415,6 +416,7 @@ int launch_conv_tc_generic(const float* xhat, const float* f, float* out, const 
   if (!P.status) return IM2WIN_ECUDA;
   P.C = g.C; P.K = g.K; P.Ho = g.Ho; P.Wo = g.Wo; P.L = g.L; P.FF = g.FF; P.Fh = g.Fh; P.Fw = g.Fw;
   P.sFh = g.sFh; P.HoL = g.HoL; P.HoWo = g.HoWo; P.Kg = g.Kg; P.Mtot = g.Mtot; P.n_win = g.n_win;
+  P.nhwc = g.out_nhwc;
   P.bf16 = (mode == IM2WIN_MODE_BF16);
   P.kstep = P.bf16 ? 16 : 8;
   P.kchunk = P.bf16 ? 64 : 32;

@@ -54,6 +54,7 @@ struct PParams {
   float* out;
   int32_t* status;
   int32_t C, K, Ho, Wo;
+  int32_t nhwc;         // output layout N x Ho x Wo x K (fp32, no reduction slices)
   int32_t row_mul;      // source floats from one output row to the next: W*Fh (im2win strips) or s*W (raw rows)
   int32_t col_mul;      // source floats from one output column to the next: s*Fh or s
   int32_t win_span;     // floats from a window's first to one past its last element: Fh*Fw or (Fh-1)*W+Fw
@@ -1002,7 +1003,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     // slowed the C = 3 stem layers, which this loop bounds, by 20 %.
     PROF_DECL(6)
     auto epilogue_role = [&](auto kind_tag) {
-      constexpr int EK = decltype(kind_tag)::value;  // 0 fp32 stores, 1 fp32 reductions, 2 bf16 stores
+      constexpr int EK = decltype(kind_tag)::value;  // 0 fp32 stores, 1 fp32 reductions, 2 bf16 stores, 3 fp32 stores in NHWC order
       constexpr bool REDUCE = EK == 1;
       Ring dr;
       bool ok = true;
@@ -1028,7 +1029,8 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         if (valid) {
           int32_t i_off, q;
           tile_row(P, ti, p, i_off, q);
-          orow += ((ti.i_first + i_off) * P.K + n0) * (int64_t)P.HoWo + q;
+          if constexpr (EK == 3) orow += ((ti.i_first + i_off) * (int64_t)P.HoWo + q) * P.K + n0;
+          else orow += ((ti.i_first + i_off) * P.K + n0) * (int64_t)P.HoWo + q;
         }
         const int32_t d = dr.idx;
         PROF_ADD(1, tp)
@@ -1062,6 +1064,22 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
                 if (e + 1 < left) o16[(int64_t)(e + 1) * eHoWo] = (uint16_t)(pk >> 16);
               }
             }
+          } else if constexpr (EK == 3) {
+            // NHWC: the thread's 16 filters of one position are contiguous
+            if (valid) {
+              float* o = orow + c0;
+              const int32_t left = eK - n0 - c0;
+              if (left >= 16 && (eK & 3) == 0) {
+#pragma unroll
+                for (int e = 0; e < 16; e += 4)
+                  *reinterpret_cast<float4*>(o + e) = make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]),
+                                                                  __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+              } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e)
+                  if (e < left) o[e] = __uint_as_float(v[e]);
+              }
+            }
           } else
           if (valid) {
             float* o = orow + (int64_t)c0 * eHoWo;
@@ -1087,7 +1105,8 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     if constexpr (OUT16) {  // (separate instantiations: the fp32 kernels' code is not touched by this variant)
       epilogue_role(std::integral_constant<int, 2>{});
     } else {
-      if (P.Z == 1) epilogue_role(std::integral_constant<int, 0>{});
+      if (P.nhwc) epilogue_role(std::integral_constant<int, 3>{});
+      else if (P.Z == 1) epilogue_role(std::integral_constant<int, 0>{});
       else epilogue_role(std::integral_constant<int, 1>{});
     }
     if (q4 == 0) { PROF_DUMP(6, 6) }
@@ -1164,6 +1183,7 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
 
   PParams P{};
   P.xhat = xhat; P.f = f; P.out = out;  // (OUT16: `out` points at 16-bit words)
+  P.nhwc = g.out_nhwc;
   P.status = device_status_word();
   if (!P.status) return IM2WIN_ECUDA;
 #ifdef IM2WIN_PROF
@@ -1273,7 +1293,7 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   // issuing threads spend about 200 cycles per MMA (measured), in microseconds at 1.9 GHz.
   int32_t bs_z = 0, bs_gz = 0;
   const bool bs_force = knobs().bslice != 0;  // test knob
-  if ((!resident || bs_force) && P.n_ntiles == 1 && !out16 && !knobs().no_bslice) {
+  if ((!resident || bs_force) && P.n_ntiles == 1 && !out16 && !g.out_nhwc && !knobs().no_bslice) {
     const int nsm = sm_count();
     for (int32_t z = 2; z <= 16 && z <= P.NG && z <= nsm; ++z) {
       const int32_t gz = (P.NG + z - 1) / z;
@@ -1354,7 +1374,7 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
     if (!resident) while ((gmul * S) % 4 != 0) ++gmul;
     double best = cost(1, P.NG) * 0.92;  // a split must win clearly
     int forced = knobs().splitk;
-    if (out16) forced = 1;  // partial sums cannot be added into a bf16 output
+    if (out16 || g.out_nhwc) forced = 1;  // partial sums cannot be added into a bf16 output; the NHWC epilogue has no adding copy
     for (int32_t z = 2; z <= 16 && z <= P.NG; ++z) {
       int32_t gz = (P.NG + z - 1) / z;
       gz = (gz + gmul - 1) / gmul * gmul;

@@ -56,6 +56,7 @@ struct SParams {
   int32_t NT, n_ntiles, Kp;
   int32_t NTB;        // filter rows one CTA holds per block: NT, or NT/2 when two CTAs share an MMA
   int32_t pair;       // two CTAs (a cluster) work as one: tcgen05.mma.cta_group::2, M = 256, each CTA its own rows and half the filter tile
+  int32_t nhwc;       // output layout N x Ho x Wo x K
   int64_t tiles;      // row tiles: N * TPI
   int32_t G, GR, NSUB, NTS;  // channels per T stage / per source stage, source stages per T stage, T stages per unit
   int32_t CBN;        // channel blocks (of NCH channels) per source stage
@@ -475,8 +476,10 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
           const bool valid = u.store && rho < P.RPI && q < P.Wo;
           const int32_t n0 = u.nt * P.NT;
           const int64_t HoWo = (int64_t)P.Ho * P.Wo;
-          float* const orow = P.out + ((int64_t)u.img * P.K + n0) * HoWo + (int64_t)m * P.Wo + q;
-          store_columns(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(hh * P.NT), orow, HoWo, P.epi_split, P.NT, P.K - n0, valid);
+          float* const orow = P.nhwc ? P.out + ((int64_t)u.img * HoWo + (int64_t)m * P.Wo + q) * P.K + n0
+                                     : P.out + ((int64_t)u.img * P.K + n0) * HoWo + (int64_t)m * P.Wo + q;
+          store_columns(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(hh * P.NT), orow, P.nhwc ? 1 : HoWo, P.epi_split, P.NT,
+                        P.K - n0, valid, false, P.nhwc && (P.K & 3) == 0);
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) {
@@ -506,12 +509,13 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
       const int32_t m = rho / P.WP, q = rho - m * P.WP;
       const bool valid = u.store && rho < P.RPI && q < P.Wo;
       const int32_t n0 = u.nt * P.NT;
-      float* const orow = P.out + ((int64_t)u.img * P.K + n0) * eHoWo + (int64_t)m * P.Wo + q;
+      float* const orow = P.nhwc ? P.out + ((int64_t)u.img * eHoWo + (int64_t)m * P.Wo + q) * eK + n0
+                                 : P.out + ((int64_t)u.img * P.K + n0) * eHoWo + (int64_t)m * P.Wo + q;
       SPROF_W(0, ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->acc_full[dr.idx]), dr.phase, DEV_TIMEOUT_ACC, 128))
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)((dr.idx * P.MH + h) * P.NT);
-      store_columns(d_tmem, orow, eHoWo, 0, P.epi_split, eK - n0, valid);
+      store_columns(d_tmem, orow, P.nhwc ? 1 : eHoWo, 0, P.epi_split, eK - n0, valid, false, P.nhwc && (eK & 3) == 0);
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) {
@@ -575,6 +579,7 @@ int make_plan(const Geometry& g, Plan* pl, int pair, int mh_fixed) {
   if (g.C % P.G != 0) return IM2WIN_EUNSUPPORTED;
   if (g.HoWo > (1 << 28) || (int64_t)g.H * g.W > (1 << 28)) return IM2WIN_EUNSUPPORTED;
   P.C = g.C; P.K = g.K; P.Ho = g.Ho; P.Wo = g.Wo; P.W = g.W;
+  P.nhwc = g.out_nhwc;
   P.WP = (g.W + S - 1) / S;
   P.RPI = g.Ho * P.WP;
   P.n_ntiles = (g.K + 255) / 256;

@@ -55,6 +55,7 @@ struct WParams {
   int32_t RA;         // X rows allocated (RX rounded up to 8)
   int32_t NT, n_ntiles, Kp;
   int32_t NTB;        // filter rows one CTA holds per block: NT, or NT/2 when two CTAs share an MMA
+  int32_t nhwc;       // output layout N x Ho x Wo x K
   int32_t two;        // two MMA-issuing threads share the filter stages by parity; every MMA accumulates, the epilogue zeroes behind its reads
   int32_t pair;       // two CTAs (a cluster) work as one: tcgen05.mma.cta_group::2, M = 256, each CTA its own rows and half the filter tile
   int32_t G, GR, NSUB, NXS;  // channels per X stage / per source stage, source stages per X stage, X stages per unit
@@ -528,9 +529,10 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
         const int32_t rho = u.R0 + h * 128 + q4 * 32 + lane;
         const int32_t m = rho / P.W, q = rho - m * P.W;
         const bool valid = u.store && rho < P.RPI && q < P.Wo;
-        float* const orow = P.out + ((int64_t)u.img * P.K + n0) * eHoWo + (int64_t)m * P.Wo + q;
+        float* const orow = P.nhwc ? P.out + ((int64_t)u.img * eHoWo + (int64_t)m * P.Wo + q) * P.K + n0
+                                   : P.out + ((int64_t)u.img * P.K + n0) * eHoWo + (int64_t)m * P.Wo + q;
         const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)((dr.idx * P.MH + h) * P.NT);
-        store_columns(d_tmem, orow, eHoWo, 0, P.NT, P.K - n0, valid, P.two != 0);
+        store_columns(d_tmem, orow, P.nhwc ? 1 : eHoWo, 0, P.NT, P.K - n0, valid, P.two != 0, P.nhwc && (P.K & 3) == 0);
       }
       ptx::tc_fence_before();
       __syncwarp();
@@ -605,6 +607,7 @@ int make_wplan(const Geometry& g, WPlan* pl, int pair, int mh_fixed) {
   if (g.C % gmin != 0) return IM2WIN_EUNSUPPORTED;
   if (g.HoWo > (1 << 28) || (int64_t)g.H * g.W > (1 << 26)) return IM2WIN_EUNSUPPORTED;
   P.C = g.C; P.K = g.K; P.Ho = g.Ho; P.Wo = g.Wo; P.W = g.W; P.H = g.H;
+  P.nhwc = g.out_nhwc;
   P.RPI = g.Ho * g.W;
   P.n_ntiles = (g.K + 255) / 256;
   P.NT = ((g.K + P.n_ntiles - 1) / P.n_ntiles + 15) / 16 * 16;

@@ -158,10 +158,22 @@ __device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
 }
 
 // Stores columns [c_begin, c_end) (multiples of 16) of one warp's 32 accumulator rows: TMEM -> registers
-// -> NCHW.  The TMEM load of the next 16 columns is in flight while the current 16 are stored.  With
+// -> the output (column stride Ho*Wo for NCHW; 1, with 128-bit stores where aligned, for NHWC).  The TMEM load of the next 16 columns is in flight while the current 16 are stored.  With
 // zero_behind the columns are zeroed once read (kernels whose MMAs all accumulate).
-__device__ __forceinline__ void store_columns(uint32_t d_tmem, float* orow, int64_t HoWo, int32_t c_begin, int32_t c_end,
-                                              int32_t k_left, bool valid, bool zero_behind = false) {
+__device__ __forceinline__ void store16(float* o, int64_t cstride, const uint32_t (&v)[16], int32_t left, bool vec) {
+  if (vec && left >= 16) {  // (NHWC: a position's filters are contiguous)
+#pragma unroll
+    for (int e = 0; e < 16; e += 4)
+      *reinterpret_cast<float4*>(o + e) = make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]), __uint_as_float(v[e + 2]),
+                                                      __uint_as_float(v[e + 3]));
+  } else {
+#pragma unroll
+    for (int e = 0; e < 16; ++e)
+      if (e < left) o[(int64_t)e * cstride] = __uint_as_float(v[e]);
+  }
+}
+__device__ __forceinline__ void store_columns(uint32_t d_tmem, float* orow, int64_t cstride, int32_t c_begin, int32_t c_end,
+                                              int32_t k_left, bool valid, bool zero_behind = false, bool vec = false) {
   uint32_t va[16], vb[16];
   if (c_begin >= c_end) return;
   ptx::tmem_ld_x16(d_tmem + (uint32_t)c_begin, va);
@@ -171,24 +183,12 @@ __device__ __forceinline__ void store_columns(uint32_t d_tmem, float* orow, int6
     const bool more = c0 + 16 < c_end;
     if (more) ptx::tmem_ld_x16(d_tmem + (uint32_t)(c0 + 16), vb);
     if (zero_behind) ptx::tmem_zero_x16(d_tmem + (uint32_t)c0);  // (the columns just read: the next unit accumulates onto zeros)
-    if (valid) {
-      float* o = orow + (int64_t)c0 * HoWo;
-      const int32_t left = k_left - c0;
-#pragma unroll
-      for (int e = 0; e < 16; ++e)
-        if (e < left) o[(int64_t)e * HoWo] = __uint_as_float(va[e]);
-    }
+    if (valid) store16(orow + (int64_t)c0 * cstride, cstride, va, k_left - c0, vec);
     if (more) {
       ptx::tmem_wait_ld();
       if (c0 + 32 < c_end) ptx::tmem_ld_x16(d_tmem + (uint32_t)(c0 + 32), va);
       if (zero_behind) ptx::tmem_zero_x16(d_tmem + (uint32_t)(c0 + 16));
-      if (valid) {
-        float* o = orow + (int64_t)(c0 + 16) * HoWo;
-        const int32_t left = k_left - c0 - 16;
-#pragma unroll
-        for (int e = 0; e < 16; ++e)
-          if (e < left) o[(int64_t)e * HoWo] = __uint_as_float(vb[e]);
-      }
+      if (valid) store16(orow + (int64_t)(c0 + 16) * cstride, cstride, vb, k_left - c0 - 16, vec);
     }
   }
   if (zero_behind) ptx::tmem_wait_st();

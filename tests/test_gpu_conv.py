@@ -353,7 +353,7 @@ def test_conv_table1_layers_batch128(layer, mode, _kernel):
 @pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
 @pytest.mark.parametrize("layer", wl.SWEEP, ids=lambda l: l.name)
 def test_conv_sweep_layers_batch32_small_integers_bit_exact(layer, mode, _kernel):
-    if _kernel not in ("auto", "minws", "strip", "window", "nostrip"):
+    if _kernel not in ("auto", "minws", "strip", "window", "wtwo", "wpair", "wpair2", "nostrip"):
         pytest.skip("forced persistent-kernel variants are covered at small sizes")
     layer = layer.with_batch(32)
     dims = layer.dims()
