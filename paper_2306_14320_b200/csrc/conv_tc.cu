@@ -116,7 +116,7 @@ __device__ __forceinline__ bool wait_bar(const ConvParams& P, Misc* misc, uint64
   return false;
 }
 
-// The same for a whole warp: every lane polls, the verdict is made uniform so that the
+// The same for a whole warp: every lane polls, the outcome is made uniform so that the
 // warp-collective tcgen05 instructions that follow run converged.
 __device__ __forceinline__ bool wait_bar_warp(const ConvParams& P, Misc* misc, uint64_t* bar, uint32_t parity,
                                               int32_t code) {
