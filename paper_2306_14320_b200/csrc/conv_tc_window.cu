@@ -62,6 +62,8 @@ struct WParams {
   int32_t TPS;        // taps per filter stage (Fw: one filter row per stage; 1: one tap per stage)
   int32_t SR, SB, ND;
   int32_t n_epi;      // epilogue warps in use
+  int32_t epi_split;  // the epilogue warps store columns [0, epi_split); with one accumulator buffer the (then idle)
+                      // interleaver warps store [epi_split, NT); epi_split == NT: no help
   int32_t box;        // source stages come as 2-D TMA boxes
   int32_t NBX, BXE;   // boxes per source stage; elements per box row (bulk copies: one "box" of CP elements)
   int32_t pm;         // plane length modulo the elements of a 16-byte chunk (bulk copies: per-channel phase)
@@ -245,7 +247,7 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
       ptx::mbar_init(ptx::smem_u32(&bars->t_full[i]), kTW * kShare);
       ptx::mbar_init(ptx::smem_u32(&bars->t_empty[i]), 1u + (uint32_t)P.two);
       ptx::mbar_init(ptx::smem_u32(&bars->acc_full[i]), 1u + (uint32_t)P.two);
-      ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), (uint32_t)P.n_epi * kShare);
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[i]), (uint32_t)P.n_epi * kShare * (P.epi_split < P.NT ? 2u : 1u));
     }
     ptx::fence_mbar_init();
     misc->abort = 0;
@@ -411,6 +413,7 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
     bool ok = true;
     SPROF_DECL
     const uint32_t x_full_lead0 = remote ? mapa(ptx::smem_u32(&bars->t_full[0]), 0) : ptx::smem_u32(&bars->t_full[0]);
+    uint32_t hphase = 0;  // (epilogue help) phase of the single accumulator buffer's "full" barrier
     for (int64_t it = 0; ok; ++it) {
       WUnit u;
       if (!wunit_at<PAIR>(P, it, rank, u)) break;
@@ -507,6 +510,33 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
           }
         }
       }
+      // One accumulator buffer: the next unit's MMAs cannot start before this unit's results are stored, so
+      // this warp stores the upper columns of its TMEM lane quarter meanwhile.
+      if (ok && P.epi_split < P.NT) {
+        const int32_t hh = (warp - kTWarp0) >> 2, q4 = warp & 3;
+        ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->acc_full[0]), hphase, DEV_TIMEOUT_ACC, 128);
+        if (!ok) break;
+        hphase ^= 1u;
+        ptx::tc_fence_after();
+        if (hh < P.MH) {
+          const int32_t rho = u.R0 + hh * 128 + q4 * 32 + lane;
+          const int32_t m = rho / P.W, q = rho - m * P.W;
+          const bool valid = u.store && rho < P.RPI && q < P.Wo;
+          const int32_t n0 = u.nt * P.NT;
+          const int64_t HoWo = (int64_t)P.Ho * P.Wo;
+          float* const orow = P.nhwc ? P.out + ((int64_t)u.img * HoWo + (int64_t)m * P.Wo + q) * P.K + n0
+                                     : P.out + ((int64_t)u.img * P.K + n0) * HoWo + (int64_t)m * P.Wo + q;
+          store_columns(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(hh * P.NT), orow, P.nhwc ? 1 : HoWo, P.epi_split, P.NT,
+                        P.K - n0, valid, false, P.nhwc && (P.K & 3) == 0);
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            const uint32_t ae = ptx::smem_u32(&bars->acc_empty[0]);
+            if (remote) arrive_cluster(mapa(ae, 0));
+            else ptx::mbar_arrive(ae);
+          }
+        }
+      }
     }
     if (warp == kTWarp0) { SPROF_DUMP(2) }
   } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + P.n_epi) {
@@ -532,7 +562,7 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
         float* const orow = P.nhwc ? P.out + ((int64_t)u.img * eHoWo + (int64_t)m * P.Wo + q) * P.K + n0
                                    : P.out + ((int64_t)u.img * P.K + n0) * eHoWo + (int64_t)m * P.Wo + q;
         const uint32_t d_tmem = tmem_base + lane_base + (uint32_t)((dr.idx * P.MH + h) * P.NT);
-        store_columns(d_tmem, orow, P.nhwc ? 1 : eHoWo, 0, P.NT, P.K - n0, valid, P.two != 0, P.nhwc && (P.K & 3) == 0);
+        store_columns(d_tmem, orow, P.nhwc ? 1 : eHoWo, 0, P.epi_split, P.K - n0, valid, P.two != 0, P.nhwc && (P.K & 3) == 0);
       }
       ptx::tc_fence_before();
       __syncwarp();
@@ -633,6 +663,9 @@ int make_wplan(const Geometry& g, WPlan* pl, int pair, int mh_fixed) {
   P.units = pair ? ((P.tiles + 1) / 2) * P.n_ntiles : P.tiles * P.n_ntiles;
   P.ND = 512 / (P.MH * P.NT) >= 2 ? 2 : 1;
   P.n_epi = 4 * (P.MH < 2 ? P.MH : 2);
+  // one accumulator buffer: the interleaver warps (two sets of four, one per block) store the upper half of the
+  // columns; with one block per tile only the first set could help, so the epilogue warps keep all columns
+  P.epi_split = (P.ND == 1 && P.MH == 2 && P.NT >= 64 && !knobs().window_nohelp) ? (P.NT / 2 + 15) / 16 * 16 : P.NT;
   // source elements of one channel a tile needs at most, plus the 16-byte phase in front
   const int64_t len_max = SRCK == 1 ? P.RX : (int64_t)FH * (128 * P.MH + g.W);
   int64_t cp = len_max + 2 * EPC;
@@ -772,7 +805,7 @@ template <int FH, int FW, bool BF16, int SRCK>
 bool window_preferred(const Geometry& g, const WParams& P) {
   const int nsm = sm_count();
   if (P.units * 2 <= nsm) return false;  // under-filled launches: the persistent kernel's reduction slices
-  if (FH == 5) return BF16;               // 5x5 layers: 25 taps of one staged tile
+  if (FH == 5) return BF16 || SRCK == 0;  // 5x5 layers: 25 taps of one staged tile (TF32: from the tensor only)
   const int64_t span_tiles = (g.Mtot + 127) / 128;
   if (P.n_ntiles == 1 && span_tiles <= nsm && P.NT > 128) return false;  // one wave of the persistent kernel
   if (!BF16) {
