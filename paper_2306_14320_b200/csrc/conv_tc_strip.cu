@@ -539,21 +539,46 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
 
 // Tap-major copy of the filter for the TMA-streamed B operand:
 //   Fv[v][j][r*Fh + u] = F[j][r][u][v]   (j < K; rows K..Kp-1 are zero), fp32 or bf16 (nearest even).
-// One block row per (v, j): no division but the one by the (small) filter height.
+// One CTA per (filter j, block of 128 channels): its 128*Fh*Fw values pass through shared memory, so that both
+// the reads and the writes are contiguous and every CTA is one load - store round trip (the convolution
+// kernel's first MMA waits for this copy: its latency counts).
+constexpr int kPrepCh = 128, kPrepFF = 9;
 template <bool BF16>
-__global__ void __launch_bounds__(256) filter_tap_major_kernel(const float* __restrict__ f, void* __restrict__ o, int32_t K,
-                                                               int32_t Kp, int32_t row, int32_t FH, int32_t FW) {
+__global__ void __launch_bounds__(128) filter_tap_major_kernel(const float* __restrict__ f, void* __restrict__ o, int32_t K,
+                                                               int32_t Kp, int32_t C, int32_t FH, int32_t FW) {
   // the convolution kernel that follows may start its prologue now (it waits for this grid's completion
   // before it reads the copy)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  const int32_t vj = (int32_t)blockIdx.y;
-  const int32_t v = vj / Kp, j = vj - v * Kp;
-  const float* fj = f + (int64_t)j * row * FW + v;
-  const int64_t obase = (int64_t)vj * row;
-  for (int32_t ku = (int32_t)(blockIdx.x * 256 + threadIdx.x); ku < row; ku += (int32_t)gridDim.x * 256) {
-    const float x = j < K ? __ldg(fj + (int64_t)ku * FW) : 0.f;   // (r*Fh + u)*Fw + v = ku*Fw + v
-    if (BF16) static_cast<__nv_bfloat16*>(o)[obase + ku] = __float2bfloat16_rn(x);
-    else static_cast<float*>(o)[obase + ku] = x;
+  __shared__ float sm[kPrepCh * kPrepFF];
+  const int32_t j = (int32_t)blockIdx.x, tid = (int32_t)threadIdx.x;
+  const int32_t c0 = (int32_t)blockIdx.y * kPrepCh;
+  const int32_t nc = min(kPrepCh, C - c0);
+  const int32_t ff = FH * FW, n = nc * ff;
+  const float* fj = f + ((int64_t)j * C + c0) * ff;
+  if (j < K) {
+    float x[kPrepFF];
+#pragma unroll
+    for (int q = 0; q < kPrepFF; ++q) {  // (all loads in flight before the first use)
+      const int32_t i = tid + q * 128;
+      x[q] = (q < ff && i < n) ? __ldg(fj + i) : 0.f;
+    }
+#pragma unroll
+    for (int q = 0; q < kPrepFF; ++q) {
+      const int32_t i = tid + q * 128;
+      if (q < ff && i < n) sm[i] = x[q];
+    }
+  } else {
+    for (int32_t i = tid; i < n; i += 128) sm[i] = 0.f;
+  }
+  __syncthreads();
+  const int32_t row = C * FH, nku = nc * FH;
+  for (int32_t v = 0; v < FW; ++v) {
+    const int64_t obase = ((int64_t)v * Kp + j) * row + (int64_t)c0 * FH;
+    for (int32_t ku = tid; ku < nku; ku += 128) {
+      const float y = sm[ku * FW + v];  // (r*Fh + u)*Fw + v = ku*Fw + v
+      if (BF16) static_cast<__nv_bfloat16*>(o)[obase + ku] = __float2bfloat16_rn(y);
+      else static_cast<float*>(o)[obase + ku] = y;
+    }
   }
 }
 
@@ -585,7 +610,6 @@ int make_plan(const Geometry& g, Plan* pl, int pair, int mh_fixed) {
   P.n_ntiles = (g.K + 255) / 256;
   P.NT = ((g.K + P.n_ntiles - 1) / P.n_ntiles + 15) / 16 * 16;
   P.Kp = P.n_ntiles * P.NT;
-  if ((int64_t)FW * P.Kp > 65535) return IM2WIN_EUNSUPPORTED;  // (grid of the filter-copy kernel)
   P.pair = pair;
   P.NTB = pair ? P.NT / 2 : P.NT;
   P.NTS = g.C / P.G;
@@ -824,9 +848,9 @@ int launch_strip(const void* src, const float* f, float* out, const Geometry& g,
       P.box = 0;  // bulk copies then
   }
   {
-    const int32_t row = g.C * FH;
-    const dim3 pg((unsigned)((row + 255) / 256 < 4 ? (row + 255) / 256 : 4), (unsigned)(FW * P.Kp));
-    filter_tap_major_kernel<BF16><<<pg, 256, 0, st>>>(f, scratch.ptr, g.K, P.Kp, row, FH, FW);
+    static_assert(FH * FW <= kPrepFF, "filter-copy kernel's shared buffer");
+    const dim3 pg((unsigned)P.Kp, (unsigned)((g.C + kPrepCh - 1) / kPrepCh));
+    filter_tap_major_kernel<BF16><<<pg, 128, 0, st>>>(f, scratch.ptr, g.K, P.Kp, g.C, FH, FW);
   }
   return P.pair ? launch_kernel<FH, FW, S, BF16, SRCK, true>(P, pl, fmap, xmap, st)
                 : launch_kernel<FH, FW, S, BF16, SRCK, false>(P, pl, fmap, xmap, st);

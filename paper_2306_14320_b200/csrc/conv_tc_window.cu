@@ -587,8 +587,9 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
 
 // Tap-major copy of the filter for the TMA-streamed B operand:
 //   F9[t][j][r] = F[j][r][u][v],  t = u*Fw + v   (j < K; rows K..Kp-1 are zero), fp32 or bf16 (nearest even).
-// One CTA per filter j: its C*Fh*Fw values pass through shared memory 128 channels at a time, so that both
-// the reads and the writes are contiguous.
+// One CTA per (filter j, block of 128 channels): its 128*Fh*Fw values pass through shared memory, so that both
+// the reads and the writes are contiguous, and every CTA is one load - store round trip (the convolution
+// kernel's first MMA waits for this copy: its latency counts).
 constexpr int kPrepCh = 128, kPrepTaps = 25;
 template <bool BF16>
 __global__ void __launch_bounds__(128) filter_tap_rows_kernel(const float* __restrict__ f, void* __restrict__ o, int32_t K,
@@ -598,20 +599,33 @@ __global__ void __launch_bounds__(128) filter_tap_rows_kernel(const float* __res
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   __shared__ float sm[kPrepCh * kPrepTaps];
   const int32_t j = (int32_t)blockIdx.x, tid = (int32_t)threadIdx.x;
-  for (int32_t c0 = 0; c0 < C; c0 += kPrepCh) {
-    const int32_t nc = min(kPrepCh, C - c0);
-    const float* fj = f + ((int64_t)j * C + c0) * taps;
-    for (int32_t i = tid; i < nc * taps; i += 128) sm[i] = j < K ? __ldg(fj + i) : 0.f;
-    __syncthreads();
-    if (tid < nc) {
-      for (int32_t t = 0; t < taps; ++t) {
-        const float x = sm[tid * taps + t];
-        const int64_t oi = ((int64_t)t * Kp + j) * C + c0 + tid;
-        if (BF16) static_cast<__nv_bfloat16*>(o)[oi] = __float2bfloat16_rn(x);
-        else static_cast<float*>(o)[oi] = x;
-      }
+  const int32_t c0 = (int32_t)blockIdx.y * kPrepCh;
+  const int32_t nc = min(kPrepCh, C - c0);
+  const float* fj = f + ((int64_t)j * C + c0) * taps;
+  const int32_t n = nc * taps;
+  if (j < K) {
+    float v[kPrepTaps];
+#pragma unroll
+    for (int q = 0; q < kPrepTaps; ++q) {  // (all loads in flight before the first use)
+      const int32_t i = tid + q * 128;
+      v[q] = (q < taps && i < n) ? __ldg(fj + i) : 0.f;
     }
-    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < kPrepTaps; ++q) {
+      const int32_t i = tid + q * 128;
+      if (q < taps && i < n) sm[i] = v[q];
+    }
+  } else {
+    for (int32_t i = tid; i < n; i += 128) sm[i] = 0.f;
+  }
+  __syncthreads();
+  if (tid < nc) {
+    for (int32_t t = 0; t < taps; ++t) {
+      const float x = sm[tid * taps + t];
+      const int64_t oi = ((int64_t)t * Kp + j) * C + c0 + tid;
+      if (BF16) static_cast<__nv_bfloat16*>(o)[oi] = __float2bfloat16_rn(x);
+      else static_cast<float*>(o)[oi] = x;
+    }
   }
 }
 
@@ -908,8 +922,9 @@ int launch_window(const void* src, const float* f, float* out, const Geometry& g
       P.NBX = 1;
     }
   }
-  if (BF16) filter_tap_rows_kernel<true><<<dim3((unsigned)P.Kp), 128, 0, st>>>(f, scratch.ptr, g.K, P.Kp, g.C, FH * FW);
-  else filter_tap_rows_kernel<false><<<dim3((unsigned)P.Kp), 128, 0, st>>>(f, scratch.ptr, g.K, P.Kp, g.C, FH * FW);
+  const dim3 pgrid((unsigned)P.Kp, (unsigned)((g.C + kPrepCh - 1) / kPrepCh));
+  if (BF16) filter_tap_rows_kernel<true><<<pgrid, 128, 0, st>>>(f, scratch.ptr, g.K, P.Kp, g.C, FH * FW);
+  else filter_tap_rows_kernel<false><<<pgrid, 128, 0, st>>>(f, scratch.ptr, g.K, P.Kp, g.C, FH * FW);
   if (cudaGetLastError() != cudaSuccess) return IM2WIN_ECUDA;
   rc = P.pair ? launch_wkernel<FH, FW, BF16, SRCK, true>(P, pl, fmap, xmap, st) : launch_wkernel<FH, FW, BF16, SRCK, false>(P, pl, fmap, xmap, st);
   if (rc != IM2WIN_OK) return rc;
