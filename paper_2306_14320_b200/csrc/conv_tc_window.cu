@@ -527,7 +527,7 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
           float* const orow = P.nhwc ? P.out + ((int64_t)u.img * HoWo + (int64_t)m * P.Wo + q) * P.K + n0
                                      : P.out + ((int64_t)u.img * P.K + n0) * HoWo + (int64_t)m * P.Wo + q;
           store_columns(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(hh * P.NT), orow, P.nhwc ? 1 : HoWo, P.epi_split, P.NT,
-                        P.K - n0, valid, false, P.nhwc && (P.K & 3) == 0);
+                        P.K - n0, valid, P.two != 0, P.nhwc && (P.K & 3) == 0);
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) {

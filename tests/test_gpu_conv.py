@@ -38,6 +38,9 @@ SMALL = [
     # shapes for the window-offset kernel (stride 1, 3x3 and 5x5): a 5x5 filter, source ranges of several TMA
     # boxes, four 128-row blocks per tile with a ragged last tile
     (1, 32, 14, 15, 24, 5, 5, 1), (2, 64, 30, 28, 64, 3, 3, 1), (1, 32, 70, 66, 32, 3, 3, 1),
+    # two filter tiles of 144: two blocks per tile leave one accumulator buffer, so the interleaver warps help
+    # the epilogue (with two issuing threads they too must zero the columns they read)
+    (2, 64, 20, 30, 288, 3, 3, 1),
 ]
 STRIP_SHAPES = [d for d in SMALL if d[5] == 3 and d[6] == 3 and d[1] % 32 == 0 and d[7] in (1, 2)]
 WINDOW_SHAPES = [d for d in SMALL if (d[5], d[6]) in ((3, 3), (5, 5)) and d[1] % 32 == 0 and d[7] == 1]
