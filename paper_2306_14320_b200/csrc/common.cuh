@@ -109,6 +109,7 @@ struct Knobs {
   int window_mh = 0;         // window-offset kernel: 128-row blocks per tile (0: own choice)
   int window_plan = 0;       // window-offset kernel: forced split of shared memory (0: own choice)
   int window_pair = 0;       // window-offset kernel: 1 = CTA pairs forced, 2 = single CTAs forced, 0 = own choice
+  int window_bres = 0;       // window-offset kernel: 1 = resident filter or nothing, 2 = never resident, 0 = own choice
   int window_nohelp = 0;     // window-offset kernel: the interleaver warps never help the epilogue
   int window_two = 0;        // window-offset kernel: 1 = two MMA-issuing threads forced, 2 = one forced, 0 = own choice
 };

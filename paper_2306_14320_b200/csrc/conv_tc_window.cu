@@ -56,6 +56,7 @@ struct WParams {
   int32_t NT, n_ntiles, Kp;
   int32_t NTB;        // filter rows one CTA holds per block: NT, or NT/2 when two CTAs share an MMA
   int32_t nhwc;       // output layout N x Ho x Wo x K
+  int32_t bres;       // the whole filter tile stays in shared memory: SB stages = one unit's, loaded once per CTA
   int32_t two;        // two MMA-issuing threads share the filter stages by parity; every MMA accumulates, the epilogue zeroes behind its reads
   int32_t pair;       // two CTAs (a cluster) work as one: tcgen05.mma.cta_group::2, M = 256, each CTA its own rows and half the filter tile
   int32_t G, GR, NSUB, NXS;  // channels per X stage / per source stage, source stages per X stage, X stages per unit
@@ -131,6 +132,7 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
   Ring xr, br, dr;
   bool ok = true;
   constexpr bool two = TWO;
+  const bool bres = P.bres != 0;  // resident filter: the stages of a unit are the ring, filled once
   uint32_t bc = 0;  // filter stages so far: with two issuing threads, thread `which` takes those of its parity
   (void)bc; (void)which;
   SPROF_DECL
@@ -165,7 +167,7 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
           if constexpr (TWO) {
             if ((bc++ & 1u) != which) { br.advance(P.SB); continue; }
           }
-          SPROF_W(2, ok = wait_bar(P, misc, b_full0 + (uint32_t)br.idx * 8u, br.phase, DEV_TIMEOUT_B_FULL, 20))
+          SPROF_W(2, ok = wait_bar(P, misc, b_full0 + (uint32_t)br.idx * 8u, bres ? 0u : br.phase, DEV_TIMEOUT_B_FULL, 20))
           if (!ok) break;
           ptx::tc_fence_after();
           // (block by block: consecutive MMAs onto the same accumulator run faster than alternating ones)
@@ -198,7 +200,9 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
 #ifdef IM2WIN_PROF
           pw[3] += clock64() - cm0;
 #endif
-          SPROF_W(4, if constexpr (PAIR) mma_commit_pair(b_empty0 + (uint32_t)br.idx * 8u); else ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u))
+          if (!bres) {
+            SPROF_W(4, if constexpr (PAIR) mma_commit_pair(b_empty0 + (uint32_t)br.idx * 8u); else ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u))
+          }
           br.advance(P.SB);
         }
       }
@@ -378,10 +382,13 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
       for (int64_t it = 0; ok; ++it) {
         WUnit u;
         if (!wunit_at<PAIR>(P, it, rank, u)) break;
+        if (P.bres && it > 0) break;  // resident filter: one unit's stages are the whole (single) filter tile
         const int32_t row0 = u.nt * P.NT + (int32_t)rank * P.NTB;
         for (int32_t xs = 0; xs < P.NXS && ok; ++xs) {
           for (int32_t t0 = 0; t0 < FH * FW && ok; t0 += P.TPS, ++count, br.advance(P.SB)) {
-            SPROF_W(0, ok = wait_bar(P, misc, ptx::smem_u32(&bars->b_empty[br.idx]), br.phase ^ 1u, DEV_TIMEOUT_B_EMPTY))
+            if (!P.bres) {
+              SPROF_W(0, ok = wait_bar(P, misc, ptx::smem_u32(&bars->b_empty[br.idx]), br.phase ^ 1u, DEV_TIMEOUT_B_EMPTY))
+            }
             if (!ok) break;
             const uint32_t full = b_full_lead0 + (uint32_t)br.idx * 8u;
 #ifdef IM2WIN_PROF
@@ -400,8 +407,12 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
       SPROF_DUMP(7)
       // every copy issued must have landed before the CTA exits: the stage's release by the MMAs that read it
       // says so (in pair mode the bytes are counted on the leader's barrier, not here)
-      for (int64_t c = count > P.SB ? count - P.SB : 0; c < count; ++c)
-        wait_bar(P, misc, ptx::smem_u32(&bars->b_empty[c % P.SB]), (uint32_t)(c / P.SB) & 1u, DEV_TIMEOUT_DRAIN);
+      if (P.bres) {
+        for (int64_t c = 0; c < count; ++c) wait_bar(P, misc, ptx::smem_u32(&bars->b_full[c]), 0u, DEV_TIMEOUT_DRAIN);
+      } else {
+        for (int64_t c = count > P.SB ? count - P.SB : 0; c < count; ++c)
+          wait_bar(P, misc, ptx::smem_u32(&bars->b_empty[c % P.SB]), (uint32_t)(c / P.SB) & 1u, DEV_TIMEOUT_DRAIN);
+      }
     }
     __syncwarp();
   } else if (warp >= kTWarp0 && warp < kTWarp0 + kTW) {
@@ -701,10 +712,16 @@ int make_wplan(const Geometry& g, WPlan* pl, int pair, int mh_fixed) {
   const Try order_win16[] = {{1, FW, 32}, {1, FW, 16}, {2, 1, 16}, {1, 1, 16}, {1, 1, 8}, {1, 1, 32}};
   const Try* order = SRCK == 1 ? order_fused : (SRCK == 2 ? order_win16 : order_win);
   const int n_order = SRCK == 1 ? 9 : 6;
+  // (resident only where source stages of sixteen channels still fit: with smaller ones it was measured slower)
+  const Try order_res[] = {{2, FW, 32}, {2, FW, 16}, {1, FW, 32}, {1, FW, 16}};
   bool found = false;
-  {
-    for (int t = 0; t < n_order && !found; ++t) {
-      int nblk = order[t].nblk, tps = order[t].tps, gr = order[t].gr;
+  for (int pass = 0; pass < 2 && !found; ++pass) {  // first the resident filter, then the streamed one
+    if (pass == 0 && (pair || P.n_ntiles != 1 || knobs().window_bres == 2)) continue;
+    if (pass == 1 && knobs().window_bres == 1) break;  // (test build: resident or nothing)
+    const Try* ord = pass == 0 ? order_res : order;
+    const int n_ord = pass == 0 ? 4 : n_order;
+    for (int t = 0; t < n_ord && !found; ++t) {
+      int nblk = ord[t].nblk, tps = ord[t].tps, gr = ord[t].gr;
       if (forced_plan) {
         if (t > 0) break;
         nblk = forced_plan & 15; tps = (forced_plan >> 4) & 15; gr = forced_plan >> 8;
@@ -725,6 +742,22 @@ int make_wplan(const Geometry& g, WPlan* pl, int pair, int mh_fixed) {
       }
       const int64_t raw_bytes = (int64_t)gr * nbx * bxe * ES;
       if (raw_bytes % 128 != 0 || bxe * ES > 65536) continue;
+      // Resident filter: a single filter tile whose Fh*Fw*C/G stages all fit beside the X stages and two source
+      // stages stays in shared memory for the whole kernel (no filter stream, no release traffic).
+      const int64_t n_res = (int64_t)(g.C / G) * (FH * FW / tps);
+      const bool try_res = pass == 0 && n_res <= kMaxB && n_res * b_stage_bytes + 2 * raw_bytes <= left;
+      if (pass == 0 && !try_res) continue;
+      if (try_res) {
+        int64_t sr = 2;
+        while (sr < kMaxRaw && n_res * b_stage_bytes + (sr + 1) * raw_bytes <= left) ++sr;
+        P.G = G; P.NXS = g.C / G; P.x_stage_bytes = x_stage_bytes;
+        P.TPS = tps; P.b_stage_bytes = (uint32_t)b_stage_bytes;
+        P.GR = gr; P.NSUB = G / gr; P.box = box_ok ? 1 : 0;
+        P.NBX = (int32_t)nbx; P.BXE = (int32_t)bxe; P.raw_stage_bytes = (uint32_t)raw_bytes;
+        P.SB = (int32_t)n_res; P.SR = (int32_t)sr; P.bres = 1;
+        found = true;
+        break;
+      }
       const int64_t min_b = 2;
       if (min_b * b_stage_bytes + 2 * raw_bytes > left) continue;
       const int nsub = G / gr;
@@ -828,7 +861,7 @@ bool window_preferred(const Geometry& g, const WParams& P) {
   }
   if (SRCK == 2) return P.NT <= 192;                                   // bf16 im2win tensor
   if (SRCK == 1)                                                        // fused
-    return g.C >= 128 && (P.NT <= 192 || P.RPI < 128);
+    return (g.C >= 128 || P.NT <= 64) && (P.NT <= 192 || P.RPI < 128);
   return g.C >= 128;                                                    // fp32 im2win tensor
 }
 
@@ -930,7 +963,7 @@ int launch_window(const void* src, const float* f, float* out, const Geometry& g
   if (rc != IM2WIN_OK) return rc;
   note_kernel(KERNEL_WINDOW);
   {
-    const int v[8] = {P.MH + 10 * P.pair, P.G, P.TPS, P.GR, P.SB, P.SR, P.ND, P.box * 100 + P.NBX};
+    const int v[8] = {P.MH + 10 * P.pair + 100 * P.bres, P.G, P.TPS, P.GR, P.SB, P.SR, P.ND, P.box * 100 + P.NBX};
     note_plan(v, 8);
   }
   return IM2WIN_OK;

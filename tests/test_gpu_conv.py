@@ -153,7 +153,7 @@ def test_forced_strip_configurations_run_the_strip_kernel(dims, mode, _kernel):
 @pytest.mark.parametrize("dims", WINDOW_SHAPES)
 def test_forced_window_configurations_run_the_window_kernel(dims, mode, src_kind, _kernel):
     """The same for the window-offset kernel, from the im2win tensor and fused."""
-    if _kernel not in ("window", "window1", "window2", "wtwo", "wpair", "wpair2"):
+    if _kernel not in ("window", "window1", "window2", "wtwo", "wstream", "wpair", "wpair2"):
         pytest.skip("only for the configurations that force the window-offset kernel")
     x, f = _data(dims, 810, ints=True)
     got = gpu_conv(x, f, dims, mode, src_kind=src_kind)
