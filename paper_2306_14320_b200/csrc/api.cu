@@ -354,7 +354,7 @@ int im2win_debug_set_option(const char* name, int value) {
       {"ntiles", &Knobs::ntiles}, {"transform_gather", &Knobs::transform_gather},
       {"test_skip_copy", &Knobs::test_skip_copy}, {"strip_mh", &Knobs::strip_mh}, {"strip_pair", &Knobs::strip_pair},
       {"force_window", &Knobs::force_window}, {"no_window", &Knobs::no_window}, {"window_mh", &Knobs::window_mh},
-      {"window_plan", &Knobs::window_plan}, {"window_pair", &Knobs::window_pair}, {"window_two", &Knobs::window_two}, {"window_nohelp", &Knobs::window_nohelp}, {"window_bres", &Knobs::window_bres}};
+      {"window_plan", &Knobs::window_plan}, {"window_pair", &Knobs::window_pair}, {"window_two", &Knobs::window_two}, {"window_nohelp", &Knobs::window_nohelp}, {"window_bres", &Knobs::window_bres}, {"transform_budget_kb", &Knobs::transform_budget_kb}};
   for (const Entry& e : table)
     if (strcmp(e.name, name) == 0) { g_knobs.*(e.field) = value; return IM2WIN_OK; }
   return IM2WIN_EINVAL;

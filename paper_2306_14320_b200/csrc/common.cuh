@@ -100,6 +100,7 @@ struct Knobs {
   int no_l2ahead = 0;        // persistent kernel: no L2 prefetch of the next tile's boxes
   int no_btma = 0;           // persistent kernel: resident filter built by threads, not fetched by TMA
   int ntiles = 0;            // persistent kernel: number of filter tiles (0: own choice)
+  int transform_budget_kb = 0;  // transform tile kernel: shared-memory budget per CTA in KB (0: own choice)
   int transform_gather = 0;  // transform: the staged-gather kernel instead of the tile kernel
   int test_skip_copy = 0;    // transform tile kernel, single-CTA problems: announce the input copy, never issue it
   int strip_mh = 0;          // strip-matrix kernel: 128-row halves per tile (0: own choice)

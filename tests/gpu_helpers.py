@@ -39,7 +39,7 @@ CONV_CONFIGS = {
 _KNOB_DEFAULTS = {"force_generic": 0, "no_strip": 0, "force_strip": 0, "no_box": 0, "no_pim": 0, "bslice": 0,
                   "no_bslice": 0, "splitk": -1, "force_stream": 0, "nsets": 0, "no_l2ahead": 0, "no_btma": 0,
                   "ntiles": 0, "transform_gather": 0, "test_skip_copy": 0, "strip_mh": 0, "strip_pair": 0,
-                  "force_window": 0, "no_window": 0, "window_mh": 0, "window_plan": 0, "window_pair": 0, "window_two": 0, "window_nohelp": 0, "window_bres": 0}
+                  "force_window": 0, "no_window": 0, "window_mh": 0, "window_plan": 0, "window_pair": 0, "window_two": 0, "window_nohelp": 0, "window_bres": 0, "transform_budget_kb": 0}
 _min_workspace = False
 
 
