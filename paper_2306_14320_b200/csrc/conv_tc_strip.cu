@@ -88,26 +88,28 @@ struct Unit {
 };
 template <bool PAIR>
 __device__ __forceinline__ bool unit_at(const SParams& P, int64_t it, uint32_t rank, Unit& u) {
-  int64_t tile;
+  // (32-bit arithmetic: the host declines problems of 2^31 units or more; a 64-bit division costs a role
+  // some 250 cycles, and every role does this once per unit)
+  uint32_t tile;
   if (PAIR) {
-    const int64_t pu = (int64_t)(blockIdx.x >> 1) + it * (int64_t)(gridDim.x >> 1);
-    if (pu >= P.units) return false;
-    const int64_t half = (P.tiles + 1) >> 1;
-    const int64_t nt = pu / half;
-    tile = 2 * (pu - nt * half) + rank;
-    u.store = tile < P.tiles;
-    if (!u.store) tile = P.tiles - 1;
+    const uint32_t pu = (blockIdx.x >> 1) + (uint32_t)it * (gridDim.x >> 1);
+    if (pu >= (uint32_t)P.units) return false;
+    const uint32_t half = ((uint32_t)P.tiles + 1u) >> 1;
+    const uint32_t nt = pu / half;
+    tile = 2u * (pu - nt * half) + rank;
+    u.store = tile < (uint32_t)P.tiles;
+    if (!u.store) tile = (uint32_t)P.tiles - 1u;
     u.nt = (int32_t)nt;
   } else {
-    const int64_t t = (int64_t)blockIdx.x + it * (int64_t)gridDim.x;
-    if (t >= P.units) return false;
-    tile = t / P.n_ntiles;
-    u.nt = (int32_t)(t - tile * P.n_ntiles);
+    const uint32_t t = blockIdx.x + (uint32_t)it * gridDim.x;
+    if (t >= (uint32_t)P.units) return false;
+    if (P.n_ntiles == 1) { tile = t; u.nt = 0; }
+    else { tile = t / (uint32_t)P.n_ntiles; u.nt = (int32_t)(t - tile * (uint32_t)P.n_ntiles); }
     u.store = true;
   }
-  const int64_t img = tile / P.TPI;
+  const uint32_t img = tile / (uint32_t)P.TPI;
   u.img = (int32_t)img;
-  u.R0 = (int32_t)(tile - img * P.TPI) * 128 * P.MH;
+  u.R0 = (int32_t)(tile - img * (uint32_t)P.TPI) * 128 * P.MH;
   return true;
 }
 // Source elements [e_lo, e_hi) of a channel plane that the tile starting at T row R0 needs.
@@ -625,6 +627,7 @@ int make_plan(const Geometry& g, Plan* pl, int pair, int mh_fixed) {
   P.TPI = (P.RPI + 128 * P.MH - 1) / (128 * P.MH);
   P.tiles = (int64_t)g.N * P.TPI;
   P.units = pair ? ((P.tiles + 1) / 2) * P.n_ntiles : P.tiles * P.n_ntiles;
+  if (P.tiles * P.n_ntiles >= (1ll << 31) - 65536) return IM2WIN_EUNSUPPORTED;  // (the kernel's unit arithmetic is 32-bit)
   P.RT = 128 * P.MH + SH;
   P.RA = (P.RT + 7) / 8 * 8;
   P.NJ = P.RT * S;

@@ -89,26 +89,28 @@ struct WUnit {
 // last pair's second CTA repeats the last tile without storing.
 template <bool PAIR>
 __device__ __forceinline__ bool wunit_at(const WParams& P, int64_t it, uint32_t rank, WUnit& u) {
-  int64_t tile;
+  // (32-bit arithmetic: the host declines problems of 2^31 units or more; a 64-bit division costs a role
+  // some 250 cycles, and every role does this once per unit)
+  uint32_t tile;
   if (PAIR) {
-    const int64_t pu = (int64_t)(blockIdx.x >> 1) + it * (int64_t)(gridDim.x >> 1);
-    if (pu >= P.units) return false;
-    const int64_t half = (P.tiles + 1) >> 1;
-    const int64_t nt = pu / half;
-    tile = 2 * (pu - nt * half) + rank;
-    u.store = tile < P.tiles;
-    if (!u.store) tile = P.tiles - 1;
+    const uint32_t pu = (blockIdx.x >> 1) + (uint32_t)it * (gridDim.x >> 1);
+    if (pu >= (uint32_t)P.units) return false;
+    const uint32_t half = ((uint32_t)P.tiles + 1u) >> 1;
+    const uint32_t nt = pu / half;
+    tile = 2u * (pu - nt * half) + rank;
+    u.store = tile < (uint32_t)P.tiles;
+    if (!u.store) tile = (uint32_t)P.tiles - 1u;
     u.nt = (int32_t)nt;
   } else {
-    const int64_t t = (int64_t)blockIdx.x + it * (int64_t)gridDim.x;
-    if (t >= P.units) return false;
-    tile = t / P.n_ntiles;
-    u.nt = (int32_t)(t - tile * P.n_ntiles);
+    const uint32_t t = blockIdx.x + (uint32_t)it * gridDim.x;
+    if (t >= (uint32_t)P.units) return false;
+    if (P.n_ntiles == 1) { tile = t; u.nt = 0; }
+    else { tile = t / (uint32_t)P.n_ntiles; u.nt = (int32_t)(t - tile * (uint32_t)P.n_ntiles); }
     u.store = true;
   }
-  const int64_t img = tile / P.TPI;
+  const uint32_t img = tile / (uint32_t)P.TPI;
   u.img = (int32_t)img;
-  u.R0 = (int32_t)(tile - img * P.TPI) * 128 * P.MH;
+  u.R0 = (int32_t)(tile - img * (uint32_t)P.TPI) * 128 * P.MH;
   return true;
 }
 // Source elements [e_lo, e_hi) of a channel plane that the tile starting at position R0 needs, and (im2win
@@ -686,6 +688,7 @@ int make_wplan(const Geometry& g, WPlan* pl, int pair, int mh_fixed) {
   P.TPI = (P.RPI + 128 * P.MH - 1) / (128 * P.MH);
   P.tiles = (int64_t)g.N * P.TPI;
   P.units = pair ? ((P.tiles + 1) / 2) * P.n_ntiles : P.tiles * P.n_ntiles;
+  if (P.tiles * P.n_ntiles >= (1ll << 31) - 65536) return IM2WIN_EUNSUPPORTED;  // (the kernel's unit arithmetic is 32-bit)
   P.ND = 512 / (P.MH * P.NT) >= 2 ? 2 : 1;
   P.n_epi = 4 * (P.MH < 2 ? P.MH : 2);
   // one accumulator buffer: the interleaver warps (two sets of four, one per block) store the upper half of the
