@@ -78,6 +78,7 @@ struct PParams {
   uint64_t magic_TPI, magic_Wo;  // pim: ceil(2^32 / d); n / d == (n * magic) >> 32 while n * d < 2^32 (host check)
   int32_t nchunks;      // 128-byte filter chunks per tile
   int32_t l2_ahead;     // box mode: request the next tile's boxes into L2 one tile ahead
+  int32_t wait_prev;    // the preceding kernel in the stream is not this call's own filter copy: source reads and output writes wait for it
   int32_t bslice;       // resident filter holds only this CTA's reduction slice (grid is a multiple of Z)
   int32_t b_tma;        // resident filter fetched by TMA (TF32, dense groups) instead of built by the threads
   int32_t tmem_cols;
@@ -519,6 +520,11 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
 #ifdef IM2WIN_PROF
     prof_acc[1] = prof_t0 - prof_kernel_t0;  // prologue (barrier init, TMEM alloc, resident filter build)
 #endif
+    // The kernel is launched as a programmatic dependent of whatever precedes it in the stream: where that is
+    // the transform kernel (which lets its dependents start while it drains), the prologue above overlapped
+    // its tail, and the source is read only once that grid has completed.  After any other kernel: no effect.
+    // (Behind this call's own filter-copy kernel, an ordinary launch, everything earlier has completed already.)
+    if (P.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (P.box) {
       // One 2-D box per channel group.  The tile lies in one image: x = first needed float of the
       // plane rounded down to 16 bytes (in 8-byte elements), y = plane index of the group's first
@@ -1007,6 +1013,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
       constexpr bool REDUCE = EK == 1;
       Ring dr;
       bool ok = true;
+      if (P.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");  // (the output is written only after the preceding grid has completed)
       const int32_t eK = P.K, eNT = P.NT, eHoWo = P.HoWo;  // kept in registers for the store loop
       // hand both accumulator buffers to the MMA side zeroed: every MMA accumulates
       for (int32_t d = 0; d < P.ND; ++d) {
@@ -1465,32 +1472,31 @@ int launch_spec_impl(const void* xhat, const float* f, float* out, const Geometr
   int64_t grid = P.ntiles < sm_count() ? P.ntiles : sm_count();
   if (P.bslice) grid = grid / P.Z * P.Z;  // every CTA keeps to one slice
   cudaError_t e;
+  // Programmatic dependent launch: behind the filter-copy kernel (BF16 streamed mode) the prologue, strip copies
+  // and repacking overlap that copy, and the filter producer waits for it; behind the transform kernel the
+  // prologue overlaps that kernel's tail, and the strip producer and the epilogue wait (griddepcontrol.wait).
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)kThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  // (the filter copy itself is an ordinary launch: when it runs, everything before it has completed)
+  P.wait_prev = f_bf16 ? 0 : 1;
   if (resident) {
     auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, true, FUSED, SRC16, OUT16>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
-    kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
+    if (cudaLaunchKernelEx(&cfg, kern, P, fmap, xmap) != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
   } else {
     auto kern = conv_tc_persistent_kernel<FH, FW, CB, BF16, false, FUSED, SRC16, OUT16>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (e != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
-    if (f_bf16) {
-      // behind the filter-copy kernel as a programmatic dependent: prologue, strip copies and repacking overlap
-      // that copy; the filter producer waits for it (griddepcontrol.wait)
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3((unsigned)grid);
-      cfg.blockDim = dim3((unsigned)kThreads);
-      cfg.dynamicSmemBytes = smem_bytes;
-      cfg.stream = st;
-      cudaLaunchAttribute attr[1];
-      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-      attr[0].val.programmaticStreamSerializationAllowed = 1;
-      cfg.attrs = attr;
-      cfg.numAttrs = 1;
-      if (cudaLaunchKernelEx(&cfg, kern, P, fmap, xmap) != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
-    } else {
-      kern<<<(unsigned)grid, kThreads, smem_bytes, st>>>(P, fmap, xmap);
-    }
+    if (cudaLaunchKernelEx(&cfg, kern, P, fmap, xmap) != cudaSuccess) { cudaGetLastError(); return IM2WIN_ECUDA; }
   }
   note_kernel(KERNEL_PERSISTENT);
   return cuda_status(cudaGetLastError());

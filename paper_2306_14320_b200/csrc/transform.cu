@@ -53,6 +53,9 @@ struct Cursor {  // position of an output element inside the CTA's range
 // FHT: the filter height as a compile-time constant (division by it is then a multiplication), or 0.
 template <int FHT>
 __global__ void __launch_bounds__(kThreads) transform_smem_kernel(const TransformParams P) {
+  // a convolution launched next as a programmatic dependent may set up (barriers, tensor memory, resident
+  // filter) while this grid drains; it waits for this grid's completion before it reads the im2win tensor
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   extern __shared__ __align__(16) float smem[];
   const int32_t Fh = FHT ? FHT : P.Fh;
   const int64_t job = blockIdx.x;
@@ -187,6 +190,9 @@ __device__ __forceinline__ uint32_t bf16x2_rn(float lo, float hi) {
 __device__ __forceinline__ uint16_t bf16_rn(float x) { return (uint16_t)(bf16x2_rn(x, 0.f) & 0xffffu); }
 
 __global__ void __launch_bounds__(kThreads) transform_smem_bf16_kernel(const TransformParams P, uint16_t* out16) {
+  // a convolution launched next as a programmatic dependent may set up (barriers, tensor memory, resident
+  // filter) while this grid drains; it waits for this grid's completion before it reads the im2win tensor
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   extern __shared__ __align__(16) float smem[];
   const int64_t job = blockIdx.x;
   const int64_t pg = job / P.nblk;
@@ -315,6 +321,9 @@ struct TileParams {
 // OUT16: the output is the bf16 storage variant (P.out then points at 16-bit words).
 template <int FH, bool OUT16>
 __global__ void __launch_bounds__(kThreads) transform_tile_kernel(const TileParams P) {
+  // a convolution launched next as a programmatic dependent may set up (barriers, tensor memory, resident
+  // filter) while this grid drains; it waits for this grid's completion before it reads the im2win tensor
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   using OutT = typename std::conditional<OUT16, uint16_t, float>::type;
   constexpr int32_t OPC = OUT16 ? 8 : 4;  // output elements per 16-byte chunk
   extern __shared__ __align__(128) uint8_t smem_raw[];
