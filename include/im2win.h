@@ -115,8 +115,10 @@ int im2win_transform_bf16(const float* in_nchw, const im2win_shape* shape, uint1
  *            src_kind NCHW_FUSED: the input I; the tensor-core kernel stages the input rows a tile
  *            needs and reads the windows from them, so nothing of size Ihat is written (workspace
  *            0 bytes).  Same result as the other two kinds.  Shapes without a fused specialisation
- *            (see below) fall back to transform + convolution if a sufficient `workspace` is
- *            given, else EUNSUPPORTED; IM2WIN_MODE_FP32 always takes that fallback.
+ *            (the specialised filter sizes are 3x3, 5x5, 7x7, 11x11 and, with channel counts that are
+ *            multiples of 16, 1x1, 1x3, 3x1, 1x7, 7x1) fall back to transform + convolution if a
+ *            sufficient `workspace` is given, else EUNSUPPORTED; IM2WIN_MODE_FP32 always takes that
+ *            fallback.
  *            src_kind IM2WIN_BF16: a bf16 im2win tensor from im2win_transform_bf16; mode must be
  *            IM2WIN_MODE_BF16 (EINVAL otherwise); `workspace` optional scratch.  The MMA operands
  *            are the same bf16 values as from an fp32 im2win tensor.  Implemented where a
@@ -162,8 +164,8 @@ int im2win_conv_nhwc(const void* src, int src_kind, const float* filter_kcfhfw,
  * element: half the output footprint and half the bytes written.
  * out_nchw_bf16: device, N*K*Ho*Wo 16-bit words, every element is written; 16-byte aligned.
  * Everything else as im2win_conv.  Tensor-core modes only (IM2WIN_MODE_FP32: EINVAL), and only
- * shapes with a filter-size specialisation (EUNSUPPORTED otherwise: the generic kernel has no
- * bf16 epilogue). */
+ * square filters with a specialisation: 3x3, 5x5, 7x7, 11x11 (EUNSUPPORTED otherwise: the generic
+ * kernel and the pointwise / factorised families have no bf16 epilogue). */
 int im2win_conv_bf16out(const void* src, int src_kind, const float* filter_kcfhfw,
                         const im2win_shape* shape, int mode, uint16_t* out_nchw_bf16,
                         void* workspace, size_t workspace_bytes, void* cuda_stream);

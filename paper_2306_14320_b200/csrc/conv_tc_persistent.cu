@@ -1530,8 +1530,8 @@ int launch_spec(const void* src, const float* f, float* out, const Geometry& g, 
 // fused: `xhat` is the untransformed NCHW input and the windows are built from staged input rows
 // (no im2win tensor exists in global memory).
 // The filter-size families are separate functions so that the build can compile them as separate
-// translation units in parallel (-DIM2WIN_PART=0..3: part 0 = 3x3 + this dispatcher, 1 = 5x5,
-// 2 = 7x7, 3 = 11x11; without the macro everything is compiled here).
+// translation units in parallel (-DIM2WIN_PART=0..5: part 0 = 3x3 + this dispatcher, 1 = 5x5,
+// 2 = 7x7, 3 = 11x11, 4 = 1x1 / 1x3 / 3x1, 5 = 1x7 / 7x1; without the macro everything is compiled here).
 #ifndef IM2WIN_PART
 #define IM2WIN_PART -1
 #endif
@@ -1541,6 +1541,8 @@ int launch_spec_3x3(IM2WIN_SPEC_ARGS);
 int launch_spec_5x5(IM2WIN_SPEC_ARGS);
 int launch_spec_7x7(IM2WIN_SPEC_ARGS);
 int launch_spec_11x11(IM2WIN_SPEC_ARGS);
+int launch_spec_rect_a(IM2WIN_SPEC_ARGS);
+int launch_spec_rect_b(IM2WIN_SPEC_ARGS);
 
 #if IM2WIN_PART == -1 || IM2WIN_PART == 0
 int launch_spec_3x3(IM2WIN_SPEC_ARGS) {
@@ -1593,6 +1595,49 @@ int launch_spec_11x11(IM2WIN_SPEC_ARGS) {
 }
 #endif
 
+// Pointwise and factorised filters (1x1; 1x3 / 3x1; 1x7 / 7x1): the same kernel, from the fp32 im2win tensor or
+// fused, fp32 NCHW or NHWC output (the bf16 storage variants of these shapes go to the generic kernel).
+// Sixteen channels per group (TF32: two to six MMA steps, BF16: one to seven, no padding); 1x7 / 7x1 in TF32
+// mode: eight (seven steps).
+template <int FH, int FW>
+int launch_spec_rect(IM2WIN_SPEC_ARGS) {
+  if (kind == 2 || out_bf16 || g.C % 8 != 0) return IM2WIN_EUNSUPPORTED;
+  if constexpr (FH * FW == 1) {  // pointwise: thirty-two channels per group where they divide C
+    if (g.C % 32 == 0) {
+      int rc;
+      if (bf16) rc = kind == 1 ? launch_spec_impl<1, 1, 32, true, true>(xhat, f, out, g, st, scratch)
+                               : launch_spec_impl<1, 1, 32, true, false>(xhat, f, out, g, st, scratch);
+      else rc = kind == 1 ? launch_spec_impl<1, 1, 32, false, true>(xhat, f, out, g, st, scratch)
+                          : launch_spec_impl<1, 1, 32, false, false>(xhat, f, out, g, st, scratch);
+      if (rc != IM2WIN_EUNSUPPORTED) return rc;
+    }
+  }
+  if (bf16) {
+    if (g.C % 16 != 0) return IM2WIN_EUNSUPPORTED;
+    return kind == 1 ? launch_spec_impl<FH, FW, 16, true, true>(xhat, f, out, g, st, scratch)
+                     : launch_spec_impl<FH, FW, 16, true, false>(xhat, f, out, g, st, scratch);
+  }
+  constexpr int CBT = FH * FW >= 7 ? 8 : 16;
+  if (g.C % CBT != 0) return IM2WIN_EUNSUPPORTED;
+  return kind == 1 ? launch_spec_impl<FH, FW, CBT, false, true>(xhat, f, out, g, st, scratch)
+                   : launch_spec_impl<FH, FW, CBT, false, false>(xhat, f, out, g, st, scratch);
+}
+#if IM2WIN_PART == -1 || IM2WIN_PART == 4
+int launch_spec_rect_a(IM2WIN_SPEC_ARGS) {
+  if (g.Fh == 1 && g.Fw == 1) return launch_spec_rect<1, 1>(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh == 1 && g.Fw == 3) return launch_spec_rect<1, 3>(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh == 3 && g.Fw == 1) return launch_spec_rect<3, 1>(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  return IM2WIN_EUNSUPPORTED;
+}
+#endif
+#if IM2WIN_PART == -1 || IM2WIN_PART == 5
+int launch_spec_rect_b(IM2WIN_SPEC_ARGS) {
+  if (g.Fh == 1 && g.Fw == 7) return launch_spec_rect<1, 7>(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh == 7 && g.Fw == 1) return launch_spec_rect<7, 1>(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  return IM2WIN_EUNSUPPORTED;
+}
+#endif
+
 #if IM2WIN_PART == -1 || IM2WIN_PART == 0
 int launch_conv_tc_persistent(const void* xhat, const float* f, float* out, const Geometry& g, int mode,
                               cudaStream_t st, Scratch scratch, bool fused, bool src_bf16, bool out_bf16) {
@@ -1603,6 +1648,9 @@ int launch_conv_tc_persistent(const void* xhat, const float* f, float* out, cons
   if (g.Fh == 5 && g.Fw == 5) return launch_spec_5x5(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
   if (g.Fh == 7 && g.Fw == 7) return launch_spec_7x7(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
   if (g.Fh == 11 && g.Fw == 11) return launch_spec_11x11(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh == 1 && g.Fw == 7 || g.Fh == 7 && g.Fw == 1) return launch_spec_rect_b(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh * g.Fw <= 3 && (g.Fh == 1 || g.Fw == 1) && g.Fh * g.Fw != 2)
+    return launch_spec_rect_a(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
   return IM2WIN_EUNSUPPORTED;
 }
 
