@@ -128,7 +128,8 @@ __device__ __forceinline__ void tile_range(const SParams& P, int32_t R0, int32_t
   }
 }
 
-// The MMA-issuing thread's whole life.  A filter stage holds the NBLK blocks of one (T stage, tap),
+// The MMA-issuing warp's whole life (all lanes run it, so that the descriptor arithmetic and the waits are
+// warp-uniform work; lane 0 issues).  A filter stage holds the NBLK blocks of one (T stage, tap),
 // so there is one wait and one release per NBLK*2*MH MMAs.
 template <int FW, int S, bool BF16, int MH, int NBLK, bool PAIR>
 __device__ __forceinline__ void mma_role(const SParams& P, SBars* bars, SMisc* misc, uint32_t tmem_base, uint32_t t_sa,
@@ -146,23 +147,23 @@ __device__ __forceinline__ void mma_role(const SParams& P, SBars* bars, SMisc* m
   const uint32_t RA = (uint32_t)P.RA, NT = (uint32_t)P.NT, idesc = P.idesc;
   const uint32_t t_full0 = ptx::smem_u32(&bars->t_full[0]), t_empty0 = ptx::smem_u32(&bars->t_empty[0]);
   const uint32_t b_full0 = ptx::smem_u32(&bars->b_full[0]), b_empty0 = ptx::smem_u32(&bars->b_empty[0]);
-  const int32_t lane = 0;
-  (void)lane;
+  const int32_t lane = (int32_t)(threadIdx.x & 31);
+  const uint32_t elect = lane == 0 ? 1u : 0u;
   for (int64_t it = 0; ok; ++it, dr.advance(P.ND)) {
     Unit u;
     if (!unit_at<PAIR>(P, it, 0, u)) break;
-    SPROF_W(0, ok = wait_bar(P, misc, ptx::smem_u32(&bars->acc_empty[dr.idx]), dr.phase ^ 1u, DEV_TIMEOUT_ACC))
+    SPROF_W(0, ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->acc_empty[dr.idx]), dr.phase ^ 1u, DEV_TIMEOUT_ACC))
     if (!ok) break;
     ptx::tc_fence_after();
     const uint32_t d_tmem = tmem_base + (uint32_t)(dr.idx * MH) * NT;
     uint32_t accum = 0;
     for (int32_t ts = 0; ts < P.NTS && ok; ++ts, tr.advance(2)) {
-      SPROF_W(1, ok = wait_bar(P, misc, t_full0 + (uint32_t)tr.idx * 8u, tr.phase, DEV_TIMEOUT_A_FULL, 20))
+      SPROF_W(1, ok = wait_bar_warp(P, misc, t_full0 + (uint32_t)tr.idx * 8u, tr.phase, DEV_TIMEOUT_A_FULL, 20))
       if (!ok) break;
       const uint32_t a_stage = a_lo0 + (uint32_t)tr.idx * t16;
 #pragma unroll
       for (int v = 0; v < FW; ++v) {
-        SPROF_W(2, ok = wait_bar(P, misc, b_full0 + (uint32_t)br.idx * 8u, br.phase, DEV_TIMEOUT_B_FULL, 20))
+        SPROF_W(2, ok = wait_bar_warp(P, misc, b_full0 + (uint32_t)br.idx * 8u, br.phase, DEV_TIMEOUT_B_FULL, 20))
         if (!ok) break;
         ptx::tc_fence_after();
         uint32_t a_k = a_stage + (uint32_t)(v % S) * RA + (uint32_t)(v / S);
@@ -171,29 +172,21 @@ __device__ __forceinline__ void mma_role(const SParams& P, SBars* bars, SMisc* m
         for (int blk = 0; blk < NBLK; ++blk) {
 #pragma unroll
           for (int k2 = 0; k2 < 2; ++k2) {
-            if constexpr (PAIR) {
-              mma_ss_pair<BF16>(d_tmem, a_k, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, accum);
-              if (MH == 2) mma_ss_pair<BF16>(d_tmem + NT, a_k + 128u, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, accum);
-            } else {
-              ptx::mma_ss_lohi<BF16>(d_tmem, a_k, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, accum);
-              if (MH == 2) ptx::mma_ss_lohi<BF16>(d_tmem + NT, a_k + 128u, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, accum);
-            }
+            mma_ss_e<BF16, PAIR>(d_tmem, a_k, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, accum, elect);
+            if (MH == 2) mma_ss_e<BF16, PAIR>(d_tmem + NT, a_k + 128u, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, accum, elect);
             accum = 1;
             a_k += kstep16;
           }
           b_k += blk16;
         }
-        if constexpr (PAIR) mma_commit_pair(b_empty0 + (uint32_t)br.idx * 8u);
-        else ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u);
+        mma_commit_e<PAIR>(b_empty0 + (uint32_t)br.idx * 8u, elect);
         br.advance(P.SB);
       }
       if (!ok) break;
-      if constexpr (PAIR) mma_commit_pair(t_empty0 + (uint32_t)tr.idx * 8u);
-      else ptx::mma_commit(t_empty0 + (uint32_t)tr.idx * 8u);
+      mma_commit_e<PAIR>(t_empty0 + (uint32_t)tr.idx * 8u, elect);
     }
     if (!ok) break;
-    if constexpr (PAIR) mma_commit_pair(ptx::smem_u32(&bars->acc_full[dr.idx]));
-    else ptx::mma_commit(ptx::smem_u32(&bars->acc_full[dr.idx]));
+    mma_commit_e<PAIR>(ptx::smem_u32(&bars->acc_full[dr.idx]), elect);
   }
   SPROF_DUMP(1)
 }
@@ -316,7 +309,7 @@ conv_tc_strip_kernel(const SParams P, const __grid_constant__ CUtensorMap fmap, 
     // One thread.  Its instruction stream is what bounds narrow filter tiles, so the loop over one
     // T stage is fully unrolled for the compile-time (taps, filter blocks, halves) and steps the
     // descriptors by additions of registers computed once.
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
       if (P.MH == 1) mma_role<FW, S, BF16, 1, NBLK, PAIR>(P, bars, misc, tmem_base, t_sa, b_sa);
       else mma_role<FW, S, BF16, 2, NBLK, PAIR>(P, bars, misc, tmem_base, t_sa, b_sa);
     }
@@ -746,7 +739,7 @@ int choose_plan(const Geometry& g, Plan* best) {
 // comparison is between the two kernels' waves: small images whose tiles just fill one wave there stay
 // there.  In BF16 mode a filter small enough to stay resident in the persistent kernel's shared memory
 // also stays there.  Launches that fill less than half the SMs stay there too (reduction slices).
-template <int FH, int FW, int S, bool BF16>
+template <int FH, int FW, int S, bool BF16, int SRCK>
 bool strip_preferred(const Geometry& g, const SParams& P) {
   if (S != 1 || P.NT < 96) return false;
   if (BF16 && (int64_t)g.K * g.Kg * 2 <= 160 * 1024) return false;
@@ -760,7 +753,10 @@ bool strip_preferred(const Geometry& g, const SParams& P) {
   // (measured at batch 1 and 32 on the deepest layers)
   if (tiles * P.n_ntiles * 2 <= nsm) return false;
   const double persistent_passes = (double)((tiles * P.n_ntiles + nsm - 1) / nsm);
-  return BF16 ? strip_passes * 0.75 < persistent_passes : strip_passes * 0.8 <= persistent_passes;
+  // (BF16: a tie goes to this kernel where the source is the input itself or the bf16 tensor, a third or half of the
+  // fp32 tensor's staged bytes: sweep layer 7 fused 88 -> 77 us)
+  if (BF16) return SRCK != 0 ? strip_passes * 0.75 <= persistent_passes : strip_passes * 0.75 < persistent_passes;
+  return strip_passes * 0.8 <= persistent_passes;
 }
 
 template <int FH, int FW, int S, bool BF16, int SRCK, bool PAIR>
@@ -815,7 +811,7 @@ int launch_strip(const void* src, const float* f, float* out, const Geometry& g,
   int rc = choose_plan<FH, FW, S, BF16, SRCK>(g, &pl);
   if (rc != IM2WIN_OK) return rc;
   SParams& P = pl.P;
-  if (!even_if_slower && !knobs().force_strip && !strip_preferred<FH, FW, S, BF16>(g, P)) return IM2WIN_EUNSUPPORTED;
+  if (!even_if_slower && !knobs().force_strip && !strip_preferred<FH, FW, S, BF16, SRCK>(g, P)) return IM2WIN_EUNSUPPORTED;
   if (!scratch.ptr || scratch.bytes < pl.scratch_bytes || (reinterpret_cast<uintptr_t>(scratch.ptr) & 15u)) return IM2WIN_EUNSUPPORTED;
   EncodeTiledFn enc = encode_fn();
   if (!enc) return IM2WIN_EUNSUPPORTED;

@@ -138,8 +138,8 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
   uint32_t bc = 0;  // filter stages so far: with two issuing threads, thread `which` takes those of its parity
   (void)bc; (void)which;
   SPROF_DECL
-  const int32_t lane = 0;
-  (void)lane;
+  const int32_t lane = (int32_t)(threadIdx.x & 31);
+  const uint32_t elect = lane == 0 ? 1u : 0u;  // the whole warp runs this role; one lane issues
   const uint32_t RA = (uint32_t)P.RA, NT = (uint32_t)P.NT, idesc = P.idesc, W = (uint32_t)P.W;
   const uint64_t ad0 = ptx::smem_desc_k_chunkmajor(x_sa, RA * 16u);
   const uint64_t bd0 = ptx::smem_desc_k_sw64(b_sa);
@@ -153,13 +153,13 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
   for (int64_t it = 0; ok; ++it, dr.advance(P.ND)) {
     WUnit u;
     if (!wunit_at<PAIR>(P, it, 0, u)) break;
-    SPROF_W(0, ok = wait_bar(P, misc, ptx::smem_u32(&bars->acc_empty[dr.idx]), dr.phase ^ 1u, DEV_TIMEOUT_ACC))
+    SPROF_W(0, ok = wait_bar_warp(P, misc, ptx::smem_u32(&bars->acc_empty[dr.idx]), dr.phase ^ 1u, DEV_TIMEOUT_ACC))
     if (!ok) break;
     ptx::tc_fence_after();
     const uint32_t d_tmem = tmem_base + (uint32_t)(dr.idx * MH) * NT;
     uint32_t accum = two ? 1u : 0u;
     for (int32_t xs = 0; xs < P.NXS && ok; ++xs, xr.advance(2)) {
-      SPROF_W(1, ok = wait_bar(P, misc, x_full0 + (uint32_t)xr.idx * 8u, xr.phase, DEV_TIMEOUT_A_FULL, 20))
+      SPROF_W(1, ok = wait_bar_warp(P, misc, x_full0 + (uint32_t)xr.idx * 8u, xr.phase, DEV_TIMEOUT_A_FULL, 20))
       if (!ok) break;
       uint32_t a_u = a_lo0 + (uint32_t)xr.idx * x16;
 #pragma unroll 1
@@ -169,7 +169,7 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
           if constexpr (TWO) {
             if ((bc++ & 1u) != which) { br.advance(P.SB); continue; }
           }
-          SPROF_W(2, ok = wait_bar(P, misc, b_full0 + (uint32_t)br.idx * 8u, bres ? 0u : br.phase, DEV_TIMEOUT_B_FULL, 20))
+          SPROF_W(2, ok = wait_bar_warp(P, misc, b_full0 + (uint32_t)br.idx * 8u, bres ? 0u : br.phase, DEV_TIMEOUT_B_FULL, 20))
           if (!ok) break;
           ptx::tc_fence_after();
           // (block by block: consecutive MMAs onto the same accumulator run faster than alternating ones)
@@ -189,8 +189,7 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
               for (int blk = 0; blk < NBLK; ++blk) {
 #pragma unroll
                 for (int k2 = 0; k2 < 2; ++k2) {
-                  if constexpr (PAIR) mma_ss_pair<BF16>(d_tmem + (uint32_t)h * NT, a_k, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, acc);
-                  else ptx::mma_ss_lohi<BF16>(d_tmem + (uint32_t)h * NT, a_k, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, acc);
+                  mma_ss_e<BF16, PAIR>(d_tmem + (uint32_t)h * NT, a_k, a_hi, b_k + (uint32_t)k2 * 2u, b_hi, idesc, acc, elect);
                   acc = 1;
                   a_k += kstep16;
                 }
@@ -203,18 +202,16 @@ __device__ __forceinline__ void wmma_role(const WParams& P, SBars* bars, SMisc* 
           pw[3] += clock64() - cm0;
 #endif
           if (!bres) {
-            SPROF_W(4, if constexpr (PAIR) mma_commit_pair(b_empty0 + (uint32_t)br.idx * 8u); else ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u))
+            SPROF_W(4, mma_commit_e<PAIR>(b_empty0 + (uint32_t)br.idx * 8u, elect))
           }
           br.advance(P.SB);
         }
       }
       if (!ok) break;
-      if constexpr (PAIR) mma_commit_pair(x_empty0 + (uint32_t)xr.idx * 8u);
-      else ptx::mma_commit(x_empty0 + (uint32_t)xr.idx * 8u);
+      mma_commit_e<PAIR>(x_empty0 + (uint32_t)xr.idx * 8u, elect);
     }
     if (!ok) break;
-    if constexpr (PAIR) mma_commit_pair(ptx::smem_u32(&bars->acc_full[dr.idx]));
-    else ptx::mma_commit(ptx::smem_u32(&bars->acc_full[dr.idx]));
+    mma_commit_e<PAIR>(ptx::smem_u32(&bars->acc_full[dr.idx]), elect);
   }
   SPROF_DUMP(1)
 }
@@ -351,7 +348,7 @@ conv_tc_window_kernel(const WParams P, const __grid_constant__ CUtensorMap fmap,
       wait_bar(P, misc, ptx::smem_u32(&bars->raw_full[c % P.SR]), (uint32_t)(c / P.SR) & 1u, DEV_TIMEOUT_DRAIN);
   } else if (warp == 1 || (warp == 3 && P.two)) {
     // ================================================================ MMA ISSUER (one thread, or one each of warps 1 and 3)
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
       const uint32_t which = warp == 1 ? 0u : 1u;
       const int nblk = P.G / (4 * NCH);
 #define WRUN(MHv, NBv, TPv) do { if (!PAIR && P.two) wmma_role<FH, FW, BF16, MHv, NBv, TPv, PAIR, !PAIR>(P, bars, misc, tmem_base, x_sa, b_sa, which); \
@@ -847,10 +844,12 @@ int choose_wplan(const Geometry& g, WPlan* best) {
 // measured table (B200, batch 128, every stride-1 3x3 / 5x5 layer of the benchmark lists, three source kinds,
 // both modes).  Its strengths: the staged bytes and the interleaving work are a third of the strip-matrix
 // kernel's, and it has no per-thread window loads (the persistent kernel's bound on deep layers in BF16 mode).
-// It has no CTA-pair mode, so in TF32 mode and for the fused and bf16 sources the 256-wide filter tiles on
-// images of more than one block stay with the strip-matrix kernel; its one issuing thread is slower than the
-// persistent kernel's three on TF32 layers of 64 filters; and where the persistent kernel finishes in a single
-// wave of tiles that span images (small images, one filter tile) that kernel stays.
+// In TF32 mode and for the fused source the 256-wide filter tiles on images of more than one block stay with
+// the strip-matrix kernel's CTA pairs; TF32 layers of 64 filters from the fp32 im2win tensor stay with the
+// persistent kernel (a 64-column MMA from shared memory takes 54 cycles, that kernel's from tensor memory 32,
+// and the tensor's staged bytes are three times the input's), the same layers fused come here; and where the
+// persistent kernel finishes in a single wave of tiles that span images (small images, one filter tile) that
+// kernel stays.
 template <int FH, int FW, bool BF16, int SRCK>
 bool window_preferred(const Geometry& g, const WParams& P) {
   const int nsm = sm_count();
@@ -859,10 +858,10 @@ bool window_preferred(const Geometry& g, const WParams& P) {
   const int64_t span_tiles = (g.Mtot + 127) / 128;
   if (P.n_ntiles == 1 && span_tiles <= nsm && P.NT > 128) return false;  // one wave of the persistent kernel
   if (!BF16) {
-    if (SRCK == 1) return g.C >= 128 && P.NT >= 128 && P.NT <= 192;
+    if (SRCK == 1) return P.NT <= 64 || (g.C >= 128 && P.NT >= 128 && P.NT <= 192);
     return P.NT > 64 && P.NT <= 128;
   }
-  if (SRCK == 2) return P.NT <= 192;                                   // bf16 im2win tensor
+  if (SRCK == 2) return P.NT <= 192 || P.RPI >= 128;                   // bf16 im2win tensor
   if (SRCK == 1)                                                        // fused
     return (g.C >= 128 || P.NT <= 64) && (P.NT <= 192 || P.RPI < 128);
   return g.C >= 128;                                                    // fp32 im2win tensor

@@ -129,32 +129,40 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
-// D[tmem of both CTAs] (+)= A[each CTA's own rows] * B[each CTA holds half the N rows]; M = 256.
-template <bool BF16>
-__device__ __forceinline__ void mma_ss_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                            uint32_t idesc, uint32_t accumulate) {
-  if constexpr (BF16) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
-        "setp.ne.b32 p, %6, 0;\n\t"
-        "mov.b64 ad, {%1, %2};\n\t"
-        "mov.b64 bd, {%3, %4};\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], ad, bd, %5, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+// tcgen05.mma with both operands from shared memory (descriptors passed as 32-bit halves) and tcgen05.commit,
+// for one CTA or for a CTA pair (cta_group::2: D[tmem of both CTAs] (+)= A[each CTA's own rows] * B[each CTA
+// holds half the N rows], M = 256; the commit arrives on both CTAs' barriers).  The role that issues them is run
+// by a WHOLE warp (descriptor arithmetic and waits are then
+// warp-uniform work, which the compiler can keep in uniform registers: tcgen05.mma takes its operands from
+// those): only the lane with `elect` set issues.
+template <bool BF16, bool PAIR>
+__device__ __forceinline__ void mma_ss_e(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                         uint32_t idesc, uint32_t accumulate, uint32_t elect) {
+#define IM2WIN_MMA_E(GROUP, KIND)                                                                                   \
+  asm volatile("{\n\t.reg .pred p, q;\n\t.reg .b64 ad, bd;\n\t"                                                    \
+               "setp.ne.b32 p, %6, 0;\n\t"                                                                          \
+               "setp.ne.b32 q, %7, 0;\n\t"                                                                          \
+               "mov.b64 ad, {%1, %2};\n\t"                                                                          \
+               "mov.b64 bd, {%3, %4};\n\t"                                                                          \
+               "@q tcgen05.mma.cta_group::" GROUP ".kind::" KIND " [%0], ad, bd, %5, p;\n\t}"                        \
+               ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elect) : "memory")
+  if constexpr (PAIR) {
+    if constexpr (BF16) IM2WIN_MMA_E("2", "f16"); else IM2WIN_MMA_E("2", "tf32");
   } else {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
-        "setp.ne.b32 p, %6, 0;\n\t"
-        "mov.b64 ad, {%1, %2};\n\t"
-        "mov.b64 bd, {%3, %4};\n\t"
-        "tcgen05.mma.cta_group::2.kind::tf32 [%0], ad, bd, %5, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+    if constexpr (BF16) IM2WIN_MMA_E("1", "f16"); else IM2WIN_MMA_E("1", "tf32");
   }
+#undef IM2WIN_MMA_E
 }
-// Arrive on the barrier at the same shared-memory offset in both CTAs of the pair once every MMA issued so far is done.
-__device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-               ::"r"(bar), "h"((uint16_t)3) : "memory");
+template <bool PAIR>
+__device__ __forceinline__ void mma_commit_e(uint32_t bar, uint32_t elect) {
+  if constexpr (PAIR)
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t"
+                 "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}"
+                 ::"r"(bar), "h"((uint16_t)3), "r"(elect) : "memory");
+  else
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+                 "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+                 ::"r"(bar), "r"(elect) : "memory");
 }
 
 // Stores columns [c_begin, c_end) (multiples of 16) of one warp's 32 accumulator rows: TMEM -> registers
