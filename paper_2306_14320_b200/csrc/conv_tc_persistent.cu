@@ -692,7 +692,21 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     // barrier sees both of them in every phase.
     const uint32_t me = BRES ? (uint32_t)(warp - 1) : (warp == 3 ? 1u : 0u);
     (void)me;
-    if (lane == 0) {
+    // The whole warp runs the role and lane 0 issues: the descriptor arithmetic and the waits are then warp-uniform
+    // work (4-7 % on the TF32 layers, whose narrow MMAs the issue rate bounds).  One family keeps the one-thread
+    // form: the 7x7 three-channel stems in TF32 mode from the im2win tensor were measured 7 % slower with it.
+    constexpr bool WARP_ISSUE = !(FH == 7 && CB == 3 && !BF16 && !FUSED);
+    if (WARP_ISSUE || lane == 0) {
+      const uint32_t elect = lane == 0 ? 1u : 0u;
+      auto wait_role = [&](uint64_t* bar, uint32_t parity, int32_t code, long long* acc, uint32_t sleep_ns) -> bool {
+        if constexpr (WARP_ISSUE) return wait_bar_warp(P, misc, bar, parity, code, acc, sleep_ns);
+        else return wait_bar(P, misc, bar, parity, code, acc, sleep_ns);
+      };
+      auto poll_role = [&](uint32_t bar_addr, uint32_t parity) -> bool {
+        const bool r = ptx::mbar_try_wait(bar_addr, parity);
+        if constexpr (WARP_ISSUE) return __all_sync(0xffffffffu, r);
+        else return r;
+      };
       Ring ar0, ar1, ar2, br, dr;  // A slot (one ring per repack set), streamed filter stage, accumulator buffer
       uint32_t gset = 0;    // running group count modulo the number of sets = which set produced the group
       const uint32_t nsets = (uint32_t)P.NSETS;
@@ -708,11 +722,11 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
       const uint32_t a_full0 = ptx::smem_u32(&bars->a_full[0]), a_empty0 = ptx::smem_u32(&bars->a_empty[0]);
       const uint32_t b_full0 = ptx::smem_u32(&bars->b_full[0]), b_empty0 = ptx::smem_u32(&bars->b_empty[0]);
       (void)b_full0; (void)b_empty0;
-      if constexpr (BRES) ok = wait_bar(P, misc, &bars->b_full[0], 0u, DEV_TIMEOUT_B_FULL, PROF_SLOT(1));
+      if constexpr (BRES) ok = wait_role(&bars->b_full[0], 0u, DEV_TIMEOUT_B_FULL, PROF_SLOT(1), 64);
       for (int32_t t = blockIdx.x; t < (int32_t)P.ntiles && ok; t += gridDim.x, dr.advance(P.ND)) {
         const int32_t d = dr.idx;
         // the epilogue hands the buffer over zeroed (also before its first use)
-        ok = wait_bar(P, misc, &bars->acc_empty[d], dr.phase, DEV_TIMEOUT_ACC, PROF_SLOT(2));
+        ok = wait_role(&bars->acc_empty[d], dr.phase, DEV_TIMEOUT_ACC, PROF_SLOT(2), 64);
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(d * P.NT);
@@ -732,12 +746,12 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
               uint32_t st = st0;
               while (true) {
                 if ((st & 3u) == 0) {
-                  ok = wait_bar(P, misc, &bars->b_full[br.idx], br.phase, DEV_TIMEOUT_B_FULL, nullptr, 20);
+                  ok = wait_role(&bars->b_full[br.idx], br.phase, DEV_TIMEOUT_B_FULL, nullptr, 20);
                   if (!ok) break;
                 }
                 const uint32_t last = st | 3u;  // last step of the stage that holds step st
                 if (last >= end) break;         // the stage runs on into the next group
-                ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u);
+                ptx::mma_commit_if(b_empty0 + (uint32_t)br.idx * 8u, elect);
                 br.advance(P.SB);
                 st = last + 1u;
                 if (st >= end) break;
@@ -754,8 +768,8 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
           for (int h = 0; h < PARTS; ++h) {
             const int nst = (h == PARTS - 1) ? (S - (PARTS - 1) * SLOT_STEPS) : SLOT_STEPS;
             const int32_t slot = slot0 + ar.idx;
-            if (!ptx::mbar_try_wait(a_full0 + (uint32_t)slot * 8u, ar.phase)) {  // usually ready: one poll
-              ok = wait_bar(P, misc, &bars->a_full[slot], ar.phase, DEV_TIMEOUT_A_FULL, PROF_SLOT(0), 20);
+            if (!poll_role(a_full0 + (uint32_t)slot * 8u, ar.phase)) {  // usually ready: one poll
+              ok = wait_role(&bars->a_full[slot], ar.phase, DEV_TIMEOUT_A_FULL, PROF_SLOT(0), 20);
               if (!ok) break;
             }
             PROF_T0(tf)
@@ -774,8 +788,8 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
                   lo = lo_part + step_off[j];  // one add per MMA, no chain from step to step
                 } else {
                   if ((st & 3u) == 0) {
-                    if (!ptx::mbar_try_wait(b_full0 + (uint32_t)br.idx * 8u, br.phase)) {
-                      ok = wait_bar(P, misc, &bars->b_full[br.idx], br.phase, DEV_TIMEOUT_B_FULL, PROF_SLOT(1), 20);
+                    if (!poll_role(b_full0 + (uint32_t)br.idx * 8u, br.phase)) {
+                      ok = wait_role(&bars->b_full[br.idx], br.phase, DEV_TIMEOUT_B_FULL, PROF_SLOT(1), 20);
                       if (!ok) break;
                     }
                     ptx::tc_fence_after();
@@ -783,9 +797,9 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
                   }
                   lo = b_lo + (st & 3u) * 2u;
                 }
-                ptx::mma_ts_lohi<BF16>(d_tmem, a_addr + j * 8, lo, desc_hi, P.idesc, accum);
+                ptx::mma_ts_lohi_if<BF16>(d_tmem, a_addr + j * 8, lo, desc_hi, P.idesc, accum, elect);
                 if constexpr (!BRES) {
-                  if ((st & 3u) == 3u) { ptx::mma_commit(b_empty0 + (uint32_t)br.idx * 8u); br.advance(P.SB); }
+                  if ((st & 3u) == 3u) { ptx::mma_commit_if(b_empty0 + (uint32_t)br.idx * 8u, elect); br.advance(P.SB); }
                 }
               }
             }
@@ -793,7 +807,7 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
             PROF_ADD(4, tm)
             st0 += nst;
             PROF_T0(tc)
-            ptx::mma_commit(a_empty0 + (uint32_t)slot * 8u);
+            ptx::mma_commit_if(a_empty0 + (uint32_t)slot * 8u, elect);
             PROF_ADD(5, tc)
             ar.advance(P.NSS);
           }
@@ -801,11 +815,11 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
         }
         if (!ok) break;
         if constexpr (!BRES) {
-          if ((st0 & 3u) != 0) { ptx::mma_commit(ptx::smem_u32(&bars->b_empty[br.idx])); br.advance(P.SB); }
+          if ((st0 & 3u) != 0) { ptx::mma_commit_if(ptx::smem_u32(&bars->b_empty[br.idx]), elect); br.advance(P.SB); }
         }
-        ptx::mma_commit(ptx::smem_u32(&bars->acc_full[d]));
+        ptx::mma_commit_if(ptx::smem_u32(&bars->acc_full[d]), elect);
       }
-      if (me == 0) { PROF_DUMP(1, 7) }
+      if (me == 0 && lane == 0) { PROF_DUMP(1, 7) }
     }
     __syncwarp();
   } else if (warp == 2) {
