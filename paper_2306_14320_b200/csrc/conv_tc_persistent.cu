@@ -693,9 +693,10 @@ conv_tc_persistent_kernel(const PParams P, const __grid_constant__ CUtensorMap f
     const uint32_t me = BRES ? (uint32_t)(warp - 1) : (warp == 3 ? 1u : 0u);
     (void)me;
     // The whole warp runs the role and lane 0 issues: the descriptor arithmetic and the waits are then warp-uniform
-    // work (4-7 % on the TF32 layers, whose narrow MMAs the issue rate bounds).  One family keeps the one-thread
-    // form: the 7x7 three-channel stems in TF32 mode from the im2win tensor were measured 7 % slower with it.
-    constexpr bool WARP_ISSUE = !(FH == 7 && CB == 3 && !BF16 && !FUSED);
+    // work (4-7 % on the TF32 layers, whose narrow MMAs the issue rate bounds).  Two families keep the one-thread
+    // form, measured slower with it: the 7x7 three-channel stems in TF32 mode from the im2win tensor (7 %), and
+    // streamed filters other than 3x3 (the 5x5 layers: 18-22 %).
+    constexpr bool WARP_ISSUE = (BRES || FH == 3) && !(FH == 7 && CB == 3 && !BF16 && !FUSED);
     if (WARP_ISSUE || lane == 0) {
       const uint32_t elect = lane == 0 ? 1u : 0u;
       auto wait_role = [&](uint64_t* bar, uint32_t parity, int32_t code, long long* acc, uint32_t sleep_ns) -> bool {
