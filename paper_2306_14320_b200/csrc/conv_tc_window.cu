@@ -710,10 +710,31 @@ int make_wplan(const Geometry& g, WPlan* pl, int pair, int mh_fixed) {
   const Try order_fused[] = {{2, FW, 16}, {2, FW, 8}, {2, 1, 32}, {2, 1, 16}, {1, FW, 32}, {1, FW, 16}, {1, 1, 16}, {1, 1, 8}, {1, 1, 4}};
   const Try order_win[] = {{1, FW, 16}, {1, FW, 8}, {2, 1, 8}, {1, 1, 8}, {1, 1, 4}, {1, 1, 16}};
   const Try order_win16[] = {{1, FW, 32}, {1, FW, 16}, {2, 1, 16}, {1, 1, 16}, {1, 1, 8}, {1, 1, 32}};
-  const Try* order = SRCK == 1 ? order_fused : (SRCK == 2 ? order_win16 : order_win);
-  const int n_order = SRCK == 1 ? 9 : 6;
-  // (resident only where source stages of sixteen channels still fit: with smaller ones it was measured slower)
-  const Try order_res[] = {{2, FW, 32}, {2, FW, 16}, {1, FW, 32}, {1, FW, 16}};
+  const Try* order_tail = SRCK == 1 ? order_fused : (SRCK == 2 ? order_win16 : order_win);
+  const int n_tail = SRCK == 1 ? 9 : 6;
+  // In front of those, the measured exceptions: 256-wide filter tiles want one filter block per X stage (a stage of
+  // two blocks x Fw taps x 256 rows is 96 KB, and two of them leave the other rings too little): fused with two
+  // 128-row blocks {1,Fw,16} (the deep 3x3 layers in BF16 mode: 50 -> 43, 62 -> 56, 83 -> 74 us), with one block
+  // (images under 128 positions) {2,Fw,32}; from the fp32 tensor eight or four channels per source stage for tiles
+  // of 192 and more (TF32: 108 -> 98, 151 -> 134 us on the 384-filter layers).
+  Try order_all[12];
+  int n_order = 0;
+  if (SRCK == 1) {
+    if (P.NT >= 256) order_all[n_order++] = P.MH == 2 ? Try{1, FW, 16} : Try{2, FW, 32};
+  } else if (SRCK == 0 && P.MH == 2) {  // (images of a single block keep the general order: measured)
+    if (BF16) {
+      if (P.NT >= 256 && FH == 3) order_all[n_order++] = Try{1, 1, 16};
+      if (P.NT >= 192) order_all[n_order++] = Try{1, FW, 8};
+    } else {
+      if (P.NT >= 256 && FH == 3) order_all[n_order++] = Try{1, FW, 4};
+      if (P.NT >= 192) order_all[n_order++] = Try{1, FW, 8};
+    }
+  }
+  for (int t = 0; t < n_tail; ++t) order_all[n_order++] = order_tail[t];
+  const Try* order = order_all;
+  // (resident only where source stages of sixteen channels still fit: with smaller ones it was measured slower;
+  // one filter block per X stage first: `resnet3x3` BF16 fused 71 -> 60 us)
+  const Try order_res[] = {{1, FW, 32}, {1, FW, 16}, {2, FW, 32}, {2, FW, 16}};
   bool found = false;
   for (int pass = 0; pass < 2 && !found; ++pass) {  // first the resident filter, then the streamed one
     if (pass == 0 && (pair || P.n_ntiles != 1 || knobs().window_bres == 2)) continue;
@@ -854,16 +875,15 @@ template <int FH, int FW, bool BF16, int SRCK>
 bool window_preferred(const Geometry& g, const WParams& P) {
   const int nsm = sm_count();
   if (P.units * 2 <= nsm) return false;  // under-filled launches: the persistent kernel's reduction slices
-  if (FH == 5) return BF16 || SRCK == 0;  // 5x5 layers: 25 taps of one staged tile (TF32: from the tensor only)
+  if (FH == 5) return BF16 || (SRCK == 0 && P.RPI < 640);  // 5x5 layers: 25 taps of one staged tile (TF32: from the tensor, smaller images)
   const int64_t span_tiles = (g.Mtot + 127) / 128;
   if (P.n_ntiles == 1 && span_tiles <= nsm && P.NT > 128) return false;  // one wave of the persistent kernel
   if (!BF16) {
     if (SRCK == 1) return P.NT <= 64 || (g.C >= 128 && P.NT >= 128 && P.NT <= 192);
-    return P.NT > 64 && P.NT <= 128;
+    return P.NT > 64 && P.NT <= 192;
   }
   if (SRCK == 2) return P.NT <= 192 || P.RPI >= 128;                   // bf16 im2win tensor
-  if (SRCK == 1)                                                        // fused
-    return (g.C >= 128 || P.NT <= 64) && (P.NT <= 192 || P.RPI < 128);
+  if (SRCK == 1) return g.C >= 128 || P.NT <= 64;                      // fused
   return g.C >= 128;                                                    // fp32 im2win tensor
 }
 
