@@ -116,7 +116,7 @@ int im2win_transform_bf16(const float* in_nchw, const im2win_shape* shape, uint1
  *            needs and reads the windows from them, so nothing of size Ihat is written (workspace
  *            0 bytes).  Same result as the other two kinds.  Shapes without a fused specialisation
  *            (the specialised filter sizes are 3x3, 5x5, 7x7, 11x11 and, with channel counts that are
- *            multiples of 16, 1x1, 1x3, 3x1, 1x7, 7x1) fall back to transform + convolution if a
+ *            multiples of 16, 1x1, 1x3, 3x1, 1x7, 7x1, 2x2, 4x4, 3x5, 5x3) fall back to transform + convolution if a
  *            sufficient `workspace` is given, else EUNSUPPORTED; IM2WIN_MODE_FP32 always takes that
  *            fallback.
  *            src_kind IM2WIN_BF16: a bf16 im2win tensor from im2win_transform_bf16; mode must be

@@ -34,7 +34,7 @@ def _stale() -> bool:
 
 # conv_tc_persistent.cu holds four families of kernel instantiations (by filter size); compiled as
 # four translation units (-DIM2WIN_PART=k) they build in parallel.
-PARTS = {"conv_tc_persistent.cu": 6}
+PARTS = {"conv_tc_persistent.cu": 8}
 
 
 def build_library(force: bool = False, verbose: bool = False, out: str | None = None,

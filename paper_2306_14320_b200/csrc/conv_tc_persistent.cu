@@ -1546,7 +1546,8 @@ int launch_spec(const void* src, const float* f, float* out, const Geometry& g, 
 // (no im2win tensor exists in global memory).
 // The filter-size families are separate functions so that the build can compile them as separate
 // translation units in parallel (-DIM2WIN_PART=0..5: part 0 = 3x3 + this dispatcher, 1 = 5x5,
-// 2 = 7x7, 3 = 11x11, 4 = 1x1 / 1x3 / 3x1, 5 = 1x7 / 7x1; without the macro everything is compiled here).
+// 2 = 7x7, 3 = 11x11, 4 = 1x1 / 1x3 / 3x1, 5 = 1x7 / 7x1, 6 = 2x2 / 4x4, 7 = 3x5 / 5x3; without the macro
+// everything is compiled here).
 #ifndef IM2WIN_PART
 #define IM2WIN_PART -1
 #endif
@@ -1558,6 +1559,8 @@ int launch_spec_7x7(IM2WIN_SPEC_ARGS);
 int launch_spec_11x11(IM2WIN_SPEC_ARGS);
 int launch_spec_rect_a(IM2WIN_SPEC_ARGS);
 int launch_spec_rect_b(IM2WIN_SPEC_ARGS);
+int launch_spec_rect_c(IM2WIN_SPEC_ARGS);
+int launch_spec_rect_d(IM2WIN_SPEC_ARGS);
 
 #if IM2WIN_PART == -1 || IM2WIN_PART == 0
 int launch_spec_3x3(IM2WIN_SPEC_ARGS) {
@@ -1610,7 +1613,8 @@ int launch_spec_11x11(IM2WIN_SPEC_ARGS) {
 }
 #endif
 
-// Pointwise and factorised filters (1x1; 1x3 / 3x1; 1x7 / 7x1): the same kernel, from the fp32 im2win tensor or
+// Pointwise, factorised, patch and other small rectangular filters (1x1; 1x3 / 3x1; 1x7 / 7x1; 2x2, 4x4; 3x5 / 5x3):
+// the same kernel, from the fp32 im2win tensor or
 // fused, fp32 NCHW or NHWC output (the bf16 storage variants of these shapes go to the generic kernel).
 // Sixteen channels per group (TF32: two to six MMA steps, BF16: one to seven, no padding); 1x7 / 7x1 in TF32
 // mode: eight (seven steps).
@@ -1628,9 +1632,18 @@ int launch_spec_rect(IM2WIN_SPEC_ARGS) {
     }
   }
   if (bf16) {
-    if (g.C % 16 != 0) return IM2WIN_EUNSUPPORTED;
-    return kind == 1 ? launch_spec_impl<FH, FW, 16, true, true>(xhat, f, out, g, st, scratch)
+    int rc = IM2WIN_EUNSUPPORTED;
+    if (g.C % 16 == 0)
+      rc = kind == 1 ? launch_spec_impl<FH, FW, 16, true, true>(xhat, f, out, g, st, scratch)
                      : launch_spec_impl<FH, FW, 16, true, false>(xhat, f, out, g, st, scratch);
+    // an even number of taps: eight channels are whole MMA steps too, for strips too long for sixteen-channel
+    // stages (4x4 with stride 4: 16 floats per position)
+    if constexpr ((8 * FH * FW) % 16 == 0 && FH * FW >= 4) {
+      if (rc == IM2WIN_EUNSUPPORTED)
+        rc = kind == 1 ? launch_spec_impl<FH, FW, 8, true, true>(xhat, f, out, g, st, scratch)
+                       : launch_spec_impl<FH, FW, 8, true, false>(xhat, f, out, g, st, scratch);
+    }
+    return rc;
   }
   constexpr int CBT = FH * FW >= 7 ? 8 : 16;
   if (g.C % CBT != 0) return IM2WIN_EUNSUPPORTED;
@@ -1653,6 +1666,21 @@ int launch_spec_rect_b(IM2WIN_SPEC_ARGS) {
 }
 #endif
 
+#if IM2WIN_PART == -1 || IM2WIN_PART == 6
+int launch_spec_rect_c(IM2WIN_SPEC_ARGS) {  // the patch / downsampling filters
+  if (g.Fh == 2 && g.Fw == 2) return launch_spec_rect<2, 2>(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh == 4 && g.Fw == 4) return launch_spec_rect<4, 4>(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  return IM2WIN_EUNSUPPORTED;
+}
+#endif
+#if IM2WIN_PART == -1 || IM2WIN_PART == 7
+int launch_spec_rect_d(IM2WIN_SPEC_ARGS) {
+  if (g.Fh == 3 && g.Fw == 5) return launch_spec_rect<3, 5>(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh == 5 && g.Fw == 3) return launch_spec_rect<5, 3>(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  return IM2WIN_EUNSUPPORTED;
+}
+#endif
+
 #if IM2WIN_PART == -1 || IM2WIN_PART == 0
 int launch_conv_tc_persistent(const void* xhat, const float* f, float* out, const Geometry& g, int mode,
                               cudaStream_t st, Scratch scratch, bool fused, bool src_bf16, bool out_bf16) {
@@ -1666,6 +1694,8 @@ int launch_conv_tc_persistent(const void* xhat, const float* f, float* out, cons
   if (g.Fh == 1 && g.Fw == 7 || g.Fh == 7 && g.Fw == 1) return launch_spec_rect_b(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
   if (g.Fh * g.Fw <= 3 && (g.Fh == 1 || g.Fw == 1) && g.Fh * g.Fw != 2)
     return launch_spec_rect_a(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh == g.Fw && (g.Fh == 2 || g.Fh == 4)) return launch_spec_rect_c(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
+  if (g.Fh * g.Fw == 15 && (g.Fh == 3 || g.Fh == 5)) return launch_spec_rect_d(xhat, f, out, g, st, scratch, kind, out_bf16, bf16);
   return IM2WIN_EUNSUPPORTED;
 }
 

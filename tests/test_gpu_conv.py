@@ -45,8 +45,11 @@ SMALL = [
     # counts of 32 (the pointwise groups), 16 and 8 (TF32 1x7), strides, two filter tiles, tiles that span images
     (3, 64, 9, 11, 40, 1, 1, 1), (2, 48, 14, 13, 300, 1, 1, 2), (2, 32, 12, 17, 24, 1, 3, 1), (2, 16, 17, 12, 33, 3, 1, 2),
     (1, 24, 9, 40, 20, 1, 7, 1), (2, 16, 30, 9, 130, 7, 1, 1), (4, 8, 6, 9, 16, 1, 7, 3),
+    # patch / downsampling filters and 3x5 / 5x3 (also families of the persistent kernel)
+    (2, 32, 18, 22, 40, 2, 2, 2), (2, 16, 36, 40, 24, 4, 4, 4), (2, 16, 13, 19, 300, 3, 5, 1), (1, 32, 21, 11, 17, 5, 3, 2),
 ]
-RECT_SHAPES = [d for d in SMALL if (d[5], d[6]) in ((1, 1), (1, 3), (3, 1), (1, 7), (7, 1)) and d[1] % 8 == 0]
+RECT_FAMILIES = ((1, 1), (1, 3), (3, 1), (1, 7), (7, 1), (2, 2), (4, 4), (3, 5), (5, 3))
+RECT_SHAPES = [d for d in SMALL if (d[5], d[6]) in RECT_FAMILIES and d[1] % 8 == 0]
 STRIP_SHAPES = [d for d in SMALL if d[5] == 3 and d[6] == 3 and d[1] % 32 == 0 and d[7] in (1, 2)]
 WINDOW_SHAPES = [d for d in SMALL if (d[5], d[6]) in ((3, 3), (5, 5)) and d[1] % 32 == 0 and d[7] == 1]
 
@@ -173,15 +176,15 @@ def test_forced_window_configurations_run_the_window_kernel(dims, mode, src_kind
 @pytest.mark.parametrize("mode", [b.MODE_TF32, b.MODE_BF16], ids=MODE_ID.get)
 @pytest.mark.parametrize("dims", RECT_SHAPES)
 def test_pointwise_and_factorised_filters_run_the_persistent_kernel(dims, mode, src_kind, _kernel):
-    """1x1, 1x3 / 3x1 and 1x7 / 7x1 filters are families of the persistent kernel, not cases of the generic
-    one: the configurations that leave the choice to the library must run it (BF16 mode: channel counts
-    that are multiples of 16; TF32 1x7 / 7x1: of 8)."""
+    """1x1, 1x3 / 3x1, 1x7 / 7x1, 2x2, 4x4 and 3x5 / 5x3 filters are families of the persistent kernel, not cases
+    of the generic one: the configurations that leave the choice to the library must run it (channel counts
+    that are multiples of 16; in TF32 mode with seven or more taps: of 8)."""
     if _kernel not in ("nostrip", "nobox", "nopim", "split3", "bslice"):
         pytest.skip("only for the test-build configurations that leave the persistent kernel its own choice")
     x, f = _data(dims, 820, ints=True)
     got = gpu_conv(x, f, dims, mode, src_kind=src_kind)
     c, taps = dims[1], dims[5] * dims[6]
-    if c % 16 == 0 or (mode == b.MODE_TF32 and taps == 7):
+    if c % 16 == 0 or (mode == b.MODE_TF32 and taps >= 7):
         assert b.last_kernel() == b.KERNEL_PERSISTENT
     assert np.array_equal(got.astype(np.float64), oracle_conv(x, f, dims))
 
